@@ -1,0 +1,175 @@
+/*
+ * cudallm_gemm.h -- C ABI of the B200 (sm_100a) bf16 GEMM library.
+ *
+ * The operation is the paper's benchmark Task 2, "Matrix Multiplication":
+ * given A (M x K) and B (K x N) compute C = A x B (M x N), i.e.
+ *
+ *     C[i][j] = sum_{k=0}^{K-1} A[i][k] * B[k][j]
+ *
+ * with all three matrices stored row-major as flat arrays (the storage the
+ * paper's task descriptions state for its matrix tasks).  Here A and B hold
+ * bfloat16, products are accumulated in fp32 and C is written as fp32 or
+ * bfloat16 (rounded once, to nearest even).  Old contents of C are never
+ * read (beta = 0).
+ *
+ * The paper's programs own their buffers and transfers in host code and hand
+ * raw device pointers to one kernel launch (Section 2, "CUDA program"); the
+ * calls below keep that split: the caller owns every buffer, the library only
+ * enqueues work on the caller's stream.
+ *
+ * General conventions
+ *  - Unless a parameter says "host", pointers are DEVICE pointers.
+ *  - Leading dimensions and batch strides are in ELEMENTS, not bytes.
+ *  - Every call returns a status: 0 on success, a negative CUDALLM_ERR_* code
+ *    otherwise.  Argument errors are detected before any CUDA call is made,
+ *    and nothing is written in that case.
+ *  - Calls enqueue on `stream` (a cudaStream_t passed as void*; NULL is the
+ *    legacy default stream) and return without synchronising, except where
+ *    stated.
+ *  - Only element alignment is required (2 bytes for bf16, 4 for fp32
+ *    output).  16-byte aligned bases with leading dimensions that are
+ *    multiples of 8 elements take the direct TMA path; other operands are
+ *    first repacked into the library workspace.
+ *  - Degenerate sizes: M == 0 or N == 0 or batch == 0 -> success, nothing
+ *    written.  K == 0 -> the M x N block of C is set to zero.
+ *  - Padding columns of C (N <= j < ldc) are left untouched.
+ *  - C must not overlap A or B.
+ *  - The library is for compute capability 10.0 devices only and has no CPU
+ *    fallback.
+ *  - Calls that need the workspace (repacking, split-K) share one workspace
+ *    per device; such calls must not run concurrently on different streams.
+ */
+#ifndef CUDALLM_GEMM_H
+#define CUDALLM_GEMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* out_dtype */
+#define CUDALLM_F32  0
+#define CUDALLM_BF16 1
+
+/* status codes */
+#define CUDALLM_OK                      0
+#define CUDALLM_ERR_INVALID_POINTER    -1  /* NULL operand with a non-empty problem            */
+#define CUDALLM_ERR_INVALID_DIM        -2  /* negative size, or sizes beyond what is indexable  */
+#define CUDALLM_ERR_INVALID_LD         -3  /* lda < K, ldb < N, ldc < N, or overlapping strides */
+#define CUDALLM_ERR_INVALID_DTYPE      -4
+#define CUDALLM_ERR_INVALID_VARIANT    -5
+#define CUDALLM_ERR_UNSUPPORTED_SHAPE  -6  /* forced variant cannot run this problem            */
+#define CUDALLM_ERR_UNSUPPORTED_DEVICE -7  /* current device is not compute capability 10.0     */
+#define CUDALLM_ERR_CUDA               -8  /* a CUDA runtime/driver call failed                 */
+#define CUDALLM_ERR_DEVICE_TIMEOUT     -9  /* a bounded wait inside a kernel ran out            */
+#define CUDALLM_ERR_WORKSPACE         -10  /* workspace missing, too small or misaligned        */
+#define CUDALLM_ERR_MISALIGNED        -11  /* pointer not aligned to its element size           */
+
+/* variant id meaning "let the library choose" */
+#define CUDALLM_VARIANT_AUTO           -1
+
+/*
+ * C = A x B  (Task 2).
+ *   A : bf16, M x K, row stride lda >= K      (read only)
+ *   B : bf16, K x N, row stride ldb >= N      (read only)
+ *   C : fp32 (out_dtype 0) or bf16 (out_dtype 1), M x N, row stride ldc >= N
+ */
+int cudallm_gemm_bf16(const void *A, const void *B, void *C,
+                      int64_t M, int64_t N, int64_t K,
+                      int64_t lda, int64_t ldb, int64_t ldc,
+                      int out_dtype, void *stream);
+
+/*
+ * `batch` independent products of the same shape (Task 2 applied per item;
+ * the paper's Task 6 score matrices Q_i K_i^T are products of this kind).
+ * Item t uses A + t*strideA, B + t*strideB, C + t*strideC.  Items of C must
+ * not overlap: strideC >= (M-1)*ldc + N when batch > 1.
+ */
+int cudallm_gemm_bf16_batched(const void *A, const void *B, void *C,
+                              int64_t M, int64_t N, int64_t K,
+                              int64_t lda, int64_t ldb, int64_t ldc,
+                              int64_t strideA, int64_t strideB, int64_t strideC,
+                              int64_t batch, int out_dtype, void *stream);
+
+/*
+ * As the batched call, but runs kernel variant `variant` instead of the
+ * library's choice (CUDALLM_VARIANT_AUTO selects as the calls above do).
+ * This is the hook for the search loop of the paper's Algorithm 1: candidates
+ * are validated, timed and the fastest valid one kept.  Returns
+ * CUDALLM_ERR_UNSUPPORTED_SHAPE when the variant cannot run the problem.
+ */
+int cudallm_gemm_bf16_variant(int variant,
+                              const void *A, const void *B, void *C,
+                              int64_t M, int64_t N, int64_t K,
+                              int64_t lda, int64_t ldb, int64_t ldc,
+                              int64_t strideA, int64_t strideB, int64_t strideC,
+                              int64_t batch, int out_dtype, void *stream);
+
+/*
+ * The same product with HOST buffers (the paper's host-code pattern: copy the
+ * operands in, launch, copy the result out).  A_host, B_host and C_host are
+ * host pointers (pinned memory makes the copies asynchronous); `dev_buf` is a
+ * caller-owned DEVICE staging buffer of `dev_bytes` bytes, at least
+ * cudallm_host_staging_bytes(...) and 256-byte aligned.  The call copies
+ * M*lda and K*ldb elements in, multiplies, copies M*ldc elements out, and
+ * SYNCHRONISES `stream` before returning.
+ */
+int cudallm_gemm_bf16_host(const void *A_host, const void *B_host, void *C_host,
+                           int64_t M, int64_t N, int64_t K,
+                           int64_t lda, int64_t ldb, int64_t ldc,
+                           int out_dtype, void *dev_buf, size_t dev_bytes,
+                           void *stream);
+size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K,
+                                  int64_t lda, int64_t ldb, int64_t ldc,
+                                  int out_dtype);
+
+/* Kernel variants (the candidate set of Algorithm 1's search). */
+int cudallm_num_variants(void);
+const char *cudallm_variant_name(int variant);            /* NULL if out of range */
+/* 1 if `variant` can run the problem, 0 if not, negative status on bad args. */
+int cudallm_variant_supports(int variant,
+                             int64_t M, int64_t N, int64_t K,
+                             int64_t lda, int64_t ldb, int64_t ldc,
+                             int64_t batch, int out_dtype);
+/* Variant the library would choose for this problem (host-side decision only;
+ * no CUDA call).  `a_aligned`/`b_aligned` say whether the operand base is
+ * 16-byte aligned.  Returns a variant id or a negative status. */
+int cudallm_select_variant(int64_t M, int64_t N, int64_t K,
+                           int64_t lda, int64_t ldb, int64_t ldc,
+                           int64_t batch, int out_dtype);
+
+/*
+ * Workspace.  Upper bound of the scratch bytes any variant may need for the
+ * problem (repacked operands, split-K partial tiles, tile counters).  Without
+ * cudallm_set_workspace the library allocates (and grows) one workspace per
+ * device with cudaMalloc on demand.  A caller-provided workspace must be
+ * 256-byte aligned, zero-filled once before first use, and stay valid until
+ * replaced; pass (NULL, 0) to return to the internal one.  It applies to the
+ * device that is current at the time of the call.
+ */
+size_t cudallm_workspace_bytes(int64_t M, int64_t N, int64_t K,
+                               int64_t lda, int64_t ldb, int64_t ldc,
+                               int64_t batch, int out_dtype);
+int cudallm_set_workspace(void *dev_ptr, size_t bytes);
+
+/*
+ * Synchronises `stream`, then reads and clears the device status word that
+ * kernels set when one of their bounded waits ran out.  *code is CUDALLM_OK or
+ * CUDALLM_ERR_DEVICE_TIMEOUT, *detail identifies the wait (role and barrier).
+ * Returns *code (or CUDALLM_ERR_CUDA if the synchronisation failed).
+ */
+int cudallm_device_status(void *stream, int *code, int *detail);
+
+/* Text for a status code; for CUDALLM_ERR_CUDA includes the last CUDA error
+ * text seen by the calling thread.  Never NULL. */
+const char *cudallm_strerror(int status);
+
+/* major*10000 + minor*100 + patch */
+int cudallm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CUDALLM_GEMM_H */

@@ -1,0 +1,175 @@
+"""ctypes binding of ``libcudallm_gemm.so``: one Python function per C entry
+point, same names, argument marshalling only.
+
+Device buffers are passed as integer addresses (``tensor.data_ptr()``) or as
+torch tensors (their ``data_ptr()`` is taken); streams as integer handles
+(``torch.cuda.current_stream().cuda_stream``).  Nothing here computes: if the
+shared library is missing this module raises, it never falls back to the CPU.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+F32, BF16 = 0, 1
+VARIANT_AUTO = -1
+
+OK = 0
+ERR_INVALID_POINTER = -1
+ERR_INVALID_DIM = -2
+ERR_INVALID_LD = -3
+ERR_INVALID_DTYPE = -4
+ERR_INVALID_VARIANT = -5
+ERR_UNSUPPORTED_SHAPE = -6
+ERR_UNSUPPORTED_DEVICE = -7
+ERR_CUDA = -8
+ERR_DEVICE_TIMEOUT = -9
+ERR_WORKSPACE = -10
+ERR_MISALIGNED = -11
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libcudallm_gemm.so")
+_lib = None
+
+_i64 = ctypes.c_int64
+_vp = ctypes.c_void_p
+_int = ctypes.c_int
+_sz = ctypes.c_size_t
+
+# name -> (restype, argtypes); mirrors include/cudallm_gemm.h
+SIGNATURES = {
+    "cudallm_gemm_bf16": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp]),
+    "cudallm_gemm_bf16_batched": (_int, [_vp, _vp, _vp] + [_i64] * 10 + [_int, _vp]),
+    "cudallm_gemm_bf16_variant": (_int, [_int, _vp, _vp, _vp] + [_i64] * 10 + [_int, _vp]),
+    "cudallm_gemm_bf16_host": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp, _sz, _vp]),
+    "cudallm_host_staging_bytes": (_sz, [_i64] * 6 + [_int]),
+    "cudallm_num_variants": (_int, []),
+    "cudallm_variant_name": (ctypes.c_char_p, [_int]),
+    "cudallm_variant_supports": (_int, [_int] + [_i64] * 7 + [_int]),
+    "cudallm_select_variant": (_int, [_i64] * 7 + [_int]),
+    "cudallm_workspace_bytes": (_sz, [_i64] * 7 + [_int]),
+    "cudallm_set_workspace": (_int, [_vp, _sz]),
+    "cudallm_device_status": (_int, [_vp, ctypes.POINTER(_int), ctypes.POINTER(_int)]),
+    "cudallm_strerror": (ctypes.c_char_p, [_int]),
+    "cudallm_version": (_int, []),
+}
+
+
+class CudallmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status}: {strerror(status)}")
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2506_09092_b200.build` "
+                "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _p(x):
+    """Address of a device/host buffer: int, None, or anything with data_ptr()."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    raise TypeError(type(x))
+
+
+def _s(stream):
+    if stream is None:
+        return None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def _check(st: int, where: str, check: bool):
+    if check and st != OK:
+        raise CudallmError(st, where)
+    return st
+
+
+def gemm_bf16(A, B, C, M, N, K, lda, ldb, ldc, out_dtype, stream=None, check=True):
+    st = lib().cudallm_gemm_bf16(_p(A), _p(B), _p(C), M, N, K, lda, ldb, ldc, out_dtype, _s(stream))
+    return _check(st, "cudallm_gemm_bf16", check)
+
+
+def gemm_bf16_batched(A, B, C, M, N, K, lda, ldb, ldc, strideA, strideB, strideC, batch,
+                      out_dtype, stream=None, check=True):
+    st = lib().cudallm_gemm_bf16_batched(_p(A), _p(B), _p(C), M, N, K, lda, ldb, ldc,
+                                         strideA, strideB, strideC, batch, out_dtype, _s(stream))
+    return _check(st, "cudallm_gemm_bf16_batched", check)
+
+
+def gemm_bf16_variant(variant, A, B, C, M, N, K, lda, ldb, ldc, strideA, strideB, strideC, batch,
+                      out_dtype, stream=None, check=True):
+    st = lib().cudallm_gemm_bf16_variant(variant, _p(A), _p(B), _p(C), M, N, K, lda, ldb, ldc,
+                                         strideA, strideB, strideC, batch, out_dtype, _s(stream))
+    return _check(st, "cudallm_gemm_bf16_variant", check)
+
+
+def gemm_bf16_host(A_host, B_host, C_host, M, N, K, lda, ldb, ldc, out_dtype, dev_buf, dev_bytes,
+                   stream=None, check=True):
+    st = lib().cudallm_gemm_bf16_host(_p(A_host), _p(B_host), _p(C_host), M, N, K, lda, ldb, ldc,
+                                      out_dtype, _p(dev_buf), dev_bytes, _s(stream))
+    return _check(st, "cudallm_gemm_bf16_host", check)
+
+
+def host_staging_bytes(M, N, K, lda, ldb, ldc, out_dtype) -> int:
+    return int(lib().cudallm_host_staging_bytes(M, N, K, lda, ldb, ldc, out_dtype))
+
+
+def num_variants() -> int:
+    return int(lib().cudallm_num_variants())
+
+
+def variant_name(variant: int):
+    s = lib().cudallm_variant_name(variant)
+    return None if s is None else s.decode()
+
+
+def variant_supports(variant, M, N, K, lda, ldb, ldc, batch, out_dtype) -> int:
+    return int(lib().cudallm_variant_supports(variant, M, N, K, lda, ldb, ldc, batch, out_dtype))
+
+
+def select_variant(M, N, K, lda, ldb, ldc, batch, out_dtype) -> int:
+    return int(lib().cudallm_select_variant(M, N, K, lda, ldb, ldc, batch, out_dtype))
+
+
+def workspace_bytes(M, N, K, lda, ldb, ldc, batch, out_dtype) -> int:
+    return int(lib().cudallm_workspace_bytes(M, N, K, lda, ldb, ldc, batch, out_dtype))
+
+
+def set_workspace(dev_ptr, nbytes: int, check=True):
+    return _check(lib().cudallm_set_workspace(_p(dev_ptr), nbytes), "cudallm_set_workspace", check)
+
+
+def device_status(stream=None):
+    """(code, detail) after synchronising ``stream``."""
+    code, detail = _int(0), _int(0)
+    lib().cudallm_device_status(_s(stream), ctypes.byref(code), ctypes.byref(detail))
+    return code.value, detail.value
+
+
+def strerror(status: int) -> str:
+    return lib().cudallm_strerror(status).decode()
+
+
+def version() -> int:
+    return int(lib().cudallm_version())

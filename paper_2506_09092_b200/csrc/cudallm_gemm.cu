@@ -1,0 +1,674 @@
+// C ABI of the bf16 GEMM library: argument validation, variant table and
+// selection, workspace, tensor-map encoding and kernel launches.
+// See include/cudallm_gemm.h for the contract of every entry point.
+#include "../../include/cudallm_gemm.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "aux_kernels.cuh"
+#include "umma_gemm.cuh"
+
+using namespace cudallm;
+
+namespace {
+
+// ------------------------------------------------------------------ errors --
+thread_local char g_cuda_err[256] = "";
+
+int cuda_fail(cudaError_t e, const char *where)
+{
+    snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", where, cudaGetErrorString(e));
+    return CUDALLM_ERR_CUDA;
+}
+#define CUDA_TRY(expr)                                          \
+    do {                                                        \
+        cudaError_t e__ = (expr);                               \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #expr);   \
+    } while (0)
+
+// ----------------------------------------------------------------- problem --
+struct Problem {
+    const void *A, *B;
+    void *C;
+    int64_t M, N, K, lda, ldb, ldc, sA, sB, sC, batch;
+    int out_dtype;
+};
+
+constexpr int64_t kMaxDim = (int64_t(1) << 31) - 1024;   // kernels index tiles with int
+constexpr int64_t kMaxElems = int64_t(1) << 46;          // per operand, keeps byte offsets < 2^48
+
+int validate(const Problem &p)
+{
+    if (p.out_dtype != CUDALLM_F32 && p.out_dtype != CUDALLM_BF16) return CUDALLM_ERR_INVALID_DTYPE;
+    if (p.M < 0 || p.N < 0 || p.K < 0 || p.batch < 0) return CUDALLM_ERR_INVALID_DIM;
+    if (p.M > kMaxDim || p.N > kMaxDim || p.K > kMaxDim || p.batch > kMaxDim)
+        return CUDALLM_ERR_INVALID_DIM;
+    if (p.M == 0 || p.N == 0 || p.batch == 0) return CUDALLM_OK;   // nothing to do
+    if (p.lda < p.K || p.ldb < p.N || p.ldc < p.N) return CUDALLM_ERR_INVALID_LD;
+    if (p.lda > kMaxElems || p.ldb > kMaxElems || p.ldc > kMaxElems) return CUDALLM_ERR_INVALID_DIM;
+    if (p.batch > 1) {
+        if (p.sA < 0 || p.sB < 0 || p.sC < 0) return CUDALLM_ERR_INVALID_LD;
+        if (p.sC < (p.M - 1) * p.ldc + p.N) return CUDALLM_ERR_INVALID_LD;   // items of C overlap
+    }
+    // extents must stay indexable
+    const long double extA = (long double)(p.batch - 1) * p.sA + (long double)(p.M - 1) * p.lda + p.K;
+    const long double extB = (long double)(p.batch - 1) * p.sB + (long double)(p.K > 0 ? p.K - 1 : 0) * p.ldb + p.N;
+    const long double extC = (long double)(p.batch - 1) * p.sC + (long double)(p.M - 1) * p.ldc + p.N;
+    if (extA > (long double)kMaxElems || extB > (long double)kMaxElems || extC > (long double)kMaxElems)
+        return CUDALLM_ERR_INVALID_DIM;
+    if ((long double)p.M * p.N * p.batch > (long double)kMaxElems) return CUDALLM_ERR_INVALID_DIM;
+    if (!p.C) return CUDALLM_ERR_INVALID_POINTER;
+    if (p.K > 0 && (!p.A || !p.B)) return CUDALLM_ERR_INVALID_POINTER;
+    if (p.K > 0 && ((reinterpret_cast<uintptr_t>(p.A) & 1) || (reinterpret_cast<uintptr_t>(p.B) & 1)))
+        return CUDALLM_ERR_MISALIGNED;
+    const uintptr_t cmask = (p.out_dtype == CUDALLM_F32) ? 3 : 1;
+    if (reinterpret_cast<uintptr_t>(p.C) & cmask) return CUDALLM_ERR_MISALIGNED;
+    return CUDALLM_OK;
+}
+
+inline bool is_empty(const Problem &p) { return p.M == 0 || p.N == 0 || p.batch == 0; }
+
+// ---------------------------------------------------------------- variants --
+enum Family { kSimt = 0, kUmma = 1 };
+struct Variant {
+    char name[32];
+    Family family;
+    int block_n;
+    int split_k;
+};
+constexpr int kBlockNs[3] = {64, 128, 256};
+constexpr int kSplits[5] = {1, 2, 4, 8, 16};
+constexpr int kNumVariants = 1 + 3 * 5;
+Variant g_variants[kNumVariants];
+std::once_flag g_variants_once;
+
+void build_variants()
+{
+    std::call_once(g_variants_once, [] {
+        snprintf(g_variants[0].name, sizeof g_variants[0].name, "simt");
+        g_variants[0].family = kSimt;
+        g_variants[0].block_n = 0;
+        g_variants[0].split_k = 1;
+        int v = 1;
+        for (int bn : kBlockNs)
+            for (int sk : kSplits) {
+                if (sk == 1) snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma_n%d", bn);
+                else snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma_n%d_sk%d", bn, sk);
+                g_variants[v].family = kUmma;
+                g_variants[v].block_n = bn;
+                g_variants[v].split_k = sk;
+                ++v;
+            }
+    });
+}
+
+constexpr int kNumSMs = 148;
+constexpr int64_t kMaxCounters = 16384;              // tiles a split-K launch may have
+constexpr int64_t kMaxPartialBytes = int64_t(1) << 30;
+
+inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline int64_t round_up(int64_t a, int64_t b) { return cdiv(a, b) * b; }
+
+struct Tiling {
+    int64_t tiles_m, tiles_n, tiles, kblocks, units;
+};
+Tiling tiling_for(const Problem &p, int block_n, int split_k)
+{
+    Tiling t;
+    t.tiles_m = cdiv(p.M, kBlockM);
+    t.tiles_n = cdiv(p.N, block_n);
+    t.tiles = t.tiles_m * t.tiles_n * p.batch;
+    t.kblocks = cdiv(p.K, kBlockK);
+    t.units = t.tiles * split_k;
+    return t;
+}
+
+bool variant_supports(const Variant &v, const Problem &p)
+{
+    if (is_empty(p)) return true;
+    if (v.family == kSimt) return true;
+    if (p.K == 0) return false;                       // the zero-fill case runs on the simt kernel
+    const Tiling t = tiling_for(p, v.block_n, v.split_k);
+    if (t.units > kMaxDim) return false;
+    if (v.split_k > 1) {
+        if (v.split_k > t.kblocks) return false;
+        if (t.tiles > kMaxCounters) return false;
+        if (t.units * int64_t(kBlockM) * v.block_n * 4 > kMaxPartialBytes) return false;
+    }
+    return true;
+}
+
+// Cost model (SM clocks) behind the automatic choice.  A CTA spends, per
+// 64-deep k-block, the larger of the tensor-pipe time (2*BLOCK_N clocks for
+// four 128 x BLOCK_N x 16 MMAs) and the time to stream the block's operand
+// bytes at this SM's share of memory bandwidth; per unit it also pays an
+// epilogue, and split-K units pay for writing and re-reading partial tiles.
+double variant_cost(const Variant &v, const Problem &p)
+{
+    const Tiling t = tiling_for(p, v.block_n, v.split_k);
+    const double waves = (double)cdiv(t.units, kNumSMs);
+    const double kb_per_unit = (double)cdiv(t.kblocks, v.split_k);
+    const double rows = p.M < kBlockM ? (double)p.M : (double)kBlockM;
+    const double cols = p.N < v.block_n ? (double)p.N : (double)v.block_n;
+    const double bytes_kb = rows * 128.0 + cols * 128.0;
+    const double mem_clk = bytes_kb / 24.0;           // ~6.5 TB/s over 148 SMs at ~1.9 GHz
+    const double mma_clk = 2.0 * v.block_n;
+    const double per_kb = mma_clk > mem_clk ? mma_clk : mem_clk;
+    const double out_b = (p.out_dtype == CUDALLM_F32) ? 4.0 : 2.0;
+    double epi = rows * cols * out_b / 24.0 + 600.0;
+    if (v.split_k > 1) epi += rows * v.block_n * 4.0 * 2.0 / 24.0 + 1500.0;
+    // the epilogue of a tile overlaps the next tile's main loop except on the last wave
+    const double main = waves * kb_per_unit * per_kb;
+    return main + epi + (waves - 1.0) * (epi > kb_per_unit * per_kb ? epi - kb_per_unit * per_kb : 0.0)
+         + 3000.0;
+}
+
+int select_variant(const Problem &p)
+{
+    build_variants();
+    if (is_empty(p) || p.K == 0) return 0;
+    int best = -1;
+    double best_cost = 0;
+    for (int v = 1; v < kNumVariants; ++v) {
+        if (!variant_supports(g_variants[v], p)) continue;
+        const double c = variant_cost(g_variants[v], p);
+        if (best < 0 || c < best_cost) { best = v; best_cost = c; }
+    }
+    return best < 0 ? 0 : best;
+}
+
+// --------------------------------------------------------------- workspace --
+// Layout: [status 256 B][tile counters][split-K partials][packed A][packed B]
+constexpr size_t kStatusBytes = 256;
+constexpr size_t kCounterBytes = kMaxCounters * sizeof(int);
+constexpr size_t kHeaderBytes = kStatusBytes + kCounterBytes;
+constexpr int kMaxDevices = 64;
+
+struct DeviceState {
+    bool probed = false;
+    bool supported = false;
+    int sm_count = 0;
+    void *ws = nullptr;          // active workspace
+    size_t ws_bytes = 0;
+    bool ws_external = false;
+    void *ws_internal = nullptr; // owned allocation (kept when an external one is set)
+    size_t ws_internal_bytes = 0;
+    bool smem_attr_set[16] = {};
+};
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mutex;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int probe_device(int dev)
+{
+    DeviceState &d = g_dev[dev];
+    if (d.probed) return d.supported ? CUDALLM_OK : CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    int major = 0, minor = 0, sms = 0;
+    CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    d.probed = true;
+    d.supported = (major == 10 && minor == 0);
+    d.sm_count = sms;
+    if (!d.supported) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    if (!g_encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+        if (qres != cudaDriverEntryPointSuccess || !fn) {
+            snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled not available");
+            return CUDALLM_ERR_CUDA;
+        }
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    return CUDALLM_OK;
+}
+
+// Make sure the active workspace of `dev` holds `bytes`; allocates or grows the
+// internal one (never an external one).
+int ensure_workspace(int dev, size_t bytes, cudaStream_t stream)
+{
+    DeviceState &d = g_dev[dev];
+    if (d.ws && d.ws_bytes >= bytes) return CUDALLM_OK;
+    if (d.ws_external) return CUDALLM_ERR_WORKSPACE;
+    size_t want = bytes < (size_t(8) << 20) ? (size_t(8) << 20) : bytes + bytes / 4;
+    if (d.ws_internal) {
+        CUDA_TRY(cudaDeviceSynchronize());            // earlier launches may still use it
+        CUDA_TRY(cudaFree(d.ws_internal));
+        d.ws_internal = nullptr;
+        d.ws_internal_bytes = 0;
+        d.ws = nullptr;
+        d.ws_bytes = 0;
+    }
+    void *ptr = nullptr;
+    CUDA_TRY(cudaMalloc(&ptr, want));
+    CUDA_TRY(cudaMemsetAsync(ptr, 0, kHeaderBytes, stream));
+    // later launches on other streams must see the cleared header
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    d.ws_internal = ptr;
+    d.ws_internal_bytes = want;
+    d.ws = ptr;
+    d.ws_bytes = want;
+    return CUDALLM_OK;
+}
+
+struct Plan {
+    bool pack_a, pack_b;
+    int64_t ldap, ldbp, sAp, sBp;      // packed leading dimensions / strides (elements)
+    size_t off_partials, off_pack_a, off_pack_b, total;
+};
+
+inline bool a_operand_aligned(const Problem &p)
+{
+    return (reinterpret_cast<uintptr_t>(p.A) % 16 == 0) && (p.lda % 8 == 0)
+        && (p.batch == 1 || p.sA % 8 == 0);
+}
+inline bool b_operand_aligned(const Problem &p)
+{
+    return (reinterpret_cast<uintptr_t>(p.B) % 16 == 0) && (p.ldb % 8 == 0)
+        && (p.batch == 1 || p.sB % 8 == 0);
+}
+
+Plan make_plan(const Variant &v, const Problem &p, bool pack_a, bool pack_b)
+{
+    Plan pl{};
+    pl.pack_a = pack_a;
+    pl.pack_b = pack_b;
+    size_t off = kHeaderBytes;
+    pl.off_partials = off;
+    if (v.family == kUmma && v.split_k > 1) {
+        const Tiling t = tiling_for(p, v.block_n, v.split_k);
+        off += (size_t)t.units * kBlockM * v.block_n * 4;
+    }
+    off = (size_t)round_up((int64_t)off, 256);
+    pl.off_pack_a = off;
+    pl.ldap = round_up(p.K, 8);
+    pl.sAp = p.M * pl.ldap;
+    if (pack_a) off += (size_t)(p.batch * pl.sAp * 2);
+    off = (size_t)round_up((int64_t)off, 256);
+    pl.off_pack_b = off;
+    pl.ldbp = round_up(p.N, 8);
+    pl.sBp = p.K * pl.ldbp;
+    if (pack_b) off += (size_t)(p.batch * pl.sBp * 2);
+    pl.total = (size_t)round_up((int64_t)off, 256);
+    return pl;
+}
+
+// ------------------------------------------------------------- tensor maps --
+int encode_operand_map(CUtensorMap *tm, const void *base, int64_t inner, int64_t rows, int64_t batch,
+                       int64_t ld, int64_t stride, int box_inner, int box_rows)
+{
+    cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batch};
+    cuuint64_t item_stride = (batch > 1) ? (cuuint64_t)stride * 2 : (cuuint64_t)rows * ld * 2;
+    cuuint64_t strides[2] = {(cuuint64_t)ld * 2, item_stride};
+    cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims,
+                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return CUDALLM_ERR_CUDA;
+    }
+    return CUDALLM_OK;
+}
+
+// ---------------------------------------------------------------- launches --
+template <int BLOCK_N, int STAGES, bool OUT_BF16>
+int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &gp,
+                cudaStream_t stream)
+{
+    using L = SmemLayout<BLOCK_N, STAGES>;
+    static_assert(L::kDynamicBytes <= 232448, "shared memory budget");
+    // More than half of an SM's shared memory, so two CTAs (and their tensor
+    // memory allocations) can never share an SM.
+    static_assert(L::kDynamicBytes > 120 * 1024, "one CTA per SM");
+    auto kernel = umma_gemm_kernel<BLOCK_N, STAGES, OUT_BF16>;
+    DeviceState &d = g_dev[dev];
+    if (!d.smem_attr_set[slot]) {
+        CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      L::kDynamicBytes));
+        d.smem_attr_set[slot] = true;
+    }
+    int grid = gp.num_units < d.sm_count ? gp.num_units : d.sm_count;
+    kernel<<<grid, kNumThreads, L::kDynamicBytes, stream>>>(ta, tb, gp);
+    CUDA_TRY(cudaGetLastError());
+    return CUDALLM_OK;
+}
+
+int launch_simt(const Problem &p, cudaStream_t stream)
+{
+    dim3 block(256);
+    int64_t gy = cdiv(p.M, 16), gz = p.batch;
+    dim3 grid((unsigned)cdiv(p.N, 16), (unsigned)(gy > 65535 ? 65535 : gy), (unsigned)(gz > 65535 ? 65535 : gz));
+    const __nv_bfloat16 *A = static_cast<const __nv_bfloat16 *>(p.A);
+    const __nv_bfloat16 *B = static_cast<const __nv_bfloat16 *>(p.B);
+    if (p.out_dtype == CUDALLM_BF16)
+        simt_gemm_kernel<true><<<grid, block, 0, stream>>>(A, B, p.C, (int)p.M, (int)p.N, (int)p.K, p.lda,
+                                                           p.ldb, p.ldc, p.sA, p.sB, p.sC, (int)p.batch);
+    else
+        simt_gemm_kernel<false><<<grid, block, 0, stream>>>(A, B, p.C, (int)p.M, (int)p.N, (int)p.K, p.lda,
+                                                            p.ldb, p.ldc, p.sA, p.sB, p.sC, (int)p.batch);
+    CUDA_TRY(cudaGetLastError());
+    return CUDALLM_OK;
+}
+
+int launch_pack(const void *src, void *dst, int64_t rows, int64_t cols, int64_t ld_src, int64_t ld_dst,
+                int64_t s_src, int64_t s_dst, int64_t batch, cudaStream_t stream)
+{
+    const int64_t total = rows * cdiv(cols, 8) * batch;
+    int64_t blocks = cdiv(total, 256);
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    pack_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const uint16_t *>(src),
+                                                           static_cast<uint16_t *>(dst), (int)rows,
+                                                           (int)cols, ld_src, ld_dst, s_src, s_dst,
+                                                           (int)batch);
+    CUDA_TRY(cudaGetLastError());
+    return CUDALLM_OK;
+}
+
+int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
+{
+    const bool pack_a = !a_operand_aligned(p);
+    const bool pack_b = !b_operand_aligned(p);
+    const Plan pl = make_plan(v, p, pack_a, pack_b);
+    int st = ensure_workspace(dev, pl.total, stream);
+    if (st != CUDALLM_OK) return st;
+    DeviceState &d = g_dev[dev];
+    uint8_t *ws = static_cast<uint8_t *>(d.ws);
+
+    const void *A = p.A, *B = p.B;
+    int64_t lda = p.lda, ldb = p.ldb, sA = p.sA, sB = p.sB;
+    if (pack_a) {
+        st = launch_pack(p.A, ws + pl.off_pack_a, p.M, p.K, p.lda, pl.ldap, p.sA, pl.sAp, p.batch, stream);
+        if (st != CUDALLM_OK) return st;
+        A = ws + pl.off_pack_a; lda = pl.ldap; sA = pl.sAp;
+    }
+    if (pack_b) {
+        st = launch_pack(p.B, ws + pl.off_pack_b, p.K, p.N, p.ldb, pl.ldbp, p.sB, pl.sBp, p.batch, stream);
+        if (st != CUDALLM_OK) return st;
+        B = ws + pl.off_pack_b; ldb = pl.ldbp; sB = pl.sBp;
+    }
+
+    CUtensorMap ta, tb;
+    st = encode_operand_map(&ta, A, p.K, p.M, p.batch, lda, sA, kBlockK, kBlockM);
+    if (st != CUDALLM_OK) return st;
+    st = encode_operand_map(&tb, B, p.N, p.K, p.batch, ldb, sB, 64, kBlockK);
+    if (st != CUDALLM_OK) return st;
+
+    const Tiling t = tiling_for(p, v.block_n, v.split_k);
+    GemmParams gp{};
+    gp.C = p.C;
+    gp.ldc = p.ldc;
+    gp.strideC = p.batch > 1 ? p.sC : 0;
+    gp.M = (int)p.M; gp.N = (int)p.N; gp.K = (int)p.K; gp.batch = (int)p.batch;
+    gp.tiles_m = (int)t.tiles_m; gp.tiles_n = (int)t.tiles_n;
+    gp.split_k = v.split_k;
+    gp.kblocks = (int)t.kblocks;
+    gp.num_units = (int)t.units;
+    const int64_t vec = (p.out_dtype == CUDALLM_F32) ? 4 : 8;
+    gp.c_vec_ok = (reinterpret_cast<uintptr_t>(p.C) % 16 == 0) && (p.ldc % vec == 0)
+               && (p.batch == 1 || p.sC % vec == 0);
+    gp.partials = reinterpret_cast<float *>(ws + pl.off_partials);
+    gp.counters = reinterpret_cast<int *>(ws + kStatusBytes);
+    gp.status = reinterpret_cast<int *>(ws);
+
+    const bool bf = p.out_dtype == CUDALLM_BF16;
+    switch (v.block_n) {
+    case 64:  return bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
+                        : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream);
+    case 128: return bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
+                        : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream);
+    default:  return bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
+                        : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream);
+    }
+}
+
+int run(int variant, const Problem &p, void *stream_v)
+{
+    build_variants();
+    int st = validate(p);
+    if (st != CUDALLM_OK) return st;
+    if (variant != CUDALLM_VARIANT_AUTO && (variant < 0 || variant >= kNumVariants))
+        return CUDALLM_ERR_INVALID_VARIANT;
+    if (is_empty(p)) return CUDALLM_OK;
+    if (variant == CUDALLM_VARIANT_AUTO) variant = select_variant(p);
+    const Variant &v = g_variants[variant];
+    if (!variant_supports(v, p)) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    st = probe_device(dev);
+    if (st != CUDALLM_OK) return st;
+    if (v.family == kSimt) return launch_simt(p, stream);
+    return run_umma(dev, v, p, stream);
+}
+
+Problem make_problem(const void *A, const void *B, void *C, int64_t M, int64_t N, int64_t K, int64_t lda,
+                     int64_t ldb, int64_t ldc, int64_t sA, int64_t sB, int64_t sC, int64_t batch,
+                     int out_dtype)
+{
+    Problem p;
+    p.A = A; p.B = B; p.C = C;
+    p.M = M; p.N = N; p.K = K;
+    p.lda = lda; p.ldb = ldb; p.ldc = ldc;
+    p.sA = sA; p.sB = sB; p.sC = sC;
+    p.batch = batch;
+    p.out_dtype = out_dtype;
+    return p;
+}
+
+// Shape-only problem for the query functions: aligned dummy pointers.
+Problem shape_problem(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,
+                      int64_t batch, int out_dtype)
+{
+    void *dummy = reinterpret_cast<void *>(uintptr_t(256));
+    return make_problem(dummy, dummy, dummy, M, N, K, lda, ldb, ldc, M * lda, K * ldb, M * ldc, batch,
+                        out_dtype);
+}
+
+}  // namespace
+
+// ================================================================= C ABI ====
+extern "C" {
+
+int cudallm_gemm_bf16(const void *A, const void *B, void *C, int64_t M, int64_t N, int64_t K,
+                      int64_t lda, int64_t ldb, int64_t ldc, int out_dtype, void *stream)
+{
+    return run(CUDALLM_VARIANT_AUTO,
+               make_problem(A, B, C, M, N, K, lda, ldb, ldc, 0, 0, 0, 1, out_dtype), stream);
+}
+
+int cudallm_gemm_bf16_batched(const void *A, const void *B, void *C, int64_t M, int64_t N, int64_t K,
+                              int64_t lda, int64_t ldb, int64_t ldc, int64_t strideA, int64_t strideB,
+                              int64_t strideC, int64_t batch, int out_dtype, void *stream)
+{
+    return run(CUDALLM_VARIANT_AUTO,
+               make_problem(A, B, C, M, N, K, lda, ldb, ldc, strideA, strideB, strideC, batch, out_dtype),
+               stream);
+}
+
+int cudallm_gemm_bf16_variant(int variant, const void *A, const void *B, void *C, int64_t M, int64_t N,
+                              int64_t K, int64_t lda, int64_t ldb, int64_t ldc, int64_t strideA,
+                              int64_t strideB, int64_t strideC, int64_t batch, int out_dtype, void *stream)
+{
+    return run(variant,
+               make_problem(A, B, C, M, N, K, lda, ldb, ldc, strideA, strideB, strideC, batch, out_dtype),
+               stream);
+}
+
+size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,
+                                  int out_dtype)
+{
+    if (M < 0 || N < 0 || K < 0 || lda < K || ldb < N || ldc < N) return 0;
+    const int64_t esz = out_dtype == CUDALLM_F32 ? 4 : 2;
+    return (size_t)(round_up(M * lda * 2, 256) + round_up(K * ldb * 2, 256) + round_up(M * ldc * esz, 256));
+}
+
+int cudallm_gemm_bf16_host(const void *A_host, const void *B_host, void *C_host, int64_t M, int64_t N,
+                           int64_t K, int64_t lda, int64_t ldb, int64_t ldc, int out_dtype, void *dev_buf,
+                           size_t dev_bytes, void *stream_v)
+{
+    // Validate with stand-in device pointers first (nothing is touched on error).
+    void *dummy = reinterpret_cast<void *>(uintptr_t(256));
+    Problem p = make_problem(A_host ? dummy : nullptr, B_host ? dummy : nullptr, C_host ? dummy : nullptr,
+                             M, N, K, lda, ldb, ldc, 0, 0, 0, 1, out_dtype);
+    int st = validate(p);
+    if (st != CUDALLM_OK) return st;
+    if (is_empty(p)) return CUDALLM_OK;
+    const size_t need = cudallm_host_staging_bytes(M, N, K, lda, ldb, ldc, out_dtype);
+    if (!dev_buf || dev_bytes < need || (reinterpret_cast<uintptr_t>(dev_buf) % 256))
+        return CUDALLM_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int64_t esz = out_dtype == CUDALLM_F32 ? 4 : 2;
+    uint8_t *dA = static_cast<uint8_t *>(dev_buf);
+    uint8_t *dB = dA + round_up(M * lda * 2, 256);
+    uint8_t *dC = dB + round_up(K * ldb * 2, 256);
+    // rows are copied with their padding: (rows-1)*ld + cols elements
+    if (K > 0) {
+        CUDA_TRY(cudaMemcpyAsync(dA, A_host, (size_t)(((M - 1) * lda + K) * 2), cudaMemcpyHostToDevice, stream));
+        CUDA_TRY(cudaMemcpyAsync(dB, B_host, (size_t)(((K - 1) * ldb + N) * 2), cudaMemcpyHostToDevice, stream));
+    }
+    st = cudallm_gemm_bf16(dA, dB, dC, M, N, K, lda, ldb, ldc, out_dtype, stream_v);
+    if (st != CUDALLM_OK) return st;
+    if (ldc == N) {
+        CUDA_TRY(cudaMemcpyAsync(C_host, dC, (size_t)(M * N * esz), cudaMemcpyDeviceToHost, stream));
+    } else {
+        // keep the caller's padding columns untouched
+        CUDA_TRY(cudaMemcpy2DAsync(C_host, (size_t)(ldc * esz), dC, (size_t)(ldc * esz), (size_t)(N * esz),
+                                   (size_t)M, cudaMemcpyDeviceToHost, stream));
+    }
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    return CUDALLM_OK;
+}
+
+int cudallm_num_variants(void)
+{
+    return kNumVariants;
+}
+
+const char *cudallm_variant_name(int variant)
+{
+    build_variants();
+    if (variant < 0 || variant >= kNumVariants) return nullptr;
+    return g_variants[variant].name;
+}
+
+int cudallm_variant_supports(int variant, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
+                             int64_t ldc, int64_t batch, int out_dtype)
+{
+    build_variants();
+    if (variant < 0 || variant >= kNumVariants) return CUDALLM_ERR_INVALID_VARIANT;
+    Problem p = shape_problem(M, N, K, lda, ldb, ldc, batch, out_dtype);
+    int st = validate(p);
+    if (st != CUDALLM_OK) return st;
+    return variant_supports(g_variants[variant], p) ? 1 : 0;
+}
+
+int cudallm_select_variant(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,
+                           int64_t batch, int out_dtype)
+{
+    Problem p = shape_problem(M, N, K, lda, ldb, ldc, batch, out_dtype);
+    int st = validate(p);
+    if (st != CUDALLM_OK) return st;
+    return select_variant(p);
+}
+
+size_t cudallm_workspace_bytes(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,
+                               int64_t batch, int out_dtype)
+{
+    build_variants();
+    Problem p = shape_problem(M, N, K, lda, ldb, ldc, batch, out_dtype);
+    if (validate(p) != CUDALLM_OK || is_empty(p)) return kHeaderBytes;
+    size_t best = kHeaderBytes;
+    for (int v = 0; v < kNumVariants; ++v) {
+        if (!variant_supports(g_variants[v], p)) continue;
+        const Plan pl = make_plan(g_variants[v], p, true, true);   // worst case: both operands repacked
+        if (pl.total > best) best = pl.total;
+    }
+    return best;
+}
+
+int cudallm_set_workspace(void *dev_ptr, size_t bytes)
+{
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState &d = g_dev[dev];
+    if (!dev_ptr) {
+        d.ws = d.ws_internal;
+        d.ws_bytes = d.ws_internal_bytes;
+        d.ws_external = false;
+        return CUDALLM_OK;
+    }
+    if (bytes < kHeaderBytes || (reinterpret_cast<uintptr_t>(dev_ptr) % 256)) return CUDALLM_ERR_WORKSPACE;
+    d.ws = dev_ptr;
+    d.ws_bytes = bytes;
+    d.ws_external = true;
+    return CUDALLM_OK;
+}
+
+int cudallm_device_status(void *stream_v, int *code, int *detail)
+{
+    if (code) *code = CUDALLM_OK;
+    if (detail) *detail = 0;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState &d = g_dev[dev];
+    if (!d.ws) return CUDALLM_OK;                      // no kernel of ours has run yet
+    int host[2] = {0, 0};
+    CUDA_TRY(cudaMemcpy(host, d.ws, sizeof host, cudaMemcpyDeviceToHost));
+    if (host[0] != 0) {
+        // a kernel gave up: its tile counters may be stale; clear the whole header
+        CUDA_TRY(cudaMemset(d.ws, 0, kHeaderBytes));
+    }
+    if (code) *code = host[0];
+    if (detail) *detail = host[1];
+    return host[0];
+}
+
+const char *cudallm_strerror(int status)
+{
+    switch (status) {
+    case CUDALLM_OK: return "success";
+    case CUDALLM_ERR_INVALID_POINTER: return "null operand pointer for a non-empty problem";
+    case CUDALLM_ERR_INVALID_DIM: return "negative or too large dimension";
+    case CUDALLM_ERR_INVALID_LD: return "leading dimension smaller than the row length, or overlapping batch items of C";
+    case CUDALLM_ERR_INVALID_DTYPE: return "out_dtype must be 0 (fp32) or 1 (bf16)";
+    case CUDALLM_ERR_INVALID_VARIANT: return "variant id out of range";
+    case CUDALLM_ERR_UNSUPPORTED_SHAPE: return "the requested variant cannot run this problem";
+    case CUDALLM_ERR_UNSUPPORTED_DEVICE: return "the current device is not compute capability 10.0";
+    case CUDALLM_ERR_CUDA: return g_cuda_err[0] ? g_cuda_err : "CUDA call failed";
+    case CUDALLM_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case CUDALLM_ERR_WORKSPACE: return "workspace missing, too small or misaligned";
+    case CUDALLM_ERR_MISALIGNED: return "pointer not aligned to its element size";
+    default: return "unknown status";
+    }
+}
+
+int cudallm_version(void)
+{
+    return 100;   // 0.1.0
+}
+
+}  // extern "C"

@@ -1,0 +1,359 @@
+// Warp-specialised, persistent tcgen05 GEMM kernel for sm_100a.
+//
+//   C[i][j] = sum_k A[i][k] * B[k][j]      (Task 2: matrix multiplication)
+//
+// A is row-major M x K  -> K-major operand, TMA box 64(K) x 128(M), 128B swizzle.
+// B is row-major K x N  -> MN-major operand, TMA boxes 64(N) x 64(K), 128B swizzle.
+// One CTA owns a 128 x BLOCK_N tile of C; its fp32 accumulator lives in tensor
+// memory (two buffers, so the epilogue of one tile overlaps the main loop of
+// the next).  Roles: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM
+// owner), warps 2..5 = epilogue (TMEM -> registers -> global).
+//
+// Work is cut into units (tile, k-split); CTA b runs units b, b+grid, ...
+// With split_k > 1 every unit writes an fp32 partial tile to the workspace and
+// the unit that arrives last at the tile's counter adds the partials in split
+// order 0..S-1 (so the result does not depend on arrival order) and stores C.
+#pragma once
+#include "ptx.cuh"
+
+namespace cudallm {
+
+constexpr int kBlockM = 128;
+constexpr int kBlockK = 64;           // one 128-byte swizzle row of bf16
+constexpr int kUmmaK = 16;            // K of one tcgen05.mma for 16-bit inputs
+constexpr int kNumThreads = 192;      // 6 warps
+constexpr int kEpiThreads = 128;
+
+// status detail codes: (role << 8) | barrier kind
+enum : int { kRoleProducer = 1, kRoleMma = 2, kRoleEpilogue = 3 };
+
+struct GemmParams {
+    void *C;
+    long long ldc;          // elements
+    long long strideC;      // elements between batch items
+    int M, N, K, batch;
+    int tiles_m, tiles_n;   // tiles per batch item
+    int split_k;            // >= 1, <= kblocks
+    int kblocks;            // ceil(K / 64)
+    int num_units;          // tiles_m * tiles_n * batch * split_k
+    int c_vec_ok;           // C base, ldc, strideC allow 16-byte stores
+    float *partials;        // split-K partial tiles (workspace)
+    int *counters;          // one per tile (workspace), zero between launches
+    int *status;            // [0] = code, [1] = detail
+};
+
+template <int BLOCK_N, int STAGES>
+struct SmemLayout {
+    static constexpr int kABytes = kBlockM * kBlockK * 2;
+    static constexpr int kBBytes = kBlockK * BLOCK_N * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kBarOffset = STAGES * kStageBytes;
+    // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], epilogue group
+    static constexpr int kNumBars = 2 * STAGES + 5;
+    static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
+    static constexpr int kBytes = kMiscOffset + 64;
+    static constexpr int kDynamicBytes = kBytes + 1024;  // slack for 1024-byte alignment
+};
+
+__device__ __forceinline__ void report_timeout(int *status, int role, int what)
+{
+    if (atomicCAS(status, 0, -9 /* CUDALLM_ERR_DEVICE_TIMEOUT */) == 0)
+        status[1] = (role << 8) | what;
+}
+
+struct UnitCoord {
+    int m_tile, n_tile, b, split, tile_linear;
+    int kb_begin, kb_end;
+};
+
+__device__ __forceinline__ UnitCoord decode_unit(const GemmParams &p, int u)
+{
+    UnitCoord c;
+    c.split = u % p.split_k;
+    int t = u / p.split_k;
+    c.tile_linear = t;
+    c.m_tile = t % p.tiles_m;
+    t /= p.tiles_m;
+    c.n_tile = t % p.tiles_n;
+    c.b = t / p.tiles_n;
+    c.kb_begin = static_cast<int>((static_cast<long long>(p.kblocks) * c.split) / p.split_k);
+    c.kb_end = static_cast<int>((static_cast<long long>(p.kblocks) * (c.split + 1)) / p.split_k);
+    return c;
+}
+
+// Store 32 consecutive fp32 accumulator values of one row to C (fp32 or bf16).
+template <bool OUT_BF16>
+__device__ __forceinline__ void store_row_chunk(const GemmParams &p, const float (&v)[32],
+                                                long long row_off, int col0, bool row_ok)
+{
+    if (!row_ok) return;
+    const int n_left = p.N - col0;
+    if (n_left <= 0) return;
+    if (OUT_BF16) {
+        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.C) + row_off + col0;
+        if (p.c_vec_ok && n_left >= 32) {
+            uint4 *d4 = reinterpret_cast<uint4 *>(dst);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint4 w;
+                w.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
+                w.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
+                w.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
+                w.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
+                d4[q] = w;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (j < n_left) dst[j] = __float2bfloat16_rn(v[j]);
+        }
+    } else {
+        float *dst = reinterpret_cast<float *>(p.C) + row_off + col0;
+        if (p.c_vec_ok && n_left >= 32) {
+            float4 *d4 = reinterpret_cast<float4 *>(dst);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                d4[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (j < n_left) dst[j] = v[j];
+        }
+    }
+}
+
+template <int BLOCK_N, int STAGES, bool OUT_BF16>
+__global__ void __launch_bounds__(kNumThreads, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                 const __grid_constant__ CUtensorMap tmap_b, const GemmParams p)
+{
+    using L = SmemLayout<BLOCK_N, STAGES>;
+    static_assert(BLOCK_N % 64 == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
+    constexpr uint32_t kTmemCols = 2 * BLOCK_N;          // 128, 256 or 512: power of two
+    constexpr uint32_t kIdesc = make_idesc_bf16(kBlockM, BLOCK_N, 0, 1);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_base + L::kBarOffset;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    const uint32_t epi_bar = bar_base + 8u * (2 * STAGES + 4);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L::kMiscOffset);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kMiscOffset + 4);
+    volatile int *last_flag = reinterpret_cast<volatile int *>(smem + L::kMiscOffset + 8);
+
+    const int warp_idx = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        *last_flag = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 4);     // one arrival per epilogue warp
+        }
+        mbar_init(epi_bar, kEpiThreads);
+        fence_mbar_init();
+        fence_proxy_async_smem();
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+    }
+    if (warp_idx == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp_idx == 0) {
+        // ------------------------------------------------ TMA producer ----
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; ok && u < p.num_units; u += gridDim.x) {
+                const UnitCoord c = decode_unit(p, u);
+                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) {
+                        report_timeout(p.status, kRoleProducer, stage);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t sa = smem_base + stage * L::kStageBytes;
+                    const uint32_t sb = sa + L::kABytes;
+                    mbar_arrive_expect_tx(full_bar(stage), L::kStageBytes);
+                    tma_load_3d(sa, &tmap_a, full_bar(stage), kb * kBlockK, c.m_tile * kBlockM, c.b);
+#pragma unroll
+                    for (int j = 0; j < BLOCK_N / 64; ++j)
+                        tma_load_3d(sb + j * (64 * kBlockK * 2), &tmap_b, full_bar(stage),
+                                    c.n_tile * BLOCK_N + j * 64, kb * kBlockK, c.b);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp_idx == 1) {
+        // -------------------------------------------------- MMA issuer ----
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; ok && u < p.num_units; u += gridDim.x) {
+                const UnitCoord c = decode_unit(p, u);
+                if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag)) {
+                    report_timeout(p.status, kRoleMma, 0x40 + acc);
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
+                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+                        report_timeout(p.status, kRoleMma, stage);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = smem_base + stage * L::kStageBytes;
+                    const uint32_t sb = sa + L::kABytes;
+#pragma unroll
+                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                        // A: K-major, 8-row groups 1024 B apart; 16 K-elements = 32 B
+                        const uint64_t da = make_smem_desc_sw128(sa + k * 32, 16, 1024);
+                        // B: MN-major, 64-column chunks 8192 B apart (LBO),
+                        //    8-k groups 1024 B apart (SBO); 16 k = 2048 B
+                        const uint64_t db = make_smem_desc_sw128(sb + k * 2048, 8192, 1024);
+                        umma_bf16(d_tmem, da, db, kIdesc, (kb > c.kb_begin || k > 0) ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(stage));       // frees the stage when the MMAs retire
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                umma_commit(tfull_bar(acc));             // accumulator complete
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ---------------------------------------------------- epilogue ----
+        const int quad = warp_idx & 3;                   // TMEM lanes 32*quad .. +31
+        const int epi_tid = quad * 32 + lane;            // == row within the tile
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        uint32_t epi_phase = 0;
+        // Rendezvous of the 128 epilogue threads on an mbarrier, so that this
+        // wait is bounded like every other one in the kernel.
+        auto epi_sync = [&]() -> bool {
+            mbar_arrive(epi_bar);
+            const bool done = mbar_wait(epi_bar, epi_phase, abort_flag);
+            epi_phase ^= 1;
+            return done;
+        };
+        for (int u = blockIdx.x; u < p.num_units; u += gridDim.x) {
+            const UnitCoord c = decode_unit(p, u);
+            bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0x80 + acc);
+                break;
+            }
+            tc_fence_after();
+            const int row = c.m_tile * kBlockM + epi_tid;
+            const bool row_ok = row < p.M;
+            const long long row_off = static_cast<long long>(c.b) * p.strideC
+                                    + static_cast<long long>(row) * p.ldc;
+            const uint32_t t_addr = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(quad * 32) << 16);
+            if (p.split_k == 1) {
+#pragma unroll 1
+                for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(t_addr + ch * 32, r);
+                    tmem_ld_wait();
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+                    store_row_chunk<OUT_BF16>(p, v, row_off, c.n_tile * BLOCK_N + ch * 32, row_ok);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(acc));
+            } else {
+                // partial tile layout: float4 index ((ch*8 + q) * 128 + row)
+                float4 *part = reinterpret_cast<float4 *>(p.partials)
+                             + (static_cast<long long>(c.tile_linear) * p.split_k + c.split)
+                                   * (kBlockM * BLOCK_N / 4);
+#pragma unroll 1
+                for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(t_addr + ch * 32, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        __stcg(part + (ch * 8 + q) * kBlockM + epi_tid,
+                               make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                           __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3])));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(acc));
+                __threadfence();
+                if (!epi_sync()) {
+                    report_timeout(p.status, kRoleEpilogue, 0xC0);
+                    break;
+                }
+                if (epi_tid == 0) {
+                    const int old = atomicAdd(p.counters + c.tile_linear, 1);
+                    const int last = (old == p.split_k - 1);
+                    if (last) p.counters[c.tile_linear] = 0;   // ready for the next launch
+                    *last_flag = last;
+                }
+                if (!epi_sync()) {
+                    report_timeout(p.status, kRoleEpilogue, 0xC1);
+                    break;
+                }
+                if (*last_flag) {
+                    __threadfence();
+                    const float4 *tile0 = reinterpret_cast<const float4 *>(p.partials)
+                                        + static_cast<long long>(c.tile_linear) * p.split_k
+                                              * (kBlockM * BLOCK_N / 4);
+#pragma unroll 1
+                    for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
+                        float v[32];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                        for (int s = 0; s < p.split_k; ++s) {
+                            const float4 *ps = tile0 + static_cast<long long>(s) * (kBlockM * BLOCK_N / 4);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                const float4 t = __ldcg(ps + (ch * 8 + q) * kBlockM + epi_tid);
+                                v[4 * q] += t.x; v[4 * q + 1] += t.y;
+                                v[4 * q + 2] += t.z; v[4 * q + 3] += t.w;
+                            }
+                        }
+                        store_row_chunk<OUT_BF16>(p, v, row_off, c.n_tile * BLOCK_N + ch * 32, row_ok);
+                    }
+                }
+            }
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp_idx == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace cudallm
