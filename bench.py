@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the bf16 GEMM library on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One *step* is one call of the whole hot path -- ``cudallm_gemm_bf16`` on the
+headline workload C2 (M = N = K = 4096, bf16 in, fp32 accumulate, bf16 out) --
+on seeded synthetic operands that are already resident in HBM.  The line
+printed by rank 0 carries the device-timed TFLOP/s (``value``), the same
+metric through the host-buffer entry point with the copies inside the timed
+region (``e2e``), the roofline fraction of the GEMM kernel against the measured
+cuBLAS bf16 peak of this pool (``roofline``), the skinny HBM-bound workload C5a
+in GB/s against the measured copy bandwidth (``skinny``), and the CPU oracle
+timed on the host cores on a bounded sample (``cpu_baseline``).
+
+With N > 1 (launched by torchrun, one rank per GPU) every rank multiplies its
+own row shard of the same size: weak scaling, no data-path collective.
+
+``--impl reference`` times the CPU oracle as it stands (no GPU work).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "GEMM TFLOP/s & % of dense-bf16 peak at 4096^3; HBM GB/s & % on skinny M=16"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_BYTES = 126e6
+# DRAM traffic of one launch of the dominant kernel, from the ncu capture
+# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).
+NCU_TRAFFIC_BYTES = {"C2": None, "C5a": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------ clocks --
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _poll_once(self):
+        nv = self.nv
+        try:
+            mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                    if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons")
+                    else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            self.samples.append(mhz)
+            table = {
+                "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+                "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+                "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+                "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+            }
+            for name, bit in table.items():
+                if r & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self._poll_once()
+            time.sleep(0.001)
+
+    def start(self):
+        if self.nv is None:
+            return
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+# ------------------------------------------------------------------ helpers --
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    return rank, local, world
+
+
+def time_steps(launch, steps, warmup, barrier, sampler=None):
+    """W warm-up steps, then exactly ``steps`` timed steps with one CUDA event
+    between consecutive steps.  Returns (total seconds, per-step seconds list)."""
+    import torch
+    for i in range(warmup):
+        launch(i)
+    torch.cuda.synchronize()
+    barrier()
+    torch.cuda.synchronize()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    if sampler:
+        sampler.start()
+    evs[0].record()
+    for i in range(steps):
+        launch(warmup + i)
+        evs[i + 1].record()
+    if sampler:
+        sampler._poll_once() if sampler.nv is not None else None
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.stop()
+    barrier()
+    torch.cuda.synchronize()
+    total = evs[0].elapsed_time(evs[-1]) * 1e-3
+    per = [evs[i].elapsed_time(evs[i + 1]) * 1e-3 for i in range(steps)]
+    return total, per
+
+
+def launches_per_call(B, cfg, variant_name):
+    n = 1
+    if "_sk" in variant_name:
+        n += 1                                   # split-K reduction kernel
+    if cfg.lda_ % 8 or (cfg.batch > 1 and cfg.strideA % 8):
+        n += 1                                   # repack A
+    if cfg.ldb_ % 8 or (cfg.batch > 1 and cfg.strideB % 8):
+        n += 1                                   # repack B
+    return n
+
+
+def cpu_baseline_sample(cfg, A, Bm, target_s=12.0):
+    """The oracle as it stands, timed on the host cores on a bounded number of
+    rows of the same workload."""
+    import numpy as np
+    import oracle
+    cores = oracle.num_threads()
+    probe_rows = np.arange(min(cfg.M, 4 * cores), dtype=np.int64)
+    t0 = time.perf_counter()
+    oracle.gemm_rows(A, Bm, probe_rows, cfg.N, cfg.K, cfg.lda_, cfg.ldb_)
+    dt = max(time.perf_counter() - t0, 1e-6)
+    rate = probe_rows.size / dt
+    nrows = int(min(cfg.M, max(cores, rate * target_s)))
+    nrows = max(cores, (nrows // cores) * cores)
+    rows = np.arange(nrows, dtype=np.int64)
+    t0 = time.perf_counter()
+    oracle.gemm_rows(A, Bm, rows, cfg.N, cfg.K, cfg.lda_, cfg.ldb_)
+    dt = time.perf_counter() - t0
+    flops = 2.0 * nrows * cfg.N * cfg.K
+    return {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+            "sample": f"rows 0..{nrows - 1} of {cfg.name} ({nrows} x {cfg.N} x {cfg.K}), "
+                      f"C_ref and S in fp64, {dt:.2f} s"}
+
+
+# ------------------------------------------------------------ reference arm --
+def run_reference(args):
+    rank, local, world = dist_env()
+    if rank != 0:
+        return 0
+    import numpy as np
+    import oracle
+    from paper_2506_09092_b200 import inputs as gi
+    cfg = gi.CONFIGS["C2"]
+    A, Bm = cfg.make()
+    cores = oracle.num_threads()
+    rows_per_step = max(cores, 64)
+    rng = np.random.default_rng(0)
+
+    def step(i):
+        start = (i * rows_per_step) % (cfg.M - rows_per_step + 1)
+        rows = np.arange(start, start + rows_per_step, dtype=np.int64)
+        oracle.gemm_rows(A, Bm, rows, cfg.N, cfg.K, cfg.lda_, cfg.ldb_)
+
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    dt = time.perf_counter() - t0
+    flops = 2.0 * rows_per_step * cfg.N * cfg.K * args.steps
+    value = flops / dt / 1e12
+    sample = (f"each step = {rows_per_step} consecutive rows of {cfg.name} "
+              f"({rows_per_step} x {cfg.N} x {cfg.K}), C_ref and S in fp64")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(cfg), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def workload_name(cfg):
+    out = "bf16" if cfg.out_dtype == 1 else "fp32"
+    return (f"{cfg.name}: GEMM M={cfg.M} N={cfg.N} K={cfg.K} batch={cfg.batch}, bf16 in, "
+            f"fp32 accumulate, {out} out, row-major")
+
+
+# ------------------------------------------------------------------- our arm --
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2506_09092_b200 import binding as B
+    from paper_2506_09092_b200 import harness as H
+    from paper_2506_09092_b200 import inputs as gi
+
+    rank, local, world = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU fallback")
+    B.lib()                                            # fail loudly if the library is not built
+    torch.cuda.set_device(local)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        barrier = lambda: dist.barrier()
+    else:
+        barrier = lambda: None
+    peaks, peak_src = load_peaks()
+    stream = torch.cuda.current_stream()
+
+    # ------------------------------------------------ headline workload: C2 --
+    cfg = gi.CONFIGS["C2"]
+    A, Bm = cfg.make()
+    prob = H.DeviceProblem(cfg, A, Bm, min_bytes=3.2 * L2_BYTES)
+    vname = B.variant_name(B.select_variant(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_,
+                                            cfg.batch, cfg.out_dtype))
+    sampler = ClockSampler(local)
+    total, per = time_steps(lambda i: prob.launch(i, stream=stream), args.steps, args.warmup,
+                            barrier, sampler)
+    code, detail = B.device_status(stream)
+    if code != 0:
+        raise RuntimeError(f"device status {code} detail {detail:#x}")
+    t = torch.tensor([total], dtype=torch.float64, device="cuda")
+    if use_dist:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_max = float(t.item())
+    value = world * cfg.flops * args.steps / total_max / 1e12
+    kern_avg = sum(per) / len(per)
+    achieved = cfg.flops / kern_avg / 1e12
+    n_launch = launches_per_call(B, cfg, vname)
+
+    # -------------------------------------------- e2e: host buffers, copies --
+    hA = torch.from_numpy(A.view(np.int16)).pin_memory()
+    hB = torch.from_numpy(Bm.view(np.int16)).pin_memory()
+    hC = torch.empty(cfg.M * cfg.ldc_, dtype=torch.int16).pin_memory()
+    need = B.host_staging_bytes(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.out_dtype)
+    stage = torch.empty(need, dtype=torch.uint8, device="cuda")
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def e2e_call(i):
+        B.gemm_bf16_host(hA, hB, hC, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_,
+                         cfg.out_dtype, stage, need, stream)
+    e2e_total, _ = time_steps(e2e_call, e2e_steps, 2, barrier)
+    t = torch.tensor([e2e_total], dtype=torch.float64, device="cuda")
+    if use_dist:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = world * cfg.flops * e2e_steps / float(t.item()) / 1e12
+
+    # ------------------------------------------- skinny HBM-bound workload --
+    sk = gi.CONFIGS["C5a"]
+    sA, sB = sk.make()
+    skp = H.DeviceProblem(sk, sA, sB, min_bytes=2.2 * L2_BYTES)
+    sk_name = B.variant_name(B.select_variant(sk.M, sk.N, sk.K, sk.lda_, sk.ldb_, sk.ldc_, sk.batch,
+                                              sk.out_dtype))
+    sk_steps = max(args.steps, 20)
+    sk_total, sk_per = time_steps(lambda i: skp.launch(i, stream=stream), sk_steps, args.warmup, barrier)
+    sk_avg = sum(sk_per) / len(sk_per)
+    sk_gbs = sk.algorithmic_bytes / sk_avg / 1e9
+
+    line = None
+    if rank == 0:
+        clocks = sampler.summary()
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_max / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {
+                "workload": workload_name(cfg), "variant": vname,
+                "inputs": "A, B ~ N(0,1) rounded to bf16, numpy default_rng([1,0]) / ([1,1])",
+                "l2": f"rotating {prob.nsets} operand/output sets ({prob.nsets * prob.set_bytes / 1e6:.0f} MB)"
+                      f" > {L2_BYTES / 1e6:.0f} MB L2",
+                "sharding": "one replica of the workload per GPU (row shards of a taller product), no collective",
+            },
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": "TFLOP/s",
+                    "h2d_bytes_per_step": int(A.nbytes + Bm.nbytes),
+                    "d2h_bytes_per_step": int(cfg.M * cfg.N * cfg.out_bytes),
+                    "steps": e2e_steps, "call": "cudallm_gemm_bf16_host (pinned host buffers)"},
+            "gpu_launches": n_launch * args.steps,
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                         "traffic": NCU_TRAFFIC_BYTES["C2"], "peak_source": f"of {peak_src} (burst)",
+                         "kernel": f"umma_gemm_kernel ({vname})",
+                         "frac_of_nominal_2250": achieved / 2250.0},
+            "skinny": {"workload": workload_name(sk), "variant": sk_name, "value": sk_gbs, "unit": "GB/s",
+                       "us_per_call": sk_avg * 1e6, "steps": sk_steps,
+                       "roofline": {"bound": "hbm", "achieved": sk_gbs, "peak": peaks["hbm_gbs"],
+                                    "unit": "GB/s", "frac": sk_gbs / peaks["hbm_gbs"],
+                                    "traffic": NCU_TRAFFIC_BYTES["C5a"],
+                                    "peak_source": f"of {peak_src}",
+                                    "frac_of_nominal_8000": sk_gbs / 8000.0}},
+        }
+        if world == 1:
+            line["cpu_baseline"] = cpu_baseline_sample(cfg, A, Bm)
+    if use_dist:
+        dist.barrier()
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    args = ap.parse_args()
+    if args.steps < 1:
+        ap.error("--steps must be >= 1")
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -109,8 +109,7 @@ void build_variants()
 }
 
 constexpr int kNumSMs = 148;
-constexpr int64_t kMaxCounters = 16384;              // tiles a split-K launch may have
-constexpr int64_t kMaxPartialBytes = int64_t(1) << 30;
+constexpr int64_t kMaxPartialBytes = int64_t(1) << 30;   // split-K scratch a variant may ask for
 
 inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int64_t round_up(int64_t a, int64_t b) { return cdiv(a, b) * b; }
@@ -129,6 +128,13 @@ Tiling tiling_for(const Problem &p, int block_n, int split_k)
     return t;
 }
 
+// fp32 partial sums of a split-K run: [split][batch][M][ldp], ldp = N rounded up to 4
+inline int64_t partial_ld(const Problem &p) { return round_up(p.N, 4); }
+inline int64_t partial_bytes(const Problem &p, int split_k)
+{
+    return int64_t(split_k) * p.batch * p.M * partial_ld(p) * 4;
+}
+
 bool variant_supports(const Variant &v, const Problem &p)
 {
     if (is_empty(p)) return true;
@@ -138,35 +144,39 @@ bool variant_supports(const Variant &v, const Problem &p)
     if (t.units > kMaxDim) return false;
     if (v.split_k > 1) {
         if (v.split_k > t.kblocks) return false;
-        if (t.tiles > kMaxCounters) return false;
-        if (t.units * int64_t(kBlockM) * v.block_n * 4 > kMaxPartialBytes) return false;
+        if (partial_bytes(p, v.split_k) > kMaxPartialBytes) return false;
     }
     return true;
 }
 
-// Cost model (SM clocks) behind the automatic choice.  A CTA spends, per
-// 64-deep k-block, the larger of the tensor-pipe time (2*BLOCK_N clocks for
-// four 128 x BLOCK_N x 16 MMAs) and the time to stream the block's operand
-// bytes at this SM's share of memory bandwidth; per unit it also pays an
-// epilogue, and split-K units pay for writing and re-reading partial tiles.
+// Cost model (SM clocks) behind the automatic choice: the larger of a compute
+// estimate and a memory estimate, plus fixed launch costs.
+//  compute: waves x (k-blocks per unit x 2*BLOCK_N clocks for the four
+//           128 x BLOCK_N x 16 MMAs of a k-block) plus one exposed epilogue;
+//  memory : compulsory bytes (A, B once; C once; split-K partials written and
+//           read) over the bandwidth the active SMs can draw, capped by HBM.
 double variant_cost(const Variant &v, const Problem &p)
 {
     const Tiling t = tiling_for(p, v.block_n, v.split_k);
     const double waves = (double)cdiv(t.units, kNumSMs);
     const double kb_per_unit = (double)cdiv(t.kblocks, v.split_k);
     const double rows = p.M < kBlockM ? (double)p.M : (double)kBlockM;
-    const double cols = p.N < v.block_n ? (double)p.N : (double)v.block_n;
-    const double bytes_kb = rows * 128.0 + cols * 128.0;
-    const double mem_clk = bytes_kb / 24.0;           // ~6.5 TB/s over 148 SMs at ~1.9 GHz
-    const double mma_clk = 2.0 * v.block_n;
-    const double per_kb = mma_clk > mem_clk ? mma_clk : mem_clk;
     const double out_b = (p.out_dtype == CUDALLM_F32) ? 4.0 : 2.0;
-    double epi = rows * cols * out_b / 24.0 + 600.0;
-    if (v.split_k > 1) epi += rows * v.block_n * 4.0 * 2.0 / 24.0 + 1500.0;
-    // the epilogue of a tile overlaps the next tile's main loop except on the last wave
-    const double main = waves * kb_per_unit * per_kb;
-    return main + epi + (waves - 1.0) * (epi > kb_per_unit * per_kb ? epi - kb_per_unit * per_kb : 0.0)
-         + 3000.0;
+    const double epi = rows * v.block_n * (v.split_k > 1 ? 4.0 : out_b) / 32.0 + 1500.0;
+    // measured on 4096^3: a k-block costs about 300 + 0.83 * BLOCK_N clocks
+    const double mainloop = kb_per_unit * (300.0 + 0.83 * v.block_n);
+    const double compute = waves * (mainloop > epi ? mainloop : epi) + epi;
+    const double active = t.units < kNumSMs ? (double)t.units : (double)kNumSMs;
+    double bw = active * 40.0;                         // bytes per clock the active SMs can pull
+    if (bw > 3500.0) bw = 3500.0;                      // ~6.5 TB/s at ~1.9 GHz
+    double bytes = (double)p.batch * (2.0 * p.M * p.K + 2.0 * p.K * p.N + out_b * p.M * p.N);
+    double fixed = 4000.0;
+    if (v.split_k > 1) {
+        bytes += 2.0 * (double)partial_bytes(p, v.split_k);
+        fixed += 6000.0;                               // second launch (the reduction)
+    }
+    const double memory = bytes / bw;
+    return (compute > memory ? compute : memory) + fixed;
 }
 
 int select_variant(const Problem &p)
@@ -184,10 +194,8 @@ int select_variant(const Problem &p)
 }
 
 // --------------------------------------------------------------- workspace --
-// Layout: [status 256 B][tile counters][split-K partials][packed A][packed B]
-constexpr size_t kStatusBytes = 256;
-constexpr size_t kCounterBytes = kMaxCounters * sizeof(int);
-constexpr size_t kHeaderBytes = kStatusBytes + kCounterBytes;
+// Layout: [status 256 B][split-K partials][packed A][packed B]
+constexpr size_t kHeaderBytes = 256;
 constexpr int kMaxDevices = 64;
 
 struct DeviceState {
@@ -287,10 +295,7 @@ Plan make_plan(const Variant &v, const Problem &p, bool pack_a, bool pack_b)
     pl.pack_b = pack_b;
     size_t off = kHeaderBytes;
     pl.off_partials = off;
-    if (v.family == kUmma && v.split_k > 1) {
-        const Tiling t = tiling_for(p, v.block_n, v.split_k);
-        off += (size_t)t.units * kBlockM * v.block_n * 4;
-    }
+    if (v.family == kUmma && v.split_k > 1) off += (size_t)partial_bytes(p, v.split_k);
     off = (size_t)round_up((int64_t)off, 256);
     pl.off_pack_a = off;
     pl.ldap = round_up(p.K, 8);
@@ -403,7 +408,10 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     }
 
     CUtensorMap ta, tb;
-    st = encode_operand_map(&ta, A, p.K, p.M, p.batch, lda, sA, kBlockK, kBlockM);
+    // Rows of A beyond M only feed rows of C that are never stored, so the box
+    // need not cover (and zero-fill) them.
+    const int a_box_rows = p.M >= kBlockM ? kBlockM : (int)round_up(p.M, 8);
+    st = encode_operand_map(&ta, A, p.K, p.M, p.batch, lda, sA, kBlockK, a_box_rows);
     if (st != CUDALLM_OK) return st;
     st = encode_operand_map(&tb, B, p.N, p.K, p.batch, ldb, sB, 64, kBlockK);
     if (st != CUDALLM_OK) return st;
@@ -421,19 +429,37 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     const int64_t vec = (p.out_dtype == CUDALLM_F32) ? 4 : 8;
     gp.c_vec_ok = (reinterpret_cast<uintptr_t>(p.C) % 16 == 0) && (p.ldc % vec == 0)
                && (p.batch == 1 || p.sC % vec == 0);
+    gp.a_box_bytes = a_box_rows * 128;
     gp.partials = reinterpret_cast<float *>(ws + pl.off_partials);
-    gp.counters = reinterpret_cast<int *>(ws + kStatusBytes);
+    gp.ldp = partial_ld(p);
     gp.status = reinterpret_cast<int *>(ws);
 
     const bool bf = p.out_dtype == CUDALLM_BF16;
     switch (v.block_n) {
-    case 64:  return bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
-                        : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream);
-    case 128: return bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
-                        : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream);
-    default:  return bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
-                        : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream);
+    case 64:  st = bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
+                      : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream); break;
+    case 128: st = bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
+                      : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream); break;
+    default:  st = bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
+                      : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream); break;
     }
+    if (st != CUDALLM_OK || v.split_k == 1) return st;
+
+    // split-K: add the slices in fixed order and write C
+    const int64_t groups = p.batch * p.M * cdiv(p.N, 4);
+    int64_t blocks = cdiv(groups, 256);
+    if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
+    const int64_t al = bf ? 8 : 16;
+    const int vec4 = (reinterpret_cast<uintptr_t>(p.C) % al == 0) && (p.ldc % 4 == 0)
+                  && (p.batch == 1 || p.sC % 4 == 0);
+    if (bf)
+        splitk_reduce_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>(
+            gp.partials, p.C, gp.M, gp.N, gp.batch, v.split_k, gp.ldp, p.ldc, gp.strideC, vec4);
+    else
+        splitk_reduce_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>(
+            gp.partials, p.C, gp.M, gp.N, gp.batch, v.split_k, gp.ldp, p.ldc, gp.strideC, vec4);
+    CUDA_TRY(cudaGetLastError());
+    return CUDALLM_OK;
 }
 
 int run(int variant, const Problem &p, void *stream_v)

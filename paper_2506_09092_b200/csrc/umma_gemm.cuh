@@ -10,9 +10,10 @@
 // owner), warps 2..5 = epilogue (TMEM -> registers -> global).
 //
 // Work is cut into units (tile, k-split); CTA b runs units b, b+grid, ...
-// With split_k > 1 every unit writes an fp32 partial tile to the workspace and
-// the unit that arrives last at the tile's counter adds the partials in split
-// order 0..S-1 (so the result does not depend on arrival order) and stores C.
+// With split_k > 1 every unit writes its fp32 partial sums to slice `split` of
+// a workspace shaped [split][batch][M][ldp]; splitk_reduce_kernel then adds the
+// slices in split order 0..S-1 (a fixed order, so results are reproducible)
+// and writes C, rounding once.
 #pragma once
 #include "ptx.cuh"
 
@@ -37,8 +38,9 @@ struct GemmParams {
     int kblocks;            // ceil(K / 64)
     int num_units;          // tiles_m * tiles_n * batch * split_k
     int c_vec_ok;           // C base, ldc, strideC allow 16-byte stores
-    float *partials;        // split-K partial tiles (workspace)
-    int *counters;          // one per tile (workspace), zero between launches
+    int a_box_bytes;        // bytes one TMA box of A delivers (box rows * 128)
+    float *partials;        // split-K partial sums [split][batch][M][ldp] (workspace)
+    long long ldp;          // row stride of the partial slices (multiple of 4)
     int *status;            // [0] = code, [1] = detail
 };
 
@@ -48,8 +50,8 @@ struct SmemLayout {
     static constexpr int kBBytes = kBlockK * BLOCK_N * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kBarOffset = STAGES * kStageBytes;
-    // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], epilogue group
-    static constexpr int kNumBars = 2 * STAGES + 5;
+    // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
+    static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
     static constexpr int kBytes = kMiscOffset + 64;
     static constexpr int kDynamicBytes = kBytes + 1024;  // slack for 1024-byte alignment
@@ -81,17 +83,17 @@ __device__ __forceinline__ UnitCoord decode_unit(const GemmParams &p, int u)
     return c;
 }
 
-// Store 32 consecutive fp32 accumulator values of one row to C (fp32 or bf16).
+// Store 32 consecutive fp32 accumulator values of one row, starting at column
+// col0 of an n_cols-wide matrix, to `row_ptr + col0` (fp32 or bf16 elements).
 template <bool OUT_BF16>
-__device__ __forceinline__ void store_row_chunk(const GemmParams &p, const float (&v)[32],
-                                                long long row_off, int col0, bool row_ok)
+__device__ __forceinline__ void store_row_chunk(void *row_ptr, const float (&v)[32], int col0,
+                                                int n_cols, bool vec_ok)
 {
-    if (!row_ok) return;
-    const int n_left = p.N - col0;
+    const int n_left = n_cols - col0;
     if (n_left <= 0) return;
     if (OUT_BF16) {
-        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.C) + row_off + col0;
-        if (p.c_vec_ok && n_left >= 32) {
+        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(row_ptr) + col0;
+        if (vec_ok && n_left >= 32) {
             uint4 *d4 = reinterpret_cast<uint4 *>(dst);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -108,8 +110,8 @@ __device__ __forceinline__ void store_row_chunk(const GemmParams &p, const float
                 if (j < n_left) dst[j] = __float2bfloat16_rn(v[j]);
         }
     } else {
-        float *dst = reinterpret_cast<float *>(p.C) + row_off + col0;
-        if (p.c_vec_ok && n_left >= 32) {
+        float *dst = reinterpret_cast<float *>(row_ptr) + col0;
+        if (vec_ok && n_left >= 32) {
             float4 *d4 = reinterpret_cast<float4 *>(dst);
 #pragma unroll
             for (int q = 0; q < 8; ++q)
@@ -141,17 +143,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
-    const uint32_t epi_bar = bar_base + 8u * (2 * STAGES + 4);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L::kMiscOffset);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kMiscOffset + 4);
-    volatile int *last_flag = reinterpret_cast<volatile int *>(smem + L::kMiscOffset + 8);
 
     const int warp_idx = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        *last_flag = 0;
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
@@ -160,7 +159,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             mbar_init(tfull_bar(a), 1);
             mbar_init(tempty_bar(a), 4);     // one arrival per epilogue warp
         }
-        mbar_init(epi_bar, kEpiThreads);
         fence_mbar_init();
         fence_proxy_async_smem();
         prefetch_tensormap(&tmap_a);
@@ -191,7 +189,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     }
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
                     const uint32_t sb = sa + L::kABytes;
-                    mbar_arrive_expect_tx(full_bar(stage), L::kStageBytes);
+                    mbar_arrive_expect_tx(full_bar(stage), p.a_box_bytes + L::kBBytes);
                     tma_load_3d(sa, &tmap_a, full_bar(stage), kb * kBlockK, c.m_tile * kBlockM, c.b);
 #pragma unroll
                     for (int j = 0; j < BLOCK_N / 64; ++j)
@@ -249,15 +247,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         const int epi_tid = quad * 32 + lane;            // == row within the tile
         int acc = 0;
         uint32_t acc_phase = 0;
-        uint32_t epi_phase = 0;
-        // Rendezvous of the 128 epilogue threads on an mbarrier, so that this
-        // wait is bounded like every other one in the kernel.
-        auto epi_sync = [&]() -> bool {
-            mbar_arrive(epi_bar);
-            const bool done = mbar_wait(epi_bar, epi_phase, abort_flag);
-            epi_phase ^= 1;
-            return done;
-        };
         for (int u = blockIdx.x; u < p.num_units; u += gridDim.x) {
             const UnitCoord c = decode_unit(p, u);
             bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
@@ -269,80 +258,39 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tc_fence_after();
             const int row = c.m_tile * kBlockM + epi_tid;
             const bool row_ok = row < p.M;
-            const long long row_off = static_cast<long long>(c.b) * p.strideC
-                                    + static_cast<long long>(row) * p.ldc;
             const uint32_t t_addr = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(quad * 32) << 16);
+            // destination row: C itself, or this split's slice of the partial sums
+            void *row_ptr;
+            bool vec_ok;
             if (p.split_k == 1) {
+                const long long off = static_cast<long long>(c.b) * p.strideC
+                                    + static_cast<long long>(row) * p.ldc;
+                row_ptr = OUT_BF16 ? static_cast<void *>(reinterpret_cast<__nv_bfloat16 *>(p.C) + off)
+                                   : static_cast<void *>(reinterpret_cast<float *>(p.C) + off);
+                vec_ok = p.c_vec_ok != 0;
+            } else {
+                row_ptr = p.partials
+                        + ((static_cast<long long>(c.split) * p.batch + c.b) * p.M + row) * p.ldp;
+                vec_ok = true;
+            }
 #pragma unroll 1
-                for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
-                    uint32_t r[32];
-                    tmem_ld_32x32b_x32(t_addr + ch * 32, r);
-                    tmem_ld_wait();
+            for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(t_addr + ch * 32, r);
+                tmem_ld_wait();
+                if (row_ok) {
                     float v[32];
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-                    store_row_chunk<OUT_BF16>(p, v, row_off, c.n_tile * BLOCK_N + ch * 32, row_ok);
+                    const int col0 = c.n_tile * BLOCK_N + ch * 32;
+                    if (p.split_k == 1) store_row_chunk<OUT_BF16>(row_ptr, v, col0, p.N, vec_ok);
+                    else                store_row_chunk<false>(row_ptr, v, col0, p.N, vec_ok);
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar(acc));
-            } else {
-                // partial tile layout: float4 index ((ch*8 + q) * 128 + row)
-                float4 *part = reinterpret_cast<float4 *>(p.partials)
-                             + (static_cast<long long>(c.tile_linear) * p.split_k + c.split)
-                                   * (kBlockM * BLOCK_N / 4);
-#pragma unroll 1
-                for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
-                    uint32_t r[32];
-                    tmem_ld_32x32b_x32(t_addr + ch * 32, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        __stcg(part + (ch * 8 + q) * kBlockM + epi_tid,
-                               make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
-                                           __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3])));
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar(acc));
-                __threadfence();
-                if (!epi_sync()) {
-                    report_timeout(p.status, kRoleEpilogue, 0xC0);
-                    break;
-                }
-                if (epi_tid == 0) {
-                    const int old = atomicAdd(p.counters + c.tile_linear, 1);
-                    const int last = (old == p.split_k - 1);
-                    if (last) p.counters[c.tile_linear] = 0;   // ready for the next launch
-                    *last_flag = last;
-                }
-                if (!epi_sync()) {
-                    report_timeout(p.status, kRoleEpilogue, 0xC1);
-                    break;
-                }
-                if (*last_flag) {
-                    __threadfence();
-                    const float4 *tile0 = reinterpret_cast<const float4 *>(p.partials)
-                                        + static_cast<long long>(c.tile_linear) * p.split_k
-                                              * (kBlockM * BLOCK_N / 4);
-#pragma unroll 1
-                    for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
-                        float v[32];
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = 0.f;
-                        for (int s = 0; s < p.split_k; ++s) {
-                            const float4 *ps = tile0 + static_cast<long long>(s) * (kBlockM * BLOCK_N / 4);
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                const float4 t = __ldcg(ps + (ch * 8 + q) * kBlockM + epi_tid);
-                                v[4 * q] += t.x; v[4 * q + 1] += t.y;
-                                v[4 * q + 2] += t.z; v[4 * q + 3] += t.w;
-                            }
-                        }
-                        store_row_chunk<OUT_BF16>(p, v, row_off, c.n_tile * BLOCK_N + ch * 32, row_ok);
-                    }
-                }
+                __syncwarp();                            // tcgen05.ld needs the whole warp
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
     }
@@ -353,6 +301,54 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// Adds the S slices of split-K partial sums in order s = 0..S-1 and writes C
+// (fp32, or bf16 rounded once).  One thread handles 4 consecutive columns.
+template <bool OUT_BF16>
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float *__restrict__ partials, void *C, int M, int N, int batch, int split_k,
+                     long long ldp, long long ldc, long long strideC, int c_vec4_ok)
+{
+    const int groups = (N + 3) >> 2;
+    const long long rows = static_cast<long long>(batch) * M;
+    const long long total = rows * groups;
+    const long long slice = rows * ldp;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long br = i / groups;                 // b * M + row
+        const int col = static_cast<int>(i - br * groups) * 4;
+        const int b = static_cast<int>(br / M);
+        const int row = static_cast<int>(br - static_cast<long long>(b) * M);
+        const float *src = partials + br * ldp + col;
+        float4 acc = __ldcg(reinterpret_cast<const float4 *>(src));
+        for (int s = 1; s < split_k; ++s) {
+            const float4 t = __ldcg(reinterpret_cast<const float4 *>(src + s * slice));
+            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        }
+        const long long off = b * strideC + row * ldc + col;
+        const int n_left = N - col;
+        if (OUT_BF16) {
+            __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(C) + off;
+            if (c_vec4_ok && n_left >= 4) {
+                uint2 w;
+                w.x = pack_bf16x2(acc.x, acc.y);
+                w.y = pack_bf16x2(acc.z, acc.w);
+                *reinterpret_cast<uint2 *>(dst) = w;
+            } else {
+                const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+                for (int j = 0; j < 4 && j < n_left; ++j) dst[j] = __float2bfloat16_rn(a[j]);
+            }
+        } else {
+            float *dst = reinterpret_cast<float *>(C) + off;
+            if (c_vec4_ok && n_left >= 4) {
+                *reinterpret_cast<float4 *>(dst) = acc;
+            } else {
+                const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+                for (int j = 0; j < 4 && j < n_left; ++j) dst[j] = a[j];
+            }
+        }
     }
 }
 

@@ -1,0 +1,149 @@
+"""CPU-only checks of the C ABI: the library loads, exports every symbol the
+header declares, and rejects bad arguments before touching CUDA; plus the
+host-side variant table, selection and the search loop."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2506_09092_b200 import binding as B
+from paper_2506_09092_b200 import build as libbuild
+from paper_2506_09092_b200 import harness as H
+from paper_2506_09092_b200 import inputs as gi
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    libbuild.build()
+
+
+def header_symbols():
+    text = open(os.path.join(ROOT, "include", "cudallm_gemm.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cudallm_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    syms = header_symbols()
+    assert len(syms) >= 14
+    L = ctypes.CDLL(B.LIB_PATH)
+    for s in syms:
+        assert hasattr(L, s), s
+    assert sorted(B.SIGNATURES) == syms          # the binding covers the same set
+
+
+def test_version_and_variant_table():
+    assert B.version() >= 100
+    n = B.num_variants()
+    names = [B.variant_name(v) for v in range(n)]
+    assert names[0] == "simt" and len(set(names)) == n
+    assert B.variant_name(n) is None and B.variant_name(-1) is None
+    assert any(nm.startswith("umma_n256") for nm in names)
+
+
+def test_argument_errors_are_reported_before_any_cuda_call():
+    p = 4096            # a non-null, aligned stand-in address; never dereferenced on error
+    g = lambda *a, **k: B.gemm_bf16(*a, check=False, **k)
+    assert g(None, p, p, 4, 4, 4, 4, 4, 4, 0) == B.ERR_INVALID_POINTER
+    assert g(p, None, p, 4, 4, 4, 4, 4, 4, 0) == B.ERR_INVALID_POINTER
+    assert g(p, p, None, 4, 4, 4, 4, 4, 4, 0) == B.ERR_INVALID_POINTER
+    assert g(p, p, p, -1, 4, 4, 4, 4, 4, 0) == B.ERR_INVALID_DIM
+    assert g(p, p, p, 4, 4, 1 << 40, 1 << 40, 4, 4, 0) == B.ERR_INVALID_DIM
+    assert g(p, p, p, 4, 4, 4, 3, 4, 4, 0) == B.ERR_INVALID_LD
+    assert g(p, p, p, 4, 4, 4, 4, 3, 4, 0) == B.ERR_INVALID_LD
+    assert g(p, p, p, 4, 4, 4, 4, 4, 3, 0) == B.ERR_INVALID_LD
+    assert g(p, p, p, 4, 4, 4, 4, 4, 4, 2) == B.ERR_INVALID_DTYPE
+    assert g(p + 1, p, p, 4, 4, 4, 4, 4, 4, 0) == B.ERR_MISALIGNED
+    assert g(p, p, p + 2, 4, 4, 4, 4, 4, 4, 0) == B.ERR_MISALIGNED     # fp32 C needs 4 bytes
+    # empty problems succeed without a device, even with null pointers
+    assert g(None, None, None, 0, 4, 4, 4, 4, 4, 0) == B.OK
+    assert g(None, None, None, 4, 0, 4, 4, 0, 0, 1) == B.OK
+    # batched: overlapping items of C are refused
+    st = B.gemm_bf16_batched(p, p, p, 4, 4, 4, 4, 4, 4, 16, 16, 15, 2, 0, check=False)
+    assert st == B.ERR_INVALID_LD
+    assert B.gemm_bf16_batched(p, p, p, 4, 4, 4, 4, 4, 4, 16, 16, 16, 0, 0, check=False) == B.OK
+    st = B.gemm_bf16_variant(999, p, p, p, 4, 4, 4, 4, 4, 4, 16, 16, 16, 1, 0, check=False)
+    assert st == B.ERR_INVALID_VARIANT
+    assert "leading dimension" in B.strerror(B.ERR_INVALID_LD)
+    assert B.strerror(12345) == "unknown status"
+
+
+def test_host_entry_point_validates_first():
+    p = 4096
+    assert B.gemm_bf16_host(None, p, p, 4, 4, 4, 4, 4, 4, 0, p, 1 << 20, check=False) == B.ERR_INVALID_POINTER
+    assert B.gemm_bf16_host(p, p, p, 4, 4, 4, 4, 4, 4, 0, None, 0, check=False) == B.ERR_WORKSPACE
+    need = B.host_staging_bytes(4, 4, 4, 4, 4, 4, 0)
+    assert need == 3 * 256
+    assert B.gemm_bf16_host(p, p, p, 4, 4, 4, 4, 4, 4, 0, p, need - 1, check=False) == B.ERR_WORKSPACE
+
+
+def test_variant_support_rules():
+    table = {B.variant_name(v): v for v in range(B.num_variants())}
+    # split-K needs at least one 64-deep k-block per split
+    assert B.variant_supports(table["umma_n64_sk16"], 128, 128, 64, 64, 128, 128, 1, 0) == 0
+    assert B.variant_supports(table["umma_n64_sk16"], 128, 128, 1024, 1024, 128, 128, 1, 0) == 1
+    assert B.variant_supports(table["simt"], 1, 1, 0, 0, 1, 1, 1, 0) == 1
+    assert B.variant_supports(table["umma_n128"], 1, 1, 0, 0, 1, 1, 1, 0) == 0      # K == 0
+    assert B.variant_supports(-3, 1, 1, 1, 1, 1, 1, 1, 0) == B.ERR_INVALID_VARIANT
+    assert B.variant_supports(0, 4, 4, 4, 3, 4, 4, 1, 0) == B.ERR_INVALID_LD
+
+
+def test_selection_and_workspace_queries():
+    for cfg in gi.CONFIGS.values():
+        v = B.select_variant(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype)
+        assert 0 < v < B.num_variants()
+        assert B.variant_supports(v, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch,
+                                  cfg.out_dtype) == 1
+        ws = B.workspace_bytes(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype)
+        assert ws >= 256 and ws % 256 == 0
+    c2 = gi.CONFIGS["C2"]
+    assert B.variant_name(B.select_variant(c2.M, c2.N, c2.K, c2.K, c2.N, c2.N, 1, 1)).startswith("umma_n256")
+    assert B.select_variant(4, 4, 0, 0, 4, 4, 1, 0) == 0          # K == 0 runs on the simt kernel
+
+
+# ------------------------------------------------------------ search loop ----
+
+class _Case:
+    def __init__(self, name):
+        self.name = name
+
+
+def test_search_keeps_fastest_valid_candidate():
+    lat = {0: 5.0, 1: 1.0, 2: 2.0, 3: 0.5}
+    broken = {1: H.MISMATCH, 3: H.LAUNCH_FAIL}
+
+    def validate(k):
+        return H.ValidationReport(broken.get(k, H.OK))
+
+    res = H.search([0, 1, 2, 3], validate, lambda k: lat[k])
+    assert res.valid == [0, 2] and res.best == 2 and res.best_latency == 2.0
+    assert res.reports[1].status == H.MISMATCH and 3 not in res.latencies
+
+
+def test_search_with_no_valid_candidate_reports_failure_and_terminates():
+    res = H.search([0, 1], lambda k: H.ValidationReport(H.MISMATCH), lambda k: 1.0)
+    assert res.best is None and res.best_latency == float("inf") and res.valid == []
+
+
+def test_search_tie_keeps_earlier_candidate():
+    res = H.search([4, 2], lambda k: H.ValidationReport(H.OK), lambda k: 1.0)
+    assert res.best == 4
+
+
+def test_function_validator_failure_classes():
+    cases = [_Case("a"), _Case("b"), _Case("c")]
+    good = lambda k, c: (0, 1.0)
+    cmp_ok = lambda c, out: (True, 1e-6, "")
+    assert H.function_validator(0, cases, good, cmp_ok).status == H.OK
+    rep = H.function_validator(0, cases, lambda k, c: (-8, None) if c.name == "b" else (0, 1.0), cmp_ok)
+    assert rep.status == H.LAUNCH_FAIL and rep.failed_case == "b" and rep.cases == 1
+    rep = H.function_validator(0, cases, lambda k, c: (-9, None), cmp_ok)
+    assert rep.status == H.TIMEOUT
+    rep = H.function_validator(0, cases, lambda k, c: ("unsupported", None), cmp_ok)
+    assert rep.status == H.UNSUPPORTED
+    rep = H.function_validator(0, cases, good, lambda c, out: (c.name != "c", 0.5, "edge column stale"))
+    assert rep.status == H.MISMATCH and rep.failed_case == "c" and rep.detail == "edge column stale"

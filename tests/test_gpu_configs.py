@@ -1,0 +1,82 @@
+"""The benchmark configurations at full size, in the launch configuration the
+benchmark times (automatic variant choice, device-resident operands).
+
+C1, C4, C5a and C5b are compared with the oracle on every element.  C2 and C3
+are compared on a seeded sample of full rows (the oracle needs tens of seconds
+for the whole product) and, on every element, against the integer rank-1
+closed form, which holds at any size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import gpu_util as G
+from paper_2506_09092_b200 import binding as B
+from paper_2506_09092_b200 import inputs as gi
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, A, Bm, variant=B.VARIANT_AUTO):
+    vals, raw, guards = G.run_config(cfg, variant, (A, Bm))
+    assert guards
+    return vals, raw
+
+
+@pytest.mark.parametrize("name", ["C1", "C4", "C5a", "C5b"])
+def test_config_every_element(name):
+    cfg = gi.CONFIGS[name]
+    A, Bm = cfg.make()
+    vals, _ = _run(cfg, A, Bm)
+    if cfg.batch > 1:
+        Cref, S = oracle.gemm_batched(A, Bm, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_,
+                                      cfg.strideA, cfg.strideB, cfg.batch)
+        r = oracle.check(vals, Cref, S, G.tol_for(cfg.out_dtype))
+    else:
+        Cref, S = oracle.gemm(A, Bm, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_)
+        r = oracle.check(vals[0], Cref, S, G.tol_for(cfg.out_dtype))
+    assert r.ok, (name, r)
+
+
+@pytest.mark.parametrize("name,nrows", [("C2", 384), ("C3", 96)])
+def test_config_sampled_rows(name, nrows):
+    cfg = gi.CONFIGS[name]
+    A, Bm = cfg.make()
+    vals, _ = _run(cfg, A, Bm)
+    rng = np.random.default_rng([cfg.seed, 99])
+    rows = np.sort(rng.choice(cfg.M, size=nrows, replace=False))
+    rows[0], rows[-1] = 0, cfg.M - 1                      # always include the edges
+    rows[1] = 127; rows[2] = 128                          # and a tile boundary
+    Cref, S = oracle.gemm_rows(A, Bm, rows, cfg.N, cfg.K, cfg.lda_, cfg.ldb_)
+    r = oracle.check(vals[0][rows], Cref, S, G.tol_for(cfg.out_dtype))
+    assert r.ok, (name, r)
+    assert np.isfinite(vals[0]).all()
+
+
+@pytest.mark.parametrize("name", ["C2", "C3", "C5a", "C5b"])
+def test_config_size_integer_closed_form(name):
+    """A = u p^T, B = q v^T with small integers: C = (p.q) u v^T exactly, at the
+    configuration's full size and strides, every element."""
+    cfg = gi.CONFIGS[name]
+    u, v_, p, q = gi.rank1_int_factors(cfg.M, cfg.N, cfg.K, seed=cfg.seed + 50)
+    A = gi.embed(gi.int_to_bf16_bits(np.outer(u, p)), cfg.lda_)
+    Bm = gi.embed(gi.int_to_bf16_bits(np.outer(q, v_)), cfg.ldb_)
+    exact = np.outer(u, v_).astype(np.float64) * float(np.dot(p, q))
+    vals, raw = _run(cfg, A, Bm)
+    if cfg.out_dtype == gi.F32:
+        assert np.array_equal(vals[0], exact)
+    else:
+        want = oracle.f64_to_bf16_bits(exact)
+        assert ((raw[0] == want) | ((exact == 0) & (vals[0] == 0))).all()
+
+
+def test_paper_task2_ladder_first_two_sizes():
+    """The paper's own Task 2 shapes (A size x 4096, B 4096 x 2048), the two
+    smallest sizes, sampled rows."""
+    for step in (0, 1):
+        cfg = gi.task2_ladder(step)
+        A, Bm = cfg.make()
+        vals, _ = _run(cfg, A, Bm)
+        rows = np.random.default_rng(step).choice(cfg.M, size=64, replace=False)
+        Cref, S = oracle.gemm_rows(A, Bm, rows, cfg.N, cfg.K, cfg.lda_, cfg.ldb_)
+        assert oracle.check(vals[0][rows], Cref, S, G.tol_for(cfg.out_dtype)).ok
