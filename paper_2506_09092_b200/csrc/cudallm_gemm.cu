@@ -149,12 +149,13 @@ bool variant_supports(const Variant &v, const Problem &p)
     return true;
 }
 
-// Cost model (SM clocks) behind the automatic choice: the larger of a compute
-// estimate and a memory estimate, plus fixed launch costs.
-//  compute: waves x (k-blocks per unit x 2*BLOCK_N clocks for the four
-//           128 x BLOCK_N x 16 MMAs of a k-block) plus one exposed epilogue;
-//  memory : compulsory bytes (A, B once; C once; split-K partials written and
-//           read) over the bandwidth the active SMs can draw, capped by HBM.
+// Cost model (SM clocks) behind the automatic choice.
+//  main kernel: the larger of a compute estimate -- waves x k-blocks per unit x
+//      clocks per k-block (measured on 4096^3: about 300 + 0.83 * BLOCK_N),
+//      plus one exposed epilogue -- and a memory estimate: A and B read once
+//      and C (or the split-K partial sums) written once, over the bandwidth
+//      the active SMs can draw (about 40 B/clock each), capped by HBM.
+//  split-K adds the reduction kernel: partial sums read, C written, a launch.
 double variant_cost(const Variant &v, const Problem &p)
 {
     const Tiling t = tiling_for(p, v.block_n, v.split_k);
@@ -163,20 +164,18 @@ double variant_cost(const Variant &v, const Problem &p)
     const double rows = p.M < kBlockM ? (double)p.M : (double)kBlockM;
     const double out_b = (p.out_dtype == CUDALLM_F32) ? 4.0 : 2.0;
     const double epi = rows * v.block_n * (v.split_k > 1 ? 4.0 : out_b) / 32.0 + 1500.0;
-    // measured on 4096^3: a k-block costs about 300 + 0.83 * BLOCK_N clocks
     const double mainloop = kb_per_unit * (300.0 + 0.83 * v.block_n);
     const double compute = waves * (mainloop > epi ? mainloop : epi) + epi;
+    const double hbm = 3500.0;                         // bytes per clock: ~6.5 TB/s at ~1.9 GHz
     const double active = t.units < kNumSMs ? (double)t.units : (double)kNumSMs;
-    double bw = active * 40.0;                         // bytes per clock the active SMs can pull
-    if (bw > 3500.0) bw = 3500.0;                      // ~6.5 TB/s at ~1.9 GHz
-    double bytes = (double)p.batch * (2.0 * p.M * p.K + 2.0 * p.K * p.N + out_b * p.M * p.N);
-    double fixed = 4000.0;
-    if (v.split_k > 1) {
-        bytes += 2.0 * (double)partial_bytes(p, v.split_k);
-        fixed += 6000.0;                               // second launch (the reduction)
-    }
-    const double memory = bytes / bw;
-    return (compute > memory ? compute : memory) + fixed;
+    const double bw = active * 40.0 < hbm ? active * 40.0 : hbm;
+    const double ab_bytes = (double)p.batch * (2.0 * p.M * p.K + 2.0 * p.K * p.N);
+    const double c_bytes = (double)p.batch * out_b * p.M * p.N;
+    const double part_bytes = v.split_k > 1 ? (double)partial_bytes(p, v.split_k) : 0.0;
+    const double main_mem = (ab_bytes + (v.split_k > 1 ? part_bytes : c_bytes)) / bw;
+    double cost = (compute > main_mem ? compute : main_mem) + 4000.0;
+    if (v.split_k > 1) cost += (part_bytes + c_bytes) / hbm + 6000.0;
+    return cost;
 }
 
 int select_variant(const Problem &p)

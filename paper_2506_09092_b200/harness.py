@@ -171,3 +171,45 @@ class DeviceProblem:
         torch.cuda.synchronize()
         raw = self.sets[i % self.nsets][2].cpu().numpy()
         return raw.view(np.float32 if cfg.out_dtype == 0 else np.uint16)
+
+
+def _main(argv=None):
+    """``python -m paper_2506_09092_b200.harness --config C2``: run one benchmark
+    configuration a few times and print its timing (also the command that ncu
+    captures are taken from)."""
+    import argparse
+    import json
+    import torch
+    from . import binding as B
+    from . import inputs as gi
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default="C2", choices=sorted(gi.CONFIGS))
+    ap.add_argument("--variant", default="auto")
+    ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--sets", type=int, default=None, help="rotating buffer sets (default: > L2)")
+    ap.add_argument("--all-variants", action="store_true", help="time every variant that supports the shape")
+    args = ap.parse_args(argv)
+    cfg = gi.CONFIGS[args.config]
+    names = {B.variant_name(v): v for v in range(B.num_variants())}
+    prob = DeviceProblem(cfg, nsets=args.sets)
+    if args.all_variants:
+        todo = [v for v in range(1, B.num_variants())
+                if B.variant_supports(v, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch,
+                                      cfg.out_dtype) == 1]
+    elif args.variant == "auto":
+        todo = [B.select_variant(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype)]
+    else:
+        todo = [names[args.variant]]
+    for v in todo:
+        t = performance_profiler(lambda i: prob.launch(i, v), iters=args.iters, warmup=args.warmup)
+        code, detail = B.device_status(torch.cuda.current_stream())
+        print(json.dumps({"config": cfg.name, "variant": B.variant_name(v), "status": code,
+                          "us_min": t["min_s"] * 1e6, "us_median": t["median_s"] * 1e6,
+                          "tflops": cfg.flops / t["median_s"] / 1e12,
+                          "gbs": cfg.algorithmic_bytes / t["median_s"] / 1e9}), flush=True)
+
+
+if __name__ == "__main__":
+    _main()

@@ -165,11 +165,13 @@ def test_rank1_integer_closed_form_bf16_rounds_to_nearest_even():
 
 
 def test_bf16_ties_round_to_even():
-    # C[i][j] = i * j style integers in [256, 512): odd values are exact ties
+    # C[i][j] = 256 + (i % 128) + j lies in [256, 512) where bf16 has spacing 2:
+    # every odd value is an exact tie.  All operand entries are exact in bf16.
     M, N, K = 130, 70, 64
     Am = np.zeros((M, K)); Bmat = np.zeros((K, N))
-    Am[:, 0] = 1.0; Am[:, 1] = np.arange(M) % 128          # C = 256 + (i%128) + j
-    Bmat[0, :] = 256.0 + np.arange(N); Bmat[1, :] = 1.0
+    Am[:, 0] = 1.0; Bmat[0, :] = 256.0
+    Am[:, 1] = np.arange(M) % 128; Bmat[1, :] = 1.0
+    Am[:, 2] = 1.0; Bmat[2, :] = np.arange(N)
     exact = 256.0 + (np.arange(M) % 128)[:, None] + np.arange(N)[None, :]
     expect_bits = oracle.f64_to_bf16_bits(exact)
     assert oracle.bf16_bits_to_f64(oracle.f64_to_bf16_bits(np.array([257.0, 259.0]))).tolist() == [256.0, 260.0]
