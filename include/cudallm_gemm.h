@@ -134,8 +134,8 @@ int cudallm_variant_supports(int variant,
                              int64_t lda, int64_t ldb, int64_t ldc,
                              int64_t batch, int out_dtype);
 /* Variant the library would choose for this problem (host-side decision only;
- * no CUDA call).  `a_aligned`/`b_aligned` say whether the operand base is
- * 16-byte aligned.  Returns a variant id or a negative status. */
+ * no CUDA call; operand bases are assumed 16-byte aligned).  Returns a variant
+ * id or a negative status. */
 int cudallm_select_variant(int64_t M, int64_t N, int64_t K,
                            int64_t lda, int64_t ldb, int64_t ldc,
                            int64_t batch, int out_dtype);
