@@ -66,6 +66,7 @@ extern "C" {
 #define CUDALLM_ERR_DEVICE_TIMEOUT     -9  /* a bounded wait inside a kernel ran out            */
 #define CUDALLM_ERR_WORKSPACE         -10  /* workspace missing, too small or misaligned        */
 #define CUDALLM_ERR_MISALIGNED        -11  /* pointer not aligned to its element size           */
+#define CUDALLM_ERR_TOO_LARGE         -12  /* problem exceeds a built-in, fixed-size scratch    */
 
 /* variant id meaning "let the library choose" */
 #define CUDALLM_VARIANT_AUTO           -1
@@ -124,6 +125,47 @@ int cudallm_gemm_bf16_host(const void *A_host, const void *B_host, void *C_host,
 size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K,
                                   int64_t lda, int64_t ldb, int64_t ldc,
                                   int out_dtype);
+
+/*
+ * Split-K product for callers that must not allocate.  (The paper has no
+ * counterpart for this call: its programs allocate freely in host code.)
+ *
+ * Who needs it: a process whose device memory is entirely owned by someone
+ * else's allocator (an inference server that reserved the whole GPU at start,
+ * a framework plug-in that may only use the tensors it is handed), or code on
+ * a path where a cudaMalloc -- which may synchronise the device or fail when
+ * memory is exhausted -- is not acceptable.  The other entry points obtain
+ * their split-K scratch from a workspace that the library allocates with
+ * cudaMalloc on first need; this one calls no cudaMalloc, cudaFree or any
+ * other allocating routine, ever.
+ *
+ * Its scratch is an array compiled into the library's device image
+ * (CUDALLM_NOALLOC_SCRATCH_BYTES, 8 MiB, resident on every GPU that loads the
+ * library until the process exits).  The product is split along K into
+ * `split_k` parts (2, 4, 8 or 16, at most ceil(K/64)); the fp32 partial sums
+ * go to that array and a second kernel adds them in fixed order and writes C.
+ *
+ *  - A, B, C, sizes, leading dimensions and out_dtype as cudallm_gemm_bf16.
+ *    A and B must take the direct TMA path: 16-byte aligned bases, lda and ldb
+ *    multiples of 8 (else CUDALLM_ERR_UNSUPPORTED_SHAPE; repacking would need
+ *    more scratch).
+ *  - Limit: 256 + split_k * M * round_up(N, 4) * 4 bytes must not exceed
+ *    CUDALLM_NOALLOC_SCRATCH_BYTES, else CUDALLM_ERR_TOO_LARGE and nothing runs.
+ *  - The call SYNCHRONISES `stream` before it returns and reports a kernel
+ *    whose bounded wait ran out as CUDALLM_ERR_DEVICE_TIMEOUT.
+ *  - The first call on each device looks up the array's device address (and,
+ *    like any first launch, lets the driver load the kernels).  Make that
+ *    first call outside any stream capture.
+ *  - All calls on a device share the one array, which keeps whatever the last
+ *    call left in it; the call clears the words that must start at zero.  Two
+ *    calls that overlap on the GPU (different streams, or different host
+ *    threads) race on it: serialise them.
+ */
+#define CUDALLM_NOALLOC_SCRATCH_BYTES (8u << 20)
+int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C,
+                                     int64_t M, int64_t N, int64_t K,
+                                     int64_t lda, int64_t ldb, int64_t ldc,
+                                     int out_dtype, int split_k, void *stream);
 
 /* Kernel variants (the candidate set of Algorithm 1's search). */
 int cudallm_num_variants(void);

@@ -26,6 +26,8 @@ ERR_CUDA = -8
 ERR_DEVICE_TIMEOUT = -9
 ERR_WORKSPACE = -10
 ERR_MISALIGNED = -11
+ERR_TOO_LARGE = -12
+NOALLOC_SCRATCH_BYTES = 8 << 20
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libcudallm_gemm.so")
@@ -43,6 +45,7 @@ SIGNATURES = {
     "cudallm_gemm_bf16_variant": (_int, [_int, _vp, _vp, _vp] + [_i64] * 10 + [_int, _vp]),
     "cudallm_gemm_bf16_host": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp, _sz, _vp]),
     "cudallm_host_staging_bytes": (_sz, [_i64] * 6 + [_int]),
+    "cudallm_gemm_bf16_splitk_noalloc": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _int, _vp]),
     "cudallm_num_variants": (_int, []),
     "cudallm_variant_name": (ctypes.c_char_p, [_int]),
     "cudallm_variant_supports": (_int, [_int] + [_i64] * 7 + [_int]),
@@ -129,6 +132,17 @@ def gemm_bf16_host(A_host, B_host, C_host, M, N, K, lda, ldb, ldc, out_dtype, de
     st = lib().cudallm_gemm_bf16_host(_p(A_host), _p(B_host), _p(C_host), M, N, K, lda, ldb, ldc,
                                       out_dtype, _p(dev_buf), dev_bytes, _s(stream))
     return _check(st, "cudallm_gemm_bf16_host", check)
+
+
+def gemm_bf16_splitk_noalloc(A, B, C, M, N, K, lda, ldb, ldc, out_dtype, split_k, stream=None,
+                             check=True):
+    """Split-K product whose scratch is an array built into the library: for
+    callers that may not allocate device memory (see the header).  Synchronises
+    ``stream``; the first call per device should come before any stream capture;
+    calls that overlap on the GPU race on the shared scratch."""
+    st = lib().cudallm_gemm_bf16_splitk_noalloc(_p(A), _p(B), _p(C), M, N, K, lda, ldb, ldc,
+                                                out_dtype, split_k, _s(stream))
+    return _check(st, "cudallm_gemm_bf16_splitk_noalloc", check)
 
 
 def host_staging_bytes(M, N, K, lda, ldb, ldc, out_dtype) -> int:

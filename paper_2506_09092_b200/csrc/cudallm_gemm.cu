@@ -582,6 +582,103 @@ int cudallm_gemm_bf16_host(const void *A_host, const void *B_host, void *C_host,
     return CUDALLM_OK;
 }
 
+// ---------------------------------------------------------------------------
+// Split-K without any allocation: the scratch is part of the device image.
+// `g_noalloc_scratch` names the array for device code; on the host the same
+// name is only a handle for cudaGetSymbolAddress, never a device address.
+// Layout: [status word, 256 B][fp32 partial sums: split_k x M x ldp].
+static __device__ __align__(256) unsigned char g_noalloc_scratch[CUDALLM_NOALLOC_SCRATCH_BYTES];
+static void *g_noalloc_scratch_addr[kMaxDevices] = {};   // per device, filled on first use
+
+int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int64_t M, int64_t N,
+                                     int64_t K, int64_t lda, int64_t ldb, int64_t ldc, int out_dtype,
+                                     int split_k, void *stream_v)
+{
+    build_variants();
+    const Problem p = make_problem(A, B, C, M, N, K, lda, ldb, ldc, 0, 0, 0, 1, out_dtype);
+    int st = validate(p);
+    if (st != CUDALLM_OK) return st;
+    if (split_k != 2 && split_k != 4 && split_k != 8 && split_k != 16) return CUDALLM_ERR_INVALID_VARIANT;
+    if (is_empty(p)) return CUDALLM_OK;
+    if (cdiv(K, kBlockK) < split_k) return CUDALLM_ERR_UNSUPPORTED_SHAPE;   // also covers K == 0
+    if (!a_operand_aligned(p) || !b_operand_aligned(p)) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+    if ((long double)partial_bytes(p, split_k) + 256.0L > (long double)CUDALLM_NOALLOC_SCRATCH_BYTES)
+        return CUDALLM_ERR_TOO_LARGE;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    st = probe_device(dev);
+    if (st != CUDALLM_OK) return st;
+    if (!g_noalloc_scratch_addr[dev]) {
+        // once per device, with that device current
+        void *addr = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&addr, g_noalloc_scratch));
+        g_noalloc_scratch_addr[dev] = addr;
+    }
+    uint8_t *scratch = static_cast<uint8_t *>(g_noalloc_scratch_addr[dev]);
+
+    // widest tile that still gives every SM a unit, else the narrowest
+    int block_n = 64;
+    for (int bn : kBlockNs) {
+        if (tiling_for(p, bn, split_k).units >= kNumSMs) block_n = bn;
+    }
+
+    CUtensorMap ta, tb;
+    const int a_box_rows = p.M >= kBlockM ? kBlockM : (int)round_up(p.M, 8);
+    st = encode_operand_map(&ta, A, p.K, p.M, 1, lda, 0, kBlockK, a_box_rows);
+    if (st != CUDALLM_OK) return st;
+    st = encode_operand_map(&tb, B, p.N, p.K, 1, ldb, 0, 64, kBlockK);
+    if (st != CUDALLM_OK) return st;
+
+    const Tiling t = tiling_for(p, block_n, split_k);
+    GemmParams gp{};
+    gp.C = p.C;
+    gp.ldc = p.ldc;
+    gp.strideC = 0;
+    gp.M = (int)p.M; gp.N = (int)p.N; gp.K = (int)p.K; gp.batch = 1;
+    gp.tiles_m = (int)t.tiles_m; gp.tiles_n = (int)t.tiles_n;
+    gp.split_k = split_k;
+    gp.kblocks = (int)t.kblocks;
+    gp.num_units = (int)t.units;
+    gp.c_vec_ok = 0;                                    // unused: every unit writes partial sums
+    gp.a_box_bytes = a_box_rows * 128;
+    gp.partials = reinterpret_cast<float *>(scratch + 256);
+    gp.ldp = partial_ld(p);
+    gp.status = reinterpret_cast<int *>(scratch);
+
+    // the status word must start at zero; the partial sums are fully overwritten
+    CUDA_TRY(cudaMemsetAsync(scratch, 0, 256, stream));
+    const bool bf = p.out_dtype == CUDALLM_BF16;
+    switch (block_n) {
+    case 64:  st = bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
+                      : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream); break;
+    case 128: st = bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
+                      : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream); break;
+    default:  st = bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
+                      : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream); break;
+    }
+    if (st != CUDALLM_OK) return st;
+    const int64_t groups = p.M * cdiv(p.N, 4);
+    int64_t blocks = cdiv(groups, 256);
+    if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
+    const int64_t al = bf ? 8 : 16;
+    const int vec4 = (reinterpret_cast<uintptr_t>(p.C) % al == 0) && (p.ldc % 4 == 0);
+    if (bf)
+        splitk_reduce_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>(
+            gp.partials, p.C, gp.M, gp.N, 1, split_k, gp.ldp, p.ldc, 0, vec4);
+    else
+        splitk_reduce_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>(
+            gp.partials, p.C, gp.M, gp.N, 1, split_k, gp.ldp, p.ldc, 0, vec4);
+    CUDA_TRY(cudaGetLastError());
+    int host_status[2] = {0, 0};
+    CUDA_TRY(cudaMemcpyAsync(host_status, scratch, sizeof host_status, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    return host_status[0] == 0 ? CUDALLM_OK : CUDALLM_ERR_DEVICE_TIMEOUT;
+}
+
 int cudallm_num_variants(void)
 {
     return kNumVariants;
@@ -687,6 +784,7 @@ const char *cudallm_strerror(int status)
     case CUDALLM_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
     case CUDALLM_ERR_WORKSPACE: return "workspace missing, too small or misaligned";
     case CUDALLM_ERR_MISALIGNED: return "pointer not aligned to its element size";
+    case CUDALLM_ERR_TOO_LARGE: return "problem exceeds the fixed-size built-in scratch of this entry point";
     default: return "unknown status";
     }
 }
