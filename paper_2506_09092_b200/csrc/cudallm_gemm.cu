@@ -13,6 +13,7 @@
 
 #include "aux_kernels.cuh"
 #include "umma_gemm.cuh"
+#include "umma_gemm_2cta.cuh"
 
 using namespace cudallm;
 
@@ -75,7 +76,7 @@ int validate(const Problem &p)
 inline bool is_empty(const Problem &p) { return p.M == 0 || p.N == 0 || p.batch == 0; }
 
 // ---------------------------------------------------------------- variants --
-enum Family { kSimt = 0, kUmma = 1 };
+enum Family { kSimt = 0, kUmma = 1, kUmmaPair = 2 };
 struct Variant {
     char name[32];
     Family family;
@@ -84,7 +85,7 @@ struct Variant {
 };
 constexpr int kBlockNs[3] = {64, 128, 256};
 constexpr int kSplits[5] = {1, 2, 4, 8, 16};
-constexpr int kNumVariants = 1 + 3 * 5;
+constexpr int kNumVariants = 1 + 3 * 5 + 5;
 Variant g_variants[kNumVariants];
 std::once_flag g_variants_once;
 
@@ -105,6 +106,15 @@ void build_variants()
                 g_variants[v].split_k = sk;
                 ++v;
             }
+        // CTA pairs (cta_group::2), 256 x 256 tile per pair
+        for (int sk : kSplits) {
+            if (sk == 1) snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma2_n256");
+            else snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma2_n256_sk%d", sk);
+            g_variants[v].family = kUmmaPair;
+            g_variants[v].block_n = 256;
+            g_variants[v].split_k = sk;
+            ++v;
+        }
     });
 }
 
@@ -117,10 +127,10 @@ inline int64_t round_up(int64_t a, int64_t b) { return cdiv(a, b) * b; }
 struct Tiling {
     int64_t tiles_m, tiles_n, tiles, kblocks, units;
 };
-Tiling tiling_for(const Problem &p, int block_n, int split_k)
+Tiling tiling_for(const Problem &p, int block_n, int split_k, int block_m = kBlockM)
 {
     Tiling t;
-    t.tiles_m = cdiv(p.M, kBlockM);
+    t.tiles_m = cdiv(p.M, block_m);
     t.tiles_n = cdiv(p.N, block_n);
     t.tiles = t.tiles_m * t.tiles_n * p.batch;
     t.kblocks = cdiv(p.K, kBlockK);
@@ -140,7 +150,7 @@ bool variant_supports(const Variant &v, const Problem &p)
     if (is_empty(p)) return true;
     if (v.family == kSimt) return true;
     if (p.K == 0) return false;                       // the zero-fill case runs on the simt kernel
-    const Tiling t = tiling_for(p, v.block_n, v.split_k);
+    const Tiling t = tiling_for(p, v.block_n, v.split_k, v.family == kUmmaPair ? kPairM : kBlockM);
     if (t.units > kMaxDim) return false;
     if (v.split_k > 1) {
         if (v.split_k > t.kblocks) return false;
@@ -148,6 +158,8 @@ bool variant_supports(const Variant &v, const Problem &p)
     }
     return true;
 }
+
+constexpr double kPairClocksPerKBlock = 540.0;       // 256 x 256 x 64 on a CTA pair
 
 // Cost model (SM clocks) behind the automatic choice.
 //  main kernel: the larger of a compute estimate -- waves x k-blocks per unit x
@@ -158,16 +170,18 @@ bool variant_supports(const Variant &v, const Problem &p)
 //  split-K adds the reduction kernel: partial sums read, C written, a launch.
 double variant_cost(const Variant &v, const Problem &p)
 {
-    const Tiling t = tiling_for(p, v.block_n, v.split_k);
-    const double waves = (double)cdiv(t.units, kNumSMs);
+    const bool pair = v.family == kUmmaPair;
+    const Tiling t = tiling_for(p, v.block_n, v.split_k, pair ? kPairM : kBlockM);
+    const int slots = pair ? kNumSMs / 2 : kNumSMs;    // units that run at once
+    const double waves = (double)cdiv(t.units, slots);
     const double kb_per_unit = (double)cdiv(t.kblocks, v.split_k);
     const double rows = p.M < kBlockM ? (double)p.M : (double)kBlockM;
     const double out_b = (p.out_dtype == CUDALLM_F32) ? 4.0 : 2.0;
     const double epi = rows * v.block_n * (v.split_k > 1 ? 4.0 : out_b) / 32.0 + 1500.0;
-    const double mainloop = kb_per_unit * (300.0 + 0.83 * v.block_n);
+    const double mainloop = kb_per_unit * (pair ? kPairClocksPerKBlock : 300.0 + 0.83 * v.block_n);
     const double compute = waves * (mainloop > epi ? mainloop : epi) + epi;
     const double hbm = 3500.0;                         // bytes per clock: ~6.5 TB/s at ~1.9 GHz
-    const double active = t.units < kNumSMs ? (double)t.units : (double)kNumSMs;
+    const double active = (pair ? 2.0 : 1.0) * (t.units < slots ? (double)t.units : (double)slots);
     const double bw = active * 40.0 < hbm ? active * 40.0 : hbm;
     const double ab_bytes = (double)p.batch * (2.0 * p.M * p.K + 2.0 * p.K * p.N);
     const double c_bytes = (double)p.batch * out_b * p.M * p.N;
@@ -207,6 +221,7 @@ struct DeviceState {
     void *ws_internal = nullptr; // owned allocation (kept when an external one is set)
     size_t ws_internal_bytes = 0;
     bool smem_attr_set[16] = {};
+    int max_pairs = 0;           // co-resident 2-CTA clusters of the pair kernel (0 = not asked yet)
 };
 DeviceState g_dev[kMaxDevices];
 std::mutex g_mutex;
@@ -294,7 +309,7 @@ Plan make_plan(const Variant &v, const Problem &p, bool pack_a, bool pack_b)
     pl.pack_b = pack_b;
     size_t off = kHeaderBytes;
     pl.off_partials = off;
-    if (v.family == kUmma && v.split_k > 1) off += (size_t)partial_bytes(p, v.split_k);
+    if (v.family != kSimt && v.split_k > 1) off += (size_t)partial_bytes(p, v.split_k);
     off = (size_t)round_up((int64_t)off, 256);
     pl.off_pack_a = off;
     pl.ldap = round_up(p.K, 8);
@@ -348,6 +363,43 @@ int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb,
     }
     int grid = gp.num_units < d.sm_count ? gp.num_units : d.sm_count;
     kernel<<<grid, kNumThreads, L::kDynamicBytes, stream>>>(ta, tb, gp);
+    CUDA_TRY(cudaGetLastError());
+    return CUDALLM_OK;
+}
+
+template <int STAGES, bool OUT_BF16>
+int launch_umma_pair(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &gp,
+                     cudaStream_t stream)
+{
+    using L = PairSmemLayout<STAGES>;
+    static_assert(L::kDynamicBytes <= 232448, "shared memory budget");
+    static_assert(L::kDynamicBytes > 120 * 1024, "one CTA per SM");
+    auto kernel = umma_gemm_2cta_kernel<STAGES, OUT_BF16>;
+    DeviceState &d = g_dev[dev];
+    if (!d.smem_attr_set[slot]) {
+        CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      L::kDynamicBytes));
+        d.smem_attr_set[slot] = true;
+    }
+    if (d.max_pairs == 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * (d.sm_count / 2));
+        cfg.blockDim = dim3(kNumThreads);
+        cfg.dynamicSmemBytes = L::kDynamicBytes;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, kernel, &cfg));
+        d.max_pairs = n > 0 ? n : 1;
+        if (d.max_pairs > d.sm_count / 2) d.max_pairs = d.sm_count / 2;
+    }
+    const int pairs = gp.num_units < d.max_pairs ? gp.num_units : d.max_pairs;
+    kernel<<<2 * pairs, kNumThreads, L::kDynamicBytes, stream>>>(ta, tb, gp);
     CUDA_TRY(cudaGetLastError());
     return CUDALLM_OK;
 }
@@ -408,14 +460,15 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
 
     CUtensorMap ta, tb;
     // Rows of A beyond M only feed rows of C that are never stored, so the box
-    // need not cover (and zero-fill) them.
-    const int a_box_rows = p.M >= kBlockM ? kBlockM : (int)round_up(p.M, 8);
+    // need not cover (and zero-fill) them.  (CTA pairs always use full boxes.)
+    const bool pair = v.family == kUmmaPair;
+    const int a_box_rows = (p.M >= kBlockM || pair) ? kBlockM : (int)round_up(p.M, 8);
     st = encode_operand_map(&ta, A, p.K, p.M, p.batch, lda, sA, kBlockK, a_box_rows);
     if (st != CUDALLM_OK) return st;
     st = encode_operand_map(&tb, B, p.N, p.K, p.batch, ldb, sB, 64, kBlockK);
     if (st != CUDALLM_OK) return st;
 
-    const Tiling t = tiling_for(p, v.block_n, v.split_k);
+    const Tiling t = tiling_for(p, v.block_n, v.split_k, pair ? kPairM : kBlockM);
     GemmParams gp{};
     gp.C = p.C;
     gp.ldc = p.ldc;
@@ -434,13 +487,18 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     gp.status = reinterpret_cast<int *>(ws);
 
     const bool bf = p.out_dtype == CUDALLM_BF16;
-    switch (v.block_n) {
-    case 64:  st = bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
-                      : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream); break;
-    case 128: st = bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
-                      : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream); break;
-    default:  st = bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
-                      : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream); break;
+    if (pair) {
+        st = bf ? launch_umma_pair<6, true>(dev, 6, ta, tb, gp, stream)
+                : launch_umma_pair<6, false>(dev, 7, ta, tb, gp, stream);
+    } else {
+        switch (v.block_n) {
+        case 64:  st = bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
+                          : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream); break;
+        case 128: st = bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
+                          : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream); break;
+        default:  st = bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
+                          : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream); break;
+        }
     }
     if (st != CUDALLM_OK || v.split_k == 1) return st;
 
@@ -481,7 +539,7 @@ int run(int variant, const Problem &p, void *stream_v)
     st = probe_device(dev);
     if (st != CUDALLM_OK) return st;
     if (v.family == kSimt) return launch_simt(p, stream);
-    return run_umma(dev, v, p, stream);
+    return run_umma(dev, v, p, stream);       // both tcgen05 families
 }
 
 Problem make_problem(const void *A, const void *B, void *C, int64_t M, int64_t N, int64_t K, int64_t lda,

@@ -124,6 +124,45 @@ __device__ __forceinline__ void store_row_chunk(void *row_ptr, const float (&v)[
     }
 }
 
+// Epilogue of one unit for one thread: `row` is this thread's row of C, `t_addr`
+// the TMEM address of its lane at the accumulator's first column.  Reads the
+// BLOCK_N accumulator columns 32 at a time and stores them to C (split_k == 1)
+// or to this split's slice of the partial sums.  Must be called by whole warps.
+template <int BLOCK_N, bool OUT_BF16>
+__device__ __forceinline__ void epilogue_tile(const GemmParams &p, const UnitCoord &c, int row,
+                                              uint32_t t_addr)
+{
+    const bool row_ok = row < p.M;
+    void *row_ptr;
+    bool vec_ok;
+    if (p.split_k == 1) {
+        const long long off = static_cast<long long>(c.b) * p.strideC
+                            + static_cast<long long>(row) * p.ldc;
+        row_ptr = OUT_BF16 ? static_cast<void *>(reinterpret_cast<__nv_bfloat16 *>(p.C) + off)
+                           : static_cast<void *>(reinterpret_cast<float *>(p.C) + off);
+        vec_ok = p.c_vec_ok != 0;
+    } else {
+        row_ptr = p.partials
+                + ((static_cast<long long>(c.split) * p.batch + c.b) * p.M + row) * p.ldp;
+        vec_ok = true;
+    }
+#pragma unroll 1
+    for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(t_addr + ch * 32, r);
+        tmem_ld_wait();
+        if (row_ok) {
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+            const int col0 = c.n_tile * BLOCK_N + ch * 32;
+            if (p.split_k == 1) store_row_chunk<OUT_BF16>(row_ptr, v, col0, p.N, vec_ok);
+            else                store_row_chunk<false>(row_ptr, v, col0, p.N, vec_ok);
+        }
+        __syncwarp();                                    // tcgen05.ld needs the whole warp
+    }
+}
+
 template <int BLOCK_N, int STAGES, bool OUT_BF16>
 __global__ void __launch_bounds__(kNumThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
@@ -256,38 +295,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 break;
             }
             tc_fence_after();
-            const int row = c.m_tile * kBlockM + epi_tid;
-            const bool row_ok = row < p.M;
-            const uint32_t t_addr = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(quad * 32) << 16);
-            // destination row: C itself, or this split's slice of the partial sums
-            void *row_ptr;
-            bool vec_ok;
-            if (p.split_k == 1) {
-                const long long off = static_cast<long long>(c.b) * p.strideC
-                                    + static_cast<long long>(row) * p.ldc;
-                row_ptr = OUT_BF16 ? static_cast<void *>(reinterpret_cast<__nv_bfloat16 *>(p.C) + off)
-                                   : static_cast<void *>(reinterpret_cast<float *>(p.C) + off);
-                vec_ok = p.c_vec_ok != 0;
-            } else {
-                row_ptr = p.partials
-                        + ((static_cast<long long>(c.split) * p.batch + c.b) * p.M + row) * p.ldp;
-                vec_ok = true;
-            }
-#pragma unroll 1
-            for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
-                uint32_t r[32];
-                tmem_ld_32x32b_x32(t_addr + ch * 32, r);
-                tmem_ld_wait();
-                if (row_ok) {
-                    float v[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-                    const int col0 = c.n_tile * BLOCK_N + ch * 32;
-                    if (p.split_k == 1) store_row_chunk<OUT_BF16>(row_ptr, v, col0, p.N, vec_ok);
-                    else                store_row_chunk<false>(row_ptr, v, col0, p.N, vec_ok);
-                }
-                __syncwarp();                            // tcgen05.ld needs the whole warp
-            }
+            epilogue_tile<BLOCK_N, OUT_BF16>(p, c, c.m_tile * kBlockM + epi_tid,
+                                             tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(quad * 32) << 16));
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));

@@ -1,0 +1,238 @@
+// tcgen05 GEMM with CTA pairs (cta_group::2): a cluster of two CTAs on two SMs
+// owns one 256 x 256 tile of C.
+//
+//   C[i][j] = sum_k A[i][k] * B[k][j]      (Task 2: matrix multiplication)
+//
+// CTA r of the pair stages rows [128 r, 128 r + 128) of the tile's A panel and
+// columns [128 r, 128 r + 128) of its B panel (32 KB per 64-deep k-block per
+// CTA instead of 48 KB for a lone 128 x 256 tile, so six stages fit and the
+// bytes that each SM must pull per MMA clock drop by a third).  The leader CTA
+// (rank 0) issues one 256 x 256 x 16 MMA for both; each CTA's tensor core
+// reads its own A rows and both halves of B, and accumulates its 128 rows x
+// 256 columns in its own tensor memory.
+//
+// Synchronisation (no multicast anywhere):
+//  * full[s]  lives in the leader.  Both producers' TMA loads complete their
+//    bytes on it (the peer's through the cluster address of that barrier).
+//  * empty[s] lives in each CTA; the leader commits the stage's MMAs to its
+//    own and to the peer's barrier (two commits).
+//  * tmem_full[a] likewise: one commit per CTA.
+//  * tmem_empty[a] lives in the leader and counts the 8 epilogue warps of both
+//    CTAs (the peer's arrive through the cluster address).
+#pragma once
+#include "umma_gemm.cuh"
+
+namespace cudallm {
+
+constexpr int kPairM = 256;
+constexpr int kPairN = 256;
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;"
+                 ::: "memory");
+}
+// address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// TMA load issued by either CTA of a pair; `bar` is a cluster address (the
+// leader's barrier), `dst` this CTA's own shared memory.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *tm, uint32_t bar,
+                                                 int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar_cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];"
+                 ::"r"(bar_cluster_addr) : "memory");
+}
+
+template <int STAGES>
+struct PairSmemLayout {
+    static constexpr int kABytes = kBlockM * kBlockK * 2;            // 128 rows of A
+    static constexpr int kBBytes = kBlockK * (kPairN / 2) * 2;       // 128 columns of B
+    static constexpr int kStageBytes = kABytes + kBBytes;            // 32 KB
+    static constexpr int kBarOffset = STAGES * kStageBytes;
+    static constexpr int kNumBars = 2 * STAGES + 4;
+    static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
+    static constexpr int kBytes = kMiscOffset + 64;
+    static constexpr int kDynamicBytes = kBytes + 1024;
+};
+
+template <int STAGES, bool OUT_BF16>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
+umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                      const __grid_constant__ CUtensorMap tmap_b, const GemmParams p)
+{
+    using L = PairSmemLayout<STAGES>;
+    constexpr uint32_t kTmemCols = 2 * kPairN;                       // 512: two accumulators
+    constexpr uint32_t kIdesc = make_idesc_bf16(kPairM, kPairN, 0, 1);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_base + L::kBarOffset;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L::kMiscOffset);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kMiscOffset + 4);
+
+    const int warp_idx = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                         // 0 = leader
+    const int pair = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);       // leader's is used: one expect_tx arrival + bytes
+            mbar_init(empty_bar(s), 1);      // one commit from the leader
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);      // one commit from the leader
+            mbar_init(tempty_bar(a), 8);     // leader's is used: 4 epilogue warps x 2 CTAs
+        }
+        fence_mbar_init();
+        fence_proxy_async_smem();
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+    }
+    if (warp_idx == 1) {
+        tmem_alloc_2cta(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+        tmem_relinquish_2cta();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();              // both CTAs' barriers exist before anyone signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp_idx == 0) {
+        // ------------------------------------------------ TMA producer ----
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int u = pair; ok && u < p.num_units; u += num_pairs) {
+                const UnitCoord c = decode_unit(p, u);
+                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                    if (!mbar_wait<true>(empty_bar(stage), phase ^ 1, abort_flag)) {
+                        report_timeout(p.status, kRoleProducer, stage);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t sa = smem_base + stage * L::kStageBytes;
+                    const uint32_t sb = sa + L::kABytes;
+                    const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * L::kStageBytes);
+                    tma_load_3d_pair(sa, &tmap_a, leader_full, kb * kBlockK,
+                                     c.m_tile * kPairM + static_cast<int>(rank) * kBlockM, c.b);
+#pragma unroll
+                    for (int j = 0; j < 2; ++j)
+                        tma_load_3d_pair(sb + j * (64 * kBlockK * 2), &tmap_b, leader_full,
+                                         c.n_tile * kPairN + static_cast<int>(rank) * 128 + j * 64,
+                                         kb * kBlockK, c.b);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp_idx == 1) {
+        // ------------------------------------- MMA issuer (leader only) ----
+        if (lane == 0 && rank == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int u = pair; ok && u < p.num_units; u += num_pairs) {
+                const UnitCoord c = decode_unit(p, u);
+                if (!mbar_wait<true>(tempty_bar(acc), acc_phase ^ 1, abort_flag)) {
+                    report_timeout(p.status, kRoleMma, 0x40 + acc);
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kPairN;
+                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                    if (!mbar_wait<true>(full_bar(stage), phase, abort_flag)) {
+                        report_timeout(p.status, kRoleMma, stage);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = smem_base + stage * L::kStageBytes;
+                    const uint32_t sb = sa + L::kABytes;
+#pragma unroll
+                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                        const uint64_t da = make_smem_desc_sw128(sa + k * 32, 16, 1024);
+                        const uint64_t db = make_smem_desc_sw128(sb + k * 2048, 8192, 1024);
+                        umma_bf16_2cta(d_tmem, da, db, kIdesc, (kb > c.kb_begin || k > 0) ? 1u : 0u);
+                    }
+                    umma_commit_pair(map_to_cta(empty_bar(stage), 0));
+                    umma_commit_pair(map_to_cta(empty_bar(stage), 1));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                umma_commit_pair(map_to_cta(tfull_bar(acc), 0));
+                umma_commit_pair(map_to_cta(tfull_bar(acc), 1));
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ---------------------------------------------------- epilogue ----
+        const int quad = warp_idx & 3;
+        const int epi_tid = quad * 32 + lane;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int u = pair; u < p.num_units; u += num_pairs) {
+            const UnitCoord c = decode_unit(p, u);
+            bool ok = mbar_wait<true>(tfull_bar(acc), acc_phase, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0x80 + acc);
+                break;
+            }
+            tc_fence_after();
+            epilogue_tile<kPairN, OUT_BF16>(p, c, c.m_tile * kPairM + static_cast<int>(rank) * kBlockM + epi_tid,
+                                            tmem_base + acc * kPairN + (static_cast<uint32_t>(quad * 32) << 16));
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(map_to_cta(tempty_bar(acc), 0));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();              // nobody leaves while the peer may still signal or read it
+    if (warp_idx == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc_2cta(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace cudallm
