@@ -38,6 +38,10 @@
  *    fallback.
  *  - Calls that need the workspace (repacking, split-K) share one workspace
  *    per device; such calls must not run concurrently on different streams.
+ *  - Split-K variants make some CTAs wait (with a time limit) for partial
+ *    results of other CTAs of the same launch; they assume that the launch has
+ *    the GPU to itself.  If another kernel holds SMs for seconds, such a wait
+ *    can run out and is reported as CUDALLM_ERR_DEVICE_TIMEOUT.
  */
 #ifndef CUDALLM_GEMM_H
 #define CUDALLM_GEMM_H
@@ -141,27 +145,31 @@ size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K,
  *
  * Its scratch is an array compiled into the library's device image
  * (CUDALLM_NOALLOC_SCRATCH_BYTES, 8 MiB, resident on every GPU that loads the
- * library until the process exits).  The product is split along K into
- * `split_k` parts (2, 4, 8 or 16, at most ceil(K/64)); the fp32 partial sums
- * go to that array and a second kernel adds them in fixed order and writes C.
+ * library until the process exits).  C is cut into tiles of 128 x 64 and each
+ * tile's K range into `split_k` parts (2, 4, 8 or 16, at most ceil(K/64));
+ * split_k - 1 of them leave an fp32 partial tile of 32 KiB in that array and
+ * the last one adds them in fixed order and writes C.
  *
  *  - A, B, C, sizes, leading dimensions and out_dtype as cudallm_gemm_bf16.
  *    A and B must take the direct TMA path: 16-byte aligned bases, lda and ldb
  *    multiples of 8 (else CUDALLM_ERR_UNSUPPORTED_SHAPE; repacking would need
  *    more scratch).
- *  - Limit: 256 + split_k * M * round_up(N, 4) * 4 bytes must not exceed
- *    CUDALLM_NOALLOC_SCRATCH_BYTES, else CUDALLM_ERR_TOO_LARGE and nothing runs.
+ *  - Limit: P = ceil(M/128) * ceil(N/64) * (split_k - 1) partial tiles; the
+ *    call needs P <= 4080 and CUDALLM_NOALLOC_HEADER_BYTES + P * 32 KiB <=
+ *    CUDALLM_NOALLOC_SCRATCH_BYTES (P <= 253), else it returns
+ *    CUDALLM_ERR_TOO_LARGE and nothing runs.
  *  - The call SYNCHRONISES `stream` before it returns and reports a kernel
  *    whose bounded wait ran out as CUDALLM_ERR_DEVICE_TIMEOUT.
  *  - The first call on each device looks up the array's device address (and,
  *    like any first launch, lets the driver load the kernels).  Make that
  *    first call outside any stream capture.
  *  - All calls on a device share the one array, which keeps whatever the last
- *    call left in it; the call clears the words that must start at zero.  Two
- *    calls that overlap on the GPU (different streams, or different host
- *    threads) race on it: serialise them.
+ *    call left in it; each call clears the words that must start at zero (the
+ *    status word and the helper flags).  Two calls that overlap on the GPU
+ *    (different streams, or different host threads) race on it: serialise them.
  */
 #define CUDALLM_NOALLOC_SCRATCH_BYTES (8u << 20)
+#define CUDALLM_NOALLOC_HEADER_BYTES  (64u << 10)   /* status word + helper flags */
 int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C,
                                      int64_t M, int64_t N, int64_t K,
                                      int64_t lda, int64_t ldb, int64_t ldc,
@@ -184,7 +192,7 @@ int cudallm_select_variant(int64_t M, int64_t N, int64_t K,
 
 /*
  * Workspace.  Upper bound of the scratch bytes any variant may need for the
- * problem (repacked operands, split-K partial tiles, tile counters).  Without
+ * problem (repacked operands, split-K partial tiles and their flags).  Without
  * cudallm_set_workspace the library allocates (and grows) one workspace per
  * device with cudaMalloc on demand.  A caller-provided workspace must be
  * 256-byte aligned, zero-filled once before first use, and stay valid until

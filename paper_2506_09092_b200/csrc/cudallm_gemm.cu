@@ -77,17 +77,25 @@ inline bool is_empty(const Problem &p) { return p.M == 0 || p.N == 0 || p.batch 
 
 // ---------------------------------------------------------------- variants --
 enum Family { kSimt = 0, kUmma = 1, kUmmaPair = 2 };
+constexpr int kTailSplit = 0;          // Variant::split_k value: cut the ragged last wave's tiles along N
 struct Variant {
     char name[32];
     Family family;
     int block_n;
-    int split_k;
+    int split_k;                       // 1 = none, 2..16 = every tile along K, kTailSplit = see above
 };
 constexpr int kBlockNs[3] = {64, 128, 256};
-constexpr int kSplits[5] = {1, 2, 4, 8, 16};
-constexpr int kNumVariants = 1 + 3 * 5 + 5;
+constexpr int kSplits[6] = {1, 2, 4, 8, 16, kTailSplit};
+constexpr int kNumVariants = 1 + 3 * 6 + 6;
 Variant g_variants[kNumVariants];
 std::once_flag g_variants_once;
+
+void name_variant(Variant &v, const char *stem, int bn, int sk)
+{
+    if (sk == 1) snprintf(v.name, sizeof v.name, "%s_n%d", stem, bn);
+    else if (sk == kTailSplit) snprintf(v.name, sizeof v.name, "%s_n%d_ts", stem, bn);
+    else snprintf(v.name, sizeof v.name, "%s_n%d_sk%d", stem, bn, sk);
+}
 
 void build_variants()
 {
@@ -99,8 +107,7 @@ void build_variants()
         int v = 1;
         for (int bn : kBlockNs)
             for (int sk : kSplits) {
-                if (sk == 1) snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma_n%d", bn);
-                else snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma_n%d_sk%d", bn, sk);
+                name_variant(g_variants[v], "umma", bn, sk);
                 g_variants[v].family = kUmma;
                 g_variants[v].block_n = bn;
                 g_variants[v].split_k = sk;
@@ -108,8 +115,7 @@ void build_variants()
             }
         // CTA pairs (cta_group::2), 256 x 256 tile per pair
         for (int sk : kSplits) {
-            if (sk == 1) snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma2_n256");
-            else snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma2_n256_sk%d", sk);
+            name_variant(g_variants[v], "umma2", 256, sk);
             g_variants[v].family = kUmmaPair;
             g_variants[v].block_n = 256;
             g_variants[v].split_k = sk;
@@ -120,76 +126,116 @@ void build_variants()
 
 constexpr int kNumSMs = 148;
 constexpr int64_t kMaxPartialBytes = int64_t(1) << 30;   // split-K scratch a variant may ask for
+constexpr int64_t kMaxHelperTiles = 65536;               // helper partial tiles per launch (4 flags each)
 
 inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int64_t round_up(int64_t a, int64_t b) { return cdiv(a, b) * b; }
 
+// How a variant cuts a problem into units.
 struct Tiling {
-    int64_t tiles_m, tiles_n, tiles, kblocks, units;
+    int64_t tiles_m, tiles_n, tiles, kblocks;
+    int64_t dp_tiles;        // leading tiles that are one unit each
+    int split;               // K parts per remaining tile
+    int nsplit;              // N parts per remaining tile (never together with split > 1)
+    int64_t units;           // dp_tiles + (tiles - dp_tiles) * split * nsplit
+    int64_t helper_tiles;    // partial tiles in the workspace: (tiles - dp_tiles) * (split - 1) * CTAs per tile
+    int64_t partial_bytes;
 };
-Tiling tiling_for(const Problem &p, int block_n, int split_k, int block_m = kBlockM)
+
+// `slots` = units that run at once (CTAs, or CTA pairs, of the persistent grid).
+Tiling tiling_for(const Variant &v, const Problem &p, int slots)
 {
-    Tiling t;
-    t.tiles_m = cdiv(p.M, block_m);
-    t.tiles_n = cdiv(p.N, block_n);
+    const bool pair = v.family == kUmmaPair;
+    Tiling t{};
+    if (v.family == kSimt) return t;                  // no tiles, no scratch
+    t.tiles_m = cdiv(p.M, pair ? kPairM : kBlockM);
+    t.tiles_n = cdiv(p.N, v.block_n);
     t.tiles = t.tiles_m * t.tiles_n * p.batch;
     t.kblocks = cdiv(p.K, kBlockK);
-    t.units = t.tiles * split_k;
+    t.split = 1;
+    t.nsplit = 1;
+    t.dp_tiles = t.tiles;
+    if (v.split_k == kTailSplit) {
+        // Cut the tiles of the ragged last wave into narrower ones (64-column
+        // granularity per CTA) so that they fill the grid about once.
+        const int64_t tail = t.tiles % slots;
+        const int max_parts = pair ? 2 : v.block_n / 64;
+        int parts = 1;
+        while (tail > 0 && parts * 2 <= max_parts && tail * parts * 2 <= slots) parts *= 2;
+        if (parts > 1) {
+            t.nsplit = parts;
+            t.dp_tiles = t.tiles - tail;
+        }
+    } else if (v.split_k > 1) {
+        t.split = v.split_k;
+        t.dp_tiles = 0;
+    }
+    t.units = t.dp_tiles + (t.tiles - t.dp_tiles) * t.split * t.nsplit;
+    t.helper_tiles = (t.tiles - t.dp_tiles) * (t.split - 1) * (pair ? 2 : 1);
+    t.partial_bytes = t.helper_tiles * int64_t(kBlockM) * v.block_n * 4;
     return t;
 }
-
-// fp32 partial sums of a split-K run: [split][batch][M][ldp], ldp = N rounded up to 4
-inline int64_t partial_ld(const Problem &p) { return round_up(p.N, 4); }
-inline int64_t partial_bytes(const Problem &p, int split_k)
-{
-    return int64_t(split_k) * p.batch * p.M * partial_ld(p) * 4;
-}
+inline int default_slots(const Variant &v) { return v.family == kUmmaPair ? kNumSMs / 2 : kNumSMs; }
 
 bool variant_supports(const Variant &v, const Problem &p)
 {
     if (is_empty(p)) return true;
     if (v.family == kSimt) return true;
     if (p.K == 0) return false;                       // the zero-fill case runs on the simt kernel
-    const Tiling t = tiling_for(p, v.block_n, v.split_k, v.family == kUmmaPair ? kPairM : kBlockM);
+    const Tiling t = tiling_for(v, p, default_slots(v));
     if (t.units > kMaxDim) return false;
-    if (v.split_k > 1) {
-        if (v.split_k > t.kblocks) return false;
-        if (partial_bytes(p, v.split_k) > kMaxPartialBytes) return false;
-    }
+    if (v.split_k > 1 && v.split_k > t.kblocks) return false;
+    // bounds that must hold for any grid size the device may give
+    // (tail-split variants have at most one grid's worth of helper tiles)
+    if (v.split_k > 1 && (t.helper_tiles > kMaxHelperTiles || t.partial_bytes > kMaxPartialBytes))
+        return false;
     return true;
 }
 
-constexpr double kPairClocksPerKBlock = 540.0;       // 256 x 256 x 64 on a CTA pair
+constexpr double kPairClocksPerKBlock = 455.0;       // 256 x 256 x 64 on a CTA pair (measured: 0.89 x a lone CTA's 128 x 256 x 64)
 
-// Cost model (SM clocks) behind the automatic choice.
-//  main kernel: the larger of a compute estimate -- waves x k-blocks per unit x
-//      clocks per k-block (measured on 4096^3: about 300 + 0.83 * BLOCK_N),
-//      plus one exposed epilogue -- and a memory estimate: A and B read once
-//      and C (or the split-K partial sums) written once, over the bandwidth
-//      the active SMs can draw (about 40 B/clock each), capped by HBM.
-//  split-K adds the reduction kernel: partial sums read, C written, a launch.
+// Cost model (SM clocks) behind the automatic choice: the larger of
+//  compute: rounds of units x k-blocks per unit x clocks per k-block (measured
+//      on 4096^3: about 300 + 0.83 * BLOCK_N for a lone CTA, 540 for a pair),
+//      plus one exposed epilogue; a split tile's owner also reads its helpers'
+//      partial tiles from L2;
+//  memory: A and B read once, C written once (partial tiles stay in L2), over
+//      the bandwidth the active SMs can draw (about 40 B/clock each), capped
+//      by HBM.
 double variant_cost(const Variant &v, const Problem &p)
 {
     const bool pair = v.family == kUmmaPair;
-    const Tiling t = tiling_for(p, v.block_n, v.split_k, pair ? kPairM : kBlockM);
-    const int slots = pair ? kNumSMs / 2 : kNumSMs;    // units that run at once
-    const double waves = (double)cdiv(t.units, slots);
-    const double kb_per_unit = (double)cdiv(t.kblocks, v.split_k);
+    const int slots = default_slots(v);
+    const Tiling t = tiling_for(v, p, slots);
+    const double per_kb = pair ? kPairClocksPerKBlock : 300.0 + 0.83 * v.block_n;
     const double rows = p.M < kBlockM ? (double)p.M : (double)kBlockM;
     const double out_b = (p.out_dtype == CUDALLM_F32) ? 4.0 : 2.0;
-    const double epi = rows * v.block_n * (v.split_k > 1 ? 4.0 : out_b) / 32.0 + 1500.0;
-    const double mainloop = kb_per_unit * (pair ? kPairClocksPerKBlock : 300.0 + 0.83 * v.block_n);
-    const double compute = waves * (mainloop > epi ? mainloop : epi) + epi;
+    const double epi = rows * v.block_n * out_b / 32.0 + 1500.0;
+    const double full_main = (double)t.kblocks * per_kb;
+    const double dp_rounds = (double)cdiv(t.dp_tiles, slots);
+    double compute = dp_rounds * (full_main > epi ? full_main : epi);
+    if (t.nsplit > 1) {
+        // narrower tiles: fewer MMA clocks per k-block, same A traffic
+        const double rounds = (double)cdiv((t.tiles - t.dp_tiles) * t.nsplit, slots);
+        const int w = v.block_n / t.nsplit;
+        const double narrow = (double)t.kblocks * (pair ? 300.0 + 0.83 * w : 300.0 + 0.83 * w);
+        compute += rounds * narrow;
+    }
+    if (t.split > 1) {
+        const double split_units = (double)(t.tiles - t.dp_tiles) * t.split;
+        const double rounds = (double)cdiv((int64_t)split_units, slots);
+        const double part_main = (double)cdiv(t.kblocks, t.split) * per_kb;
+        // measured: an owner spends about 8 us (15000 clocks) per helper tile it adds
+        const double fix = (t.split - 1) * 15000.0;
+        compute += rounds * (part_main > epi + fix ? part_main : epi + fix) + fix;
+    }
+    compute += epi;
     const double hbm = 3500.0;                         // bytes per clock: ~6.5 TB/s at ~1.9 GHz
     const double active = (pair ? 2.0 : 1.0) * (t.units < slots ? (double)t.units : (double)slots);
     const double bw = active * 40.0 < hbm ? active * 40.0 : hbm;
-    const double ab_bytes = (double)p.batch * (2.0 * p.M * p.K + 2.0 * p.K * p.N);
-    const double c_bytes = (double)p.batch * out_b * p.M * p.N;
-    const double part_bytes = v.split_k > 1 ? (double)partial_bytes(p, v.split_k) : 0.0;
-    const double main_mem = (ab_bytes + (v.split_k > 1 ? part_bytes : c_bytes)) / bw;
-    double cost = (compute > main_mem ? compute : main_mem) + 4000.0;
-    if (v.split_k > 1) cost += (part_bytes + c_bytes) / hbm + 6000.0;
-    return cost;
+    const double bytes = (double)p.batch * (2.0 * p.M * p.K + 2.0 * p.K * p.N + out_b * p.M * p.N);
+    const double memory = bytes / bw;
+    return (compute > memory ? compute : memory) + 4000.0;
 }
 
 int select_variant(const Problem &p)
@@ -207,8 +253,9 @@ int select_variant(const Problem &p)
 }
 
 // --------------------------------------------------------------- workspace --
-// Layout: [status 256 B][split-K partials][packed A][packed B]
-constexpr size_t kHeaderBytes = 256;
+// Layout: [status 256 B][split-K flags][split-K partial tiles][packed A][packed B]
+constexpr size_t kFlagBytes = kMaxHelperTiles * 4 * sizeof(int);
+constexpr size_t kHeaderBytes = 256 + kFlagBytes;    // zeroed when a workspace is created
 constexpr int kMaxDevices = 64;
 
 struct DeviceState {
@@ -222,6 +269,7 @@ struct DeviceState {
     size_t ws_internal_bytes = 0;
     bool smem_attr_set[16] = {};
     int max_pairs = 0;           // co-resident 2-CTA clusters of the pair kernel (0 = not asked yet)
+    int epoch = 0;               // last split-K flag value used on this device
 };
 DeviceState g_dev[kMaxDevices];
 std::mutex g_mutex;
@@ -302,14 +350,14 @@ inline bool b_operand_aligned(const Problem &p)
         && (p.batch == 1 || p.sB % 8 == 0);
 }
 
-Plan make_plan(const Variant &v, const Problem &p, bool pack_a, bool pack_b)
+Plan make_plan(const Tiling &t, const Problem &p, bool pack_a, bool pack_b)
 {
     Plan pl{};
     pl.pack_a = pack_a;
     pl.pack_b = pack_b;
     size_t off = kHeaderBytes;
     pl.off_partials = off;
-    if (v.family != kSimt && v.split_k > 1) off += (size_t)partial_bytes(p, v.split_k);
+    off += (size_t)t.partial_bytes;
     off = (size_t)round_up((int64_t)off, 256);
     pl.off_pack_a = off;
     pl.ldap = round_up(p.K, 8);
@@ -367,14 +415,15 @@ int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb,
     return CUDALLM_OK;
 }
 
-template <int STAGES, bool OUT_BF16>
-int launch_umma_pair(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &gp,
-                     cudaStream_t stream)
+// Sets the pair kernel's shared-memory attribute and asks how many CTA pairs
+// the device can hold at once (the persistent grid of the pair kernels).
+template <int STAGES, int KSUB, bool OUT_BF16>
+int prepare_umma_pair(int dev, int slot)
 {
-    using L = PairSmemLayout<STAGES>;
+    using L = PairSmemLayout<STAGES, KSUB>;
     static_assert(L::kDynamicBytes <= 232448, "shared memory budget");
     static_assert(L::kDynamicBytes > 120 * 1024, "one CTA per SM");
-    auto kernel = umma_gemm_2cta_kernel<STAGES, OUT_BF16>;
+    auto kernel = umma_gemm_2cta_kernel<STAGES, KSUB, OUT_BF16>;
     DeviceState &d = g_dev[dev];
     if (!d.smem_attr_set[slot]) {
         CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -398,6 +447,16 @@ int launch_umma_pair(int dev, int slot, const CUtensorMap &ta, const CUtensorMap
         d.max_pairs = n > 0 ? n : 1;
         if (d.max_pairs > d.sm_count / 2) d.max_pairs = d.sm_count / 2;
     }
+    return CUDALLM_OK;
+}
+
+template <int STAGES, int KSUB, bool OUT_BF16>
+int launch_umma_pair(int dev, const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &gp,
+                     cudaStream_t stream)
+{
+    using L = PairSmemLayout<STAGES, KSUB>;
+    auto kernel = umma_gemm_2cta_kernel<STAGES, KSUB, OUT_BF16>;
+    DeviceState &d = g_dev[dev];
     const int pairs = gp.num_units < d.max_pairs ? gp.num_units : d.max_pairs;
     kernel<<<2 * pairs, kNumThreads, L::kDynamicBytes, stream>>>(ta, tb, gp);
     CUDA_TRY(cudaGetLastError());
@@ -435,14 +494,53 @@ int launch_pack(const void *src, void *dst, int64_t rows, int64_t cols, int64_t 
     return CUDALLM_OK;
 }
 
+// Fills the kernel parameters that depend only on the problem and the tiling.
+GemmParams make_params(const Problem &p, const Tiling &t, int a_box_rows)
+{
+    GemmParams gp{};
+    gp.C = p.C;
+    gp.ldc = p.ldc;
+    gp.strideC = p.batch > 1 ? p.sC : 0;
+    gp.M = (int)p.M; gp.N = (int)p.N; gp.K = (int)p.K; gp.batch = (int)p.batch;
+    gp.tiles_m = (int)t.tiles_m; gp.tiles_n = (int)t.tiles_n;
+    gp.kblocks = (int)t.kblocks;
+    gp.dp_tiles = (int)t.dp_tiles;
+    gp.split_k = t.split;
+    gp.tail_nsplit = t.nsplit;
+    gp.num_units = (int)t.units;
+    const int64_t vec = (p.out_dtype == CUDALLM_F32) ? 4 : 8;
+    gp.c_vec_ok = (reinterpret_cast<uintptr_t>(p.C) % 16 == 0) && (p.ldc % vec == 0)
+               && (p.batch == 1 || p.sC % vec == 0);
+    gp.a_box_bytes = a_box_rows * 128;
+    return gp;
+}
+
+int next_epoch(DeviceState &d)
+{
+    d.epoch = (d.epoch == 0x7fffffff) ? 1 : d.epoch + 1;
+    return d.epoch;
+}
+
 int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
 {
+    DeviceState &d = g_dev[dev];
+    const bool pair = v.family == kUmmaPair;
+    const bool bf = p.out_dtype == CUDALLM_BF16;
+    int st;
+    if (pair) {
+        st = bf ? prepare_umma_pair<3, 2, true>(dev, 6) : prepare_umma_pair<3, 2, false>(dev, 7);
+        if (st != CUDALLM_OK) return st;
+    }
+    const int slots = pair ? d.max_pairs : d.sm_count;
+    const Tiling t = tiling_for(v, p, slots);
+    if (t.helper_tiles > kMaxHelperTiles || t.partial_bytes > kMaxPartialBytes)
+        return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+
     const bool pack_a = !a_operand_aligned(p);
     const bool pack_b = !b_operand_aligned(p);
-    const Plan pl = make_plan(v, p, pack_a, pack_b);
-    int st = ensure_workspace(dev, pl.total, stream);
+    const Plan pl = make_plan(t, p, pack_a, pack_b);
+    st = ensure_workspace(dev, pl.total, stream);
     if (st != CUDALLM_OK) return st;
-    DeviceState &d = g_dev[dev];
     uint8_t *ws = static_cast<uint8_t *>(d.ws);
 
     const void *A = p.A, *B = p.B;
@@ -461,62 +559,29 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     CUtensorMap ta, tb;
     // Rows of A beyond M only feed rows of C that are never stored, so the box
     // need not cover (and zero-fill) them.  (CTA pairs always use full boxes.)
-    const bool pair = v.family == kUmmaPair;
     const int a_box_rows = (p.M >= kBlockM || pair) ? kBlockM : (int)round_up(p.M, 8);
     st = encode_operand_map(&ta, A, p.K, p.M, p.batch, lda, sA, kBlockK, a_box_rows);
     if (st != CUDALLM_OK) return st;
     st = encode_operand_map(&tb, B, p.N, p.K, p.batch, ldb, sB, 64, kBlockK);
     if (st != CUDALLM_OK) return st;
 
-    const Tiling t = tiling_for(p, v.block_n, v.split_k, pair ? kPairM : kBlockM);
-    GemmParams gp{};
-    gp.C = p.C;
-    gp.ldc = p.ldc;
-    gp.strideC = p.batch > 1 ? p.sC : 0;
-    gp.M = (int)p.M; gp.N = (int)p.N; gp.K = (int)p.K; gp.batch = (int)p.batch;
-    gp.tiles_m = (int)t.tiles_m; gp.tiles_n = (int)t.tiles_n;
-    gp.split_k = v.split_k;
-    gp.kblocks = (int)t.kblocks;
-    gp.num_units = (int)t.units;
-    const int64_t vec = (p.out_dtype == CUDALLM_F32) ? 4 : 8;
-    gp.c_vec_ok = (reinterpret_cast<uintptr_t>(p.C) % 16 == 0) && (p.ldc % vec == 0)
-               && (p.batch == 1 || p.sC % vec == 0);
-    gp.a_box_bytes = a_box_rows * 128;
+    GemmParams gp = make_params(p, t, a_box_rows);
+    gp.epoch = t.split > 1 ? next_epoch(d) : 0;
     gp.partials = reinterpret_cast<float *>(ws + pl.off_partials);
-    gp.ldp = partial_ld(p);
+    gp.flags = reinterpret_cast<int *>(ws + 256);
     gp.status = reinterpret_cast<int *>(ws);
 
-    const bool bf = p.out_dtype == CUDALLM_BF16;
-    if (pair) {
-        st = bf ? launch_umma_pair<6, true>(dev, 6, ta, tb, gp, stream)
-                : launch_umma_pair<6, false>(dev, 7, ta, tb, gp, stream);
-    } else {
-        switch (v.block_n) {
-        case 64:  st = bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
-                          : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream); break;
-        case 128: st = bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
-                          : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream); break;
-        default:  st = bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
-                          : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream); break;
-        }
+    if (pair)
+        return bf ? launch_umma_pair<3, 2, true>(dev, ta, tb, gp, stream)
+                  : launch_umma_pair<3, 2, false>(dev, ta, tb, gp, stream);
+    switch (v.block_n) {
+    case 64:  return bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
+                        : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream);
+    case 128: return bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
+                        : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream);
+    default:  return bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
+                        : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream);
     }
-    if (st != CUDALLM_OK || v.split_k == 1) return st;
-
-    // split-K: add the slices in fixed order and write C
-    const int64_t groups = p.batch * p.M * cdiv(p.N, 4);
-    int64_t blocks = cdiv(groups, 256);
-    if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
-    const int64_t al = bf ? 8 : 16;
-    const int vec4 = (reinterpret_cast<uintptr_t>(p.C) % al == 0) && (p.ldc % 4 == 0)
-                  && (p.batch == 1 || p.sC % 4 == 0);
-    if (bf)
-        splitk_reduce_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>(
-            gp.partials, p.C, gp.M, gp.N, gp.batch, v.split_k, gp.ldp, p.ldc, gp.strideC, vec4);
-    else
-        splitk_reduce_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>(
-            gp.partials, p.C, gp.M, gp.N, gp.batch, v.split_k, gp.ldp, p.ldc, gp.strideC, vec4);
-    CUDA_TRY(cudaGetLastError());
-    return CUDALLM_OK;
 }
 
 int run(int variant, const Problem &p, void *stream_v)
@@ -644,9 +709,12 @@ int cudallm_gemm_bf16_host(const void *A_host, const void *B_host, void *C_host,
 // Split-K without any allocation: the scratch is part of the device image.
 // `g_noalloc_scratch` names the array for device code; on the host the same
 // name is only a handle for cudaGetSymbolAddress, never a device address.
-// Layout: [status word, 256 B][fp32 partial sums: split_k x M x ldp].
+// Layout: [status word, 256 B][helper flags, 64 KiB][helper partial tiles].
 static __device__ __align__(256) unsigned char g_noalloc_scratch[CUDALLM_NOALLOC_SCRATCH_BYTES];
 static void *g_noalloc_scratch_addr[kMaxDevices] = {};   // per device, filled on first use
+static int g_noalloc_epoch[kMaxDevices] = {};
+constexpr size_t kNoallocHeaderBytes = CUDALLM_NOALLOC_HEADER_BYTES;   // status + flags
+constexpr int64_t kNoallocMaxHelperTiles = (kNoallocHeaderBytes - 256) / 16;
 
 int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int64_t M, int64_t N,
                                      int64_t K, int64_t lda, int64_t ldb, int64_t ldc, int out_dtype,
@@ -660,7 +728,16 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     if (is_empty(p)) return CUDALLM_OK;
     if (cdiv(K, kBlockK) < split_k) return CUDALLM_ERR_UNSUPPORTED_SHAPE;   // also covers K == 0
     if (!a_operand_aligned(p) || !b_operand_aligned(p)) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
-    if ((long double)partial_bytes(p, split_k) + 256.0L > (long double)CUDALLM_NOALLOC_SCRATCH_BYTES)
+
+    // always 128 x 64 tiles, every tile split: split_k - 1 partial tiles of 32 KiB each
+    Variant v{};
+    v.family = kUmma;
+    v.block_n = 64;
+    v.split_k = split_k;
+    const Tiling t = tiling_for(v, p, kNumSMs);
+    if (t.units > kMaxDim || t.helper_tiles > kNoallocMaxHelperTiles
+        || (long double)t.partial_bytes + (long double)kNoallocHeaderBytes
+               > (long double)CUDALLM_NOALLOC_SCRATCH_BYTES)
         return CUDALLM_ERR_TOO_LARGE;
 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
@@ -678,12 +755,6 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     }
     uint8_t *scratch = static_cast<uint8_t *>(g_noalloc_scratch_addr[dev]);
 
-    // widest tile that still gives every SM a unit, else the narrowest
-    int block_n = 64;
-    for (int bn : kBlockNs) {
-        if (tiling_for(p, bn, split_k).units >= kNumSMs) block_n = bn;
-    }
-
     CUtensorMap ta, tb;
     const int a_box_rows = p.M >= kBlockM ? kBlockM : (int)round_up(p.M, 8);
     st = encode_operand_map(&ta, A, p.K, p.M, 1, lda, 0, kBlockK, a_box_rows);
@@ -691,46 +762,19 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     st = encode_operand_map(&tb, B, p.N, p.K, 1, ldb, 0, 64, kBlockK);
     if (st != CUDALLM_OK) return st;
 
-    const Tiling t = tiling_for(p, block_n, split_k);
-    GemmParams gp{};
-    gp.C = p.C;
-    gp.ldc = p.ldc;
-    gp.strideC = 0;
-    gp.M = (int)p.M; gp.N = (int)p.N; gp.K = (int)p.K; gp.batch = 1;
-    gp.tiles_m = (int)t.tiles_m; gp.tiles_n = (int)t.tiles_n;
-    gp.split_k = split_k;
-    gp.kblocks = (int)t.kblocks;
-    gp.num_units = (int)t.units;
-    gp.c_vec_ok = 0;                                    // unused: every unit writes partial sums
-    gp.a_box_bytes = a_box_rows * 128;
-    gp.partials = reinterpret_cast<float *>(scratch + 256);
-    gp.ldp = partial_ld(p);
+    GemmParams gp = make_params(p, t, a_box_rows);
+    g_noalloc_epoch[dev] = (g_noalloc_epoch[dev] == 0x7fffffff) ? 1 : g_noalloc_epoch[dev] + 1;
+    gp.epoch = g_noalloc_epoch[dev];
     gp.status = reinterpret_cast<int *>(scratch);
+    gp.flags = reinterpret_cast<int *>(scratch + 256);
+    gp.partials = reinterpret_cast<float *>(scratch + kNoallocHeaderBytes);
 
-    // the status word must start at zero; the partial sums are fully overwritten
-    CUDA_TRY(cudaMemsetAsync(scratch, 0, 256, stream));
-    const bool bf = p.out_dtype == CUDALLM_BF16;
-    switch (block_n) {
-    case 64:  st = bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
-                      : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream); break;
-    case 128: st = bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
-                      : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream); break;
-    default:  st = bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
-                      : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream); break;
-    }
+    // The array keeps the last call's contents.  The status word and the flags
+    // must start at zero; partial tiles are written before they are read.
+    CUDA_TRY(cudaMemsetAsync(scratch, 0, kNoallocHeaderBytes, stream));
+    st = (p.out_dtype == CUDALLM_BF16) ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
+                                       : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream);
     if (st != CUDALLM_OK) return st;
-    const int64_t groups = p.M * cdiv(p.N, 4);
-    int64_t blocks = cdiv(groups, 256);
-    if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
-    const int64_t al = bf ? 8 : 16;
-    const int vec4 = (reinterpret_cast<uintptr_t>(p.C) % al == 0) && (p.ldc % 4 == 0);
-    if (bf)
-        splitk_reduce_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>(
-            gp.partials, p.C, gp.M, gp.N, 1, split_k, gp.ldp, p.ldc, 0, vec4);
-    else
-        splitk_reduce_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>(
-            gp.partials, p.C, gp.M, gp.N, 1, split_k, gp.ldp, p.ldc, 0, vec4);
-    CUDA_TRY(cudaGetLastError());
     int host_status[2] = {0, 0};
     CUDA_TRY(cudaMemcpyAsync(host_status, scratch, sizeof host_status, cudaMemcpyDeviceToHost, stream));
     CUDA_TRY(cudaStreamSynchronize(stream));
@@ -778,7 +822,8 @@ size_t cudallm_workspace_bytes(int64_t M, int64_t N, int64_t K, int64_t lda, int
     size_t best = kHeaderBytes;
     for (int v = 0; v < kNumVariants; ++v) {
         if (!variant_supports(g_variants[v], p)) continue;
-        const Plan pl = make_plan(g_variants[v], p, true, true);   // worst case: both operands repacked
+        // worst case: both operands repacked
+        const Plan pl = make_plan(tiling_for(g_variants[v], p, default_slots(g_variants[v])), p, true, true);
         if (pl.total > best) best = pl.total;
     }
     return best;

@@ -77,6 +77,27 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     return ok != 0;
 }
 
+// Non-blocking probe of a barrier phase (1 = complete).  Probing a barrier
+// takes a few hundred clocks while the tensor core is reading operands from
+// shared memory, so the hot loops probe the NEXT stage's barrier first, issue
+// their work for the current stage, and only then look at the result.
+template <bool kCluster = false>
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    if (kCluster)
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+
 // Wall-clock limit of every in-kernel wait.  Far above any legitimate wait
 // (a whole GEMM takes well under a second), short enough that a logic error
 // ends the kernel instead of hanging the device.
@@ -195,6 +216,140 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)
           "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
           "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
+}
+
+
+// ------------------------------------------------- fused hot-loop steps --
+// Any instruction whose result the issuing thread has to wait for (a barrier
+// probe, even a plain shared-memory load) costs the MMA thread about 100 ns
+// while the tensor core streams operands out of shared memory, on top of
+// about 36 ns per tcgen05.mma it issues.  The hot loops therefore do ONE
+// barrier round trip per stage and put as much work behind it as a stage
+// holds (one or two 64-deep k-blocks); each step is a single asm block that
+// probes the NEXT stage first, issues the current stage's work, and reads the
+// probe's predicate last (through a branch, which cannot be hoisted).
+
+// MMA step for one stage of `nsub` (1 or 2) 64-deep k-blocks: four K=16 MMAs
+// per k-block, then the commit(s) that free the stage when they retire.
+//   returns 1 if `next_bar` has completed phase `next_parity`.
+//   first_acc: 0 -> the first MMA overwrites the accumulator.
+//   da0 / db0: descriptors of the first k-block; the second one lies
+//   `sub_bytes` further in shared memory.  commit_b is used by pairs only.
+template <bool kPair>
+__device__ __forceinline__ uint32_t umma_stage_step(uint32_t next_bar, uint32_t next_parity,
+                                                    uint32_t d_tmem, uint32_t idesc, uint32_t first_acc,
+                                                    uint64_t da0, uint64_t db0, uint32_t sub_bytes,
+                                                    int nsub, uint32_t commit_a, uint32_t commit_b)
+{
+    uint32_t tok;
+    const uint64_t sub = static_cast<uint64_t>(sub_bytes >> 4);
+#define CUDALLM_MMA_STEP(GROUP, TESTW, TRYW, COMMIT2)                                              \
+    asm volatile(                                                                                  \
+        "{\n\t"                                                                                    \
+        ".reg .pred pn, p0, pt, p2;\n\t"                                                           \
+        ".reg .b64 a1, a2, a3, a4, a5, a6, a7, b1, b2, b3, b4, b5, b6, b7;\n\t"                    \
+        TESTW " pn, [%1], %2;\n\t"                                                                 \
+        "tcgen05.fence::after_thread_sync;\n\t"                                                    \
+        "setp.ne.b32 p0, %5, 0;\n\t"                                                               \
+        "setp.eq.b32 pt, %5, %5;\n\t"                                                              \
+        "setp.gt.s32 p2, %9, 1;\n\t"                                                               \
+        "add.u64 a1, %6, 2;\n\t add.u64 a2, %6, 4;\n\t add.u64 a3, %6, 6;\n\t"                   \
+        "add.u64 b1, %7, 128;\n\t add.u64 b2, %7, 256;\n\t add.u64 b3, %7, 384;\n\t"             \
+        "add.u64 a4, %6, %8;\n\t add.u64 a5, a1, %8;\n\t add.u64 a6, a2, %8;\n\t add.u64 a7, a3, %8;\n\t" \
+        "add.u64 b4, %7, %8;\n\t add.u64 b5, b1, %8;\n\t add.u64 b6, b2, %8;\n\t add.u64 b7, b3, %8;\n\t" \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%3], %6, %7, %4, p0;\n\t"                     \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%3], a1, b1, %4, pt;\n\t"                     \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%3], a2, b2, %4, pt;\n\t"                     \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%3], a3, b3, %4, pt;\n\t"                     \
+        "@p2 tcgen05.mma.cta_group::" GROUP ".kind::f16 [%3], a4, b4, %4, pt;\n\t"                 \
+        "@p2 tcgen05.mma.cta_group::" GROUP ".kind::f16 [%3], a5, b5, %4, pt;\n\t"                 \
+        "@p2 tcgen05.mma.cta_group::" GROUP ".kind::f16 [%3], a6, b6, %4, pt;\n\t"                 \
+        "@p2 tcgen05.mma.cta_group::" GROUP ".kind::f16 [%3], a7, b7, %4, pt;\n\t"                 \
+        "tcgen05.commit.cta_group::" GROUP ".mbarrier::arrive::one.shared::cluster.b64 [%10];\n\t" \
+        COMMIT2                                                                                    \
+        "@pn bra LDONE;\n\t"                                                                       \
+        TRYW " pn, [%1], %2;\n\t"                                                                  \
+        "LDONE:\n\t"                                                                               \
+        "selp.u32 %0, 1, 0, pn;\n\t"                                                               \
+        "}"                                                                                        \
+        : "=r"(tok)                                                                                \
+        : "r"(next_bar), "r"(next_parity), "r"(d_tmem), "r"(idesc), "r"(first_acc), "l"(da0),      \
+          "l"(db0), "l"(sub), "r"(nsub), "r"(commit_a), "r"(commit_b)                              \
+        : "memory")
+    if (kPair) {
+        CUDALLM_MMA_STEP("2", "mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64",
+                         "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64",
+                         "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%11];\n\t");
+    } else {
+        CUDALLM_MMA_STEP("1", "mbarrier.test_wait.parity.shared::cta.b64",
+                         "mbarrier.try_wait.parity.shared::cta.b64", "");
+    }
+#undef CUDALLM_MMA_STEP
+    return tok;
+}
+
+// Producer step for one stage of `nsub` (1 or 2) k-blocks: arm `full_bar` with
+// `tx_bytes` (if arm != 0); per k-block load one box of A and `boxes` boxes of
+// B (64 columns wide, 8 KB apart in shared memory; up to 4 for the first
+// k-block, up to 2 for the second).  The second k-block's tiles lie
+// `sub_bytes` after the first's.  Returns 1 if `next_bar` has completed phase
+// `next_parity`.  `signal_bar` is where the loads complete their bytes (the
+// leader's barrier for CTA pairs).
+template <bool kPair>
+__device__ __forceinline__ uint32_t tma_stage_step(uint32_t next_bar, uint32_t next_parity,
+                                                   uint32_t full_bar, uint32_t arm, uint32_t tx_bytes,
+                                                   uint32_t signal_bar, const CUtensorMap *tm_a,
+                                                   const CUtensorMap *tm_b, uint32_t sa, uint32_t sb,
+                                                   int k0, int row0, int col0, int batch, int boxes,
+                                                   int nsub, uint32_t sub_bytes)
+{
+    uint32_t tok;
+    const uint64_t ta = reinterpret_cast<uint64_t>(tm_a), tb = reinterpret_cast<uint64_t>(tm_b);
+#define CUDALLM_TMA_STEP(TESTW, TRYW, LOAD)                                                        \
+    asm volatile(                                                                                  \
+        "{\n\t"                                                                                    \
+        ".reg .pred pn, pa, p1, p2, p3, q0, q1;\n\t"                                               \
+        ".reg .b32 c1, c2, c3, s1, s2, s3, k1, ta1, tb1, tb2;\n\t"                                 \
+        TESTW " pn, [%1], %2;\n\t"                                                                 \
+        "setp.ne.b32 pa, %4, 0;\n\t"                                                               \
+        "setp.gt.s32 p1, %15, 1;\n\t"                                                              \
+        "setp.gt.s32 p2, %15, 2;\n\t"                                                              \
+        "setp.gt.s32 p3, %15, 3;\n\t"                                                              \
+        "setp.gt.s32 q0, %16, 1;\n\t"                                                              \
+        "and.pred q1, q0, p1;\n\t"                                                                 \
+        "add.s32 c1, %13, 64;\n\t add.s32 c2, %13, 128;\n\t add.s32 c3, %13, 192;\n\t"           \
+        "add.u32 s1, %10, 8192;\n\t add.u32 s2, %10, 16384;\n\t add.u32 s3, %10, 24576;\n\t"     \
+        "add.s32 k1, %11, 64;\n\t add.u32 ta1, %9, %17;\n\t add.u32 tb1, %10, %17;\n\t add.u32 tb2, s1, %17;\n\t" \
+        "@pa mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %5;\n\t"                           \
+        LOAD " [%9], [%7, {%11, %12, %14}], [%6];\n\t"                                             \
+        LOAD " [%10], [%8, {%13, %11, %14}], [%6];\n\t"                                            \
+        "@p1 " LOAD " [s1], [%8, {c1, %11, %14}], [%6];\n\t"                                       \
+        "@p2 " LOAD " [s2], [%8, {c2, %11, %14}], [%6];\n\t"                                       \
+        "@p3 " LOAD " [s3], [%8, {c3, %11, %14}], [%6];\n\t"                                       \
+        "@q0 " LOAD " [ta1], [%7, {k1, %12, %14}], [%6];\n\t"                                      \
+        "@q0 " LOAD " [tb1], [%8, {%13, k1, %14}], [%6];\n\t"                                      \
+        "@q1 " LOAD " [tb2], [%8, {c1, k1, %14}], [%6];\n\t"                                       \
+        "@pn bra LDONE;\n\t"                                                                       \
+        TRYW " pn, [%1], %2;\n\t"                                                                  \
+        "LDONE:\n\t"                                                                               \
+        "selp.u32 %0, 1, 0, pn;\n\t"                                                               \
+        "}"                                                                                        \
+        : "=r"(tok)                                                                                \
+        : "r"(next_bar), "r"(next_parity), "r"(full_bar), "r"(arm), "r"(tx_bytes), "r"(signal_bar), \
+          "l"(ta), "l"(tb), "r"(sa), "r"(sb), "r"(k0), "r"(row0), "r"(col0), "r"(batch), "r"(boxes), \
+          "r"(nsub), "r"(sub_bytes)                                                                \
+        : "memory")
+    if (kPair) {
+        CUDALLM_TMA_STEP("mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64",
+                         "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64",
+                         "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes");
+    } else {
+        CUDALLM_TMA_STEP("mbarrier.test_wait.parity.shared::cta.b64",
+                         "mbarrier.try_wait.parity.shared::cta.b64",
+                         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes");
+    }
+#undef CUDALLM_TMA_STEP
+    return tok;
 }
 
 // ---------------------------------------------------------- descriptors --

@@ -9,11 +9,22 @@
 // the next).  Roles: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM
 // owner), warps 2..5 = epilogue (TMEM -> registers -> global).
 //
-// Work is cut into units (tile, k-split); CTA b runs units b, b+grid, ...
-// With split_k > 1 every unit writes its fp32 partial sums to slice `split` of
-// a workspace shaped [split][batch][M][ldp]; splitk_reduce_kernel then adds the
-// slices in split order 0..S-1 (a fixed order, so results are reproducible)
-// and writes C, rounding once.
+// Work is cut into units; CTA b runs units b, b+grid, ... in that order.  The
+// first dp_tiles tiles are one unit each.  Every later tile is cut along K into
+// split_k units with consecutive indices: the first split_k-1 ("helpers") write
+// their fp32 partial tile to the workspace and raise a flag; the last one (the
+// "owner") waits for those flags, adds the partial tiles to its own accumulator
+// in split order 0..S-2 -- a fixed order, so results are reproducible -- and
+// stores C, rounding once.  A unit only ever waits for units with smaller
+// indices, which run earlier on the same CTA or on other CTAs, so the waits
+// cannot form a cycle; they are bounded like every other wait in the kernel.
+// dp_tiles = 0 is plain split-K.
+//
+// Tiles >= dp_tiles can instead be cut along N into tail_nsplit narrower units
+// (BLOCK_N / tail_nsplit columns each, no partial sums needed): with dp_tiles =
+// tiles - tiles % grid this makes the ragged last wave of a launch take about
+// 1/tail_nsplit of a tile's time.  The MMA's N, the number of B boxes and the
+// epilogue's column count are per-unit values for that reason.
 #pragma once
 #include "ptx.cuh"
 
@@ -34,13 +45,16 @@ struct GemmParams {
     long long strideC;      // elements between batch items
     int M, N, K, batch;
     int tiles_m, tiles_n;   // tiles per batch item
-    int split_k;            // >= 1, <= kblocks
     int kblocks;            // ceil(K / 64)
-    int num_units;          // tiles_m * tiles_n * batch * split_k
+    int dp_tiles;           // leading tiles that are not split
+    int split_k;            // K parts per tile for tiles >= dp_tiles (1 = none), <= kblocks
+    int tail_nsplit;        // N parts per tile for tiles >= dp_tiles (1 = none); not with split_k > 1
+    int num_units;          // dp_tiles + (tiles - dp_tiles) * split_k * tail_nsplit
     int c_vec_ok;           // C base, ldc, strideC allow 16-byte stores
     int a_box_bytes;        // bytes one TMA box of A delivers (box rows * 128)
-    float *partials;        // split-K partial sums [split][batch][M][ldp] (workspace)
-    long long ldp;          // row stride of the partial slices (multiple of 4)
+    int epoch;              // value that marks a flag as raised in this launch (never 0)
+    float *partials;        // helper partial tiles (workspace), 128 x BLOCK_N fp32 each
+    int *flags;             // one per (helper partial tile, epilogue warp) (workspace)
     int *status;            // [0] = code, [1] = detail
 };
 
@@ -64,23 +78,77 @@ __device__ __forceinline__ void report_timeout(int *status, int role, int what)
 }
 
 struct UnitCoord {
-    int m_tile, n_tile, b, split, tile_linear;
+    int m_tile, b;
+    int n0, width;          // first column and number of columns (multiple of 64) of this unit
+    int split, nsplit;      // this unit's part of K and how many parts its tile has
+    int helper_index;       // (tile - dp_tiles) * (split_k - 1): first partial tile of this unit's tile
     int kb_begin, kb_end;
 };
 
+template <int BLOCK_N>
 __device__ __forceinline__ UnitCoord decode_unit(const GemmParams &p, int u)
 {
     UnitCoord c;
-    c.split = u % p.split_k;
-    int t = u / p.split_k;
-    c.tile_linear = t;
+    int t;
+    int part = 0;
+    c.width = BLOCK_N;
+    if (u < p.dp_tiles) {
+        t = u;
+        c.split = 0;
+        c.nsplit = 1;
+        c.helper_index = 0;
+    } else if (p.tail_nsplit > 1) {
+        const int r = u - p.dp_tiles;
+        const int ts = r / p.tail_nsplit;
+        t = p.dp_tiles + ts;
+        part = r - ts * p.tail_nsplit;
+        c.width = BLOCK_N / p.tail_nsplit;
+        c.split = 0;
+        c.nsplit = 1;
+        c.helper_index = 0;
+    } else {
+        const int r = u - p.dp_tiles;
+        const int ts = r / p.split_k;
+        t = p.dp_tiles + ts;
+        c.split = r - ts * p.split_k;
+        c.nsplit = p.split_k;
+        c.helper_index = ts * (p.split_k - 1);
+    }
     c.m_tile = t % p.tiles_m;
     t /= p.tiles_m;
-    c.n_tile = t % p.tiles_n;
+    c.n0 = (t % p.tiles_n) * BLOCK_N + part * c.width;
     c.b = t / p.tiles_n;
-    c.kb_begin = static_cast<int>((static_cast<long long>(p.kblocks) * c.split) / p.split_k);
-    c.kb_end = static_cast<int>((static_cast<long long>(p.kblocks) * (c.split + 1)) / p.split_k);
+    c.kb_begin = static_cast<int>((static_cast<long long>(p.kblocks) * c.split) / c.nsplit);
+    c.kb_end = static_cast<int>((static_cast<long long>(p.kblocks) * (c.split + 1)) / c.nsplit);
     return c;
+}
+
+__device__ __forceinline__ int ld_acquire_gpu(const int *p)
+{
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(int *p, int v)
+{
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// Bounded wait until *flag == epoch.
+__device__ __forceinline__ bool wait_flag(const int *flag, int epoch, volatile int *abort_flag)
+{
+    if (ld_acquire_gpu(flag) == epoch) return true;
+    const uint64_t t0 = globaltimer_ns();
+    while (true) {
+        for (int i = 0; i < 16; ++i) {
+            if (ld_acquire_gpu(flag) == epoch) return true;
+            __nanosleep(100);
+        }
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
 }
 
 // Store 32 consecutive fp32 accumulator values of one row, starting at column
@@ -124,30 +192,67 @@ __device__ __forceinline__ void store_row_chunk(void *row_ptr, const float (&v)[
     }
 }
 
-// Epilogue of one unit for one thread: `row` is this thread's row of C, `t_addr`
-// the TMEM address of its lane at the accumulator's first column.  Reads the
-// BLOCK_N accumulator columns 32 at a time and stores them to C (split_k == 1)
-// or to this split's slice of the partial sums.  Must be called by whole warps.
+// Epilogue of one unit, called by the four epilogue warps.  `row` is this
+// thread's row of C, `t_addr` the TMEM address of its lane at the accumulator's
+// first column, `quad`/`lane` identify the thread (row within the tile =
+// 32*quad + lane), `cta_slot` = index of this CTA among the CTAs that share a
+// tile (0 for lone CTAs, the cluster rank for pairs) and `ctas_per_tile` their
+// number.  Reads the BLOCK_N accumulator columns 32 at a time and
+//   - stores them to C (unsplit tile),
+//   - or writes them to this helper's partial tile and raises its flag,
+//   - or (owner) adds the helpers' partial tiles in split order and stores C.
+// Partial tile layout: float4 index ((chunk*8 + q) * 128 + row_in_tile), so
+// that a warp writes and reads 512 contiguous bytes.
 template <int BLOCK_N, bool OUT_BF16>
-__device__ __forceinline__ void epilogue_tile(const GemmParams &p, const UnitCoord &c, int row,
-                                              uint32_t t_addr)
+__device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoord &c, int row,
+                                              uint32_t t_addr, int quad, int lane, int cta_slot,
+                                              int ctas_per_tile, volatile int *abort_flag)
 {
+    constexpr int kTileF4 = kBlockM * BLOCK_N / 4;
     const bool row_ok = row < p.M;
-    void *row_ptr;
-    bool vec_ok;
-    if (p.split_k == 1) {
-        const long long off = static_cast<long long>(c.b) * p.strideC
-                            + static_cast<long long>(row) * p.ldc;
-        row_ptr = OUT_BF16 ? static_cast<void *>(reinterpret_cast<__nv_bfloat16 *>(p.C) + off)
-                           : static_cast<void *>(reinterpret_cast<float *>(p.C) + off);
-        vec_ok = p.c_vec_ok != 0;
-    } else {
-        row_ptr = p.partials
-                + ((static_cast<long long>(c.split) * p.batch + c.b) * p.M + row) * p.ldp;
-        vec_ok = true;
+    const int row_in_tile = quad * 32 + lane;
+    const bool helper = c.split + 1 < c.nsplit;
+    const bool owner = c.nsplit > 1 && !helper;
+    bool ok = true;
+
+    if (helper) {
+        const long long slot = static_cast<long long>(c.helper_index + c.split) * ctas_per_tile + cta_slot;
+        float4 *part = reinterpret_cast<float4 *>(p.partials) + slot * kTileF4;
+#pragma unroll 1
+        for (int ch = 0; ch < c.width / 32; ++ch) {
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(t_addr + ch * 32, r);
+            tmem_ld_wait();
+            if (row_ok) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    __stcg(part + (ch * 8 + q) * kBlockM + row_in_tile,
+                           make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                       __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3])));
+            }
+            __syncwarp();                                // tcgen05.ld needs the whole warp
+        }
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) st_release_gpu(p.flags + slot * 4 + quad, p.epoch);
+        return true;
+    }
+
+    const long long off = static_cast<long long>(c.b) * p.strideC + static_cast<long long>(row) * p.ldc;
+    void *row_ptr = OUT_BF16 ? static_cast<void *>(reinterpret_cast<__nv_bfloat16 *>(p.C) + off)
+                             : static_cast<void *>(reinterpret_cast<float *>(p.C) + off);
+    const bool vec_ok = p.c_vec_ok != 0;
+    if (owner) {
+        // the same epilogue warp of every helper wrote the rows this warp needs
+        for (int s = 0; s + 1 < c.nsplit; ++s) {
+            const long long slot = static_cast<long long>(c.helper_index + s) * ctas_per_tile + cta_slot;
+            ok = wait_flag(p.flags + slot * 4 + quad, p.epoch, abort_flag) && ok;
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        __threadfence();
     }
 #pragma unroll 1
-    for (int ch = 0; ch < BLOCK_N / 32; ++ch) {
+    for (int ch = 0; ch < c.width / 32; ++ch) {
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_addr + ch * 32, r);
         tmem_ld_wait();
@@ -155,12 +260,22 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams &p, const UnitCoo
             float v[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            const int col0 = c.n_tile * BLOCK_N + ch * 32;
-            if (p.split_k == 1) store_row_chunk<OUT_BF16>(row_ptr, v, col0, p.N, vec_ok);
-            else                store_row_chunk<false>(row_ptr, v, col0, p.N, vec_ok);
+            if (owner) {
+                for (int s = 0; s + 1 < c.nsplit; ++s) {
+                    const long long slot = static_cast<long long>(c.helper_index + s) * ctas_per_tile + cta_slot;
+                    const float4 *part = reinterpret_cast<const float4 *>(p.partials) + slot * kTileF4;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 t = __ldcg(part + (ch * 8 + q) * kBlockM + row_in_tile);
+                        v[4 * q] += t.x; v[4 * q + 1] += t.y; v[4 * q + 2] += t.z; v[4 * q + 3] += t.w;
+                    }
+                }
+            }
+            store_row_chunk<OUT_BF16>(row_ptr, v, c.n0 + ch * 32, p.N, vec_ok);
         }
         __syncwarp();                                    // tcgen05.ld needs the whole warp
     }
+    return ok;
 }
 
 template <int BLOCK_N, int STAGES, bool OUT_BF16>
@@ -171,7 +286,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     using L = SmemLayout<BLOCK_N, STAGES>;
     static_assert(BLOCK_N % 64 == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
     constexpr uint32_t kTmemCols = 2 * BLOCK_N;          // 128, 256 or 512: power of two
-    constexpr uint32_t kIdesc = make_idesc_bf16(kBlockM, BLOCK_N, 0, 1);
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
@@ -218,23 +332,26 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
+            uint32_t tok = 1;                            // the first STAGES stages start out free
             for (int u = blockIdx.x; ok && u < p.num_units; u += gridDim.x) {
-                const UnitCoord c = decode_unit(p, u);
+                const UnitCoord c = decode_unit<BLOCK_N>(p, u);
+                const int boxes = c.width / 64;
                 for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) {
+                    if (!tok && !mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) {
                         report_timeout(p.status, kRoleProducer, stage);
                         ok = false;
                         break;
                     }
+                    // probes the next stage, then issues this stage's loads (one asm block)
+                    const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
+                    const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
-                    const uint32_t sb = sa + L::kABytes;
-                    mbar_arrive_expect_tx(full_bar(stage), p.a_box_bytes + L::kBBytes);
-                    tma_load_3d(sa, &tmap_a, full_bar(stage), kb * kBlockK, c.m_tile * kBlockM, c.b);
-#pragma unroll
-                    for (int j = 0; j < BLOCK_N / 64; ++j)
-                        tma_load_3d(sb + j * (64 * kBlockK * 2), &tmap_b, full_bar(stage),
-                                    c.n_tile * BLOCK_N + j * 64, kb * kBlockK, c.b);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    tok = tma_stage_step<false>(empty_bar(nstage), nphase ^ 1, full_bar(stage), 1,
+                                                p.a_box_bytes + boxes * (64 * kBlockK * 2), full_bar(stage),
+                                                &tmap_a, &tmap_b, sa, sa + L::kABytes, kb * kBlockK,
+                                                c.m_tile * kBlockM, c.n0, c.b, boxes, 1, 0);
+                    stage = nstage;
+                    phase = nphase;
                 }
             }
         }
@@ -246,34 +363,36 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
+            uint32_t tok = 0;                            // answer of the probe of full[stage]
             for (int u = blockIdx.x; ok && u < p.num_units; u += gridDim.x) {
-                const UnitCoord c = decode_unit(p, u);
+                const UnitCoord c = decode_unit<BLOCK_N>(p, u);
+                const uint32_t idesc = make_idesc_bf16(kBlockM, c.width, 0, 1);
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag)) {
                     report_timeout(p.status, kRoleMma, 0x40 + acc);
                     break;
                 }
-                tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
                 for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+                    if (!tok && !mbar_wait(full_bar(stage), phase, abort_flag)) {
                         report_timeout(p.status, kRoleMma, stage);
                         ok = false;
                         break;
                     }
-                    tc_fence_after();
+                    // probes the next stage, then issues this stage's four MMAs and the
+                    // commit that frees the stage when they retire (one asm block).
+                    // A: K-major, 8-row groups 1024 B apart (SBO); 16 K-elements = 32 B.
+                    // B: MN-major, 64-column chunks 8192 B apart (LBO), 8-k groups
+                    //    1024 B apart (SBO); 16 k = 2048 B.
+                    const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
+                    const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
-                    const uint32_t sb = sa + L::kABytes;
-#pragma unroll
-                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        // A: K-major, 8-row groups 1024 B apart; 16 K-elements = 32 B
-                        const uint64_t da = make_smem_desc_sw128(sa + k * 32, 16, 1024);
-                        // B: MN-major, 64-column chunks 8192 B apart (LBO),
-                        //    8-k groups 1024 B apart (SBO); 16 k = 2048 B
-                        const uint64_t db = make_smem_desc_sw128(sb + k * 2048, 8192, 1024);
-                        umma_bf16(d_tmem, da, db, kIdesc, (kb > c.kb_begin || k > 0) ? 1u : 0u);
-                    }
-                    umma_commit(empty_bar(stage));       // frees the stage when the MMAs retire
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    tok = umma_stage_step<false>(full_bar(nstage), nphase, d_tmem, idesc,
+                                                 kb > c.kb_begin ? 1u : 0u,
+                                                 make_smem_desc_sw128(sa, 16, 1024),
+                                                 make_smem_desc_sw128(sa + L::kABytes, 8192, 1024),
+                                                 0, 1, empty_bar(stage), 0);
+                    stage = nstage;
+                    phase = nphase;
                 }
                 if (!ok) break;
                 umma_commit(tfull_bar(acc));             // accumulator complete
@@ -287,7 +406,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int u = blockIdx.x; u < p.num_units; u += gridDim.x) {
-            const UnitCoord c = decode_unit(p, u);
+            const UnitCoord c = decode_unit<BLOCK_N>(p, u);
             bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
@@ -295,8 +414,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 break;
             }
             tc_fence_after();
-            epilogue_tile<BLOCK_N, OUT_BF16>(p, c, c.m_tile * kBlockM + epi_tid,
-                                             tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(quad * 32) << 16));
+            if (!epilogue_tile<BLOCK_N, OUT_BF16>(p, c, c.m_tile * kBlockM + epi_tid,
+                                                  tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(quad * 32) << 16),
+                                                  quad, lane, 0, 1, abort_flag)) {
+                if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0xC0);
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -310,54 +432,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
-    }
-}
-
-// Adds the S slices of split-K partial sums in order s = 0..S-1 and writes C
-// (fp32, or bf16 rounded once).  One thread handles 4 consecutive columns.
-template <bool OUT_BF16>
-__global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const float *__restrict__ partials, void *C, int M, int N, int batch, int split_k,
-                     long long ldp, long long ldc, long long strideC, int c_vec4_ok)
-{
-    const int groups = (N + 3) >> 2;
-    const long long rows = static_cast<long long>(batch) * M;
-    const long long total = rows * groups;
-    const long long slice = rows * ldp;
-    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
-         i += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const long long br = i / groups;                 // b * M + row
-        const int col = static_cast<int>(i - br * groups) * 4;
-        const int b = static_cast<int>(br / M);
-        const int row = static_cast<int>(br - static_cast<long long>(b) * M);
-        const float *src = partials + br * ldp + col;
-        float4 acc = __ldcg(reinterpret_cast<const float4 *>(src));
-        for (int s = 1; s < split_k; ++s) {
-            const float4 t = __ldcg(reinterpret_cast<const float4 *>(src + s * slice));
-            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
-        }
-        const long long off = b * strideC + row * ldc + col;
-        const int n_left = N - col;
-        if (OUT_BF16) {
-            __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(C) + off;
-            if (c_vec4_ok && n_left >= 4) {
-                uint2 w;
-                w.x = pack_bf16x2(acc.x, acc.y);
-                w.y = pack_bf16x2(acc.z, acc.w);
-                *reinterpret_cast<uint2 *>(dst) = w;
-            } else {
-                const float a[4] = {acc.x, acc.y, acc.z, acc.w};
-                for (int j = 0; j < 4 && j < n_left; ++j) dst[j] = __float2bfloat16_rn(a[j]);
-            }
-        } else {
-            float *dst = reinterpret_cast<float *>(C) + off;
-            if (c_vec4_ok && n_left >= 4) {
-                *reinterpret_cast<float4 *>(dst) = acc;
-            } else {
-                const float a[4] = {acc.x, acc.y, acc.z, acc.w};
-                for (int j = 0; j < 4 && j < n_left; ++j) dst[j] = a[j];
-            }
-        }
     }
 }
 

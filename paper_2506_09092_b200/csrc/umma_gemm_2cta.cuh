@@ -67,11 +67,13 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t bar_cluster_addr)
                  ::"r"(bar_cluster_addr) : "memory");
 }
 
-template <int STAGES>
+// A stage holds KSUB (1 or 2) 64-deep k-blocks, each [A 128 x 64 | B 64 x 128].
+template <int STAGES, int KSUB>
 struct PairSmemLayout {
     static constexpr int kABytes = kBlockM * kBlockK * 2;            // 128 rows of A
     static constexpr int kBBytes = kBlockK * (kPairN / 2) * 2;       // 128 columns of B
-    static constexpr int kStageBytes = kABytes + kBBytes;            // 32 KB
+    static constexpr int kSubBytes = kABytes + kBBytes;              // 32 KB per k-block
+    static constexpr int kStageBytes = KSUB * kSubBytes;
     static constexpr int kBarOffset = STAGES * kStageBytes;
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
@@ -79,14 +81,13 @@ struct PairSmemLayout {
     static constexpr int kDynamicBytes = kBytes + 1024;
 };
 
-template <int STAGES, bool OUT_BF16>
+template <int STAGES, int KSUB, bool OUT_BF16>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
 umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
                       const __grid_constant__ CUtensorMap tmap_b, const GemmParams p)
 {
-    using L = PairSmemLayout<STAGES>;
+    using L = PairSmemLayout<STAGES, KSUB>;
     constexpr uint32_t kTmemCols = 2 * kPairN;                       // 512: two accumulators
-    constexpr uint32_t kIdesc = make_idesc_bf16(kPairM, kPairN, 0, 1);
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
@@ -137,26 +138,32 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
+            uint32_t tok = 1;                            // the first STAGES stages start out free
+            const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
             for (int u = pair; ok && u < p.num_units; u += num_pairs) {
-                const UnitCoord c = decode_unit(p, u);
-                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
-                    if (!mbar_wait<true>(empty_bar(stage), phase ^ 1, abort_flag)) {
+                const UnitCoord c = decode_unit<kPairN>(p, u);
+                const int half = c.width / 2;            // columns of B this CTA stages: 128 or 64
+                const int boxes = half / 64;
+                for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
+                    if (!tok && !mbar_wait<true>(empty_bar(stage), phase ^ 1, abort_flag)) {
                         report_timeout(p.status, kRoleProducer, stage);
                         ok = false;
                         break;
                     }
+                    const int nsub = (c.kb_end - kb) < KSUB ? (c.kb_end - kb) : KSUB;
+                    const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
+                    const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
-                    const uint32_t sb = sa + L::kABytes;
-                    const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
-                    if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * L::kStageBytes);
-                    tma_load_3d_pair(sa, &tmap_a, leader_full, kb * kBlockK,
-                                     c.m_tile * kPairM + static_cast<int>(rank) * kBlockM, c.b);
-#pragma unroll
-                    for (int j = 0; j < 2; ++j)
-                        tma_load_3d_pair(sb + j * (64 * kBlockK * 2), &tmap_b, leader_full,
-                                         c.n_tile * kPairN + static_cast<int>(rank) * 128 + j * 64,
-                                         kb * kBlockK, c.b);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    tok = tma_stage_step<true>(empty_bar(nstage), nphase ^ 1, full_bar(stage),
+                                               rank == 0 ? 1u : 0u,
+                                               2 * nsub * (L::kABytes + boxes * (64 * kBlockK * 2)),
+                                               leader_full0 + 8u * stage, &tmap_a, &tmap_b, sa,
+                                               sa + L::kABytes, kb * kBlockK,
+                                               c.m_tile * kPairM + static_cast<int>(rank) * kBlockM,
+                                               c.n0 + static_cast<int>(rank) * half, c.b, boxes, nsub,
+                                               L::kSubBytes);
+                    stage = nstage;
+                    phase = nphase;
                 }
             }
         }
@@ -168,36 +175,42 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
+            uint32_t tok = 0;                            // answer of the probe of full[stage]
+            // cluster addresses of the barriers this thread signals in both CTAs
+            const uint32_t empty0_cta0 = map_to_cta(empty_bar(0), 0);
+            const uint32_t empty0_cta1 = map_to_cta(empty_bar(0), 1);
+            const uint32_t tfull0_cta0 = map_to_cta(tfull_bar(0), 0);
+            const uint32_t tfull0_cta1 = map_to_cta(tfull_bar(0), 1);
             for (int u = pair; ok && u < p.num_units; u += num_pairs) {
-                const UnitCoord c = decode_unit(p, u);
+                const UnitCoord c = decode_unit<kPairN>(p, u);
+                const uint32_t idesc = make_idesc_bf16(kPairM, c.width, 0, 1);
                 if (!mbar_wait<true>(tempty_bar(acc), acc_phase ^ 1, abort_flag)) {
                     report_timeout(p.status, kRoleMma, 0x40 + acc);
                     break;
                 }
-                tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kPairN;
-                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
-                    if (!mbar_wait<true>(full_bar(stage), phase, abort_flag)) {
+                for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
+                    if (!tok && !mbar_wait<true>(full_bar(stage), phase, abort_flag)) {
                         report_timeout(p.status, kRoleMma, stage);
                         ok = false;
                         break;
                     }
-                    tc_fence_after();
+                    const int nsub = (c.kb_end - kb) < KSUB ? (c.kb_end - kb) : KSUB;
+                    const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
+                    const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
-                    const uint32_t sb = sa + L::kABytes;
-#pragma unroll
-                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        const uint64_t da = make_smem_desc_sw128(sa + k * 32, 16, 1024);
-                        const uint64_t db = make_smem_desc_sw128(sb + k * 2048, 8192, 1024);
-                        umma_bf16_2cta(d_tmem, da, db, kIdesc, (kb > c.kb_begin || k > 0) ? 1u : 0u);
-                    }
-                    umma_commit_pair(map_to_cta(empty_bar(stage), 0));
-                    umma_commit_pair(map_to_cta(empty_bar(stage), 1));
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    tok = umma_stage_step<true>(full_bar(nstage), nphase, d_tmem, idesc,
+                                                kb > c.kb_begin ? 1u : 0u,
+                                                make_smem_desc_sw128(sa, 16, 1024),
+                                                make_smem_desc_sw128(sa + L::kABytes, 8192, 1024),
+                                                L::kSubBytes, nsub, empty0_cta0 + 8u * stage,
+                                                empty0_cta1 + 8u * stage);
+                    stage = nstage;
+                    phase = nphase;
                 }
                 if (!ok) break;
-                umma_commit_pair(map_to_cta(tfull_bar(acc), 0));
-                umma_commit_pair(map_to_cta(tfull_bar(acc), 1));
+                umma_commit_pair(tfull0_cta0 + 8u * acc);
+                umma_commit_pair(tfull0_cta1 + 8u * acc);
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             }
         }
@@ -208,7 +221,7 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int u = pair; u < p.num_units; u += num_pairs) {
-            const UnitCoord c = decode_unit(p, u);
+            const UnitCoord c = decode_unit<kPairN>(p, u);
             bool ok = mbar_wait<true>(tfull_bar(acc), acc_phase, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
@@ -216,8 +229,11 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 break;
             }
             tc_fence_after();
-            epilogue_tile<kPairN, OUT_BF16>(p, c, c.m_tile * kPairM + static_cast<int>(rank) * kBlockM + epi_tid,
-                                            tmem_base + acc * kPairN + (static_cast<uint32_t>(quad * 32) << 16));
+            if (!epilogue_tile<kPairN, OUT_BF16>(p, c, c.m_tile * kPairM + static_cast<int>(rank) * kBlockM + epi_tid,
+                                                 tmem_base + acc * kPairN + (static_cast<uint32_t>(quad * 32) << 16),
+                                                 quad, lane, static_cast<int>(rank), 2, abort_flag)) {
+                if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0xC0);
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(map_to_cta(tempty_bar(acc), 0));

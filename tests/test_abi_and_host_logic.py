@@ -85,6 +85,8 @@ def test_variant_support_rules():
     table = {B.variant_name(v): v for v in range(B.num_variants())}
     # split-K needs at least one 64-deep k-block per split
     assert B.variant_supports(table["umma_n64_sk16"], 128, 128, 64, 64, 128, 128, 1, 0) == 0
+    assert B.variant_supports(table["umma2_n256_sk4"], 512, 512, 128, 128, 512, 512, 1, 0) == 0
+    assert B.variant_supports(table["umma2_n256_ts"], 512, 512, 128, 128, 512, 512, 1, 0) == 1
     assert B.variant_supports(table["umma_n64_sk16"], 128, 128, 1024, 1024, 128, 128, 1, 0) == 1
     assert B.variant_supports(table["simt"], 1, 1, 0, 0, 1, 1, 1, 0) == 1
     assert B.variant_supports(table["umma_n128"], 1, 1, 0, 0, 1, 1, 1, 0) == 0      # K == 0
@@ -101,7 +103,9 @@ def test_selection_and_workspace_queries():
         ws = B.workspace_bytes(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype)
         assert ws >= 256 and ws % 256 == 0
     c2 = gi.CONFIGS["C2"]
-    assert B.variant_name(B.select_variant(c2.M, c2.N, c2.K, c2.K, c2.N, c2.N, 1, 1)).startswith("umma_n256")
+    # the large square problem goes to 256-wide tiles (CTA pairs), never to plain split-K
+    name = B.variant_name(B.select_variant(c2.M, c2.N, c2.K, c2.K, c2.N, c2.N, 1, 1))
+    assert "n256" in name and "_sk" not in name
     assert B.select_variant(4, 4, 0, 0, 4, 4, 1, 0) == 0          # K == 0 runs on the simt kernel
 
 

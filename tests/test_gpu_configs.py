@@ -80,3 +80,26 @@ def test_paper_task2_ladder_first_two_sizes():
         rows = np.random.default_rng(step).choice(cfg.M, size=64, replace=False)
         Cref, S = oracle.gemm_rows(A, Bm, rows, cfg.N, cfg.K, cfg.lda_, cfg.ldb_)
         assert oracle.check(vals[0][rows], Cref, S, G.tol_for(cfg.out_dtype)).ok
+
+
+@pytest.mark.parametrize("name,variants", [
+    ("C2", ["umma2_n256", "umma2_n256_ts", "umma_n256_ts"]),
+    ("C5b", ["umma2_n256_ts", "umma_n256_ts", "umma_n128", "umma2_n256_sk2"]),
+    ("C5a", ["umma_n128", "umma_n256_sk2", "umma_n64_sk4"]),
+])
+def test_config_size_closed_form_on_named_variants(name, variants):
+    """The tile-splitting variants at full size: tail tiles cut along N, tiles cut
+    along K with in-kernel fix-up, CTA pairs.  Integer closed form, every element."""
+    cfg = gi.CONFIGS[name]
+    table = {B.variant_name(v): v for v in range(B.num_variants())}
+    u, v_, p, q = gi.rank1_int_factors(cfg.M, cfg.N, cfg.K, seed=cfg.seed + 70)
+    A = gi.embed(gi.int_to_bf16_bits(np.outer(u, p)), cfg.lda_)
+    Bm = gi.embed(gi.int_to_bf16_bits(np.outer(q, v_)), cfg.ldb_)
+    exact = np.outer(u, v_).astype(np.float64) * float(np.dot(p, q))
+    for vn in variants:
+        vals, raw = _run(cfg, A, Bm, table[vn])
+        if cfg.out_dtype == gi.F32:
+            assert np.array_equal(vals[0], exact), vn
+        else:
+            want = oracle.f64_to_bf16_bits(exact)
+            assert ((raw[0] == want) | ((exact == 0) & (vals[0] == 0))).all(), vn

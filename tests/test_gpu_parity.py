@@ -49,7 +49,8 @@ def test_shape_grid(M):
     on the automatic choice, the CUDA-core kernel and one tcgen05 variant per
     tile width (plus a split-K one where K allows)."""
     rng = np.random.default_rng(1000 + M)
-    names = ["simt", "umma_n64", "umma_n128", "umma_n256", "umma_n64_sk2", "umma_n256_sk4"]
+    names = ["simt", "umma_n64", "umma_n128", "umma_n256", "umma_n64_sk2", "umma_n256_sk4",
+             "umma2_n256", "umma2_n256_sk2", "umma_n256_ts", "umma2_n256_ts"]
     for ni, N in enumerate(DIMS):
         for ki in range(3):
             K = KS[(ni * 3 + ki + M) % len(KS)]
@@ -73,7 +74,7 @@ def test_padded_leading_dimensions_and_offset_bases(pad, out_dtype):
         ref = oracle.gemm(A, Bm, M, N, K)
         lda, ldb, ldc = K + pad, N + pad, N + pad
         Ap, Bp = gi.embed(A, lda), gi.embed(Bm, ldb)       # NaN padding: reading it poisons C
-        for v in [B.VARIANT_AUTO] + variant_ids("simt", "umma_n128", "umma_n256_sk2"):
+        for v in [B.VARIANT_AUTO] + variant_ids("simt", "umma_n128", "umma_n256_sk2", "umma2_n256", "umma2_n256_ts"):
             if v >= 0 and B.variant_supports(v, M, N, K, lda, ldb, ldc, 1, out_dtype) != 1:
                 continue
             check_case(Ap, Bp, M, N, K, out_dtype, v, lda, ldb, ldc, ref=ref)
@@ -109,7 +110,8 @@ def test_batched(batch, out_dtype):
         cfgA = gi.random_operand(batch * 7 + M, 0, M, K, lda, batch=batch, stride=sA)
         cfgB = gi.random_operand(batch * 7 + M, 1, K, N, ldb, batch=batch, stride=sB)
         Cref, S = oracle.gemm_batched(cfgA, cfgB, M, N, K, lda, ldb, sA, sB, batch)
-        for v in [B.VARIANT_AUTO] + variant_ids("simt", "umma_n64", "umma_n128", "umma_n128_sk2"):
+        for v in [B.VARIANT_AUTO] + variant_ids("simt", "umma_n64", "umma_n128", "umma_n128_sk2", "umma2_n256",
+                                                "umma2_n256_sk2", "umma_n128_ts", "umma2_n256_ts"):
             if v >= 0 and B.variant_supports(v, M, N, K, lda, ldb, ldc, batch, out_dtype) != 1:
                 continue
             vals, raw, guards = G.run_gemm(cfgA, cfgB, M, N, K, lda, ldb, ldc, out_dtype, batch,
@@ -215,7 +217,8 @@ def test_power_of_two_scaling_bitwise_and_run_to_run_identical():
     M, N, K = 260, 390, 777
     A = bits(rng.standard_normal((M, K))); Bm = bits(rng.standard_normal((K, N)))
     for out_dtype in (gi.F32, gi.BF16):
-        for v in [B.VARIANT_AUTO] + variant_ids("umma_n128", "umma_n256_sk4", "umma_n64_sk8"):
+        for v in [B.VARIANT_AUTO] + variant_ids("umma_n128", "umma_n256_sk4", "umma_n64_sk8", "umma2_n256_sk4",
+                                                "umma2_n256_ts"):
             _, raw0, _ = G.run_gemm(A.ravel(), Bm.ravel(), M, N, K, K, N, N, out_dtype, variant=v)
             _, raw1, _ = G.run_gemm(A.ravel(), Bm.ravel(), M, N, K, K, N, N, out_dtype, variant=v)
             assert np.array_equal(raw0, raw1)                       # deterministic
