@@ -146,17 +146,17 @@ size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K,
  * Its scratch is an array compiled into the library's device image
  * (CUDALLM_NOALLOC_SCRATCH_BYTES, 8 MiB, resident on every GPU that loads the
  * library until the process exits).  C is cut into tiles of 128 x 64 and each
- * tile's K range into `split_k` parts (2, 4, 8 or 16, at most ceil(K/64));
- * split_k - 1 of them leave an fp32 partial tile of 32 KiB in that array and
- * the last one adds them in fixed order and writes C.
+ * tile's K range into `split_k` parts (2, 4, 8 or 16, at most ceil(K/64)) that
+ * run as separate units; the units of a tile exchange their fp32 partial sums
+ * through 32 KiB slots of that array, add them in fixed order and write C.
  *
  *  - A, B, C, sizes, leading dimensions and out_dtype as cudallm_gemm_bf16.
  *    A and B must take the direct TMA path: 16-byte aligned bases, lda and ldb
  *    multiples of 8 (else CUDALLM_ERR_UNSUPPORTED_SHAPE; repacking would need
  *    more scratch).
- *  - Limit: P = ceil(M/128) * ceil(N/64) * (split_k - 1) partial tiles; the
- *    call needs P <= 4080 and CUDALLM_NOALLOC_HEADER_BYTES + P * 32 KiB <=
- *    CUDALLM_NOALLOC_SCRATCH_BYTES (P <= 253), else it returns
+ *  - Limit: P = ceil(M/128) * ceil(N/64) * split_k slots of 32 KiB must fit
+ *    behind the header: CUDALLM_NOALLOC_HEADER_BYTES + P * 32 KiB <=
+ *    CUDALLM_NOALLOC_SCRATCH_BYTES, i.e. P <= 254; else the call returns
  *    CUDALLM_ERR_TOO_LARGE and nothing runs.
  *  - The call SYNCHRONISES `stream` before it returns and reports a kernel
  *    whose bounded wait ran out as CUDALLM_ERR_DEVICE_TIMEOUT.

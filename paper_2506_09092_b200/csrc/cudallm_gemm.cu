@@ -77,7 +77,7 @@ inline bool is_empty(const Problem &p) { return p.M == 0 || p.N == 0 || p.batch 
 
 // ---------------------------------------------------------------- variants --
 enum Family { kSimt = 0, kUmma = 1, kUmmaPair = 2 };
-constexpr int kTailSplit = 0;          // Variant::split_k value: cut the ragged last wave's tiles along N
+constexpr int kTailSplit = 0;          // Variant::split_k value: split only the tiles of the ragged last wave
 struct Variant {
     char name[32];
     Family family;
@@ -136,9 +136,8 @@ struct Tiling {
     int64_t tiles_m, tiles_n, tiles, kblocks;
     int64_t dp_tiles;        // leading tiles that are one unit each
     int split;               // K parts per remaining tile
-    int nsplit;              // N parts per remaining tile (never together with split > 1)
-    int64_t units;           // dp_tiles + (tiles - dp_tiles) * split * nsplit
-    int64_t helper_tiles;    // partial tiles in the workspace: (tiles - dp_tiles) * (split - 1) * CTAs per tile
+    int64_t units;           // dp_tiles + (tiles - dp_tiles) * split
+    int64_t helper_tiles;    // partial tiles in the workspace: (tiles - dp_tiles) * split * CTAs per tile
     int64_t partial_bytes;
 };
 
@@ -153,25 +152,24 @@ Tiling tiling_for(const Variant &v, const Problem &p, int slots)
     t.tiles = t.tiles_m * t.tiles_n * p.batch;
     t.kblocks = cdiv(p.K, kBlockK);
     t.split = 1;
-    t.nsplit = 1;
     t.dp_tiles = t.tiles;
     if (v.split_k == kTailSplit) {
-        // Cut the tiles of the ragged last wave into narrower ones (64-column
-        // granularity per CTA) so that they fill the grid about once.
+        // Split the tiles of the ragged last wave along K so that they fill the
+        // grid about once: up to 4 parts, each at least 8 k-blocks deep.
         const int64_t tail = t.tiles % slots;
-        const int max_parts = pair ? 2 : v.block_n / 64;
-        int parts = 1;
-        while (tail > 0 && parts * 2 <= max_parts && tail * parts * 2 <= slots) parts *= 2;
+        int64_t parts = tail > 0 ? slots / tail : 1;
+        if (parts > 4) parts = 4;
+        while (parts > 1 && t.kblocks / parts < 8) --parts;
         if (parts > 1) {
-            t.nsplit = parts;
+            t.split = (int)parts;
             t.dp_tiles = t.tiles - tail;
         }
     } else if (v.split_k > 1) {
         t.split = v.split_k;
         t.dp_tiles = 0;
     }
-    t.units = t.dp_tiles + (t.tiles - t.dp_tiles) * t.split * t.nsplit;
-    t.helper_tiles = (t.tiles - t.dp_tiles) * (t.split - 1) * (pair ? 2 : 1);
+    t.units = t.dp_tiles + (t.tiles - t.dp_tiles) * t.split;
+    t.helper_tiles = t.split > 1 ? (t.tiles - t.dp_tiles) * t.split * (pair ? 2 : 1) : 0;
     t.partial_bytes = t.helper_tiles * int64_t(kBlockM) * v.block_n * 4;
     return t;
 }
@@ -214,20 +212,15 @@ double variant_cost(const Variant &v, const Problem &p)
     const double full_main = (double)t.kblocks * per_kb;
     const double dp_rounds = (double)cdiv(t.dp_tiles, slots);
     double compute = dp_rounds * (full_main > epi ? full_main : epi);
-    if (t.nsplit > 1) {
-        // narrower tiles: fewer MMA clocks per k-block, same A traffic
-        const double rounds = (double)cdiv((t.tiles - t.dp_tiles) * t.nsplit, slots);
-        const int w = v.block_n / t.nsplit;
-        const double narrow = (double)t.kblocks * (pair ? 300.0 + 0.83 * w : 300.0 + 0.83 * w);
-        compute += rounds * narrow;
-    }
     if (t.split > 1) {
         const double split_units = (double)(t.tiles - t.dp_tiles) * t.split;
         const double rounds = (double)cdiv((int64_t)split_units, slots);
         const double part_main = (double)cdiv(t.kblocks, t.split) * per_kb;
-        // measured: an owner spends about 8 us (15000 clocks) per helper tile it adds
-        const double fix = (t.split - 1) * 15000.0;
-        compute += rounds * (part_main > epi + fix ? part_main : epi + fix) + fix;
+        // exchange of partial chunks between the units of a tile: each unit writes
+        // and reads (S-1)/S of a tile through L2; measured a few microseconds per
+        // unit, growing with the number of partners
+        const double fix = 2500.0 + (t.split - 1) * 3500.0;
+        compute += rounds * (part_main + fix);
     }
     compute += epi;
     const double hbm = 3500.0;                         // bytes per clock: ~6.5 TB/s at ~1.9 GHz
@@ -506,7 +499,6 @@ GemmParams make_params(const Problem &p, const Tiling &t, int a_box_rows)
     gp.kblocks = (int)t.kblocks;
     gp.dp_tiles = (int)t.dp_tiles;
     gp.split_k = t.split;
-    gp.tail_nsplit = t.nsplit;
     gp.num_units = (int)t.units;
     const int64_t vec = (p.out_dtype == CUDALLM_F32) ? 4 : 8;
     gp.c_vec_ok = (reinterpret_cast<uintptr_t>(p.C) % 16 == 0) && (p.ldc % vec == 0)

@@ -11,20 +11,17 @@
 //
 // Work is cut into units; CTA b runs units b, b+grid, ... in that order.  The
 // first dp_tiles tiles are one unit each.  Every later tile is cut along K into
-// split_k units with consecutive indices: the first split_k-1 ("helpers") write
-// their fp32 partial tile to the workspace and raise a flag; the last one (the
-// "owner") waits for those flags, adds the partial tiles to its own accumulator
-// in split order 0..S-2 -- a fixed order, so results are reproducible -- and
-// stores C, rounding once.  A unit only ever waits for units with smaller
-// indices, which run earlier on the same CTA or on other CTAs, so the waits
-// cannot form a cycle; they are bounded like every other wait in the kernel.
-// dp_tiles = 0 is plain split-K.
-//
-// Tiles >= dp_tiles can instead be cut along N into tail_nsplit narrower units
-// (BLOCK_N / tail_nsplit columns each, no partial sums needed): with dp_tiles =
-// tiles - tiles % grid this makes the ragged last wave of a launch take about
-// 1/tail_nsplit of a tile's time.  The MMA's N, the number of B boxes and the
-// epilogue's column count are per-unit values for that reason.
+// split_k units with consecutive indices, and its 32-column chunks are dealt
+// round-robin to those units: unit j owns chunk c iff c mod split_k == j.  In
+// its epilogue a unit first writes the chunks it does not own (its fp32 partial
+// sums) to the workspace and raises a flag; then, for each chunk it owns, it
+// waits for the other units' flags, adds the partial chunks in split order
+// 0..S-1 -- a fixed order, so results are reproducible -- and stores C, rounding
+// once.  The units of a tile thus exchange data among themselves; a unit never
+// waits for a tile with a larger index, so the waits cannot form a cycle, and
+// they are bounded like every other wait in the kernel.
+// dp_tiles = 0 is plain split-K; dp_tiles = tiles - tiles % grid splits only the
+// ragged last wave of a launch so that it takes about 1/split_k of a tile's time.
 #pragma once
 #include "ptx.cuh"
 
@@ -48,13 +45,12 @@ struct GemmParams {
     int kblocks;            // ceil(K / 64)
     int dp_tiles;           // leading tiles that are not split
     int split_k;            // K parts per tile for tiles >= dp_tiles (1 = none), <= kblocks
-    int tail_nsplit;        // N parts per tile for tiles >= dp_tiles (1 = none); not with split_k > 1
-    int num_units;          // dp_tiles + (tiles - dp_tiles) * split_k * tail_nsplit
+    int num_units;          // dp_tiles + (tiles - dp_tiles) * split_k
     int c_vec_ok;           // C base, ldc, strideC allow 16-byte stores
     int a_box_bytes;        // bytes one TMA box of A delivers (box rows * 128)
     int epoch;              // value that marks a flag as raised in this launch (never 0)
-    float *partials;        // helper partial tiles (workspace), 128 x BLOCK_N fp32 each
-    int *flags;             // one per (helper partial tile, epilogue warp) (workspace)
+    float *partials;        // partial tiles of split units (workspace), 128 x BLOCK_N fp32 each
+    int *flags;             // one per (partial tile, epilogue warp) (workspace)
     int *status;            // [0] = code, [1] = detail
 };
 
@@ -78,45 +74,32 @@ __device__ __forceinline__ void report_timeout(int *status, int role, int what)
 }
 
 struct UnitCoord {
-    int m_tile, b;
-    int n0, width;          // first column and number of columns (multiple of 64) of this unit
+    int m_tile, n_tile, b;
     int split, nsplit;      // this unit's part of K and how many parts its tile has
-    int helper_index;       // (tile - dp_tiles) * (split_k - 1): first partial tile of this unit's tile
+    int slot0;              // (tile - dp_tiles) * split_k: partial-tile index of this tile's split 0
     int kb_begin, kb_end;
 };
 
-template <int BLOCK_N>
 __device__ __forceinline__ UnitCoord decode_unit(const GemmParams &p, int u)
 {
     UnitCoord c;
     int t;
-    int part = 0;
-    c.width = BLOCK_N;
     if (u < p.dp_tiles) {
         t = u;
         c.split = 0;
         c.nsplit = 1;
-        c.helper_index = 0;
-    } else if (p.tail_nsplit > 1) {
-        const int r = u - p.dp_tiles;
-        const int ts = r / p.tail_nsplit;
-        t = p.dp_tiles + ts;
-        part = r - ts * p.tail_nsplit;
-        c.width = BLOCK_N / p.tail_nsplit;
-        c.split = 0;
-        c.nsplit = 1;
-        c.helper_index = 0;
+        c.slot0 = 0;
     } else {
         const int r = u - p.dp_tiles;
         const int ts = r / p.split_k;
         t = p.dp_tiles + ts;
         c.split = r - ts * p.split_k;
         c.nsplit = p.split_k;
-        c.helper_index = ts * (p.split_k - 1);
+        c.slot0 = ts * p.split_k;
     }
     c.m_tile = t % p.tiles_m;
     t /= p.tiles_m;
-    c.n0 = (t % p.tiles_n) * BLOCK_N + part * c.width;
+    c.n_tile = t % p.tiles_n;
     c.b = t / p.tiles_n;
     c.kb_begin = static_cast<int>((static_cast<long long>(p.kblocks) * c.split) / c.nsplit);
     c.kb_end = static_cast<int>((static_cast<long long>(p.kblocks) * (c.split + 1)) / c.nsplit);
@@ -197,36 +180,36 @@ __device__ __forceinline__ void store_row_chunk(void *row_ptr, const float (&v)[
 // first column, `quad`/`lane` identify the thread (row within the tile =
 // 32*quad + lane), `cta_slot` = index of this CTA among the CTAs that share a
 // tile (0 for lone CTAs, the cluster rank for pairs) and `ctas_per_tile` their
-// number.  Reads the BLOCK_N accumulator columns 32 at a time and
-//   - stores them to C (unsplit tile),
-//   - or writes them to this helper's partial tile and raises its flag,
-//   - or (owner) adds the helpers' partial tiles in split order and stores C.
+// number.  Works on the BLOCK_N accumulator columns 32 at a time (a "chunk").
 // Partial tile layout: float4 index ((chunk*8 + q) * 128 + row_in_tile), so
-// that a warp writes and reads 512 contiguous bytes.
+// that a warp writes and reads 512 contiguous bytes.  Returns false if a wait
+// for another unit's flag ran out.
 template <int BLOCK_N, bool OUT_BF16>
 __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoord &c, int row,
                                               uint32_t t_addr, int quad, int lane, int cta_slot,
                                               int ctas_per_tile, volatile int *abort_flag)
 {
     constexpr int kTileF4 = kBlockM * BLOCK_N / 4;
+    constexpr int kChunks = BLOCK_N / 32;
     const bool row_ok = row < p.M;
     const int row_in_tile = quad * 32 + lane;
-    const bool helper = c.split + 1 < c.nsplit;
-    const bool owner = c.nsplit > 1 && !helper;
+    const int S = c.nsplit;
     bool ok = true;
 
-    if (helper) {
-        const long long slot = static_cast<long long>(c.helper_index + c.split) * ctas_per_tile + cta_slot;
-        float4 *part = reinterpret_cast<float4 *>(p.partials) + slot * kTileF4;
+    if (S > 1) {
+        // 1. hand the chunks other units own to them
+        const long long my_slot = static_cast<long long>(c.slot0 + c.split) * ctas_per_tile + cta_slot;
+        float4 *mine = reinterpret_cast<float4 *>(p.partials) + my_slot * kTileF4;
 #pragma unroll 1
-        for (int ch = 0; ch < c.width / 32; ++ch) {
+        for (int ch = 0; ch < kChunks; ++ch) {
+            if (ch % S == c.split) continue;
             uint32_t r[32];
             tmem_ld_32x32b_x32(t_addr + ch * 32, r);
             tmem_ld_wait();
             if (row_ok) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
-                    __stcg(part + (ch * 8 + q) * kBlockM + row_in_tile,
+                    __stcg(mine + (ch * 8 + q) * kBlockM + row_in_tile,
                            make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
                                        __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3])));
             }
@@ -234,44 +217,57 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
         }
         __threadfence();
         __syncwarp();
-        if (lane == 0) st_release_gpu(p.flags + slot * 4 + quad, p.epoch);
-        return true;
+        if (lane == 0) st_release_gpu(p.flags + my_slot * 4 + quad, p.epoch);
+        if (c.split >= kChunks) return true;             // this unit owns no chunk
+        // 2. the same epilogue warp of every other unit wrote the rows this warp needs
+        for (int s = 0; s < S; ++s) {
+            if (s == c.split) continue;
+            const long long slot = static_cast<long long>(c.slot0 + s) * ctas_per_tile + cta_slot;
+            ok = wait_flag(p.flags + slot * 4 + quad, p.epoch, abort_flag) && ok;
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        __threadfence();
     }
 
     const long long off = static_cast<long long>(c.b) * p.strideC + static_cast<long long>(row) * p.ldc;
     void *row_ptr = OUT_BF16 ? static_cast<void *>(reinterpret_cast<__nv_bfloat16 *>(p.C) + off)
                              : static_cast<void *>(reinterpret_cast<float *>(p.C) + off);
     const bool vec_ok = p.c_vec_ok != 0;
-    if (owner) {
-        // the same epilogue warp of every helper wrote the rows this warp needs
-        for (int s = 0; s + 1 < c.nsplit; ++s) {
-            const long long slot = static_cast<long long>(c.helper_index + s) * ctas_per_tile + cta_slot;
-            ok = wait_flag(p.flags + slot * 4 + quad, p.epoch, abort_flag) && ok;
-        }
-        ok = __all_sync(0xffffffffu, ok);
-        __threadfence();
-    }
+    const float4 *tile0 = reinterpret_cast<const float4 *>(p.partials)
+                        + (static_cast<long long>(c.slot0) * ctas_per_tile + cta_slot) * kTileF4;
 #pragma unroll 1
-    for (int ch = 0; ch < c.width / 32; ++ch) {
+    for (int ch = (S > 1 ? c.split : 0); ch < kChunks; ch += S) {
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_addr + ch * 32, r);
         tmem_ld_wait();
         if (row_ok) {
             float v[32];
+            if (S == 1) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            if (owner) {
-                for (int s = 0; s + 1 < c.nsplit; ++s) {
-                    const long long slot = static_cast<long long>(c.helper_index + s) * ctas_per_tile + cta_slot;
-                    const float4 *part = reinterpret_cast<const float4 *>(p.partials) + slot * kTileF4;
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+            } else {
+                // sum over the splits in index order; this unit's own term comes from TMEM
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 t = __ldcg(part + (ch * 8 + q) * kBlockM + row_in_tile);
-                        v[4 * q] += t.x; v[4 * q + 1] += t.y; v[4 * q + 2] += t.z; v[4 * q + 3] += t.w;
+                for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                for (int s = 0; s < S; ++s) {
+                    if (s == c.split) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(r[j]);
+                    } else {
+                        const float4 *part = tile0 + static_cast<long long>(s) * ctas_per_tile * kTileF4
+                                           + (ch * 8) * kBlockM + row_in_tile;
+                        float4 t[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) t[q] = __ldcg(part + q * kBlockM);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            v[4 * q] += t[q].x; v[4 * q + 1] += t[q].y;
+                            v[4 * q + 2] += t[q].z; v[4 * q + 3] += t[q].w;
+                        }
                     }
                 }
             }
-            store_row_chunk<OUT_BF16>(row_ptr, v, c.n0 + ch * 32, p.N, vec_ok);
+            store_row_chunk<OUT_BF16>(row_ptr, v, c.n_tile * BLOCK_N + ch * 32, p.N, vec_ok);
         }
         __syncwarp();                                    // tcgen05.ld needs the whole warp
     }
@@ -334,8 +330,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             bool ok = true;
             uint32_t tok = 1;                            // the first STAGES stages start out free
             for (int u = blockIdx.x; ok && u < p.num_units; u += gridDim.x) {
-                const UnitCoord c = decode_unit<BLOCK_N>(p, u);
-                const int boxes = c.width / 64;
+                const UnitCoord c = decode_unit(p, u);
+                constexpr int boxes = BLOCK_N / 64;
                 for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
                     if (!tok && !mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) {
                         report_timeout(p.status, kRoleProducer, stage);
@@ -349,7 +345,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     tok = tma_stage_step<false>(empty_bar(nstage), nphase ^ 1, full_bar(stage), 1,
                                                 p.a_box_bytes + boxes * (64 * kBlockK * 2), full_bar(stage),
                                                 &tmap_a, &tmap_b, sa, sa + L::kABytes, kb * kBlockK,
-                                                c.m_tile * kBlockM, c.n0, c.b, boxes, 1, 0);
+                                                c.m_tile * kBlockM, c.n_tile * BLOCK_N, c.b, boxes, 1, 0);
                     stage = nstage;
                     phase = nphase;
                 }
@@ -365,8 +361,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             bool ok = true;
             uint32_t tok = 0;                            // answer of the probe of full[stage]
             for (int u = blockIdx.x; ok && u < p.num_units; u += gridDim.x) {
-                const UnitCoord c = decode_unit<BLOCK_N>(p, u);
-                const uint32_t idesc = make_idesc_bf16(kBlockM, c.width, 0, 1);
+                const UnitCoord c = decode_unit(p, u);
+                constexpr uint32_t idesc = make_idesc_bf16(kBlockM, BLOCK_N, 0, 1);
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag)) {
                     report_timeout(p.status, kRoleMma, 0x40 + acc);
                     break;
@@ -406,7 +402,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int u = blockIdx.x; u < p.num_units; u += gridDim.x) {
-            const UnitCoord c = decode_unit<BLOCK_N>(p, u);
+            const UnitCoord c = decode_unit(p, u);
             bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {

@@ -141,9 +141,9 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
             uint32_t tok = 1;                            // the first STAGES stages start out free
             const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
             for (int u = pair; ok && u < p.num_units; u += num_pairs) {
-                const UnitCoord c = decode_unit<kPairN>(p, u);
-                const int half = c.width / 2;            // columns of B this CTA stages: 128 or 64
-                const int boxes = half / 64;
+                const UnitCoord c = decode_unit(p, u);
+                constexpr int half = kPairN / 2;         // columns of B this CTA stages
+                constexpr int boxes = half / 64;
                 for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
                     if (!tok && !mbar_wait<true>(empty_bar(stage), phase ^ 1, abort_flag)) {
                         report_timeout(p.status, kRoleProducer, stage);
@@ -160,7 +160,7 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                                leader_full0 + 8u * stage, &tmap_a, &tmap_b, sa,
                                                sa + L::kABytes, kb * kBlockK,
                                                c.m_tile * kPairM + static_cast<int>(rank) * kBlockM,
-                                               c.n0 + static_cast<int>(rank) * half, c.b, boxes, nsub,
+                                               c.n_tile * kPairN + static_cast<int>(rank) * half, c.b, boxes, nsub,
                                                L::kSubBytes);
                     stage = nstage;
                     phase = nphase;
@@ -182,8 +182,8 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
             const uint32_t tfull0_cta0 = map_to_cta(tfull_bar(0), 0);
             const uint32_t tfull0_cta1 = map_to_cta(tfull_bar(0), 1);
             for (int u = pair; ok && u < p.num_units; u += num_pairs) {
-                const UnitCoord c = decode_unit<kPairN>(p, u);
-                const uint32_t idesc = make_idesc_bf16(kPairM, c.width, 0, 1);
+                const UnitCoord c = decode_unit(p, u);
+                constexpr uint32_t idesc = make_idesc_bf16(kPairM, kPairN, 0, 1);
                 if (!mbar_wait<true>(tempty_bar(acc), acc_phase ^ 1, abort_flag)) {
                     report_timeout(p.status, kRoleMma, 0x40 + acc);
                     break;
@@ -221,7 +221,7 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int u = pair; u < p.num_units; u += num_pairs) {
-            const UnitCoord c = decode_unit<kPairN>(p, u);
+            const UnitCoord c = decode_unit(p, u);
             bool ok = mbar_wait<true>(tfull_bar(acc), acc_phase, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
