@@ -237,6 +237,7 @@ def run_ours(args):
     from paper_2506_09092_b200 import binding as B
     from paper_2506_09092_b200 import harness as H
     from paper_2506_09092_b200 import inputs as gi
+    from paper_2506_09092_b200 import sharding
 
     rank, local, world = dist_env()
     if not torch.cuda.is_available():
@@ -265,11 +266,8 @@ def run_ours(args):
     code, detail = B.device_status(stream)
     if code != 0:
         raise RuntimeError(f"device status {code} detail {detail:#x}")
-    t = torch.tensor([total], dtype=torch.float64, device="cuda")
-    if use_dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_max = float(t.item())
-    value = world * cfg.flops * args.steps / total_max / 1e12
+    total_max = sharding.max_over_ranks(total, device="cuda")
+    value = sharding.aggregate_throughput(cfg.flops * args.steps, world, total_max) / 1e12
     kern_avg = sum(per) / len(per)
     achieved = cfg.flops / kern_avg / 1e12
     n_launch = launches_per_call(B, cfg, vname)
@@ -286,10 +284,8 @@ def run_ours(args):
         B.gemm_bf16_host(hA, hB, hC, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_,
                          cfg.out_dtype, stage, need, stream)
     e2e_total, _ = time_steps(e2e_call, e2e_steps, 2, barrier)
-    t = torch.tensor([e2e_total], dtype=torch.float64, device="cuda")
-    if use_dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_value = world * cfg.flops * e2e_steps / float(t.item()) / 1e12
+    e2e_value = sharding.aggregate_throughput(cfg.flops * e2e_steps, world,
+                                              sharding.max_over_ranks(e2e_total, device="cuda")) / 1e12
 
     # ------------------------------------------- skinny HBM-bound workload --
     sk = gi.CONFIGS["C5a"]
@@ -315,7 +311,8 @@ def run_ours(args):
                 "inputs": "A, B ~ N(0,1) rounded to bf16, numpy default_rng([1,0]) / ([1,1])",
                 "l2": f"rotating {prob.nsets} operand/output sets ({prob.nsets * prob.set_bytes / 1e6:.0f} MB)"
                       f" > {L2_BYTES / 1e6:.0f} MB L2",
-                "sharding": "one replica of the workload per GPU (row shards of a taller product), no collective",
+                "sharding": f"rank r owns rows [{cfg.M}*r, {cfg.M}*(r+1)) of a {sharding.weak_scaling_rows(cfg.M, world)}-row product "
+                            "(B replicated), no data-path collective",
             },
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "TFLOP/s",

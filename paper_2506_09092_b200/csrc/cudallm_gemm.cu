@@ -496,6 +496,13 @@ GemmParams make_params(const Problem &p, const Tiling &t, int a_box_rows)
     gp.strideC = p.batch > 1 ? p.sC : 0;
     gp.M = (int)p.M; gp.N = (int)p.N; gp.K = (int)p.K; gp.batch = (int)p.batch;
     gp.tiles_m = (int)t.tiles_m; gp.tiles_n = (int)t.tiles_n;
+    // raster groups: as many tile rows as keep the group's slice of A within about 32 MB
+    // (half of what one L2 partition holds), so that it stays resident while B streams by
+    const int64_t tile_rows = cdiv(p.M, t.tiles_m);
+    int64_t group = (int64_t(32) << 20) / (tile_rows * p.K * 2 + 1);
+    if (group < 1) group = 1;
+    if (group > t.tiles_m) group = t.tiles_m;
+    gp.group_m = (int)group;
     gp.kblocks = (int)t.kblocks;
     gp.dp_tiles = (int)t.dp_tiles;
     gp.split_k = t.split;

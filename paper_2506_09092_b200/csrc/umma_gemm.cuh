@@ -42,6 +42,7 @@ struct GemmParams {
     long long strideC;      // elements between batch items
     int M, N, K, batch;
     int tiles_m, tiles_n;   // tiles per batch item
+    int group_m;            // tile rows per raster group (see decode_unit)
     int kblocks;            // ceil(K / 64)
     int dp_tiles;           // leading tiles that are not split
     int split_k;            // K parts per tile for tiles >= dp_tiles (1 = none), <= kblocks
@@ -97,10 +98,18 @@ __device__ __forceinline__ UnitCoord decode_unit(const GemmParams &p, int u)
         c.nsplit = p.split_k;
         c.slot0 = ts * p.split_k;
     }
-    c.m_tile = t % p.tiles_m;
-    t /= p.tiles_m;
-    c.n_tile = t % p.tiles_n;
-    c.b = t / p.tiles_n;
+    // Raster order inside a batch item: groups of group_m tile rows; inside a
+    // group the row index runs fastest, then the column.  The CTAs that run at
+    // the same time then share one slice of A (group_m tile rows, sized by the
+    // host to stay in L2) and a few column panels of B.
+    const int per_item = p.tiles_m * p.tiles_n;
+    c.b = t / per_item;
+    const int r = t - c.b * per_item;
+    const int g = r / (p.group_m * p.tiles_n);
+    const int r2 = r - g * p.group_m * p.tiles_n;
+    const int gm = min(p.group_m, p.tiles_m - g * p.group_m);
+    c.n_tile = r2 / gm;
+    c.m_tile = g * p.group_m + (r2 - c.n_tile * gm);
     c.kb_begin = static_cast<int>((static_cast<long long>(p.kblocks) * c.split) / c.nsplit);
     c.kb_end = static_cast<int>((static_cast<long long>(p.kblocks) * (c.split + 1)) / c.nsplit);
     return c;
