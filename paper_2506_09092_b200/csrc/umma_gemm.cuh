@@ -64,7 +64,8 @@ struct SmemLayout {
     // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
-    static constexpr int kBytes = kMiscOffset + 64;
+    static constexpr int kEpiOffset = (kMiscOffset + 64 + 15) / 16 * 16;
+    static constexpr int kBytes = kEpiOffset + 18432;    // + epilogue staging (kEpiStageBytes)
     static constexpr int kDynamicBytes = kBytes + 1024;  // slack for 1024-byte alignment
 };
 
@@ -143,45 +144,79 @@ __device__ __forceinline__ bool wait_flag(const int *flag, int epoch, volatile i
     }
 }
 
-// Store 32 consecutive fp32 accumulator values of one row, starting at column
-// col0 of an n_cols-wide matrix, to `row_ptr + col0` (fp32 or bf16 elements).
+// Shared-memory staging of the epilogue: one 32 x 32 fp32 block per epilogue
+// warp, rows 36 floats apart (conflict-free for the accesses below).
+constexpr int kEpiPitch = 36;
+constexpr int kEpiStageBytes = 4 * 32 * kEpiPitch * 4;
+static_assert(kEpiStageBytes == 18432, "SmemLayout reserves this many bytes");
+
+// Stores one 32 x 32 block of the accumulator (this warp's 32 rows, 32
+// consecutive columns from col0) to C.  Each thread arrives with the 32 values
+// of ITS row (v); writing them as they are would make every store instruction
+// touch 32 different rows.  The block is therefore transposed through shared
+// memory so that the lanes of a store instruction run along a row: 16-byte
+// stores covering whole 128-byte (fp32) or 64-byte (bf16) row segments when C's
+// alignment allows, else element stores that are still contiguous per row.
+// row0 = global row of lane 0; rows >= M and columns >= N are skipped.
 template <bool OUT_BF16>
-__device__ __forceinline__ void store_row_chunk(void *row_ptr, const float (&v)[32], int col0,
-                                                int n_cols, bool vec_ok)
+__device__ __forceinline__ void store_block_staged(const GemmParams &p, float *stage, const float (&v)[32],
+                                                   long long batch_off, int row0, int col0, int lane)
 {
-    const int n_left = n_cols - col0;
-    if (n_left <= 0) return;
-    if (OUT_BF16) {
-        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(row_ptr) + col0;
-        if (vec_ok && n_left >= 32) {
-            uint4 *d4 = reinterpret_cast<uint4 *>(dst);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint4 w;
-                w.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
-                w.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
-                w.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
-                w.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
-                d4[q] = w;
+    for (int q = 0; q < 8; ++q)
+        *reinterpret_cast<float4 *>(stage + lane * kEpiPitch + 4 * q) =
+            make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    __syncwarp();
+    const int rows = min(32, p.M - row0);                // > 0 for at least lane 0's row by construction
+    const bool full_cols = col0 + 32 <= p.N;
+    if (OUT_BF16) {
+        __nv_bfloat16 *C = reinterpret_cast<__nv_bfloat16 *>(p.C) + batch_off;
+        if (p.c_vec_ok && full_cols) {
+            // lane -> row r = 8 i + lane / 4, 8 columns from 8 * (lane % 4): one 16-byte store
+            const int piece = (lane & 3) * 8;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = 8 * i + (lane >> 2);
+                const float4 x = *reinterpret_cast<const float4 *>(stage + r * kEpiPitch + piece);
+                const float4 y = *reinterpret_cast<const float4 *>(stage + r * kEpiPitch + piece + 4);
+                if (r < rows) {
+                    uint4 w;
+                    w.x = pack_bf16x2(x.x, x.y); w.y = pack_bf16x2(x.z, x.w);
+                    w.z = pack_bf16x2(y.x, y.y); w.w = pack_bf16x2(y.z, y.w);
+                    *reinterpret_cast<uint4 *>(C + static_cast<long long>(row0 + r) * p.ldc + col0 + piece) = w;
+                }
             }
         } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (j < n_left) dst[j] = __float2bfloat16_rn(v[j]);
+            const bool col_ok = col0 + lane < p.N;
+#pragma unroll 4
+            for (int r = 0; r < 32; ++r) {
+                const float x = stage[r * kEpiPitch + lane];
+                if (r < rows && col_ok)
+                    C[static_cast<long long>(row0 + r) * p.ldc + col0 + lane] = __float2bfloat16_rn(x);
+            }
         }
     } else {
-        float *dst = reinterpret_cast<float *>(row_ptr) + col0;
-        if (vec_ok && n_left >= 32) {
-            float4 *d4 = reinterpret_cast<float4 *>(dst);
+        float *C = reinterpret_cast<float *>(p.C) + batch_off;
+        if (p.c_vec_ok && full_cols) {
+            // lane -> row r = 4 i + lane / 8, 4 columns from 4 * (lane % 8): one 16-byte store
+            const int piece = (lane & 7) * 4;
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-                d4[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            for (int i = 0; i < 8; ++i) {
+                const int r = 4 * i + (lane >> 3);
+                const float4 x = *reinterpret_cast<const float4 *>(stage + r * kEpiPitch + piece);
+                if (r < rows)
+                    *reinterpret_cast<float4 *>(C + static_cast<long long>(row0 + r) * p.ldc + col0 + piece) = x;
+            }
         } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (j < n_left) dst[j] = v[j];
+            const bool col_ok = col0 + lane < p.N;
+#pragma unroll 4
+            for (int r = 0; r < 32; ++r) {
+                const float x = stage[r * kEpiPitch + lane];
+                if (r < rows && col_ok) C[static_cast<long long>(row0 + r) * p.ldc + col0 + lane] = x;
+            }
         }
     }
+    __syncwarp();                                        // the block is reused for the next chunk
 }
 
 // Epilogue of one unit, called by the four epilogue warps.  `row` is this
@@ -196,7 +231,7 @@ __device__ __forceinline__ void store_row_chunk(void *row_ptr, const float (&v)[
 template <int BLOCK_N, bool OUT_BF16>
 __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoord &c, int row,
                                               uint32_t t_addr, int quad, int lane, int cta_slot,
-                                              int ctas_per_tile, volatile int *abort_flag)
+                                              int ctas_per_tile, volatile int *abort_flag, float *stage)
 {
     constexpr int kTileF4 = kBlockM * BLOCK_N / 4;
     constexpr int kChunks = BLOCK_N / 32;
@@ -238,47 +273,45 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
         __threadfence();
     }
 
-    const long long off = static_cast<long long>(c.b) * p.strideC + static_cast<long long>(row) * p.ldc;
-    void *row_ptr = OUT_BF16 ? static_cast<void *>(reinterpret_cast<__nv_bfloat16 *>(p.C) + off)
-                             : static_cast<void *>(reinterpret_cast<float *>(p.C) + off);
-    const bool vec_ok = p.c_vec_ok != 0;
+    const long long batch_off = static_cast<long long>(c.b) * p.strideC;
+    const int row0 = row - lane;                         // global row of this warp's lane 0
+    if (row0 >= p.M) return ok;                          // the whole warp is below the matrix
     const float4 *tile0 = reinterpret_cast<const float4 *>(p.partials)
                         + (static_cast<long long>(c.slot0) * ctas_per_tile + cta_slot) * kTileF4;
 #pragma unroll 1
     for (int ch = (S > 1 ? c.split : 0); ch < kChunks; ch += S) {
+        const int col0 = c.n_tile * BLOCK_N + ch * 32;
+        if (col0 >= p.N) break;                          // warp-uniform: nothing further to store
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_addr + ch * 32, r);
         tmem_ld_wait();
-        if (row_ok) {
-            float v[32];
-            if (S == 1) {
+        float v[32];
+        if (S == 1) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            } else {
-                // sum over the splits in index order; this unit's own term comes from TMEM
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+        } else {
+            // sum over the splits in index order; this unit's own term comes from TMEM
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = 0.f;
-                for (int s = 0; s < S; ++s) {
-                    if (s == c.split) {
+            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+            for (int s = 0; s < S; ++s) {
+                if (s == c.split) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(r[j]);
-                    } else {
-                        const float4 *part = tile0 + static_cast<long long>(s) * ctas_per_tile * kTileF4
-                                           + (ch * 8) * kBlockM + row_in_tile;
-                        float4 t[8];
+                    for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(r[j]);
+                } else if (row_ok) {
+                    const float4 *part = tile0 + static_cast<long long>(s) * ctas_per_tile * kTileF4
+                                       + (ch * 8) * kBlockM + row_in_tile;
+                    float4 t[8];
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) t[q] = __ldcg(part + q * kBlockM);
+                    for (int q = 0; q < 8; ++q) t[q] = __ldcg(part + q * kBlockM);
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            v[4 * q] += t[q].x; v[4 * q + 1] += t[q].y;
-                            v[4 * q + 2] += t[q].z; v[4 * q + 3] += t[q].w;
-                        }
+                    for (int q = 0; q < 8; ++q) {
+                        v[4 * q] += t[q].x; v[4 * q + 1] += t[q].y;
+                        v[4 * q + 2] += t[q].z; v[4 * q + 3] += t[q].w;
                     }
                 }
             }
-            store_row_chunk<OUT_BF16>(row_ptr, v, c.n_tile * BLOCK_N + ch * 32, p.N, vec_ok);
         }
-        __syncwarp();                                    // tcgen05.ld needs the whole warp
+        store_block_staged<OUT_BF16>(p, stage, v, batch_off, row0, col0, lane);
     }
     return ok;
 }
@@ -421,7 +454,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tc_fence_after();
             if (!epilogue_tile<BLOCK_N, OUT_BF16>(p, c, c.m_tile * kBlockM + epi_tid,
                                                   tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(quad * 32) << 16),
-                                                  quad, lane, 0, 1, abort_flag)) {
+                                                  quad, lane, 0, 1, abort_flag,
+                                                  reinterpret_cast<float *>(smem + L::kEpiOffset)
+                                                      + quad * 32 * kEpiPitch)) {
                 if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0xC0);
             }
             tc_fence_before();

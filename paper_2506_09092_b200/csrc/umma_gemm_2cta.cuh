@@ -77,7 +77,8 @@ struct PairSmemLayout {
     static constexpr int kBarOffset = STAGES * kStageBytes;
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
-    static constexpr int kBytes = kMiscOffset + 64;
+    static constexpr int kEpiOffset = (kMiscOffset + 64 + 15) / 16 * 16;
+    static constexpr int kBytes = kEpiOffset + kEpiStageBytes;
     static constexpr int kDynamicBytes = kBytes + 1024;
 };
 
@@ -231,7 +232,9 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tc_fence_after();
             if (!epilogue_tile<kPairN, OUT_BF16>(p, c, c.m_tile * kPairM + static_cast<int>(rank) * kBlockM + epi_tid,
                                                  tmem_base + acc * kPairN + (static_cast<uint32_t>(quad * 32) << 16),
-                                                 quad, lane, static_cast<int>(rank), 2, abort_flag)) {
+                                                 quad, lane, static_cast<int>(rank), 2, abort_flag,
+                                                 reinterpret_cast<float *>(smem + L::kEpiOffset)
+                                                     + quad * 32 * kEpiPitch)) {
                 if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0xC0);
             }
             tc_fence_before();
