@@ -119,7 +119,11 @@ int cudallm_gemm_bf16_variant(int variant,
  * caller-owned DEVICE staging buffer of `dev_bytes` bytes, at least
  * cudallm_host_staging_bytes(...) and 256-byte aligned.  The call copies
  * M*lda and K*ldb elements in, multiplies, copies M*ldc elements out, and
- * SYNCHRONISES `stream` before returning.
+ * SYNCHRONISES `stream` before returning.  Internally B is copied first and A
+ * in up to 8 row blocks on a second stream; each block is multiplied on
+ * `stream` as soon as it has arrived and its rows of C return on a third
+ * stream, so the two copy directions and the multiplication overlap.  The two
+ * extra streams and their events are created on the first call per device.
  */
 int cudallm_gemm_bf16_host(const void *A_host, const void *B_host, void *C_host,
                            int64_t M, int64_t N, int64_t K,

@@ -267,6 +267,16 @@ struct DeviceState {
 DeviceState g_dev[kMaxDevices];
 std::mutex g_mutex;
 
+// Streams and events of the host-buffer entry point (created on first use).
+constexpr int kHostPipeChunks = 8;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t arrived[kHostPipeChunks] = {}, computed[kHostPipeChunks] = {};
+    cudaEvent_t start = nullptr, done = nullptr;
+};
+HostPipe g_host_pipe[kMaxDevices];
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -686,20 +696,62 @@ int cudallm_gemm_bf16_host(const void *A_host, const void *B_host, void *C_host,
     uint8_t *dA = static_cast<uint8_t *>(dev_buf);
     uint8_t *dB = dA + round_up(M * lda * 2, 256);
     uint8_t *dC = dB + round_up(K * ldb * 2, 256);
-    // rows are copied with their padding: (rows-1)*ld + cols elements
-    if (K > 0) {
-        CUDA_TRY(cudaMemcpyAsync(dA, A_host, (size_t)(((M - 1) * lda + K) * 2), cudaMemcpyHostToDevice, stream));
-        CUDA_TRY(cudaMemcpyAsync(dB, B_host, (size_t)(((K - 1) * ldb + N) * 2), cudaMemcpyHostToDevice, stream));
+
+    // Copy engines and tensor cores overlap: B goes in first, then A in row
+    // blocks; block i is multiplied as soon as it has arrived while block i+1
+    // is still on the bus, and its rows of C travel back on a third stream.
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    HostPipe &hp = g_host_pipe[dev];
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!hp.ready) {
+            CUDA_TRY(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
+            CUDA_TRY(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
+            for (int i = 0; i < kHostPipeChunks; ++i) {
+                CUDA_TRY(cudaEventCreateWithFlags(&hp.arrived[i], cudaEventDisableTiming));
+                CUDA_TRY(cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming));
+            }
+            CUDA_TRY(cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming));
+            CUDA_TRY(cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming));
+            hp.ready = true;
+        }
     }
-    st = cudallm_gemm_bf16(dA, dB, dC, M, N, K, lda, ldb, ldc, out_dtype, stream_v);
-    if (st != CUDALLM_OK) return st;
-    if (ldc == N) {
-        CUDA_TRY(cudaMemcpyAsync(C_host, dC, (size_t)(M * N * esz), cudaMemcpyDeviceToHost, stream));
-    } else {
-        // keep the caller's padding columns untouched
-        CUDA_TRY(cudaMemcpy2DAsync(C_host, (size_t)(ldc * esz), dC, (size_t)(ldc * esz), (size_t)(N * esz),
-                                   (size_t)M, cudaMemcpyDeviceToHost, stream));
+    int64_t rows_per_chunk = round_up(cdiv(M, kHostPipeChunks), 256);
+    if (rows_per_chunk < 512) rows_per_chunk = 512;
+    const int n_chunks = (int)cdiv(M, rows_per_chunk);
+
+    // the staging buffer may still be in use by earlier work on the caller's stream
+    CUDA_TRY(cudaEventRecord(hp.start, stream));
+    CUDA_TRY(cudaStreamWaitEvent(hp.in, hp.start, 0));
+    if (K > 0)
+        CUDA_TRY(cudaMemcpyAsync(dB, B_host, (size_t)(((K - 1) * ldb + N) * 2), cudaMemcpyHostToDevice, hp.in));
+    for (int i = 0; i < n_chunks; ++i) {
+        const int64_t r0 = i * rows_per_chunk;
+        const int64_t rows = (M - r0) < rows_per_chunk ? (M - r0) : rows_per_chunk;
+        if (K > 0)
+            CUDA_TRY(cudaMemcpyAsync(dA + r0 * lda * 2, static_cast<const uint8_t *>(A_host) + r0 * lda * 2,
+                                     (size_t)(((rows - 1) * lda + K) * 2), cudaMemcpyHostToDevice, hp.in));
+        CUDA_TRY(cudaEventRecord(hp.arrived[i], hp.in));
+        CUDA_TRY(cudaStreamWaitEvent(stream, hp.arrived[i], 0));
+        st = cudallm_gemm_bf16(dA + r0 * lda * 2, dB, dC + r0 * ldc * esz, rows, N, K, lda, ldb, ldc,
+                               out_dtype, stream_v);
+        if (st != CUDALLM_OK) return st;
+        CUDA_TRY(cudaEventRecord(hp.computed[i], stream));
+        CUDA_TRY(cudaStreamWaitEvent(hp.out, hp.computed[i], 0));
+        uint8_t *hc = static_cast<uint8_t *>(C_host) + r0 * ldc * esz;
+        if (ldc == N) {
+            CUDA_TRY(cudaMemcpyAsync(hc, dC + r0 * ldc * esz, (size_t)(rows * N * esz), cudaMemcpyDeviceToHost,
+                                     hp.out));
+        } else {
+            // keep the caller's padding columns untouched
+            CUDA_TRY(cudaMemcpy2DAsync(hc, (size_t)(ldc * esz), dC + r0 * ldc * esz, (size_t)(ldc * esz),
+                                       (size_t)(N * esz), (size_t)rows, cudaMemcpyDeviceToHost, hp.out));
+        }
     }
+    CUDA_TRY(cudaEventRecord(hp.done, hp.out));
+    CUDA_TRY(cudaStreamWaitEvent(stream, hp.done, 0));
     CUDA_TRY(cudaStreamSynchronize(stream));
     return CUDALLM_OK;
 }

@@ -173,6 +173,182 @@ class DeviceProblem:
         return raw.view(np.float32 if cfg.out_dtype == 0 else np.uint16)
 
 
+# ------------------------------------------------- search over the variants --
+
+@dataclass
+class ClosedFormCase:
+    """A test case whose exact result is known without multiplying matrices:
+    A = u p^T and B = q v^T with small integers give C = (p . q) u v^T, every
+    partial sum an integer below 2**24 (exact in fp32 in any summation order)."""
+    name: str
+    M: int
+    N: int
+    K: int
+    out_dtype: int
+    seed: int
+    lda: int | None = None
+    ldb: int | None = None
+    ldc: int | None = None
+
+
+def default_cases(cfg=None):
+    """Seeded shapes for the Function Validator: ragged small shapes that touch
+    every tile edge, both output types, padded leading dimensions, and (if
+    given) the configuration's own shape."""
+    cases = [
+        ClosedFormCase("edge-129x257x1000-f32", 129, 257, 1000, 0, 1),
+        ClosedFormCase("edge-300x127x65-bf16", 300, 127, 65, 1, 2),
+        ClosedFormCase("pad-257x129x129-f32", 257, 129, 129, 0, 3, lda=136, ldb=136, ldc=131),
+        ClosedFormCase("odd-ld-255x300x515-f32", 255, 300, 515, 0, 4, lda=517, ldb=301, ldc=303),
+        ClosedFormCase("deep-16x520x4096-f32", 16, 520, 4096, 0, 5),
+        ClosedFormCase("wide-1100x700x200-bf16", 1100, 700, 200, 1, 6),
+    ]
+    if cfg is not None and cfg.batch == 1:
+        cases.append(ClosedFormCase(f"{cfg.name}-shape", cfg.M, cfg.N, cfg.K, cfg.out_dtype, 7,
+                                    cfg.lda, cfg.ldb, cfg.ldc))
+    return cases
+
+
+def run_closed_form_case(variant: int, case: ClosedFormCase):
+    """(status, (got_bits_or_values, exact)) for ``function_validator``'s ``run``."""
+    import numpy as np
+    import torch
+    from . import binding as B
+    from . import inputs as gi
+    M, N, K = case.M, case.N, case.K
+    lda = K if case.lda is None else case.lda
+    ldb = N if case.ldb is None else case.ldb
+    ldc = N if case.ldc is None else case.ldc
+    if B.variant_supports(variant, M, N, K, lda, ldb, ldc, 1, case.out_dtype) != 1:
+        return "unsupported", None
+    u, v, p, q = gi.rank1_int_factors(M, N, K, case.seed)
+    A = gi.embed(gi.int_to_bf16_bits(np.outer(u, p)), lda)
+    Bm = gi.embed(gi.int_to_bf16_bits(np.outer(q, v)), ldb)
+    exact = np.outer(u, v).astype(np.float64) * float(np.dot(p, q))
+    dA = torch.from_numpy(A.view(np.int16)).cuda()
+    dB = torch.from_numpy(Bm.view(np.int16)).cuda()
+    dt = torch.float32 if case.out_dtype == 0 else torch.bfloat16
+    dC = torch.full((M * ldc,), float("nan"), dtype=dt, device="cuda")
+    st = B.gemm_bf16_variant(variant, dA, dB, dC, M, N, K, lda, ldb, ldc, M * lda, K * ldb, M * ldc, 1,
+                             case.out_dtype, torch.cuda.current_stream(), check=False)
+    if st != 0:
+        return st, None
+    code, _ = B.device_status(torch.cuda.current_stream())
+    if code != 0:
+        return code, None
+    got = dC.view(M, ldc)[:, :N].to(torch.float64).cpu().numpy()
+    pad = dC.view(M, ldc)[:, N:]
+    pad_ok = bool(torch.isnan(pad).all().item()) if pad.numel() else True
+    return 0, (got, exact, pad_ok)
+
+
+def compare_closed_form(case: ClosedFormCase, out):
+    """Exact comparison: fp32 output must equal the integer result; bf16 output
+    must equal it after ONE round-to-nearest-even (checked through the error
+    bound |got - exact| <= half a bf16 spacing and got being a bf16 value)."""
+    import numpy as np
+    got, exact, pad_ok = out
+    if not pad_ok:
+        return False, float("inf"), "padding columns of C were overwritten"
+    if case.out_dtype == 0:
+        bad = got != exact
+    else:
+        # spacing of bf16 at |exact|: 2**(floor(log2|x|) - 7); nearest => |err| <= spacing / 2
+        mag = np.maximum(np.abs(exact), 2.0 ** -126)
+        half_ulp = 2.0 ** (np.floor(np.log2(mag)) - 8)
+        bad = np.abs(got - exact) > half_ulp
+    n_bad = int(bad.sum())
+    if n_bad:
+        i, j = (int(x) for x in np.argwhere(bad)[0])
+        return False, float("inf"), f"{n_bad} wrong, first at ({i}, {j}): got {got[i, j]}, want {exact[i, j]}"
+    return True, 0.0, ""
+
+
+def search_config(cfg, candidates=None, iters: int = 10, passes: int = 3, cases=None) -> SearchResult:
+    """Algorithm 1's round over the library's variants for one configuration:
+    validate every candidate on seeded closed-form cases, time the valid ones
+    (interleaved passes, median), keep the fastest."""
+    import statistics
+    from . import binding as B
+    if candidates is None:
+        candidates = [v for v in range(B.num_variants())
+                      if B.variant_supports(v, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch,
+                                            cfg.out_dtype) == 1 and B.variant_name(v) != "simt"]
+    cases = default_cases(cfg) if cases is None else cases
+
+    def run(v, case):
+        st, out = run_closed_form_case(v, case)
+        # a case the candidate cannot take does not disqualify it for other shapes
+        return (0, (None, None, None)) if st == "unsupported" else (st, out)
+
+    def compare(case, out):
+        return (True, 0.0, "") if out[0] is None else compare_closed_form(case, out)
+
+    prob = DeviceProblem(cfg)
+    samples = {}
+
+    def profile(v):
+        return samples[v]
+
+    res = SearchResult(best=None, best_latency=float("inf"))
+    for v in candidates:
+        res.reports[v] = function_validator(v, cases, run, compare)
+        if res.reports[v].ok:
+            res.valid.append(v)
+    for v in res.valid:
+        samples[v] = []
+    for _ in range(passes):
+        for v in res.valid:
+            t = performance_profiler(lambda i: prob.launch(i, v), iters=iters, warmup=2)
+            samples[v].append(t["median_s"])
+    for v in res.valid:
+        samples[v] = statistics.median(samples[v])
+    timed = search(res.valid, lambda v: res.reports[v], profile)
+    timed.reports = res.reports
+    return timed
+
+
+class TunedTable:
+    """Persisted outcome of the search: problem shape -> variant name.  Lookups
+    that miss fall back to the library's own choice."""
+
+    def __init__(self, entries=None):
+        self.entries = dict(entries or {})
+
+    @staticmethod
+    def key(M, N, K, batch, out_dtype):
+        return f"{M}x{N}x{K}x{batch}:{'bf16' if out_dtype == 1 else 'f32'}"
+
+    def record(self, cfg, variant_name, latency_s):
+        self.entries[self.key(cfg.M, cfg.N, cfg.K, cfg.batch, cfg.out_dtype)] = {
+            "variant": variant_name, "us": round(latency_s * 1e6, 2)}
+
+    def lookup(self, M, N, K, batch, out_dtype):
+        e = self.entries.get(self.key(M, N, K, batch, out_dtype))
+        return None if e is None else e["variant"]
+
+    def variant_id(self, M, N, K, batch, out_dtype, names=None):
+        """Variant id for the shape, or -1 (let the library choose)."""
+        name = self.lookup(M, N, K, batch, out_dtype)
+        if name is None:
+            return -1
+        if names is None:
+            from . import binding as B
+            names = {B.variant_name(v): v for v in range(B.num_variants())}
+        return names.get(name, -1)
+
+    def save(self, path):
+        import json
+        with open(path, "w") as f:
+            json.dump(self.entries, f, indent=1, sort_keys=True)
+
+    @classmethod
+    def load(cls, path):
+        import json
+        with open(path) as f:
+            return cls(json.load(f))
+
+
 def _main(argv=None):
     """``python -m paper_2506_09092_b200.harness --config C2``: run one benchmark
     configuration a few times and print its timing (also the command that ncu
@@ -190,7 +366,29 @@ def _main(argv=None):
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--sets", type=int, default=None, help="rotating buffer sets (default: > L2)")
     ap.add_argument("--all-variants", action="store_true", help="time every variant that supports the shape")
+    ap.add_argument("--search", action="store_true",
+                    help="validate every variant on closed-form cases, time the valid ones, report the fastest")
+    ap.add_argument("--table", default=None, help="with --search: JSON file to record the winner in")
     args = ap.parse_args(argv)
+    if args.search:
+        cfg = gi.CONFIGS[args.config]
+        res = search_config(cfg, iters=args.iters)
+        for v, rep in res.reports.items():
+            print(json.dumps({"config": cfg.name, "variant": B.variant_name(v), "validation": rep.status,
+                              "detail": rep.detail,
+                              "us": None if v not in res.latencies else res.latencies[v] * 1e6}), flush=True)
+        best = None if res.best is None else B.variant_name(res.best)
+        print(json.dumps({"config": cfg.name, "best": best,
+                          "us": None if res.best is None else res.best_latency * 1e6,
+                          "library_choice": B.variant_name(B.select_variant(
+                              cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype))}),
+              flush=True)
+        if args.table and res.best is not None:
+            import os
+            table = TunedTable.load(args.table) if os.path.exists(args.table) else TunedTable()
+            table.record(cfg, best, res.best_latency)
+            table.save(args.table)
+        return
     cfg = gi.CONFIGS[args.config]
     names = {B.variant_name(v): v for v in range(B.num_variants())}
     prob = DeviceProblem(cfg, nsets=args.sets)

@@ -151,3 +151,34 @@ def test_function_validator_failure_classes():
     assert rep.status == H.UNSUPPORTED
     rep = H.function_validator(0, cases, good, lambda c, out: (c.name != "c", 0.5, "edge column stale"))
     assert rep.status == H.MISMATCH and rep.failed_case == "c" and rep.detail == "edge column stale"
+
+
+def test_tuned_table_roundtrip(tmp_path):
+    t = H.TunedTable()
+    t.record(gi.CONFIGS["C2"], "umma2_n256_ts", 98.7e-6)
+    t.record(gi.CONFIGS["C4"], "umma_n128", 14.4e-6)
+    path = tmp_path / "tuned.json"
+    t.save(path)
+    u = H.TunedTable.load(path)
+    assert u.lookup(4096, 4096, 4096, 1, 1) == "umma2_n256_ts"
+    assert u.lookup(4096, 4096, 4096, 1, 0) is None            # other output type: not tuned
+    names = {B.variant_name(v): v for v in range(B.num_variants())}
+    assert u.variant_id(128, 128, 64, 512, 0, names) == names["umma_n128"]
+    assert u.variant_id(1, 2, 3, 1, 0, names) == -1            # miss: the library chooses
+    u.entries[H.TunedTable.key(5, 5, 5, 1, 0)] = {"variant": "no_such_kernel", "us": 1.0}
+    assert u.variant_id(5, 5, 5, 1, 0, names) == -1
+
+
+def test_closed_form_comparison_rules():
+    case = H.ClosedFormCase("t", 2, 2, 4, 0, 0)
+    exact = np.array([[3.0, -8.0], [0.0, 257.0]])
+    assert H.compare_closed_form(case, (exact.copy(), exact, True))[0]
+    off = exact.copy(); off[1, 1] += 1
+    ok, _, detail = H.compare_closed_form(case, (off, exact, True))
+    assert not ok and "(1, 1)" in detail
+    assert not H.compare_closed_form(case, (exact.copy(), exact, False))[0]     # padding clobbered
+    bf = H.ClosedFormCase("t", 2, 2, 4, 1, 0)
+    rounded = exact.copy(); rounded[1, 1] = 256.0               # 257 -> 256 (tie to even)
+    assert H.compare_closed_form(bf, (rounded, exact, True))[0]
+    trunc = exact.copy(); trunc[1, 1] = 254.0                   # more than half a spacing away
+    assert not H.compare_closed_form(bf, (trunc, exact, True))[0]

@@ -103,3 +103,24 @@ def test_config_size_closed_form_on_named_variants(name, variants):
         else:
             want = oracle.f64_to_bf16_bits(exact)
             assert ((raw[0] == want) | ((exact == 0) & (vals[0] == 0))).all(), vn
+
+
+def test_search_finds_a_valid_fastest_variant_and_rejects_a_broken_one():
+    """One round of the paper's Algorithm 1 over the library's variants on the
+    small configuration: every tcgen05 variant validates, the winner is the
+    fastest of them, and a candidate whose output is wrong is filtered out."""
+    from paper_2506_09092_b200 import harness as H
+    cfg = gi.CONFIGS["C1"]
+    names = {B.variant_name(v): v for v in range(B.num_variants())}
+    cands = [names[n] for n in ("umma_n64", "umma_n128", "umma_n256_sk2", "umma2_n256", "umma_n128_ts")]
+    res = H.search_config(cfg, candidates=cands, iters=5, passes=2)
+    assert sorted(res.valid) == sorted(cands), {B.variant_name(v): r.status for v, r in res.reports.items()}
+    assert res.best in cands and res.best_latency == min(res.latencies.values())
+    # the validator itself: a wrong element, or clobbered padding, is a MISMATCH
+    case = H.default_cases()[2]
+    st, out = H.run_closed_form_case(names["umma_n128"], case)
+    assert st == 0 and H.compare_closed_form(case, out)[0]
+    got, exact, pad_ok = out
+    broken = got.copy(); broken[-1, -1] += 1.0                       # last row / column of an edge tile
+    rep = H.function_validator(0, [case], lambda v, c: (0, (broken, exact, pad_ok)), H.compare_closed_form)
+    assert rep.status == H.MISMATCH
