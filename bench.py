@@ -119,21 +119,23 @@ def dist_env():
 
 
 def time_steps(launch, steps, warmup, barrier, sampler=None):
-    """W warm-up steps, then exactly ``steps`` timed steps with one CUDA event
-    between consecutive steps.  Returns (total seconds, per-step seconds list)."""
+    """W warm-up steps, then exactly ``steps`` timed steps between two CUDA
+    events on the launching stream (nothing else is enqueued in between, so
+    consecutive launches follow each other as they would in an application).
+    Returns (total seconds, average seconds per step)."""
     import torch
     for i in range(warmup):
         launch(i)
     torch.cuda.synchronize()
     barrier()
     torch.cuda.synchronize()
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if sampler:
         sampler.start()
-    evs[0].record()
+    e0.record()
     for i in range(steps):
         launch(warmup + i)
-        evs[i + 1].record()
+    e1.record()
     if sampler:
         sampler._poll_once() if sampler.nv is not None else None
     torch.cuda.synchronize()
@@ -141,9 +143,8 @@ def time_steps(launch, steps, warmup, barrier, sampler=None):
         sampler.stop()
     barrier()
     torch.cuda.synchronize()
-    total = evs[0].elapsed_time(evs[-1]) * 1e-3
-    per = [evs[i].elapsed_time(evs[i + 1]) * 1e-3 for i in range(steps)]
-    return total, per
+    total = e0.elapsed_time(e1) * 1e-3
+    return total, total / steps
 
 
 def launches_per_call(B, cfg, variant_name):
@@ -261,15 +262,14 @@ def run_ours(args):
     vname = B.variant_name(B.select_variant(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_,
                                             cfg.batch, cfg.out_dtype))
     sampler = ClockSampler(local)
-    total, per = time_steps(lambda i: prob.launch(i, stream=stream), args.steps, args.warmup,
-                            barrier, sampler)
+    total, kern_avg = time_steps(lambda i: prob.launch(i, stream=stream), args.steps, args.warmup,
+                                 barrier, sampler)
     code, detail = B.device_status(stream)
     if code != 0:
         raise RuntimeError(f"device status {code} detail {detail:#x}")
     total_max = sharding.max_over_ranks(total, device="cuda")
     value = sharding.aggregate_throughput(cfg.flops * args.steps, world, total_max) / 1e12
-    kern_avg = sum(per) / len(per)
-    achieved = cfg.flops / kern_avg / 1e12
+    achieved = cfg.flops / kern_avg / 1e12             # one kernel per step: step time = launch duration
     n_launch = launches_per_call(B, cfg, vname)
 
     # -------------------------------------------- e2e: host buffers, copies --
@@ -294,8 +294,7 @@ def run_ours(args):
     sk_name = B.variant_name(B.select_variant(sk.M, sk.N, sk.K, sk.lda_, sk.ldb_, sk.ldc_, sk.batch,
                                               sk.out_dtype))
     sk_steps = max(args.steps, 20)
-    sk_total, sk_per = time_steps(lambda i: skp.launch(i, stream=stream), sk_steps, args.warmup, barrier)
-    sk_avg = sum(sk_per) / len(sk_per)
+    sk_total, sk_avg = time_steps(lambda i: skp.launch(i, stream=stream), sk_steps, args.warmup, barrier)
     sk_gbs = sk.algorithmic_bytes / sk_avg / 1e9
 
     line = None

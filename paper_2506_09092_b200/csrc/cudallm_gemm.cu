@@ -396,6 +396,27 @@ int encode_operand_map(CUtensorMap *tm, const void *base, int64_t inner, int64_t
 }
 
 // ---------------------------------------------------------------- launches --
+// Launch with programmatic stream serialisation: the kernel may begin while the
+// previous kernel of the stream drains; it waits (griddepcontrol.wait) before it
+// touches global memory.
+template <typename Kernel>
+int launch_overlapped(Kernel kernel, int grid, int smem_bytes, cudaStream_t stream, const CUtensorMap &ta,
+                      const CUtensorMap &tb, const GemmParams &gp)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kNumThreads);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ta, tb, gp));
+    return CUDALLM_OK;
+}
+
 template <int BLOCK_N, int STAGES, bool OUT_BF16>
 int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &gp,
                 cudaStream_t stream)
@@ -413,9 +434,7 @@ int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb,
         d.smem_attr_set[slot] = true;
     }
     int grid = gp.num_units < d.sm_count ? gp.num_units : d.sm_count;
-    kernel<<<grid, kNumThreads, L::kDynamicBytes, stream>>>(ta, tb, gp);
-    CUDA_TRY(cudaGetLastError());
-    return CUDALLM_OK;
+    return launch_overlapped(kernel, grid, L::kDynamicBytes, stream, ta, tb, gp);
 }
 
 // Sets the pair kernel's shared-memory attribute and asks how many CTA pairs
@@ -461,9 +480,7 @@ int launch_umma_pair(int dev, const CUtensorMap &ta, const CUtensorMap &tb, cons
     auto kernel = umma_gemm_2cta_kernel<STAGES, KSUB, OUT_BF16>;
     DeviceState &d = g_dev[dev];
     const int pairs = gp.num_units < d.max_pairs ? gp.num_units : d.max_pairs;
-    kernel<<<2 * pairs, kNumThreads, L::kDynamicBytes, stream>>>(ta, tb, gp);
-    CUDA_TRY(cudaGetLastError());
-    return CUDALLM_OK;
+    return launch_overlapped(kernel, 2 * pairs, L::kDynamicBytes, stream, ta, tb, gp);
 }
 
 int launch_simt(const Problem &p, cudaStream_t stream)

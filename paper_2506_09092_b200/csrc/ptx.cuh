@@ -29,6 +29,22 @@ __device__ __forceinline__ bool elect_one()
     return pred != 0;
 }
 
+// ----------------------------------------- programmatic dependent launch --
+// The GEMM kernels are launched with programmatic stream serialisation: their
+// CTAs may start while the previous kernel of the stream is still running (as
+// soon as SMs free up), set up barriers and tensor memory, and then wait here
+// until every earlier kernel has completed and its writes are visible.  No
+// global memory is touched before this wait.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+// Lets the next kernel of the stream start launching (it will wait as above).
+__device__ __forceinline__ void grid_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ------------------------------------------------------------- mbarrier --
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {

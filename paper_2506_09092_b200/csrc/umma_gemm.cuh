@@ -363,6 +363,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    grid_launch_dependents();
+    grid_dependency_wait();          // from here on global memory may be read and written
 
     if (warp_idx == 0) {
         // ------------------------------------------------ TMA producer ----
