@@ -253,7 +253,7 @@ def run_ours(args):
     else:
         barrier = lambda: None
     peaks, peak_src = load_peaks()
-    stream = torch.cuda.current_stream()
+    stream = torch.cuda.current_stream().cuda_stream    # raw handle: no per-step Python lookups
 
     # ------------------------------------------------ headline workload: C2 --
     cfg = gi.CONFIGS["C2"]

@@ -231,7 +231,7 @@ double variant_cost(const Variant &v, const Problem &p)
     return (compute > memory ? compute : memory) + 4000.0;
 }
 
-int select_variant(const Problem &p)
+int select_variant_uncached(const Problem &p)
 {
     build_variants();
     if (is_empty(p) || p.K == 0) return 0;
@@ -243,6 +243,20 @@ int select_variant(const Problem &p)
         if (best < 0 || c < best_cost) { best = v; best_cost = c; }
     }
     return best < 0 ? 0 : best;
+}
+
+// The choice depends only on the shape; repeated calls with the same shape (the
+// common case) reuse the previous answer.
+int select_variant(const Problem &p)
+{
+    struct Last { int64_t M, N, K, batch; int out_dtype, variant; };
+    static thread_local Last last = {-1, -1, -1, -1, -1, 0};
+    if (last.M == p.M && last.N == p.N && last.K == p.K && last.batch == p.batch
+        && last.out_dtype == p.out_dtype)
+        return last.variant;
+    const int v = select_variant_uncached(p);
+    last = Last{p.M, p.N, p.K, p.batch, p.out_dtype, v};
+    return v;
 }
 
 // --------------------------------------------------------------- workspace --
@@ -376,9 +390,38 @@ Plan make_plan(const Tiling &t, const Problem &p, bool pack_a, bool pack_b)
 }
 
 // ------------------------------------------------------------- tensor maps --
-int encode_operand_map(CUtensorMap *tm, const void *base, int64_t inner, int64_t rows, int64_t batch,
-                       int64_t ld, int64_t stride, int box_inner, int box_rows)
+// Encoding a tensor map costs about a microsecond on the host, which is a large
+// share of a small GEMM; the last few are kept and reused when the same operand
+// (same base, extents, strides and box) comes back.  Called with g_mutex held.
+struct MapKey {
+    const void *base;
+    int64_t inner, rows, batch, ld, stride;
+    int box_inner, box_rows;
+    bool operator==(const MapKey &o) const
+    {
+        return base == o.base && inner == o.inner && rows == o.rows && batch == o.batch && ld == o.ld
+            && stride == o.stride && box_inner == o.box_inner && box_rows == o.box_rows;
+    }
+};
+constexpr int kMapCacheSize = 16;
+struct MapCache {
+    MapKey key[kMapCacheSize] = {};
+    CUtensorMap map[kMapCacheSize];
+    bool used[kMapCacheSize] = {};
+    int next = 0;
+};
+MapCache g_map_cache[kMaxDevices];
+
+int encode_operand_map(int dev, CUtensorMap *tm, const void *base, int64_t inner, int64_t rows,
+                       int64_t batch, int64_t ld, int64_t stride, int box_inner, int box_rows)
 {
+    MapCache &mc = g_map_cache[dev];
+    const MapKey k{base, inner, rows, batch, ld, batch > 1 ? stride : 0, box_inner, box_rows};
+    for (int i = 0; i < kMapCacheSize; ++i)
+        if (mc.used[i] && mc.key[i] == k) {
+            *tm = mc.map[i];
+            return CUDALLM_OK;
+        }
     cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batch};
     cuuint64_t item_stride = (batch > 1) ? (cuuint64_t)stride * 2 : (cuuint64_t)rows * ld * 2;
     cuuint64_t strides[2] = {(cuuint64_t)ld * 2, item_stride};
@@ -392,6 +435,11 @@ int encode_operand_map(CUtensorMap *tm, const void *base, int64_t inner, int64_t
         snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
         return CUDALLM_ERR_CUDA;
     }
+    const int slot = mc.next;
+    mc.next = (mc.next + 1) % kMapCacheSize;
+    mc.key[slot] = k;
+    mc.map[slot] = *tm;
+    mc.used[slot] = true;
     return CUDALLM_OK;
 }
 
@@ -586,9 +634,9 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     // Rows of A beyond M only feed rows of C that are never stored, so the box
     // need not cover (and zero-fill) them.  (CTA pairs always use full boxes.)
     const int a_box_rows = (p.M >= kBlockM || pair) ? kBlockM : (int)round_up(p.M, 8);
-    st = encode_operand_map(&ta, A, p.K, p.M, p.batch, lda, sA, kBlockK, a_box_rows);
+    st = encode_operand_map(dev, &ta, A, p.K, p.M, p.batch, lda, sA, kBlockK, a_box_rows);
     if (st != CUDALLM_OK) return st;
-    st = encode_operand_map(&tb, B, p.N, p.K, p.batch, ldb, sB, 64, kBlockK);
+    st = encode_operand_map(dev, &tb, B, p.N, p.K, p.batch, ldb, sB, 64, kBlockK);
     if (st != CUDALLM_OK) return st;
 
     GemmParams gp = make_params(p, t, a_box_rows);
@@ -825,9 +873,9 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
 
     CUtensorMap ta, tb;
     const int a_box_rows = p.M >= kBlockM ? kBlockM : (int)round_up(p.M, 8);
-    st = encode_operand_map(&ta, A, p.K, p.M, 1, lda, 0, kBlockK, a_box_rows);
+    st = encode_operand_map(dev, &ta, A, p.K, p.M, 1, lda, 0, kBlockK, a_box_rows);
     if (st != CUDALLM_OK) return st;
-    st = encode_operand_map(&tb, B, p.N, p.K, 1, ldb, 0, 64, kBlockK);
+    st = encode_operand_map(dev, &tb, B, p.N, p.K, 1, ldb, 0, 64, kBlockK);
     if (st != CUDALLM_OK) return st;
 
     GemmParams gp = make_params(p, t, a_box_rows);

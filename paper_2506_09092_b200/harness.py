@@ -147,21 +147,46 @@ class DeviceProblem:
         a0 = torch.from_numpy(A_bits.view(np.int16)).cuda()
         b0 = torch.from_numpy(B_bits.view(np.int16)).cuda()
         self.sets = []
+        self._calls = {}
+        self.stream_handle = torch.cuda.current_stream().cuda_stream
         for i in range(nsets):
             a = a0 if i == 0 else a0.clone()
             b = b0 if i == 0 else b0.clone()
             c = torch.empty(nC * esz, dtype=torch.uint8, device="cuda")
             self.sets.append((a, b, c))
 
-    def launch(self, i: int, variant: int = -1, stream=None, check: bool = True) -> int:
-        import torch
+    def _bound(self, variant: int, stream_handle):
+        """Per buffer set, the C call with its arguments already converted (the
+        conversion costs more than a small GEMM takes on the device)."""
+        import ctypes
         from . import binding as B
-        cfg = self.cfg
-        a, b, c = self.sets[i % self.nsets]
-        return B.gemm_bf16_variant(variant, a, b, c, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_,
-                                   cfg.strideA, cfg.strideB, cfg.strideC, cfg.batch, cfg.out_dtype,
-                                   stream if stream is not None else torch.cuda.current_stream(),
-                                   check=check)
+        key = (variant, stream_handle)
+        calls = self._calls.get(key)
+        if calls is None:
+            cfg = self.cfg
+            fn = B.lib().cudallm_gemm_bf16_variant
+            i64 = ctypes.c_int64
+            calls = []
+            for a, b, c in self.sets:
+                args = (ctypes.c_int(variant), ctypes.c_void_p(a.data_ptr()), ctypes.c_void_p(b.data_ptr()),
+                        ctypes.c_void_p(c.data_ptr()), i64(cfg.M), i64(cfg.N), i64(cfg.K), i64(cfg.lda_),
+                        i64(cfg.ldb_), i64(cfg.ldc_), i64(cfg.strideA), i64(cfg.strideB), i64(cfg.strideC),
+                        i64(cfg.batch), ctypes.c_int(cfg.out_dtype), ctypes.c_void_p(stream_handle or None))
+                calls.append((fn, args))
+            self._calls[key] = calls
+        return calls
+
+    def launch(self, i: int, variant: int = -1, stream=None, check: bool = True) -> int:
+        from . import binding as B
+        if stream is None:
+            handle = self.stream_handle          # torch's current stream when the problem was built
+        else:
+            handle = stream if isinstance(stream, int) else stream.cuda_stream
+        fn, args = self._bound(variant, handle)[i % self.nsets]
+        st = fn(*args)
+        if check and st != 0:
+            raise B.CudallmError(st, "cudallm_gemm_bf16_variant")
+        return st
 
     def output(self, i: int = 0):
         """C of set ``i`` as a host numpy array of raw elements [batch, M, ldc-strided]."""
