@@ -11,7 +11,8 @@
 //
 // Work is cut into units; CTA b runs units b, b+grid, ... in that order.  The
 // first dp_tiles tiles are one unit each.  Every later tile is cut along K into
-// split_k units with consecutive indices, and its 32-column chunks are dealt
+// split_k units with consecutive indices (these units come first in the unit
+// order, so their epilogues overlap later main loops), and its 32-column chunks are dealt
 // round-robin to those units: unit j owns chunk c iff c mod split_k == j.  In
 // its epilogue a unit first writes the chunks it does not own (its fp32 partial
 // sums) to the workspace and raises a flag; then, for each chunk it owns, it
@@ -86,16 +87,19 @@ __device__ __forceinline__ UnitCoord decode_unit(const GemmParams &p, int u)
 {
     UnitCoord c;
     int t;
-    if (u < p.dp_tiles) {
-        t = u;
+    // Split units come FIRST in the unit order (their tiles are the last
+    // tiles - dp_tiles ones): the exchange of partial sums in their epilogue
+    // then overlaps with the main loops of the unsplit tiles that follow.
+    const int split_units = p.num_units - p.dp_tiles;
+    if (u >= split_units) {
+        t = u - split_units;
         c.split = 0;
         c.nsplit = 1;
         c.slot0 = 0;
     } else {
-        const int r = u - p.dp_tiles;
-        const int ts = r / p.split_k;
+        const int ts = u / p.split_k;
         t = p.dp_tiles + ts;
-        c.split = r - ts * p.split_k;
+        c.split = u - ts * p.split_k;
         c.nsplit = p.split_k;
         c.slot0 = ts * p.split_k;
     }
