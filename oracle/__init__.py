@@ -8,7 +8,8 @@ this package imports nothing from the CUDA side.
 Contents
 --------
 * ``gemm`` / ``gemm_naive`` / ``gemm_rows`` / ``gemm_batched`` -- thin ctypes
-  wrappers over ``oracle_gemm.c`` (the plain triple loop, in two loop orders).
+  wrappers over ``oracle_gemm.c`` (the plain triple loop, in two loop orders);
+  ``gemm_f32`` / ``gemm_f32_rows`` -- the same for float32 operands.
 * ``bf16_bits_to_f64`` / ``f64_to_bf16_bits`` -- exact widening and
   round-to-nearest-even narrowing, written with integer bit operations.
 * ``check`` -- the element-wise acceptance rule
@@ -67,6 +68,13 @@ def _load():
     lib.oracle_gemm_bf16_batched.argtypes = [u16p, u16p, f64p, f64p, i64, i64,
                                              i64, i64, i64, i64, i64, i64]
     lib.oracle_gemm_bf16_batched.restype = None
+    f32p = ctypes.POINTER(ctypes.c_float)
+    for name in ("oracle_gemm_f32", "oracle_gemm_f32_naive"):
+        fn = getattr(lib, name)
+        fn.argtypes = [f32p, f32p, f64p, f64p, i64, i64, i64, i64, i64]
+        fn.restype = None
+    lib.oracle_gemm_f32_rows.argtypes = [f32p, f32p, f64p, f64p, i64p, i64, i64, i64, i64, i64]
+    lib.oracle_gemm_f32_rows.restype = None
     lib.oracle_num_threads.restype = ctypes.c_int
     lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
     _lib = lib
@@ -186,6 +194,58 @@ def gemm_batched(A, B, M, N, K, lda, ldb, strideA, strideB, batch):
                                  _ptr(C, ctypes.c_double), _ptr(S, ctypes.c_double),
                                  M, N, K, lda, ldb, strideA, strideB, batch)
     return C, S
+
+
+# --------------------------------------------------------------------------
+# fp32 operands (the paper's Task 2 as printed)
+
+def _f32_view(X, rows, cols, ld):
+    X = np.asarray(X)
+    if X.dtype != np.float32:
+        raise TypeError("operands are float32")
+    if X.ndim == 2:
+        if X.shape[0] < rows or X.shape[1] < cols:
+            raise ValueError("operand smaller than rows x cols")
+        if X.strides[1] != 4 or X.strides[0] % 4 or X.strides[0] < 0:
+            X = np.ascontiguousarray(X)
+        ldx = X.strides[0] // 4 if X.shape[0] > 1 else max(X.shape[1], cols, 1)
+        return X, (ldx or max(cols, 1))
+    ld = max(cols, 1) if ld is None else ld
+    need = (rows - 1) * ld + cols if rows > 0 and cols > 0 else 0
+    if X.ndim != 1 or ld < cols or X.size < need:
+        raise ValueError("flat float32 operand does not fit rows, cols, ld")
+    return np.ascontiguousarray(X), ld
+
+
+def gemm_f32(A, B, M, N, K, lda=None, ldb=None, naive=False):
+    """(C_ref, S) in fp64 for row-major float32 operands (Task 2 as the paper
+    states it).  ``naive=True`` runs the scalar i-j-k brute force."""
+    lib = _load()
+    Ab, lda = _f32_view(A, M, K, lda)
+    Bb, ldb = _f32_view(B, K, N, ldb)
+    C = np.empty((M, N), dtype=np.float64)
+    S = np.empty((M, N), dtype=np.float64)
+    fn = lib.oracle_gemm_f32_naive if naive else lib.oracle_gemm_f32
+    fn(_ptr(Ab, ctypes.c_float), _ptr(Bb, ctypes.c_float), _ptr(C, ctypes.c_double),
+       _ptr(S, ctypes.c_double), M, N, K, lda, ldb)
+    return C, S
+
+
+def gemm_f32_rows(A, B, rows, N, K, lda=None, ldb=None):
+    """Rows ``rows`` of the float32 product.  Returns (C_ref, S)."""
+    lib = _load()
+    rows = np.ascontiguousarray(np.asarray(rows, dtype=np.int64))
+    Mmax = int(rows.max()) + 1 if rows.size else 0
+    Ab, lda = _f32_view(A, Mmax, K, lda)
+    Bb, ldb = _f32_view(B, K, N, ldb)
+    C = np.empty((rows.size, N), dtype=np.float64)
+    S = np.empty((rows.size, N), dtype=np.float64)
+    lib.oracle_gemm_f32_rows(_ptr(Ab, ctypes.c_float), _ptr(Bb, ctypes.c_float), _ptr(C, ctypes.c_double),
+                             _ptr(S, ctypes.c_double), _ptr(rows, ctypes.c_int64), rows.size, N, K, lda, ldb)
+    return C, S
+
+
+TOL_F32_IN = 1e-5    # |C_gpu - C_ref| <= 1e-5 * S for the fp32-operand path (see DESIGN.md)
 
 
 # --------------------------------------------------------------------------

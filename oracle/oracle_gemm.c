@@ -146,6 +146,77 @@ void oracle_gemm_bf16_batched(const uint16_t *A, const uint16_t *B,
                          M, N, K, lda, ldb);
 }
 
+/*
+ * The paper's Task 2 as printed: both operands hold 32-bit floating point
+ * numbers.  C[i][j] = sum_{k<K} A[i][k] * B[k][j] with the fp32 values widened
+ * to double (exact) -- a product of two fp32 values has at most 48 significant
+ * bits and is exact in double; the only rounding is in the fp64 running sum,
+ * taken in ascending k.  S as above.  i - k - j order, rows over the threads.
+ */
+void oracle_gemm_f32(const float *A, const float *B, double *C, double *S,
+                     int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < M; ++i) {
+        double *c = C + i * N;
+        double *s = S ? S + i * N : NULL;
+        for (int64_t j = 0; j < N; ++j) c[j] = 0.0;
+        if (s) for (int64_t j = 0; j < N; ++j) s[j] = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            const double a = (double)A[i * lda + k];
+            const double aa = fabs(a);
+            const float *b = B + k * ldb;
+            for (int64_t j = 0; j < N; ++j) {
+                const double bj = (double)b[j];
+                c[j] += a * bj;
+                if (s) s[j] += aa * fabs(bj);
+            }
+        }
+    }
+}
+
+/* The same, one element at a time (i - j - k), single-threaded: brute force. */
+void oracle_gemm_f32_naive(const float *A, const float *B, double *C, double *S,
+                           int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb)
+{
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            double c = 0.0, s = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                const double a = (double)A[i * lda + k], b = (double)B[k * ldb + j];
+                c += a * b;
+                s += fabs(a) * fabs(b);
+            }
+            C[i * N + j] = c;
+            if (S) S[i * N + j] = s;
+        }
+}
+
+/* Selected rows of the fp32 product (see oracle_gemm_bf16_rows). */
+void oracle_gemm_f32_rows(const float *A, const float *B, double *C, double *S,
+                          const int64_t *rows, int64_t nrows, int64_t N, int64_t K,
+                          int64_t lda, int64_t ldb)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < nrows; ++r) {
+        const int64_t i = rows[r];
+        double *c = C + r * N;
+        double *s = S ? S + r * N : NULL;
+        for (int64_t j = 0; j < N; ++j) c[j] = 0.0;
+        if (s) for (int64_t j = 0; j < N; ++j) s[j] = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            const double a = (double)A[i * lda + k];
+            const double aa = fabs(a);
+            const float *b = B + k * ldb;
+            for (int64_t j = 0; j < N; ++j) {
+                const double bj = (double)b[j];
+                c[j] += a * bj;
+                if (s) s[j] += aa * fabs(bj);
+            }
+        }
+    }
+}
+
 /* Number of host threads the parallel loops above will use. */
 int oracle_num_threads(void)
 {

@@ -397,3 +397,76 @@ def test_check_rule():
     assert oracle.check(g, Cref, S, 1e-3)
     g = Cref.copy(); g[1, 1] = np.nan
     assert not oracle.check(g, Cref, S, 1e-3)
+
+
+# --------------------------------------------- float32 operands (Task 2) ----
+
+def test_f32_hand_computed_and_golden():
+    A = np.array([[1, 2], [3, 4]], dtype=np.float32)
+    Bm = np.array([[5, 6], [7, 8]], dtype=np.float32)
+    for naive in (False, True):
+        C, S = oracle.gemm_f32(A, Bm, 2, 2, 2, naive=naive)
+        assert C.tolist() == [[19.0, 22.0], [43.0, 50.0]] and S.tolist() == C.tolist()
+    A = np.array([[1, -2, 3], [0, 4, -1]], dtype=np.float32)
+    Bm = np.array([[2, 1], [-1, 0], [0.5, -3]], dtype=np.float32)
+    C, S = oracle.gemm_f32(A, Bm, 2, 2, 3)
+    assert C.tolist() == [[5.5, -8.0], [-4.5, 3.0]] and S.tolist() == [[5.5, 10.0], [4.5, 3.0]]
+    # a value that needs all 24 bits: (1 + 2^-23) * (1 - 2^-23) = 1 - 2^-46 exactly in fp64
+    a = np.array([[1 + 2.0 ** -23]], dtype=np.float32); b = np.array([[1 - 2.0 ** -23]], dtype=np.float32)
+    C, _ = oracle.gemm_f32(a, b, 1, 1, 1)
+    assert C.item() == 1.0 - 2.0 ** -46
+
+
+def test_f32_identity_permutation_and_roles():
+    rng = np.random.default_rng(1)
+    M, N = 33, 47
+    X = rng.standard_normal((M, N)).astype(np.float32)
+    C, S = oracle.gemm_f32(np.eye(M, dtype=np.float32), X, M, N, M)
+    assert np.array_equal(C, X.astype(np.float64)) and np.array_equal(S, np.abs(X).astype(np.float64))
+    C, _ = oracle.gemm_f32(X, np.eye(N, dtype=np.float32), M, N, N)
+    assert np.array_equal(C, X.astype(np.float64))
+    pi = rng.permutation(M)
+    P = np.zeros((M, M), dtype=np.float32); P[np.arange(M), pi] = 1
+    C, _ = oracle.gemm_f32(P, X, M, N, M)
+    assert np.array_equal(C, X[pi].astype(np.float64))
+    A = np.array([[0, 1], [0, 0]], dtype=np.float32); Bm = np.array([[0, 0], [1, 0]], dtype=np.float32)
+    assert oracle.gemm_f32(A, Bm, 2, 2, 2)[0].tolist() == [[1.0, 0.0], [0.0, 0.0]]
+    assert oracle.gemm_f32(Bm, A, 2, 2, 2)[0].tolist() == [[0.0, 0.0], [0.0, 1.0]]
+
+
+@pytest.mark.parametrize("M,N,K", [(3, 5, 7), (70, 45, 300), (16, 300, 4096)])
+def test_f32_rank1_integer_closed_form(M, N, K):
+    u, v, p, q = gi.rank1_int_factors(M, N, K, seed=M + K, umax=20, pmax=3)   # entries up to 60: not bf16-exact
+    A = np.outer(u, p).astype(np.float32); Bm = np.outer(q, v).astype(np.float32)
+    C, S = oracle.gemm_f32(A, Bm, M, N, K)
+    assert np.array_equal(C, np.outer(u, v).astype(np.float64) * float(np.dot(p, q)))
+    assert np.array_equal(S, np.outer(np.abs(u), np.abs(v)).astype(np.float64) * float(np.dot(np.abs(p), np.abs(q))))
+
+
+def test_f32_library_loop_orders_strides_rows():
+    rng = np.random.default_rng(6)
+    M, N, K = 41, 29, 130
+    A = rng.standard_normal((M, K)).astype(np.float32); Bm = rng.uniform(-1, 1, (K, N)).astype(np.float32)
+    C, S = oracle.gemm_f32(A, Bm, M, N, K)
+    bound = 2.0 * K * 2.0 ** -53 * S + 1e-300
+    assert np.all(np.abs(C - A.astype(np.float64) @ Bm.astype(np.float64)) <= bound)
+    Ct = (torch.from_numpy(A).double() @ torch.from_numpy(Bm).double()).numpy()
+    assert np.all(np.abs(C - Ct) <= bound)
+    Cn, Sn = oracle.gemm_f32(A, Bm, M, N, K, naive=True)
+    assert C.tobytes() == Cn.tobytes() and S.tobytes() == Sn.tobytes()
+    # leading dimensions with NaN padding
+    Ap = np.full(M * (K + 3), np.nan, dtype=np.float32); Ap.reshape(M, K + 3)[:, :K] = A
+    Bp = np.full(K * (N + 5), np.nan, dtype=np.float32); Bp.reshape(K, N + 5)[:, :N] = Bm
+    C2, S2 = oracle.gemm_f32(Ap, Bp, M, N, K, lda=K + 3, ldb=N + 5)
+    assert C.tobytes() == C2.tobytes() and S.tobytes() == S2.tobytes()
+    rows = [40, 0, 7, 7]
+    Cr, Sr = oracle.gemm_f32_rows(A, Bm, rows, N, K)
+    assert np.array_equal(Cr, C[rows]) and np.array_equal(Sr, S[rows])
+    # bf16-representable inputs: the fp32 oracle and the bf16 oracle agree bit for bit
+    Ab = gi.f32_to_bf16_bits(A); Bb = gi.f32_to_bf16_bits(Bm)
+    C16, S16 = oracle.gemm(Ab, Bb, M, N, K)
+    C32, S32 = oracle.gemm_f32(gi.bf16_bits_to_f32(Ab), gi.bf16_bits_to_f32(Bb), M, N, K)
+    assert C16.tobytes() == C32.tobytes() and S16.tobytes() == S32.tobytes()
+    # degenerate K
+    C0, S0 = oracle.gemm_f32(A, Bm, M, N, 0)
+    assert not C0.any() and not S0.any()
