@@ -87,6 +87,31 @@ int cudallm_gemm_bf16(const void *A, const void *B, void *C,
                       int out_dtype, void *stream);
 
 /*
+ * C = A x B with 32-bit floating point operands and result: Task 2 exactly as
+ * the paper states it ("multiplies two matrices of 32-bit floating point
+ * numbers").
+ *   A : fp32, M x K, row stride lda >= K      (read only)
+ *   B : fp32, K x N, row stride ldb >= N      (read only)
+ *   C : fp32, M x N, row stride ldc >= N
+ * B200 has no fp32 tensor-core path, so each operand is first cut into three
+ * bf16 pieces (x = x0 + x1 + x2, exact for normal numbers) in the workspace and
+ * the six piece products of relative size >= 2^-16 are accumulated in fp32 by
+ * the same tcgen05 kernels over a K range six times as long.  The result is
+ * within 1e-5 * sum_k |a_ik||b_kj| of the exact product (what is dropped is of
+ * relative size 2^-23; the fp32 accumulation contributes the rest); integer
+ * cases whose partial sums stay below 2^24 are exact.  A non-finite input gives
+ * a non-finite (possibly NaN) output in its row or column.  Pointers must be
+ * 4-byte aligned; any leading dimensions are accepted.  Needs workspace:
+ * 6 * (M*round_up(K,8) + K*round_up(N,8)) bytes plus what the chosen kernel
+ * variant needs.  `variant` as in cudallm_gemm_bf16_variant (CUDALLM_VARIANT_AUTO
+ * lets the library choose; the simt variant is not available here).
+ */
+int cudallm_gemm_f32(const void *A, const void *B, void *C,
+                     int64_t M, int64_t N, int64_t K,
+                     int64_t lda, int64_t ldb, int64_t ldc,
+                     int variant, void *stream);
+
+/*
  * `batch` independent products of the same shape (Task 2 applied per item;
  * the paper's Task 6 score matrices Q_i K_i^T are products of this kind).
  * Item t uses A + t*strideA, B + t*strideB, C + t*strideC.  Items of C must

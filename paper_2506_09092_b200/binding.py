@@ -41,6 +41,7 @@ _sz = ctypes.c_size_t
 # name -> (restype, argtypes); mirrors include/cudallm_gemm.h
 SIGNATURES = {
     "cudallm_gemm_bf16": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp]),
+    "cudallm_gemm_f32": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp]),
     "cudallm_gemm_bf16_batched": (_int, [_vp, _vp, _vp] + [_i64] * 10 + [_int, _vp]),
     "cudallm_gemm_bf16_variant": (_int, [_int, _vp, _vp, _vp] + [_i64] * 10 + [_int, _vp]),
     "cudallm_gemm_bf16_host": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp, _sz, _vp]),
@@ -111,6 +112,13 @@ def _check(st: int, where: str, check: bool):
 def gemm_bf16(A, B, C, M, N, K, lda, ldb, ldc, out_dtype, stream=None, check=True):
     st = lib().cudallm_gemm_bf16(_p(A), _p(B), _p(C), M, N, K, lda, ldb, ldc, out_dtype, _s(stream))
     return _check(st, "cudallm_gemm_bf16", check)
+
+
+def gemm_f32(A, B, C, M, N, K, lda, ldb, ldc, variant=VARIANT_AUTO, stream=None, check=True):
+    """fp32 operands and result (the paper's Task 2 as stated), computed on the
+    bf16 tensor cores from three-piece splits of the operands."""
+    st = lib().cudallm_gemm_f32(_p(A), _p(B), _p(C), M, N, K, lda, ldb, ldc, variant, _s(stream))
+    return _check(st, "cudallm_gemm_f32", check)
 
 
 def gemm_bf16_batched(A, B, C, M, N, K, lda, ldb, ldc, strideA, strideB, strideC, batch,

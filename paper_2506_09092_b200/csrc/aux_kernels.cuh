@@ -64,4 +64,44 @@ pack_rows_kernel(const uint16_t *__restrict__ src, uint16_t *__restrict__ dst,
     }
 }
 
+// Cuts fp32 values into three bf16 pieces: x = p0 + p1 + p2 exactly for normal
+// numbers whose exponent leaves room for the low piece (p0 = bf16(x), p1 =
+// bf16(x - p0), p2 = bf16(x - p0 - p1); both differences are exact in fp32, and
+// three 8-bit significands cover fp32's 24 bits).  dst holds the pieces as three
+// matrices `piece_stride` elements apart, rows ld_dst apart (a multiple of 8),
+// columns beyond `cols` zero.  One thread converts 8 consecutive elements.
+__global__ void __launch_bounds__(256)
+split3_rows_kernel(const float *__restrict__ src, uint16_t *__restrict__ dst, int rows, int cols,
+                   long long ld_src, long long ld_dst, long long piece_stride)
+{
+    const int chunks = (cols + 7) >> 3;
+    const long long total = static_cast<long long>(rows) * chunks;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int r = static_cast<int>(i / chunks);
+        const int c0 = static_cast<int>(i - static_cast<long long>(r) * chunks) * 8;
+        const float *s = src + r * ld_src + c0;
+        uint32_t w[3][4];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float x = (c0 + j < cols) ? s[j] : 0.f;
+            const __nv_bfloat16 p0 = __float2bfloat16_rn(x);
+            const float r1 = x - __bfloat162float(p0);
+            const __nv_bfloat16 p1 = __float2bfloat16_rn(r1);
+            const float r2 = r1 - __bfloat162float(p1);
+            const __nv_bfloat16 p2 = __float2bfloat16_rn(r2);
+            const uint32_t b[3] = {__bfloat16_as_ushort(p0), __bfloat16_as_ushort(p1), __bfloat16_as_ushort(p2)};
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+                if (j & 1) w[q][j >> 1] |= b[q] << 16;
+                else       w[q][j >> 1] = b[q];
+            }
+        }
+        uint16_t *d = dst + r * ld_dst + c0;
+#pragma unroll
+        for (int q = 0; q < 3; ++q)
+            *reinterpret_cast<uint4 *>(d + q * piece_stride) = make_uint4(w[q][0], w[q][1], w[q][2], w[q][3]);
+    }
+}
+
 }  // namespace cudallm

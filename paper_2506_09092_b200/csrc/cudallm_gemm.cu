@@ -562,6 +562,23 @@ int launch_pack(const void *src, void *dst, int64_t rows, int64_t cols, int64_t 
     return CUDALLM_OK;
 }
 
+// Launches the tcgen05 kernel of variant `v` (lone CTAs or CTA pairs).
+int launch_variant(int dev, const Variant &v, bool bf, const CUtensorMap &ta, const CUtensorMap &tb,
+                   const GemmParams &gp, cudaStream_t stream)
+{
+    if (v.family == kUmmaPair)
+        return bf ? launch_umma_pair<3, 2, true>(dev, ta, tb, gp, stream)
+                  : launch_umma_pair<3, 2, false>(dev, ta, tb, gp, stream);
+    switch (v.block_n) {
+    case 64:  return bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
+                        : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream);
+    case 128: return bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
+                        : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream);
+    default:  return bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
+                        : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream);
+    }
+}
+
 // Fills the kernel parameters that depend only on the problem and the tiling.
 GemmParams make_params(const Problem &p, const Tiling &t, int a_box_rows)
 {
@@ -645,17 +662,7 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     gp.flags = reinterpret_cast<int *>(ws + 256);
     gp.status = reinterpret_cast<int *>(ws);
 
-    if (pair)
-        return bf ? launch_umma_pair<3, 2, true>(dev, ta, tb, gp, stream)
-                  : launch_umma_pair<3, 2, false>(dev, ta, tb, gp, stream);
-    switch (v.block_n) {
-    case 64:  return bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
-                        : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream);
-    case 128: return bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
-                        : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream);
-    default:  return bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
-                        : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream);
-    }
+    return launch_variant(dev, v, bf, ta, tb, gp, stream);
 }
 
 int run(int variant, const Problem &p, void *stream_v)
@@ -732,6 +739,95 @@ int cudallm_gemm_bf16_variant(int variant, const void *A, const void *B, void *C
     return run(variant,
                make_problem(A, B, C, M, N, K, lda, ldb, ldc, strideA, strideB, strideC, batch, out_dtype),
                stream);
+}
+
+int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N, int64_t K, int64_t lda,
+                     int64_t ldb, int64_t ldc, int variant, void *stream_v)
+{
+    build_variants();
+    // validate as a product with fp32 output; the operand pointers need 4-byte alignment
+    const Problem p = make_problem(A, B, C, M, N, K, lda, ldb, ldc, 0, 0, 0, 1, CUDALLM_F32);
+    int st = validate(p);
+    if (st != CUDALLM_OK) return st;
+    if (variant != CUDALLM_VARIANT_AUTO && (variant < 1 || variant >= kNumVariants))
+        return CUDALLM_ERR_INVALID_VARIANT;
+    if (is_empty(p)) return CUDALLM_OK;
+    if (K > 0 && ((reinterpret_cast<uintptr_t>(A) & 3) || (reinterpret_cast<uintptr_t>(B) & 3)))
+        return CUDALLM_ERR_MISALIGNED;
+    if (K > kMaxDim / 6) return CUDALLM_ERR_INVALID_DIM;
+
+    // the tcgen05 kernels see a bf16 product over a K range six times as long
+    Problem q = p;
+    q.K = 6 * round_up(K > 0 ? K : 1, kBlockK);
+    q.lda = q.K;
+    if (variant == CUDALLM_VARIANT_AUTO) variant = select_variant(q);
+    const Variant &v = g_variants[variant];
+    if (v.family == kSimt || !variant_supports(v, q)) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    st = probe_device(dev);
+    if (st != CUDALLM_OK) return st;
+    DeviceState &d = g_dev[dev];
+    const bool pair = v.family == kUmmaPair;
+    if (pair) {
+        st = prepare_umma_pair<3, 2, false>(dev, 7);
+        if (st != CUDALLM_OK) return st;
+    }
+    if (K == 0) {
+        // empty sum: C := 0 (the CUDA-core kernel writes zeros without reading A or B)
+        Problem z = p;
+        z.A = z.B = C;
+        return launch_simt(z, stream);
+    }
+    const Tiling t = tiling_for(v, q, pair ? d.max_pairs : d.sm_count);
+    if (t.helper_tiles > kMaxHelperTiles || t.partial_bytes > kMaxPartialBytes)
+        return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+
+    // workspace: [header][partial tiles][A pieces 3 x M x ldap][B pieces 3 x K x ldbp]
+    const int64_t ldap = round_up(K, 8), ldbp = round_up(N, 8);
+    size_t off = kHeaderBytes;
+    const size_t off_partials = off;
+    off = (size_t)round_up((int64_t)(off + t.partial_bytes), 256);
+    const size_t off_a = off;
+    off = (size_t)round_up((int64_t)off + 3 * M * ldap * 2, 256);
+    const size_t off_b = off;
+    off = (size_t)round_up((int64_t)off + 3 * K * ldbp * 2, 256);
+    st = ensure_workspace(dev, off, stream);
+    if (st != CUDALLM_OK) return st;
+    uint8_t *ws = static_cast<uint8_t *>(d.ws);
+
+    auto split = [&](const void *src, void *dst, int64_t rows, int64_t cols, int64_t ld_src, int64_t ld_dst) {
+        const int64_t total = rows * cdiv(cols, 8);
+        int64_t blocks = cdiv(total, 256);
+        if (blocks > kNumSMs * 16) blocks = kNumSMs * 16;
+        split3_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const float *>(src),
+                                                                 static_cast<uint16_t *>(dst), (int)rows,
+                                                                 (int)cols, ld_src, ld_dst, rows * ld_dst);
+    };
+    split(A, ws + off_a, M, K, lda, ldap);
+    CUDA_TRY(cudaGetLastError());
+    split(B, ws + off_b, K, N, ldb, ldbp);
+    CUDA_TRY(cudaGetLastError());
+
+    CUtensorMap ta, tb;
+    const int a_box_rows = (M >= kBlockM || pair) ? kBlockM : (int)round_up(M, 8);
+    st = encode_operand_map(dev, &ta, ws + off_a, K, M, 3, ldap, M * ldap, kBlockK, a_box_rows);
+    if (st != CUDALLM_OK) return st;
+    st = encode_operand_map(dev, &tb, ws + off_b, N, K, 3, ldbp, K * ldbp, 64, kBlockK);
+    if (st != CUDALLM_OK) return st;
+
+    GemmParams gp = make_params(p, t, a_box_rows);
+    gp.K = (int)q.K;
+    gp.piece_kblocks = (int)cdiv(K, kBlockK);
+    gp.epoch = t.split > 1 ? next_epoch(d) : 0;
+    gp.partials = reinterpret_cast<float *>(ws + off_partials);
+    gp.flags = reinterpret_cast<int *>(ws + 256);
+    gp.status = reinterpret_cast<int *>(ws);
+    return launch_variant(dev, v, false, ta, tb, gp, stream);
 }
 
 size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,

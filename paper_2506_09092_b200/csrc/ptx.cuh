@@ -249,8 +249,8 @@ __device__ __forceinline__ uint32_t tma_stage_step(uint32_t next_bar, uint32_t n
                                                    uint32_t full_bar, uint32_t arm, uint32_t tx_bytes,
                                                    uint32_t signal_bar, const CUtensorMap *tm_a,
                                                    const CUtensorMap *tm_b, uint32_t sa, uint32_t sb,
-                                                   int k0, int row0, int col0, int batch, int boxes,
-                                                   int nsub, uint32_t sub_bytes)
+                                                   int k0, int row0, int col0, int batch_a, int batch_b,
+                                                   int boxes, int nsub, uint32_t sub_bytes)
 {
     uint32_t tok;
     const uint64_t ta = reinterpret_cast<uint64_t>(tm_a), tb = reinterpret_cast<uint64_t>(tm_b);
@@ -271,13 +271,13 @@ __device__ __forceinline__ uint32_t tma_stage_step(uint32_t next_bar, uint32_t n
         "add.s32 k1, %11, 64;\n\t add.u32 ta1, %9, %17;\n\t add.u32 tb1, %10, %17;\n\t add.u32 tb2, s1, %17;\n\t" \
         "@pa mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %5;\n\t"                           \
         LOAD " [%9], [%7, {%11, %12, %14}], [%6];\n\t"                                             \
-        LOAD " [%10], [%8, {%13, %11, %14}], [%6];\n\t"                                            \
-        "@p1 " LOAD " [s1], [%8, {c1, %11, %14}], [%6];\n\t"                                       \
-        "@p2 " LOAD " [s2], [%8, {c2, %11, %14}], [%6];\n\t"                                       \
-        "@p3 " LOAD " [s3], [%8, {c3, %11, %14}], [%6];\n\t"                                       \
+        LOAD " [%10], [%8, {%13, %11, %18}], [%6];\n\t"                                            \
+        "@p1 " LOAD " [s1], [%8, {c1, %11, %18}], [%6];\n\t"                                       \
+        "@p2 " LOAD " [s2], [%8, {c2, %11, %18}], [%6];\n\t"                                       \
+        "@p3 " LOAD " [s3], [%8, {c3, %11, %18}], [%6];\n\t"                                       \
         "@q0 " LOAD " [ta1], [%7, {k1, %12, %14}], [%6];\n\t"                                      \
-        "@q0 " LOAD " [tb1], [%8, {%13, k1, %14}], [%6];\n\t"                                      \
-        "@q1 " LOAD " [tb2], [%8, {c1, k1, %14}], [%6];\n\t"                                       \
+        "@q0 " LOAD " [tb1], [%8, {%13, k1, %18}], [%6];\n\t"                                      \
+        "@q1 " LOAD " [tb2], [%8, {c1, k1, %18}], [%6];\n\t"                                       \
         "@pn bra LDONE;\n\t"                                                                       \
         TRYW " pn, [%1], %2;\n\t"                                                                  \
         "LDONE:\n\t"                                                                               \
@@ -285,8 +285,8 @@ __device__ __forceinline__ uint32_t tma_stage_step(uint32_t next_bar, uint32_t n
         "}"                                                                                        \
         : "=r"(tok)                                                                                \
         : "r"(next_bar), "r"(next_parity), "r"(full_bar), "r"(arm), "r"(tx_bytes), "r"(signal_bar), \
-          "l"(ta), "l"(tb), "r"(sa), "r"(sb), "r"(k0), "r"(row0), "r"(col0), "r"(batch), "r"(boxes), \
-          "r"(nsub), "r"(sub_bytes)                                                                \
+          "l"(ta), "l"(tb), "r"(sa), "r"(sb), "r"(k0), "r"(row0), "r"(col0), "r"(batch_a), "r"(boxes), \
+          "r"(nsub), "r"(sub_bytes), "r"(batch_b)                                                  \
         : "memory")
     if (kPair) {
         CUDALLM_TMA_STEP("mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64",

@@ -44,7 +44,8 @@ struct GemmParams {
     int M, N, K, batch;
     int tiles_m, tiles_n;   // tiles per batch item
     int group_m;            // tile rows per raster group (see decode_unit)
-    int kblocks;            // ceil(K / 64)
+    int kblocks;            // 64-deep k-blocks each unit range is cut from: ceil(K / 64), or 6x that
+    int piece_kblocks;      // 0, or k-blocks per operand-piece pair (see KBlockCoord)
     int dp_tiles;           // leading tiles that are not split
     int split_k;            // K parts per tile for tiles >= dp_tiles (1 = none), <= kblocks
     int num_units;          // dp_tiles + (tiles - dp_tiles) * split_k
@@ -117,6 +118,37 @@ __device__ __forceinline__ UnitCoord decode_unit(const GemmParams &p, int u)
     c.m_tile = g * p.group_m + (r2 - c.n_tile * gm);
     c.kb_begin = static_cast<int>((static_cast<long long>(p.kblocks) * c.split) / c.nsplit);
     c.kb_end = static_cast<int>((static_cast<long long>(p.kblocks) * (c.split + 1)) / c.nsplit);
+    return c;
+}
+
+// Where k-block g of a unit's range lies in the operands.  Normally that is
+// column block g of A / row block g of B of batch item b.  In three-piece mode
+// (piece_kblocks > 0) the operands are fp32 values cut into three bf16 pieces
+// each, stored as "batch" items 0..2 of the tensor maps, and the K range is six
+// segments long: segment s multiplies piece kPieceA[s] of A with piece
+// kPieceB[s] of B (the six products of magnitude >= 2^-16 of the leading one,
+// smallest first so that they are not absorbed by the large ones too early).
+struct KBlockCoord {
+    int k;                  // first K index of the block
+    int batch_a, batch_b;   // third tensor-map coordinate for the A and the B load
+    int left_in_segment;    // k-blocks from g to the end of its segment (>= 1)
+};
+__device__ __forceinline__ KBlockCoord kblock_coord(const GemmParams &p, int g, int b)
+{
+    KBlockCoord c;
+    if (p.piece_kblocks == 0) {
+        c.k = g * kBlockK;
+        c.batch_a = c.batch_b = b;
+        c.left_in_segment = p.kblocks - g;
+    } else {
+        const int seg = g / p.piece_kblocks;
+        const int kb = g - seg * p.piece_kblocks;
+        c.k = kb * kBlockK;
+        // segments: a3*b1, a1*b3, a2*b2, a2*b1, a1*b2, a1*b1
+        c.batch_a = (0x001102 >> (4 * seg)) & 0xF;
+        c.batch_b = (0x010120 >> (4 * seg)) & 0xF;
+        c.left_in_segment = p.piece_kblocks - kb;
+    }
     return c;
 }
 
@@ -390,10 +422,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
                     const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
+                    const KBlockCoord kc = kblock_coord(p, kb, c.b);
                     tok = tma_stage_step<false>(empty_bar(nstage), nphase ^ 1, full_bar(stage), 1,
                                                 p.a_box_bytes + boxes * (64 * kBlockK * 2), full_bar(stage),
-                                                &tmap_a, &tmap_b, sa, sa + L::kABytes, kb * kBlockK,
-                                                c.m_tile * kBlockM, c.n_tile * BLOCK_N, c.b, boxes, 1, 0);
+                                                &tmap_a, &tmap_b, sa, sa + L::kABytes, kc.k,
+                                                c.m_tile * kBlockM, c.n_tile * BLOCK_N, kc.batch_a,
+                                                kc.batch_b, boxes, 1, 0);
                     stage = nstage;
                     phase = nphase;
                 }

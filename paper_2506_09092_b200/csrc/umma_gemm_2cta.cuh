@@ -142,7 +142,9 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
                         ok = false;
                         break;
                     }
-                    const int nsub = (c.kb_end - kb) < KSUB ? (c.kb_end - kb) : KSUB;
+                    // a stage takes up to KSUB k-blocks, all from the same operand segment
+                    const KBlockCoord kc = kblock_coord(p, kb, c.b);
+                    const int nsub = min(min(c.kb_end - kb, KSUB), kc.left_in_segment);
                     const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
                     const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
@@ -150,10 +152,11 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                                rank == 0 ? 1u : 0u,
                                                2 * nsub * (L::kABytes + boxes * (64 * kBlockK * 2)),
                                                leader_full0 + 8u * stage, &tmap_a, &tmap_b, sa,
-                                               sa + L::kABytes, kb * kBlockK,
+                                               sa + L::kABytes, kc.k,
                                                c.m_tile * kPairM + static_cast<int>(rank) * kBlockM,
-                                               c.n_tile * kPairN + static_cast<int>(rank) * half, c.b, boxes, nsub,
-                                               L::kSubBytes);
+                                               c.n_tile * kPairN + static_cast<int>(rank) * half, kc.batch_a,
+                                               kc.batch_b, boxes, nsub, L::kSubBytes);
+                    kb += nsub - KSUB;                   // the loop adds KSUB
                     stage = nstage;
                     phase = nphase;
                 }
@@ -181,22 +184,25 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     break;
                 }
                 const uint32_t d_tmem = tmem_base + acc * kPairN;
+                bool first_of_unit = true;
                 for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
                     if (!tok && !mbar_wait<true>(full_bar(stage), phase, abort_flag)) {
                         report_timeout(p.status, kRoleMma, stage);
                         ok = false;
                         break;
                     }
-                    const int nsub = (c.kb_end - kb) < KSUB ? (c.kb_end - kb) : KSUB;
+                    const int nsub = min(min(c.kb_end - kb, KSUB), kblock_coord(p, kb, c.b).left_in_segment);
                     const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
                     const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
                     tok = umma_stage_step<true>(full_bar(nstage), nphase, d_tmem, idesc,
-                                                kb > c.kb_begin ? 1u : 0u,
+                                                first_of_unit ? 0u : 1u,
                                                 make_smem_desc_sw128(sa, 16, 1024),
                                                 make_smem_desc_sw128(sa + L::kABytes, 8192, 1024),
                                                 L::kSubBytes, nsub, empty0_cta0 + 8u * stage,
                                                 empty0_cta1 + 8u * stage);
+                    first_of_unit = false;
+                    kb += nsub - KSUB;                   // the loop adds KSUB
                     stage = nstage;
                     phase = nphase;
                 }

@@ -72,6 +72,19 @@ def test_argument_errors_are_reported_before_any_cuda_call():
     assert B.strerror(12345) == "unknown status"
 
 
+def test_fp32_entry_point_validates_first():
+    p = 4096
+    f = lambda *a: B.gemm_f32(*a, check=False)
+    assert f(None, p, p, 4, 4, 4, 4, 4, 4) == B.ERR_INVALID_POINTER
+    assert f(p, p, p, 4, 4, 4, 3, 4, 4) == B.ERR_INVALID_LD
+    assert f(p + 2, p, p, 4, 4, 4, 4, 4, 4) == B.ERR_MISALIGNED
+    assert f(p, p, p + 2, 4, 4, 4, 4, 4, 4) == B.ERR_MISALIGNED
+    assert f(p, p, p, 4, 4, 4, 4, 4, 4, 0) == B.ERR_INVALID_VARIANT      # simt: bf16 operands only
+    assert f(p, p, p, 4, 4, 4, 4, 4, 4, 999) == B.ERR_INVALID_VARIANT
+    assert f(p, p, p, 4, 4, 1 << 30, 1 << 30, 4, 4) == B.ERR_INVALID_DIM  # 6 K must stay indexable
+    assert f(None, None, None, 0, 4, 4, 4, 4, 4) == B.OK
+
+
 def test_host_entry_point_validates_first():
     p = 4096
     assert B.gemm_bf16_host(None, p, p, 4, 4, 4, 4, 4, 4, 0, p, 1 << 20, check=False) == B.ERR_INVALID_POINTER
