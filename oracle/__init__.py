@@ -28,7 +28,8 @@ from dataclasses import dataclass
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "oracle_gemm.c")
+_SRCS = [os.path.join(_HERE, "oracle_gemm.c"), os.path.join(_HERE, "oracle_mhsa.c")]
+_SRC = _SRCS[0]
 _LIB = os.path.join(_HERE, "liboracle_gemm.so")
 _lock = threading.Lock()
 _lib = None
@@ -38,11 +39,11 @@ def build(force: bool = False) -> str:
     """Compile ``oracle_gemm.c`` with gcc into ``liboracle_gemm.so`` beside it."""
     with _lock:
         if (not force and os.path.exists(_LIB)
-                and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+                and all(os.path.getmtime(_LIB) >= os.path.getmtime(f) for f in _SRCS)):
             return _LIB
         tmp = _LIB + f".tmp{os.getpid()}"
         cmd = ["gcc", "-O3", "-march=native", "-fopenmp", "-fPIC", "-shared",
-               "-std=c11", "-Wall", "-o", tmp, _SRC, "-lm"]
+               "-std=c11", "-Wall", "-o", tmp] + _SRCS + ["-lm"]
         subprocess.run(cmd, check=True, capture_output=True, text=True)
         os.replace(tmp, _LIB)
         return _LIB
@@ -75,6 +76,8 @@ def _load():
         fn.restype = None
     lib.oracle_gemm_f32_rows.argtypes = [f32p, f32p, f64p, f64p, i64p, i64, i64, i64, i64, i64]
     lib.oracle_gemm_f32_rows.restype = None
+    lib.oracle_mhsa_bf16.argtypes = [u16p, u16p, u16p, f64p, f64p] + [i64] * 6
+    lib.oracle_mhsa_bf16.restype = ctypes.c_int
     lib.oracle_num_threads.restype = ctypes.c_int
     lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
     _lib = lib
@@ -245,6 +248,25 @@ def gemm_f32_rows(A, B, rows, N, K, lda=None, ldb=None):
     return C, S
 
 
+def mhsa(Q, K, V, N, d_model, h, ldq=None, ldk=None, ldv=None):
+    """Task 6, multi-head self-attention, in fp64 on bfloat16 bit patterns.
+    Q, K, V: N x d_model (2-D, or flat with leading dimensions).  Returns
+    (out, T), each N x d_model, T[i][c] = sum_j p_ij |V[j][c]|."""
+    lib = _load()
+    Qb, ldq = _operand_view(Q, N, d_model, ldq)
+    Kb, ldk = _operand_view(K, N, d_model, ldk)
+    Vb, ldv = _operand_view(V, N, d_model, ldv)
+    out = np.empty((N, d_model), dtype=np.float64)
+    T = np.empty((N, d_model), dtype=np.float64)
+    rc = lib.oracle_mhsa_bf16(_ptr(Qb, ctypes.c_uint16), _ptr(Kb, ctypes.c_uint16), _ptr(Vb, ctypes.c_uint16),
+                              _ptr(out, ctypes.c_double), _ptr(T, ctypes.c_double),
+                              N, d_model, h, ldq, ldk, ldv)
+    if rc != 0:
+        raise ValueError("h must divide d_model")
+    return out, T
+
+
+TOL_MHSA = 1e-2      # |O_gpu - O_ref| <= 1e-2 * T  (probabilities are rounded to bf16 on the GPU)
 TOL_F32_IN = 1e-5    # |C_gpu - C_ref| <= 1e-5 * S for the fp32-operand path (see DESIGN.md)
 
 
