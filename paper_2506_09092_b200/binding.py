@@ -42,6 +42,7 @@ _sz = ctypes.c_size_t
 SIGNATURES = {
     "cudallm_gemm_bf16": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp]),
     "cudallm_gemm_f32": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp]),
+    "cudallm_mhsa_bf16": (_int, [_vp, _vp, _vp, _vp] + [_i64] * 7 + [_vp]),
     "cudallm_gemm_bf16_batched": (_int, [_vp, _vp, _vp] + [_i64] * 10 + [_int, _vp]),
     "cudallm_gemm_bf16_variant": (_int, [_int, _vp, _vp, _vp] + [_i64] * 10 + [_int, _vp]),
     "cudallm_gemm_bf16_host": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp, _sz, _vp]),
@@ -119,6 +120,12 @@ def gemm_f32(A, B, C, M, N, K, lda, ldb, ldc, variant=VARIANT_AUTO, stream=None,
     bf16 tensor cores from three-piece splits of the operands."""
     st = lib().cudallm_gemm_f32(_p(A), _p(B), _p(C), M, N, K, lda, ldb, ldc, variant, _s(stream))
     return _check(st, "cudallm_gemm_f32", check)
+
+
+def mhsa_bf16(Q, K, V, O, N, d_model, h, ldq, ldk, ldv, ldo, stream=None, check=True):
+    """Multi-head self-attention (Task 6): bf16 Q, K, V (N x d_model), fp32 O."""
+    st = lib().cudallm_mhsa_bf16(_p(Q), _p(K), _p(V), _p(O), N, d_model, h, ldq, ldk, ldv, ldo, _s(stream))
+    return _check(st, "cudallm_mhsa_bf16", check)
 
 
 def gemm_bf16_batched(A, B, C, M, N, K, lda, ldb, ldc, strideA, strideB, strideC, batch,

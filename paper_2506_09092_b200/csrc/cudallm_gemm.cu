@@ -14,6 +14,7 @@
 #include "aux_kernels.cuh"
 #include "umma_gemm.cuh"
 #include "umma_gemm_2cta.cuh"
+#include "mhsa.cuh"
 
 using namespace cudallm;
 
@@ -828,6 +829,58 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
     gp.flags = reinterpret_cast<int *>(ws + 256);
     gp.status = reinterpret_cast<int *>(ws);
     return launch_variant(dev, v, false, ta, tb, gp, stream);
+}
+
+int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int64_t N, int64_t d_model,
+                      int64_t h, int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo, void *stream_v)
+{
+    if (N < 0 || d_model < 0 || h < 0) return CUDALLM_ERR_INVALID_DIM;
+    if (N == 0 || d_model == 0) return CUDALLM_OK;
+    if (h == 0 || d_model % h) return CUDALLM_ERR_INVALID_DIM;
+    if (ldq < d_model || ldk < d_model || ldv < d_model || ldo < d_model) return CUDALLM_ERR_INVALID_LD;
+    if (!Q || !K || !V || !O) return CUDALLM_ERR_INVALID_POINTER;
+    if (reinterpret_cast<uintptr_t>(O) & 3) return CUDALLM_ERR_MISALIGNED;
+    if ((reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V)) & 1)
+        return CUDALLM_ERR_MISALIGNED;
+    const int64_t dk = d_model / h;
+    if (N > kMhsaMaxKeys || dk > kMhsaMaxDk || dk % 8 || h > 65535) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+    if (((reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V)) & 15)
+        || ldq % 8 || ldk % 8 || ldv % 8)
+        return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int st = probe_device(dev);
+    if (st != CUDALLM_OK) return st;
+    st = ensure_workspace(dev, kHeaderBytes, stream);          // for the status word
+    if (st != CUDALLM_OK) return st;
+    DeviceState &d = g_dev[dev];
+
+    MhsaParams mp{};
+    mp.Q = static_cast<const __nv_bfloat16 *>(Q);
+    mp.K = static_cast<const __nv_bfloat16 *>(K);
+    mp.V = static_cast<const __nv_bfloat16 *>(V);
+    mp.O = static_cast<float *>(O);
+    mp.N = (int)N; mp.h = (int)h; mp.dk = (int)dk;
+    mp.keys_pad = (int)round_up(N, 32);
+    mp.dkp = (int)round_up(dk, 16);
+    mp.tmem_cols = 32;
+    while (mp.tmem_cols < mp.keys_pad) mp.tmem_cols *= 2;
+    mp.ldq = ldq; mp.ldk = ldk; mp.ldv = ldv; mp.ldo = ldo;
+    mp.scale_log2 = 1.4426950408889634f / sqrtf((float)dk);
+    mp.status = static_cast<int *>(d.ws);
+    const MhsaSmem L = mhsa_smem_layout(mp.keys_pad, mp.dkp);
+    if (!d.smem_attr_set[8]) {
+        CUDA_TRY(cudaFuncSetAttribute(mhsa_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        d.smem_attr_set[8] = true;
+    }
+    dim3 grid((unsigned)cdiv(N, kMhsaRows), (unsigned)h);
+    mhsa_kernel<<<grid, kMhsaRows, L.total, stream>>>(mp);
+    CUDA_TRY(cudaGetLastError());
+    return CUDALLM_OK;
 }
 
 size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,

@@ -1,0 +1,247 @@
+// Fused multi-head self-attention for short sequences (the paper's Task 6):
+//
+//   head_i = softmax(Q_i K_i^T / sqrt(d_k)) V_i,   O = Concat(head_1 .. head_h)
+//
+// Q, K, V are N x d_model bf16, row-major; head i owns columns [i d_k, (i+1) d_k).
+// One CTA computes 128 query rows of one head, for N <= 512 keys and d_k <= 32
+// (the paper's sizes go up to N = 512, d_model = 512, h = 16):
+//
+//   1. all threads copy Q_i (128 x d_k), K_i (N x d_k) and V_i (N x d_k) into
+//      shared memory, directly in the tensor core's unswizzled operand layouts
+//      (8-row x 16-byte core matrices), zero-padding rows and d_k;
+//   2. one thread issues S = Q_i K_i^T with tcgen05.mma into tensor memory: all
+//      keys at once, 128 lanes x up to 512 fp32 columns -- the whole of TMEM;
+//   3. each thread owns one query row (one TMEM lane): two passes over its row
+//      of S (maximum; then p = exp2((s - max) * log2(e)/sqrt(d_k)), masked beyond
+//      N, summed, rounded to bf16 and written to shared memory as the K-major
+//      A operand of the second product);
+//   4. one thread issues O = P V_i (V_i is the MN-major B operand) into the TMEM
+//      columns that S no longer needs;
+//   5. each thread divides its row of O by its row sum and stores d_k floats.
+//
+// The two waits on tensor-core completion are bounded like those of the GEMM
+// kernels.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "ptx.cuh"
+
+namespace cudallm {
+
+constexpr int kMhsaRows = 128;        // queries per CTA
+constexpr int kMhsaMaxKeys = 512;     // = TMEM columns
+constexpr int kMhsaMaxDk = 32;
+
+struct MhsaParams {
+    const __nv_bfloat16 *Q, *K, *V;
+    float *O;
+    int N, h, dk;
+    int keys_pad;           // N rounded up to 32
+    int dkp;                // d_k rounded up to 16 (K of the first product, N of the second)
+    int tmem_cols;          // power of two >= max(keys_pad, 32): tensor-memory columns to allocate
+    long long ldq, ldk, ldv, ldo;
+    float scale_log2;       // log2(e) / sqrt(d_k)
+    int *status;
+};
+
+// Unswizzled shared-memory matrix descriptor: start address, leading-dimension
+// and stride-dimension byte offsets in 16-byte units, descriptor version 1.
+__device__ __forceinline__ uint64_t make_smem_desc_plain(uint32_t smem_addr, uint32_t lbo_bytes,
+                                                         uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
+    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    return d;
+}
+
+__device__ __forceinline__ void umma_bf16_1cta(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                               uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+struct MhsaSmem {
+    // byte offsets inside the dynamic shared memory block (all multiples of 128)
+    int q, k, v, p, bar, total;
+};
+__host__ __device__ inline MhsaSmem mhsa_smem_layout(int keys_pad, int dkp)
+{
+    MhsaSmem s;
+    s.q = 0;                                          // (dkp/8) chunks x 16 row groups x 128 B
+    s.k = s.q + (dkp / 8) * 2048;                     // (dkp/8) chunks x (keys_pad/8) row groups x 128 B
+    s.v = s.k + (dkp / 8) * keys_pad * 16;            // (keys_pad/8) k groups x (dkp/8) column groups x 128 B
+    s.p = s.v + (keys_pad / 8) * (dkp / 8) * 128;     // (keys_pad/8) chunks x 16 row groups x 128 B
+    s.bar = s.p + (keys_pad / 8) * 2048;
+    s.total = s.bar + 64;
+    return s;
+}
+
+__global__ void __launch_bounds__(kMhsaRows, 1)
+mhsa_kernel(const MhsaParams p)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    const MhsaSmem L = mhsa_smem_layout(p.keys_pad, p.dkp);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar = sbase + L.bar;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.bar + 16);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L.bar + 20);
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int head = blockIdx.y;
+    const int q0 = blockIdx.x * kMhsaRows;
+    const int col0 = head * p.dk;
+    const int kchunks = p.dkp / 8;                    // 16-byte chunks along d_k
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar, 1);
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), p.tmem_cols);
+        tmem_relinquish();
+    }
+
+    // ---- 1. operands -> shared memory, in core-matrix order -------------------
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < kMhsaRows * kchunks; i += kMhsaRows) {
+        const int c = i / kMhsaRows, r = i - c * kMhsaRows, row = q0 + r;
+        uint4 x = zero;
+        if (row < p.N && c * 8 < p.dk)
+            x = *reinterpret_cast<const uint4 *>(p.Q + row * p.ldq + col0 + c * 8);
+        *reinterpret_cast<uint4 *>(smem + L.q + c * 2048 + (r >> 3) * 128 + (r & 7) * 16) = x;
+    }
+    const int lbo_k = p.keys_pad * 16;                // bytes between d_k chunks of K
+    for (int i = tid; i < p.keys_pad * kchunks; i += kMhsaRows) {
+        const int c = i / p.keys_pad, j = i - c * p.keys_pad;
+        uint4 x = zero;
+        if (j < p.N && c * 8 < p.dk)
+            x = *reinterpret_cast<const uint4 *>(p.K + j * p.ldk + col0 + c * 8);
+        *reinterpret_cast<uint4 *>(smem + L.k + c * lbo_k + (j >> 3) * 128 + (j & 7) * 16) = x;
+    }
+    const int lbo_v = kchunks * 128;                  // bytes between groups of 8 keys of V
+    for (int i = tid; i < p.keys_pad * kchunks; i += kMhsaRows) {
+        const int j = i / kchunks, c = i - j * kchunks;
+        uint4 x = zero;
+        if (j < p.N && c * 8 < p.dk)
+            x = *reinterpret_cast<const uint4 *>(p.V + j * p.ldv + col0 + c * 8);
+        *reinterpret_cast<uint4 *>(smem + L.v + (j >> 3) * lbo_v + c * 128 + (j & 7) * 16) = x;
+    }
+    fence_proxy_async_smem();                         // make the writes visible to the tensor core
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    // ---- 2. S = Q K^T ---------------------------------------------------------
+    const int n1 = p.keys_pad < 256 ? p.keys_pad : 256;
+    const int n2 = p.keys_pad - n1;
+    if (tid == 0) {
+        for (int part = 0; part < 2; ++part) {
+            const int n = part ? n2 : n1;
+            if (n == 0) break;
+            const uint32_t idesc = make_idesc_bf16(kMhsaRows, n, 0, 0);      // both operands K-major
+            for (int ks = 0; ks < p.dkp / 16; ++ks) {
+                const uint64_t da = make_smem_desc_plain(sbase + L.q + ks * 2 * 2048, 2048, 128);
+                const uint64_t db = make_smem_desc_plain(sbase + L.k + ks * 2 * lbo_k + part * (256 / 8) * 128,
+                                                         lbo_k, 128);
+                umma_bf16_1cta(tmem + part * 256, da, db, idesc, ks > 0 ? 1u : 0u);
+            }
+        }
+        umma_commit(bar);
+    }
+    bool ok = mbar_wait(bar, 0, abort_flag);
+    ok = __all_sync(0xffffffffu, ok);
+    tc_fence_after();
+
+    // ---- 3. softmax over this thread's row ------------------------------------
+    const uint32_t t_row = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    float row_max = -INFINITY;
+    if (ok) {
+#pragma unroll 1
+        for (int ch = 0; ch < p.keys_pad / 32; ++ch) {
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(t_row + ch * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (ch * 32 + j < p.N) row_max = fmaxf(row_max, __uint_as_float(r[j]));
+        }
+    }
+    float row_sum = 0.f;
+    if (ok) {
+        const int r_off = (tid >> 3) * 128 + (tid & 7) * 16;                 // this row inside a chunk of P
+#pragma unroll 1
+        for (int ch = 0; ch < p.keys_pad / 32; ++ch) {
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(t_row + ch * 32, r);
+            tmem_ld_wait();
+            uint32_t w[16];
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+                float e0 = 0.f, e1 = 0.f;
+                if (ch * 32 + j < p.N) e0 = exp2f((__uint_as_float(r[j]) - row_max) * p.scale_log2);
+                if (ch * 32 + j + 1 < p.N) e1 = exp2f((__uint_as_float(r[j + 1]) - row_max) * p.scale_log2);
+                const uint32_t packed = pack_bf16x2(e0, e1);
+                // the row sum uses the rounded probabilities, i.e. exactly what the second product sees
+                row_sum += __uint_as_float(packed << 16) + __uint_as_float(packed & 0xFFFF0000u);
+                w[j >> 1] = packed;
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g)                                      // 8 keys = one 16-byte chunk
+                *reinterpret_cast<uint4 *>(smem + L.p + (ch * 4 + g) * 2048 + r_off) =
+                    make_uint4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+        }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();                                   // everyone is done reading S and writing P
+    tc_fence_after();
+
+    // ---- 4. O = P V -------------------------------------------------------------
+    if (tid == 0 && ok) {
+        const uint32_t idesc = make_idesc_bf16(kMhsaRows, p.dkp, 0, 1);      // V: MN-major
+        for (int ks = 0; ks < p.keys_pad / 16; ++ks) {
+            const uint64_t da = make_smem_desc_plain(sbase + L.p + ks * 2 * 2048, 2048, 128);
+            const uint64_t db = make_smem_desc_plain(sbase + L.v + ks * 2 * lbo_v, lbo_v, 128);
+            umma_bf16_1cta(tmem, da, db, idesc, ks > 0 ? 1u : 0u);
+        }
+        umma_commit(bar);
+    }
+    if (ok) {
+        ok = mbar_wait(bar, 1, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+    }
+    tc_fence_after();
+
+    // ---- 5. normalise and store -------------------------------------------------
+    if (ok) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(t_row, r);                  // d_k <= 32 columns are meaningful
+        tmem_ld_wait();
+        const int row = q0 + tid;
+        if (row < p.N) {
+            const float inv = 1.f / row_sum;
+            float *dst = p.O + row * p.ldo + col0;
+#pragma unroll
+            for (int d = 0; d < kMhsaMaxDk; ++d)
+                if (d < p.dk) dst[d] = __uint_as_float(r[d]) * inv;
+        }
+    } else if (tid == 0) {
+        if (atomicCAS(p.status, 0, -9) == 0) p.status[1] = 0x600;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem, p.tmem_cols);
+    }
+}
+
+}  // namespace cudallm

@@ -85,6 +85,20 @@ def test_fp32_entry_point_validates_first():
     assert f(None, None, None, 0, 4, 4, 4, 4, 4) == B.OK
 
 
+def test_attention_entry_point_validates_first():
+    p = 4096
+    f = lambda *a: B.mhsa_bf16(*a, check=False)
+    assert f(p, p, p, p, -1, 32, 4, 32, 32, 32, 32) == B.ERR_INVALID_DIM
+    assert f(p, p, p, p, 64, 32, 3, 32, 32, 32, 32) == B.ERR_INVALID_DIM          # h must divide d_model
+    assert f(p, p, p, p, 64, 32, 4, 32, 31, 32, 32) == B.ERR_INVALID_LD
+    assert f(p, None, p, p, 64, 32, 4, 32, 32, 32, 32) == B.ERR_INVALID_POINTER
+    assert f(p, p, p, p + 2, 64, 32, 4, 32, 32, 32, 32) == B.ERR_MISALIGNED
+    assert f(p, p, p, p, 513, 32, 4, 32, 32, 32, 32) == B.ERR_UNSUPPORTED_SHAPE    # more than 512 keys
+    assert f(p, p, p, p, 64, 160, 4, 160, 160, 160, 160) == B.ERR_UNSUPPORTED_SHAPE  # d_k = 40
+    assert f(p + 2, p, p, p, 64, 32, 4, 32, 32, 32, 32) == B.ERR_UNSUPPORTED_SHAPE  # Q not 16-byte aligned
+    assert f(None, None, None, None, 0, 32, 4, 32, 32, 32, 32) == B.OK
+
+
 def test_host_entry_point_validates_first():
     p = 4096
     assert B.gemm_bf16_host(None, p, p, 4, 4, 4, 4, 4, 4, 0, p, 1 << 20, check=False) == B.ERR_INVALID_POINTER
