@@ -65,6 +65,14 @@ __device__ __forceinline__ void umma_bf16_1cta(uint32_t d_tmem, uint64_t a_desc,
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// 2^x by the special-function unit (relative error ~2^-22; inputs <= 0 here)
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 struct MhsaSmem {
     // byte offsets inside the dynamic shared memory block (all multiples of 128)
     int q, k, v, p, bar, total;
@@ -108,30 +116,45 @@ mhsa_kernel(const MhsaParams p)
     }
 
     // ---- 1. operands -> shared memory, in core-matrix order -------------------
+    // Each thread keeps sixteen 16-byte loads in flight (the copies are latency-bound).
     const uint4 zero = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < kMhsaRows * kchunks; i += kMhsaRows) {
-        const int c = i / kMhsaRows, r = i - c * kMhsaRows, row = q0 + r;
-        uint4 x = zero;
-        if (row < p.N && c * 8 < p.dk)
-            x = *reinterpret_cast<const uint4 *>(p.Q + row * p.ldq + col0 + c * 8);
-        *reinterpret_cast<uint4 *>(smem + L.q + c * 2048 + (r >> 3) * 128 + (r & 7) * 16) = x;
-    }
     const int lbo_k = p.keys_pad * 16;                // bytes between d_k chunks of K
-    for (int i = tid; i < p.keys_pad * kchunks; i += kMhsaRows) {
-        const int c = i / p.keys_pad, j = i - c * p.keys_pad;
-        uint4 x = zero;
-        if (j < p.N && c * 8 < p.dk)
-            x = *reinterpret_cast<const uint4 *>(p.K + j * p.ldk + col0 + c * 8);
-        *reinterpret_cast<uint4 *>(smem + L.k + c * lbo_k + (j >> 3) * 128 + (j & 7) * 16) = x;
-    }
     const int lbo_v = kchunks * 128;                  // bytes between groups of 8 keys of V
-    for (int i = tid; i < p.keys_pad * kchunks; i += kMhsaRows) {
-        const int j = i / kchunks, c = i - j * kchunks;
-        uint4 x = zero;
-        if (j < p.N && c * 8 < p.dk)
-            x = *reinterpret_cast<const uint4 *>(p.V + j * p.ldv + col0 + c * 8);
-        *reinterpret_cast<uint4 *>(smem + L.v + (j >> 3) * lbo_v + c * 128 + (j & 7) * 16) = x;
-    }
+    auto copy_operand = [&](int which, int total) {
+        for (int i0 = tid; i0 < total; i0 += 16 * kMhsaRows) {
+            uint4 x[16];
+            int dst[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const int i = i0 + u * kMhsaRows;
+                x[u] = zero;
+                dst[u] = -1;
+                if (i < total) {
+                    const __nv_bfloat16 *src = nullptr;
+                    if (which == 0) {                 // Q: chunk-major, row within the block
+                        const int c = i / kMhsaRows, r = i - c * kMhsaRows, row = q0 + r;
+                        dst[u] = L.q + c * 2048 + (r >> 3) * 128 + (r & 7) * 16;
+                        if (row < p.N && c * 8 < p.dk) src = p.Q + row * p.ldq + col0 + c * 8;
+                    } else if (which == 1) {          // K: chunk-major, key
+                        const int c = i / p.keys_pad, j = i - c * p.keys_pad;
+                        dst[u] = L.k + c * lbo_k + (j >> 3) * 128 + (j & 7) * 16;
+                        if (j < p.N && c * 8 < p.dk) src = p.K + j * p.ldk + col0 + c * 8;
+                    } else {                          // V: key-major, chunk of d_k
+                        const int j = i / kchunks, c = i - j * kchunks;
+                        dst[u] = L.v + (j >> 3) * lbo_v + c * 128 + (j & 7) * 16;
+                        if (j < p.N && c * 8 < p.dk) src = p.V + j * p.ldv + col0 + c * 8;
+                    }
+                    if (src) x[u] = *reinterpret_cast<const uint4 *>(src);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 16; ++u)
+                if (dst[u] >= 0) *reinterpret_cast<uint4 *>(smem + dst[u]) = x[u];
+        }
+    };
+    copy_operand(0, kMhsaRows * kchunks);
+    copy_operand(1, p.keys_pad * kchunks);
+    copy_operand(2, p.keys_pad * kchunks);
     fence_proxy_async_smem();                         // make the writes visible to the tensor core
     tc_fence_before();
     __syncthreads();
@@ -161,41 +184,63 @@ mhsa_kernel(const MhsaParams p)
 
     // ---- 3. softmax over this thread's row ------------------------------------
     const uint32_t t_row = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    // Four 32-column loads are in flight per wait: a TMEM round trip costs far
+    // more than the arithmetic on 32 values.
     float row_max = -INFINITY;
+    const int nch = p.keys_pad / 32;
     if (ok) {
 #pragma unroll 1
-        for (int ch = 0; ch < p.keys_pad / 32; ++ch) {
-            uint32_t r[32];
-            tmem_ld_32x32b_x32(t_row + ch * 32, r);
+        for (int ch0 = 0; ch0 < nch; ch0 += 4) {
+            uint32_t r[4][32];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (ch0 + u < nch) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (ch * 32 + j < p.N) row_max = fmaxf(row_max, __uint_as_float(r[j]));
+            for (int u = 0; u < 4; ++u) {
+                if (ch0 + u < nch) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if ((ch0 + u) * 32 + j < p.N) row_max = fmaxf(row_max, __uint_as_float(r[u][j]));
+                }
+            }
         }
     }
     float row_sum = 0.f;
+    const float neg_max_scaled = -row_max * p.scale_log2;
     if (ok) {
         const int r_off = (tid >> 3) * 128 + (tid & 7) * 16;                 // this row inside a chunk of P
 #pragma unroll 1
-        for (int ch = 0; ch < p.keys_pad / 32; ++ch) {
-            uint32_t r[32];
-            tmem_ld_32x32b_x32(t_row + ch * 32, r);
+        for (int ch0 = 0; ch0 < nch; ch0 += 4) {
+            uint32_t r[4][32];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (ch0 + u < nch) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
             tmem_ld_wait();
-            uint32_t w[16];
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-                float e0 = 0.f, e1 = 0.f;
-                if (ch * 32 + j < p.N) e0 = exp2f((__uint_as_float(r[j]) - row_max) * p.scale_log2);
-                if (ch * 32 + j + 1 < p.N) e1 = exp2f((__uint_as_float(r[j + 1]) - row_max) * p.scale_log2);
-                const uint32_t packed = pack_bf16x2(e0, e1);
-                // the row sum uses the rounded probabilities, i.e. exactly what the second product sees
-                row_sum += __uint_as_float(packed << 16) + __uint_as_float(packed & 0xFFFF0000u);
-                w[j >> 1] = packed;
+            for (int u = 0; u < 4; ++u) {
+                const int ch = ch0 + u;
+                if (ch < nch) {
+                    uint32_t w[16];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        // exp2(s * c - max * c): one FMA and one ex2.approx per element
+                        float e0 = 0.f, e1 = 0.f;
+                        if (ch * 32 + j < p.N)
+                            e0 = fast_exp2(fmaf(__uint_as_float(r[u][j]), p.scale_log2, neg_max_scaled));
+                        if (ch * 32 + j + 1 < p.N)
+                            e1 = fast_exp2(fmaf(__uint_as_float(r[u][j + 1]), p.scale_log2, neg_max_scaled));
+                        const uint32_t packed = pack_bf16x2(e0, e1);
+                        // the row sum uses the rounded probabilities: exactly what the second product sees
+                        row_sum += __uint_as_float(packed << 16) + __uint_as_float(packed & 0xFFFF0000u);
+                        w[j >> 1] = packed;
+                    }
+#pragma unroll
+                    for (int g = 0; g < 4; ++g)                              // 8 keys = one 16-byte chunk
+                        *reinterpret_cast<uint4 *>(smem + L.p + (ch * 4 + g) * 2048 + r_off) =
+                            make_uint4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+                }
             }
-#pragma unroll
-            for (int g = 0; g < 4; ++g)                                      // 8 keys = one 16-byte chunk
-                *reinterpret_cast<uint4 *>(smem + L.p + (ch * 4 + g) * 2048 + r_off) =
-                    make_uint4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
         }
     }
     fence_proxy_async_smem();
