@@ -398,10 +398,11 @@ struct MapKey {
     const void *base;
     int64_t inner, rows, batch, ld, stride;
     int box_inner, box_rows;
+    int kind;                              // 0 = bf16 operand, 1 = fp32 C, 2 = bf16 C
     bool operator==(const MapKey &o) const
     {
         return base == o.base && inner == o.inner && rows == o.rows && batch == o.batch && ld == o.ld
-            && stride == o.stride && box_inner == o.box_inner && box_rows == o.box_rows;
+            && stride == o.stride && box_inner == o.box_inner && box_rows == o.box_rows && kind == o.kind;
     }
 };
 constexpr int kMapCacheSize = 16;
@@ -413,24 +414,28 @@ struct MapCache {
 };
 MapCache g_map_cache[kMaxDevices];
 
-int encode_operand_map(int dev, CUtensorMap *tm, const void *base, int64_t inner, int64_t rows,
-                       int64_t batch, int64_t ld, int64_t stride, int box_inner, int box_rows)
+// kind 0: a bf16 operand read in 128-byte-swizzled boxes; kind 1 / 2: fp32 / bf16
+// C written in boxes of 32 columns x 32 rows (128- / 64-byte swizzle).
+int encode_map(int dev, CUtensorMap *tm, const void *base, int64_t inner, int64_t rows, int64_t batch,
+               int64_t ld, int64_t stride, int box_inner, int box_rows, int kind)
 {
     MapCache &mc = g_map_cache[dev];
-    const MapKey k{base, inner, rows, batch, ld, batch > 1 ? stride : 0, box_inner, box_rows};
+    const MapKey k{base, inner, rows, batch, ld, batch > 1 ? stride : 0, box_inner, box_rows, kind};
     for (int i = 0; i < kMapCacheSize; ++i)
         if (mc.used[i] && mc.key[i] == k) {
             *tm = mc.map[i];
             return CUDALLM_OK;
         }
+    const cuuint64_t es = (kind == 1) ? 4 : 2;
     cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batch};
-    cuuint64_t item_stride = (batch > 1) ? (cuuint64_t)stride * 2 : (cuuint64_t)rows * ld * 2;
-    cuuint64_t strides[2] = {(cuuint64_t)ld * 2, item_stride};
+    cuuint64_t item_stride = (batch > 1) ? (cuuint64_t)stride * es : (cuuint64_t)rows * ld * es;
+    cuuint64_t strides[2] = {(cuuint64_t)ld * es, item_stride};
     cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims,
-                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    CUresult r = g_encode(tm, kind == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                          const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          kind == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                          kind == 0 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -443,6 +448,21 @@ int encode_operand_map(int dev, CUtensorMap *tm, const void *base, int64_t inner
     mc.used[slot] = true;
     return CUDALLM_OK;
 }
+int encode_operand_map(int dev, CUtensorMap *tm, const void *base, int64_t inner, int64_t rows,
+                       int64_t batch, int64_t ld, int64_t stride, int box_inner, int box_rows)
+{
+    return encode_map(dev, tm, base, inner, rows, batch, ld, stride, box_inner, box_rows, 0);
+}
+// Tensor map of C for the epilogue's stores; all zero (and unused) when C's
+// alignment does not allow TMA.
+int encode_c_map(int dev, CUtensorMap *tm, const Problem &p, bool c_tma)
+{
+    if (!c_tma) {
+        memset(tm, 0, sizeof *tm);
+        return CUDALLM_OK;
+    }
+    return encode_map(dev, tm, p.C, p.N, p.M, p.batch, p.ldc, p.sC, 32, 32, p.out_dtype == CUDALLM_F32 ? 1 : 2);
+}
 
 // ---------------------------------------------------------------- launches --
 // Launch with programmatic stream serialisation: the kernel may begin while the
@@ -450,7 +470,7 @@ int encode_operand_map(int dev, CUtensorMap *tm, const void *base, int64_t inner
 // touches global memory.
 template <typename Kernel>
 int launch_overlapped(Kernel kernel, int grid, int smem_bytes, cudaStream_t stream, const CUtensorMap &ta,
-                      const CUtensorMap &tb, const GemmParams &gp)
+                      const CUtensorMap &tb, const CUtensorMap &tc, const GemmParams &gp)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -462,12 +482,13 @@ int launch_overlapped(Kernel kernel, int grid, int smem_bytes, cudaStream_t stre
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ta, tb, gp));
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ta, tb, tc, gp));
     return CUDALLM_OK;
 }
 
 template <int BLOCK_N, int STAGES, bool OUT_BF16>
-int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &gp,
+int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tc,
+                const GemmParams &gp,
                 cudaStream_t stream)
 {
     using L = SmemLayout<BLOCK_N, STAGES>;
@@ -483,7 +504,7 @@ int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb,
         d.smem_attr_set[slot] = true;
     }
     int grid = gp.num_units < d.sm_count ? gp.num_units : d.sm_count;
-    return launch_overlapped(kernel, grid, L::kDynamicBytes, stream, ta, tb, gp);
+    return launch_overlapped(kernel, grid, L::kDynamicBytes, stream, ta, tb, tc, gp);
 }
 
 // Sets the pair kernel's shared-memory attribute and asks how many CTA pairs
@@ -522,14 +543,15 @@ int prepare_umma_pair(int dev, int slot)
 }
 
 template <int STAGES, int KSUB, bool OUT_BF16>
-int launch_umma_pair(int dev, const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &gp,
+int launch_umma_pair(int dev, const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tc,
+                const GemmParams &gp,
                      cudaStream_t stream)
 {
     using L = PairSmemLayout<STAGES, KSUB>;
     auto kernel = umma_gemm_2cta_kernel<STAGES, KSUB, OUT_BF16>;
     DeviceState &d = g_dev[dev];
     const int pairs = gp.num_units < d.max_pairs ? gp.num_units : d.max_pairs;
-    return launch_overlapped(kernel, 2 * pairs, L::kDynamicBytes, stream, ta, tb, gp);
+    return launch_overlapped(kernel, 2 * pairs, L::kDynamicBytes, stream, ta, tb, tc, gp);
 }
 
 int launch_simt(const Problem &p, cudaStream_t stream)
@@ -565,18 +587,18 @@ int launch_pack(const void *src, void *dst, int64_t rows, int64_t cols, int64_t 
 
 // Launches the tcgen05 kernel of variant `v` (lone CTAs or CTA pairs).
 int launch_variant(int dev, const Variant &v, bool bf, const CUtensorMap &ta, const CUtensorMap &tb,
-                   const GemmParams &gp, cudaStream_t stream)
+                   const CUtensorMap &tc, const GemmParams &gp, cudaStream_t stream)
 {
     if (v.family == kUmmaPair)
-        return bf ? launch_umma_pair<3, 2, true>(dev, ta, tb, gp, stream)
-                  : launch_umma_pair<3, 2, false>(dev, ta, tb, gp, stream);
+        return bf ? launch_umma_pair<3, 2, true>(dev, ta, tb, tc, gp, stream)
+                  : launch_umma_pair<3, 2, false>(dev, ta, tb, tc, gp, stream);
     switch (v.block_n) {
-    case 64:  return bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
-                        : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream);
-    case 128: return bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, gp, stream)
-                        : launch_umma<128, 6, false>(dev, 3, ta, tb, gp, stream);
-    default:  return bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, gp, stream)
-                        : launch_umma<256, 4, false>(dev, 5, ta, tb, gp, stream);
+    case 64:  return bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, tc, gp, stream)
+                        : launch_umma<64, 8, false>(dev, 1, ta, tb, tc, gp, stream);
+    case 128: return bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, tc, gp, stream)
+                        : launch_umma<128, 6, false>(dev, 3, ta, tb, tc, gp, stream);
+    default:  return bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, tc, gp, stream)
+                        : launch_umma<256, 4, false>(dev, 5, ta, tb, tc, gp, stream);
     }
 }
 
@@ -601,9 +623,16 @@ GemmParams make_params(const Problem &p, const Tiling &t, int a_box_rows)
     gp.split_k = t.split;
     gp.num_units = (int)t.units;
     const int64_t vec = (p.out_dtype == CUDALLM_F32) ? 4 : 8;
-    gp.c_vec_ok = (reinterpret_cast<uintptr_t>(p.C) % 16 == 0) && (p.ldc % vec == 0)
+    gp.c_tma = (reinterpret_cast<uintptr_t>(p.C) % 16 == 0) && (p.ldc % vec == 0)
                && (p.batch == 1 || p.sC % vec == 0);
+    gp.n_edge_tma = (p.N % vec == 0);
     gp.a_box_bytes = a_box_rows * 128;
+    gp.div_split = make_fast_div((uint32_t)gp.split_k);
+    gp.div_item = make_fast_div((uint32_t)(gp.tiles_m * gp.tiles_n));
+    gp.div_group = make_fast_div((uint32_t)(gp.group_m * gp.tiles_n));
+    gp.div_gm = make_fast_div((uint32_t)gp.group_m);
+    const int last_gm = gp.tiles_m % gp.group_m;
+    gp.div_gm_last = make_fast_div((uint32_t)(last_gm ? last_gm : gp.group_m));
     return gp;
 }
 
@@ -658,12 +687,15 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     if (st != CUDALLM_OK) return st;
 
     GemmParams gp = make_params(p, t, a_box_rows);
+    CUtensorMap tc;
+    st = encode_c_map(dev, &tc, p, gp.c_tma != 0);
+    if (st != CUDALLM_OK) return st;
     gp.epoch = t.split > 1 ? next_epoch(d) : 0;
     gp.partials = reinterpret_cast<float *>(ws + pl.off_partials);
     gp.flags = reinterpret_cast<int *>(ws + 256);
     gp.status = reinterpret_cast<int *>(ws);
 
-    return launch_variant(dev, v, bf, ta, tb, gp, stream);
+    return launch_variant(dev, v, bf, ta, tb, tc, gp, stream);
 }
 
 int run(int variant, const Problem &p, void *stream_v)
@@ -822,13 +854,16 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
     if (st != CUDALLM_OK) return st;
 
     GemmParams gp = make_params(p, t, a_box_rows);
+    CUtensorMap tc;
+    st = encode_c_map(dev, &tc, p, gp.c_tma != 0);
+    if (st != CUDALLM_OK) return st;
     gp.K = (int)q.K;
     gp.piece_kblocks = (int)cdiv(K, kBlockK);
     gp.epoch = t.split > 1 ? next_epoch(d) : 0;
     gp.partials = reinterpret_cast<float *>(ws + off_partials);
     gp.flags = reinterpret_cast<int *>(ws + 256);
     gp.status = reinterpret_cast<int *>(ws);
-    return launch_variant(dev, v, false, ta, tb, gp, stream);
+    return launch_variant(dev, v, false, ta, tb, tc, gp, stream);
 }
 
 int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int64_t N, int64_t d_model,
@@ -1028,6 +1063,9 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     if (st != CUDALLM_OK) return st;
 
     GemmParams gp = make_params(p, t, a_box_rows);
+    CUtensorMap tc;
+    st = encode_c_map(dev, &tc, p, gp.c_tma != 0);
+    if (st != CUDALLM_OK) return st;
     g_noalloc_epoch[dev] = (g_noalloc_epoch[dev] == 0x7fffffff) ? 1 : g_noalloc_epoch[dev] + 1;
     gp.epoch = g_noalloc_epoch[dev];
     gp.status = reinterpret_cast<int *>(scratch);
@@ -1037,8 +1075,8 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     // The array keeps the last call's contents.  The status word and the flags
     // must start at zero; partial tiles are written before they are read.
     CUDA_TRY(cudaMemsetAsync(scratch, 0, kNoallocHeaderBytes, stream));
-    st = (p.out_dtype == CUDALLM_BF16) ? launch_umma<64, 8, true>(dev, 0, ta, tb, gp, stream)
-                                       : launch_umma<64, 8, false>(dev, 1, ta, tb, gp, stream);
+    st = (p.out_dtype == CUDALLM_BF16) ? launch_umma<64, 8, true>(dev, 0, ta, tb, tc, gp, stream)
+                                       : launch_umma<64, 8, false>(dev, 1, ta, tb, tc, gp, stream);
     if (st != CUDALLM_OK) return st;
     int host_status[2] = {0, 0};
     CUDA_TRY(cudaMemcpyAsync(host_status, scratch, sizeof host_status, cudaMemcpyDeviceToHost, stream));

@@ -37,6 +37,29 @@ constexpr int kEpiThreads = 128;
 // status detail codes: (role << 8) | barrier kind
 enum : int { kRoleProducer = 1, kRoleMma = 2, kRoleEpilogue = 3 };
 
+// Division of a 32-bit unsigned number by a divisor fixed on the host (1 <= d <
+// 2^31): q = (t + ((n - t) >> sh1)) >> sh2 with t = the high half of mul * n
+// (the round-up method for invariant divisors).  Exact for every 32-bit n.
+struct FastDiv {
+    uint32_t mul;
+    uint16_t sh1, sh2;
+};
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, FastDiv d)
+{
+    const uint32_t t = __umulhi(d.mul, n);
+    return (t + ((n - t) >> d.sh1)) >> d.sh2;
+}
+inline FastDiv make_fast_div(uint32_t d)
+{
+    int l = 0;
+    while ((1ull << l) < d) ++l;                         // l = ceil(log2 d)
+    FastDiv f;
+    f.mul = static_cast<uint32_t>((((1ull << 32) * ((1ull << l) - d)) / d) + 1);
+    f.sh1 = static_cast<uint16_t>(l < 1 ? l : 1);
+    f.sh2 = static_cast<uint16_t>(l ? l - 1 : 0);
+    return f;
+}
+
 struct GemmParams {
     void *C;
     long long ldc;          // elements
@@ -49,25 +72,37 @@ struct GemmParams {
     int dp_tiles;           // leading tiles that are not split
     int split_k;            // K parts per tile for tiles >= dp_tiles (1 = none), <= kblocks
     int num_units;          // dp_tiles + (tiles - dp_tiles) * split_k
-    int c_vec_ok;           // C base, ldc, strideC allow 16-byte stores
+    int c_tma;              // C base, ldc and strideC are 16-byte aligned: the epilogue stores by TMA
+    int n_edge_tma;         // ... including the box that straddles column N (N * element size % 16 == 0)
     int a_box_bytes;        // bytes one TMA box of A delivers (box rows * 128)
     int epoch;              // value that marks a flag as raised in this launch (never 0)
     float *partials;        // partial tiles of split units (workspace), 128 x BLOCK_N fp32 each
     int *flags;             // one per (partial tile, epilogue warp) (workspace)
     int *status;            // [0] = code, [1] = detail
+    // divisors of decode_unit: split_k, tiles per item, tiles per raster group,
+    // group_m, and the height of the last (possibly shorter) raster group
+    FastDiv div_split, div_item, div_group, div_gm, div_gm_last;
 };
+
+// Epilogue staging: 8 KiB per epilogue warp, 1024-byte aligned -- two 4 KiB
+// blocks of 32 rows x 128 bytes that TMA stores read in turn, or one block of
+// 32 rows x 36 floats for the element-wise path of unaligned C.
+constexpr int kEpiPitch = 36;
+constexpr int kEpiWarpBytes = 8192;
+constexpr int kEpiStageBytes = 4 * kEpiWarpBytes;
+static_assert(32 * kEpiPitch * 4 <= kEpiWarpBytes, "element-wise staging block");
 
 template <int BLOCK_N, int STAGES>
 struct SmemLayout {
     static constexpr int kABytes = kBlockM * kBlockK * 2;
     static constexpr int kBBytes = kBlockK * BLOCK_N * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kBarOffset = STAGES * kStageBytes;
+    static constexpr int kEpiOffset = STAGES * kStageBytes;          // 1024-byte aligned (swizzled staging)
+    static constexpr int kBarOffset = kEpiOffset + kEpiStageBytes;
     // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
-    static constexpr int kEpiOffset = (kMiscOffset + 64 + 15) / 16 * 16;
-    static constexpr int kBytes = kEpiOffset + 18432;    // + epilogue staging (kEpiStageBytes)
+    static constexpr int kBytes = kMiscOffset + 64;
     static constexpr int kDynamicBytes = kBytes + 1024;  // slack for 1024-byte alignment
 };
 
@@ -97,27 +132,32 @@ __device__ __forceinline__ UnitCoord decode_unit(const GemmParams &p, int u)
         c.split = 0;
         c.nsplit = 1;
         c.slot0 = 0;
+        c.kb_begin = 0;
+        c.kb_end = p.kblocks;
     } else {
-        const int ts = u / p.split_k;
+        const int ts = static_cast<int>(fast_div(u, p.div_split));
         t = p.dp_tiles + ts;
         c.split = u - ts * p.split_k;
         c.nsplit = p.split_k;
         c.slot0 = ts * p.split_k;
+        // kblocks * split_k < 2^32 (kblocks < 6 * 2^25, split_k <= 16)
+        const uint32_t lo = static_cast<uint32_t>(p.kblocks) * static_cast<uint32_t>(c.split);
+        c.kb_begin = static_cast<int>(fast_div(lo, p.div_split));
+        c.kb_end = static_cast<int>(fast_div(lo + static_cast<uint32_t>(p.kblocks), p.div_split));
     }
     // Raster order inside a batch item: groups of group_m tile rows; inside a
     // group the row index runs fastest, then the column.  The CTAs that run at
     // the same time then share one slice of A (group_m tile rows, sized by the
     // host to stay in L2) and a few column panels of B.
     const int per_item = p.tiles_m * p.tiles_n;
-    c.b = t / per_item;
+    c.b = static_cast<int>(fast_div(t, p.div_item));
     const int r = t - c.b * per_item;
-    const int g = r / (p.group_m * p.tiles_n);
+    const int g = static_cast<int>(fast_div(r, p.div_group));
     const int r2 = r - g * p.group_m * p.tiles_n;
-    const int gm = min(p.group_m, p.tiles_m - g * p.group_m);
-    c.n_tile = r2 / gm;
+    const bool last = (g + 1) * p.group_m > p.tiles_m;   // the shorter group at the bottom
+    const int gm = last ? p.tiles_m - g * p.group_m : p.group_m;
+    c.n_tile = static_cast<int>(fast_div(r2, last ? p.div_gm_last : p.div_gm));
     c.m_tile = g * p.group_m + (r2 - c.n_tile * gm);
-    c.kb_begin = static_cast<int>((static_cast<long long>(p.kblocks) * c.split) / c.nsplit);
-    c.kb_end = static_cast<int>((static_cast<long long>(p.kblocks) * (c.split + 1)) / c.nsplit);
     return c;
 }
 
@@ -180,75 +220,79 @@ __device__ __forceinline__ bool wait_flag(const int *flag, int epoch, volatile i
     }
 }
 
-// Shared-memory staging of the epilogue: one 32 x 32 fp32 block per epilogue
-// warp, rows 36 floats apart (conflict-free for the accesses below).
-constexpr int kEpiPitch = 36;
-constexpr int kEpiStageBytes = 4 * 32 * kEpiPitch * 4;
-static_assert(kEpiStageBytes == 18432, "SmemLayout reserves this many bytes");
-
 // Stores one 32 x 32 block of the accumulator (this warp's 32 rows, 32
 // consecutive columns from col0) to C.  Each thread arrives with the 32 values
 // of ITS row (v); writing them as they are would make every store instruction
-// touch 32 different rows.  The block is therefore transposed through shared
-// memory so that the lanes of a store instruction run along a row: 16-byte
-// stores covering whole 128-byte (fp32) or 64-byte (bf16) row segments when C's
-// alignment allows, else element stores that are still contiguous per row.
-// row0 = global row of lane 0; rows >= M and columns >= N are skipped.
+// touch 32 different rows, so the block goes through shared memory.
+//  * C aligned for TMA (p.c_tma): every thread writes its row (128 bytes of
+//    fp32, 64 bytes of bf16) into one of the warp's two staging blocks in the
+//    tensor map's swizzled layout -- 16-byte piece q of row r lies at piece
+//    q ^ (r % 8) (128-byte rows) or q ^ ((r / 2) % 4) (64-byte rows), which
+//    keeps the 16-byte stores of a quarter-warp on distinct banks -- and lane 0
+//    issues one TMA store of the box; the hardware clips it at M and N.  The
+//    block is reused two stores later, after lane 0 has waited for the older
+//    store to have read it.  The clipping works in units of 16 bytes (measured:
+//    with N = 127 column 127 is written), so a box that straddles an N whose
+//    row length is not a multiple of 16 bytes takes the other path.
+//  * otherwise: rows 36 floats apart, read back one row per instruction and
+//    written with element stores that are contiguous per row.
+// `stage` = shared-memory address of the warp's 8 KiB; `sel` alternates between
+// its two blocks; row0 = global row of lane 0; b = batch item.
 template <bool OUT_BF16>
-__device__ __forceinline__ void store_block_staged(const GemmParams &p, float *stage, const float (&v)[32],
-                                                   long long batch_off, int row0, int col0, int lane)
+__device__ __forceinline__ void store_block_staged(const GemmParams &p, const CUtensorMap *tmap_c,
+                                                   uint32_t stage, uint32_t &sel, const float (&v)[32],
+                                                   int b, int row0, int col0, int lane)
 {
+    if (p.c_tma && (col0 + 32 <= p.N || p.n_edge_tma)) {
+        const uint32_t blk = stage + sel * 4096u;
+        sel ^= 1u;
+        if (lane == 0) bulk_wait_group_read<1>();        // the store before the last one has read `blk`
+        __syncwarp();
+        if (OUT_BF16) {
+            const uint32_t row = blk + lane * 64;
+            const uint32_t x = (lane >> 1) & 3;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                st_shared_v4_b32(row + ((q ^ x) << 4), pack_bf16x2(v[8 * q], v[8 * q + 1]),
+                                 pack_bf16x2(v[8 * q + 2], v[8 * q + 3]), pack_bf16x2(v[8 * q + 4], v[8 * q + 5]),
+                                 pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+        } else {
+            const uint32_t row = blk + lane * 128;
+            const uint32_t x = lane & 7;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                st_shared_v4(row + ((q ^ x) << 4), v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        }
+        fence_proxy_async_smem();                        // generic-proxy writes -> visible to the TMA unit
+        __syncwarp();
+        if (lane == 0) {
+            tma_store_3d(tmap_c, blk, col0, row0, b);
+            bulk_commit_group();
+        }
+        return;
+    }
+    if (p.c_tma) {                                       // earlier TMA stores may still read the staging blocks
+        if (lane == 0) bulk_wait_group_read<0>();
+        __syncwarp();
+    }
 #pragma unroll
     for (int q = 0; q < 8; ++q)
-        *reinterpret_cast<float4 *>(stage + lane * kEpiPitch + 4 * q) =
-            make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        st_shared_v4(stage + (lane * kEpiPitch + 4 * q) * 4, v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
     __syncwarp();
     const int rows = min(32, p.M - row0);                // > 0 for at least lane 0's row by construction
-    const bool full_cols = col0 + 32 <= p.N;
-    if (OUT_BF16) {
-        __nv_bfloat16 *C = reinterpret_cast<__nv_bfloat16 *>(p.C) + batch_off;
-        if (p.c_vec_ok && full_cols) {
-            // lane -> row r = 8 i + lane / 4, 8 columns from 8 * (lane % 4): one 16-byte store
-            const int piece = (lane & 3) * 8;
+    const bool col_ok = col0 + lane < p.N;
+    const long long off0 = static_cast<long long>(b) * p.strideC + static_cast<long long>(row0) * p.ldc + col0 + lane;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int r = 8 * i + (lane >> 2);
-                const float4 x = *reinterpret_cast<const float4 *>(stage + r * kEpiPitch + piece);
-                const float4 y = *reinterpret_cast<const float4 *>(stage + r * kEpiPitch + piece + 4);
-                if (r < rows) {
-                    uint4 w;
-                    w.x = pack_bf16x2(x.x, x.y); w.y = pack_bf16x2(x.z, x.w);
-                    w.z = pack_bf16x2(y.x, y.y); w.w = pack_bf16x2(y.z, y.w);
-                    *reinterpret_cast<uint4 *>(C + static_cast<long long>(row0 + r) * p.ldc + col0 + piece) = w;
-                }
-            }
-        } else {
-            const bool col_ok = col0 + lane < p.N;
-#pragma unroll 4
-            for (int r = 0; r < 32; ++r) {
-                const float x = stage[r * kEpiPitch + lane];
-                if (r < rows && col_ok)
-                    C[static_cast<long long>(row0 + r) * p.ldc + col0 + lane] = __float2bfloat16_rn(x);
-            }
-        }
-    } else {
-        float *C = reinterpret_cast<float *>(p.C) + batch_off;
-        if (p.c_vec_ok && full_cols) {
-            // lane -> row r = 4 i + lane / 8, 4 columns from 4 * (lane % 8): one 16-byte store
-            const int piece = (lane & 7) * 4;
+    for (int r0 = 0; r0 < 32; r0 += 8) {
+        float x[8];                                      // reads first: C may alias nothing, but the compiler cannot tell
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int r = 4 * i + (lane >> 3);
-                const float4 x = *reinterpret_cast<const float4 *>(stage + r * kEpiPitch + piece);
-                if (r < rows)
-                    *reinterpret_cast<float4 *>(C + static_cast<long long>(row0 + r) * p.ldc + col0 + piece) = x;
-            }
-        } else {
-            const bool col_ok = col0 + lane < p.N;
-#pragma unroll 4
-            for (int r = 0; r < 32; ++r) {
-                const float x = stage[r * kEpiPitch + lane];
-                if (r < rows && col_ok) C[static_cast<long long>(row0 + r) * p.ldc + col0 + lane] = x;
+        for (int i = 0; i < 8; ++i) x[i] = ld_shared_f32(stage + ((r0 + i) * kEpiPitch + lane) * 4);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (r0 + i < rows && col_ok) {
+                const long long off = off0 + static_cast<long long>(r0 + i) * p.ldc;
+                if (OUT_BF16) reinterpret_cast<__nv_bfloat16 *>(p.C)[off] = __float2bfloat16_rn(x[i]);
+                else          reinterpret_cast<float *>(p.C)[off] = x[i];
             }
         }
     }
@@ -267,7 +311,8 @@ __device__ __forceinline__ void store_block_staged(const GemmParams &p, float *s
 template <int BLOCK_N, bool OUT_BF16>
 __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoord &c, int row,
                                               uint32_t t_addr, int quad, int lane, int cta_slot,
-                                              int ctas_per_tile, volatile int *abort_flag, float *stage)
+                                              int ctas_per_tile, volatile int *abort_flag,
+                                              const CUtensorMap *tmap_c, uint32_t stage, uint32_t &sel)
 {
     constexpr int kTileF4 = kBlockM * BLOCK_N / 4;
     constexpr int kChunks = BLOCK_N / 32;
@@ -309,7 +354,6 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
         __threadfence();
     }
 
-    const long long batch_off = static_cast<long long>(c.b) * p.strideC;
     const int row0 = row - lane;                         // global row of this warp's lane 0
     if (row0 >= p.M) return ok;                          // the whole warp is below the matrix
     const float4 *tile0 = reinterpret_cast<const float4 *>(p.partials)
@@ -347,15 +391,15 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
                 }
             }
         }
-        store_block_staged<OUT_BF16>(p, stage, v, batch_off, row0, col0, lane);
+        store_block_staged<OUT_BF16>(p, tmap_c, stage, sel, v, c.b, row0, col0, lane);
     }
     return ok;
 }
 
 template <int BLOCK_N, int STAGES, bool OUT_BF16>
 __global__ void __launch_bounds__(kNumThreads, 1)
-umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
-                 const __grid_constant__ CUtensorMap tmap_b, const GemmParams p)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                 const __grid_constant__ CUtensorMap tmap_c, const GemmParams p)
 {
     using L = SmemLayout<BLOCK_N, STAGES>;
     static_assert(BLOCK_N % 64 == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
@@ -390,6 +434,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         fence_proxy_async_smem();
         prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
+        if (p.c_tma) prefetch_tensormap(&tmap_c);
     }
     if (warp_idx == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
@@ -483,6 +528,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         const int epi_tid = quad * 32 + lane;            // == row within the tile
         int acc = 0;
         uint32_t acc_phase = 0;
+        uint32_t sel = 0;                                // staging block of the next TMA store
+        const uint32_t stage_addr = smem_base + L::kEpiOffset + quad * kEpiWarpBytes;
         for (int u = blockIdx.x; u < p.num_units; u += gridDim.x) {
             const UnitCoord c = decode_unit(p, u);
             bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
@@ -494,9 +541,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tc_fence_after();
             if (!epilogue_tile<BLOCK_N, OUT_BF16>(p, c, c.m_tile * kBlockM + epi_tid,
                                                   tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(quad * 32) << 16),
-                                                  quad, lane, 0, 1, abort_flag,
-                                                  reinterpret_cast<float *>(smem + L::kEpiOffset)
-                                                      + quad * 32 * kEpiPitch)) {
+                                                  quad, lane, 0, 1, abort_flag, &tmap_c, stage_addr, sel)) {
                 if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0xC0);
             }
             tc_fence_before();
@@ -504,6 +549,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             if (lane == 0) mbar_arrive(tempty_bar(acc));
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
+        if (lane == 0) bulk_wait_group_read<0>();        // shared memory must outlive the TMA stores
     }
 
     tc_fence_before();

@@ -63,18 +63,18 @@ struct PairSmemLayout {
     static constexpr int kBBytes = kBlockK * (kPairN / 2) * 2;       // 128 columns of B
     static constexpr int kSubBytes = kABytes + kBBytes;              // 32 KB per k-block
     static constexpr int kStageBytes = KSUB * kSubBytes;
-    static constexpr int kBarOffset = STAGES * kStageBytes;
+    static constexpr int kEpiOffset = STAGES * kStageBytes;          // 1024-byte aligned
+    static constexpr int kBarOffset = kEpiOffset + kEpiStageBytes;
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
-    static constexpr int kEpiOffset = (kMiscOffset + 64 + 15) / 16 * 16;
-    static constexpr int kBytes = kEpiOffset + kEpiStageBytes;
+    static constexpr int kBytes = kMiscOffset + 64;
     static constexpr int kDynamicBytes = kBytes + 1024;
 };
 
 template <int STAGES, int KSUB, bool OUT_BF16>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
-umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
-                      const __grid_constant__ CUtensorMap tmap_b, const GemmParams p)
+umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                      const __grid_constant__ CUtensorMap tmap_c, const GemmParams p)
 {
     using L = PairSmemLayout<STAGES, KSUB>;
     constexpr uint32_t kTmemCols = 2 * kPairN;                       // 512: two accumulators
@@ -111,6 +111,7 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
         fence_proxy_async_smem();
         prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
+        if (p.c_tma) prefetch_tensormap(&tmap_c);
     }
     if (warp_idx == 1) {
         tmem_alloc_2cta(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
@@ -218,6 +219,8 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
         const int epi_tid = quad * 32 + lane;
         int acc = 0;
         uint32_t acc_phase = 0;
+        uint32_t sel = 0;
+        const uint32_t stage_addr = smem_base + L::kEpiOffset + quad * kEpiWarpBytes;
         for (int u = pair; u < p.num_units; u += num_pairs) {
             const UnitCoord c = decode_unit(p, u);
             bool ok = mbar_wait<true>(tfull_bar(acc), acc_phase, abort_flag);
@@ -229,9 +232,8 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tc_fence_after();
             if (!epilogue_tile<kPairN, OUT_BF16>(p, c, c.m_tile * kPairM + static_cast<int>(rank) * kBlockM + epi_tid,
                                                  tmem_base + acc * kPairN + (static_cast<uint32_t>(quad * 32) << 16),
-                                                 quad, lane, static_cast<int>(rank), 2, abort_flag,
-                                                 reinterpret_cast<float *>(smem + L::kEpiOffset)
-                                                     + quad * 32 * kEpiPitch)) {
+                                                 quad, lane, static_cast<int>(rank), 2, abort_flag, &tmap_c,
+                                                 stage_addr, sel)) {
                 if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0xC0);
             }
             tc_fence_before();
@@ -239,6 +241,7 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a,
             if (lane == 0) mbar_arrive_remote(map_to_cta(tempty_bar(acc), 0));
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
+        if (lane == 0) bulk_wait_group_read<0>();
     }
 
     tc_fence_before();

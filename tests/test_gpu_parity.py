@@ -120,6 +120,32 @@ def test_batched(batch, out_dtype):
             assert guards and r.ok, (B.variant_name(v), M, N, K, batch, r)
 
 
+@pytest.mark.parametrize("out_dtype", [gi.F32, gi.BF16])
+def test_aligned_c_with_ragged_edges(out_dtype):
+    """C aligned for 16-byte row stores (the epilogue's TMA path) while N and M
+    end inside a 32 x 32 store box: N a multiple of the 16-byte granule or not,
+    N just past a box boundary, M ragged, batch items with padded strides.
+    The padding columns, the rows below M and the guard bands must stay intact."""
+    rng = np.random.default_rng(4242)
+    g = 4 if out_dtype == gi.F32 else 8                    # elements per 16 bytes
+    cases = [(300, 127, 200, 128, 1), (300, 124, 64, 128, 1), (45, 33, 64, 40, 1), (129, 258, 130, 264, 1),
+             (256, 257, 64, 272, 1), (70, 100, 96, 104, 3), (128, 120, 64, 128, 5), (31, 8, 16, 8, 2)]
+    for (M, N, K, ldc, batch) in cases:
+        assert ldc % g == 0
+        sA, sB, sC = M * K, K * N, M * ldc + 3 * g
+        A = gi.random_operand(M + N, 0, M, K, K, batch=batch, stride=sA)
+        Bm = gi.random_operand(M + N, 1, K, N, N, batch=batch, stride=sB)
+        Cref, S = oracle.gemm_batched(A, Bm, M, N, K, K, N, sA, sB, batch)
+        names = ("umma_n64", "umma_n128", "umma_n256", "umma_n64_sk2", "umma2_n256", "umma2_n256_sk2", "umma2_n256_ts")
+        for v in [B.VARIANT_AUTO] + variant_ids(*names):
+            if v >= 0 and B.variant_supports(v, M, N, K, K, N, ldc, batch, out_dtype) != 1:
+                continue
+            vals, raw, guards = G.run_gemm(A, Bm, M, N, K, K, N, ldc, out_dtype, batch, sA, sB, sC, variant=v)
+            r = oracle.check(vals, Cref, S, G.tol_for(out_dtype))
+            assert guards, f"padding or guard band overwritten ({B.variant_name(v)}, {(M, N, K, ldc, batch)})"
+            assert r.ok, (B.variant_name(v), M, N, K, ldc, batch, r)
+
+
 # ------------------------------------------------ integer closed forms: exact --
 
 def all_umma_and_auto(M, N, K, out_dtype, batch=1):
