@@ -12,6 +12,8 @@ Contents
   ``gemm_f32`` / ``gemm_f32_rows`` -- the same for float32 operands.
 * ``bf16_bits_to_f64`` / ``f64_to_bf16_bits`` -- exact widening and
   round-to-nearest-even narrowing, written with integer bit operations.
+* ``transpose_f32`` / ``sum_f32`` / ``dot_f32`` / ``layernorm_f32`` -- the
+  paper's Tasks 8, 14, 15 and 4 on float32 arrays (``oracle_tasks.c``).
 * ``check`` -- the element-wise acceptance rule
   ``|C_gpu - C_ref| <= tol * S`` with ``S = sum_k |a_ik| |b_kj|``.
 
@@ -28,7 +30,7 @@ from dataclasses import dataclass
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRCS = [os.path.join(_HERE, "oracle_gemm.c"), os.path.join(_HERE, "oracle_mhsa.c")]
+_SRCS = [os.path.join(_HERE, f) for f in ("oracle_gemm.c", "oracle_mhsa.c", "oracle_tasks.c")]
 _SRC = _SRCS[0]
 _LIB = os.path.join(_HERE, "liboracle_gemm.so")
 _lock = threading.Lock()
@@ -78,6 +80,14 @@ def _load():
     lib.oracle_gemm_f32_rows.restype = None
     lib.oracle_mhsa_bf16.argtypes = [u16p, u16p, u16p, f64p, f64p] + [i64] * 6
     lib.oracle_mhsa_bf16.restype = ctypes.c_int
+    lib.oracle_transpose_f32.argtypes = [f32p, f32p, i64, i64, i64, i64]
+    lib.oracle_transpose_f32.restype = None
+    lib.oracle_sum_f32.argtypes = [f32p, i64, f64p]
+    lib.oracle_sum_f32.restype = ctypes.c_double
+    lib.oracle_dot_f32.argtypes = [f32p, f32p, i64, f64p]
+    lib.oracle_dot_f32.restype = ctypes.c_double
+    lib.oracle_layernorm_f32.argtypes = [f32p, f32p, f32p, f64p, i64, i64, ctypes.c_double, f64p, f64p]
+    lib.oracle_layernorm_f32.restype = None
     lib.oracle_num_threads.restype = ctypes.c_int
     lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
     _lib = lib
@@ -266,6 +276,74 @@ def mhsa(Q, K, V, N, d_model, h, ldq=None, ldk=None, ldv=None):
     return out, T
 
 
+# --------------------------------------------------------------------------
+# Tasks 8, 14, 15, 4: transpose, sum, dot product, LayerNorm on float32 arrays
+# --------------------------------------------------------------------------
+
+def _f32_flat(x, need: int) -> np.ndarray:
+    x = np.ascontiguousarray(np.asarray(x))
+    if x.dtype != np.float32:
+        raise TypeError("operands are float32")
+    x = x.reshape(-1)
+    if x.size < need:
+        raise ValueError("array too small")
+    return x
+
+
+def transpose_f32(A, rows: int, cols: int, lda: int | None = None, ldat: int | None = None,
+                  fill: float = np.nan) -> np.ndarray:
+    """Task 8: the ``cols x rows`` transpose of the row-major ``rows x cols`` matrix A
+    (row pitch lda).  Returns a flat float32 buffer with row pitch ldat whose
+    padding elements hold ``fill``."""
+    lda = cols if lda is None else lda
+    ldat = rows if ldat is None else ldat
+    if lda < cols or ldat < rows:
+        raise ValueError("pitch smaller than the row length")
+    need = (rows - 1) * lda + cols if rows and cols else 0
+    a = _f32_flat(A, need)
+    out = np.full((cols - 1) * ldat + rows if rows and cols else 0, fill, dtype=np.float32)
+    _load().oracle_transpose_f32(_ptr(a, ctypes.c_float), _ptr(out, ctypes.c_float), rows, cols, lda, ldat)
+    return out
+
+
+def sum_f32(x):
+    """Task 14: (sum of x in fp64, sum of |x|)."""
+    a = _f32_flat(x, 0)
+    s_abs = np.zeros(1)
+    s = _load().oracle_sum_f32(_ptr(a, ctypes.c_float), a.size, _ptr(s_abs, ctypes.c_double))
+    return float(s), float(s_abs[0])
+
+
+def dot_f32(a, b):
+    """Task 15: (a . b in fp64, sum of |a_i||b_i|)."""
+    a = _f32_flat(a, 0)
+    b = _f32_flat(b, a.size)
+    if a.size != b.size:
+        raise ValueError("vectors differ in length")
+    s_abs = np.zeros(1)
+    s = _load().oracle_dot_f32(_ptr(a, ctypes.c_float), _ptr(b, ctypes.c_float), a.size,
+                               _ptr(s_abs, ctypes.c_double))
+    return float(s), float(s_abs[0])
+
+
+def layernorm_f32(x, gamma, beta, batch: int, m: int, eps: float = 1e-5):
+    """Task 4: (y as fp64 ``batch x m``, per-sample mean, per-sample 1/sqrt(var + eps)).
+    gamma / beta: ``m`` float32 values each, or None."""
+    xs = _f32_flat(x, batch * m)
+    g = None if gamma is None else _f32_flat(gamma, m)
+    b = None if beta is None else _f32_flat(beta, m)
+    y = np.empty((batch, m), dtype=np.float64)
+    mean = np.empty(batch)
+    rstd = np.empty(batch)
+    null = ctypes.POINTER(ctypes.c_float)()
+    _load().oracle_layernorm_f32(_ptr(xs, ctypes.c_float), null if g is None else _ptr(g, ctypes.c_float),
+                                 null if b is None else _ptr(b, ctypes.c_float), _ptr(y, ctypes.c_double),
+                                 batch, m, float(eps), _ptr(mean, ctypes.c_double), _ptr(rstd, ctypes.c_double))
+    return y, mean, rstd
+
+
+TOL_SUM = 2.0 ** -23      # |s_gpu - s_ref| <= 2^-23 * sum|x_i|: fp64 accumulation, one rounding to float32
+TOL_LAYERNORM = 4e-6      # |y_gpu - y_ref| <= 4e-6 * (|x - mean| * rstd * |gamma| + |beta|) + 1e-6 * |gamma|
 TOL_MHSA = 1e-2      # |O_gpu - O_ref| <= 1e-2 * T  (probabilities are rounded to bf16 on the GPU)
 TOL_F32_IN = 1e-5    # |C_gpu - C_ref| <= 1e-5 * S for the fp32-operand path (see DESIGN.md)
 
