@@ -1,0 +1,95 @@
+/*
+ * cudallm_tasks.h -- C ABI of the bandwidth-bound benchmark tasks of the paper
+ * on arrays of 32-bit floating point numbers (its Table of task prompts):
+ *
+ *   Task 8   Matrix Transpose   AT[j][i] = A[i][j]
+ *   Task 14  Reduction          s = sum_i x_i
+ *   Task 15  Dot Product        s = sum_{i<n} A_i * B_i
+ *   Task 4   LayerNorm          per sample: normalise over all its elements,
+ *                               then scale by gamma and add beta
+ *
+ * The general conventions of cudallm_gemm.h hold (device pointers owned by the
+ * caller, pitches in elements, calls enqueue on `stream` and return without
+ * synchronising, negative CUDALLM_ERR_* status codes, argument errors found
+ * before any CUDA call, compute capability 10.0 only, no CPU fallback).  The
+ * status codes are those of cudallm_gemm.h.  A bounded wait inside the
+ * transpose or the LayerNorm kernel that runs out is reported through
+ * cudallm_device_status().
+ *
+ * cudallm_sum_f32 / cudallm_dot_f32 keep their per-block partial sums in one
+ * fixed scratch area per device, and cudallm_layernorm_f32 keeps its per-sample
+ * partial statistics in the library workspace: calls of these functions must
+ * not run concurrently on different streams of one device.
+ */
+#ifndef CUDALLM_TASKS_H
+#define CUDALLM_TASKS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#include "cudallm_gemm.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/*
+ * Task 8: AT = transpose(A).
+ *   A  : fp32, rows x cols, row-major, row pitch lda  >= cols   (read only)
+ *   AT : fp32, cols x rows, row-major, row pitch ldat >= rows   (written; padding
+ *        columns rows <= i < ldat are left untouched); must not overlap A.
+ * Values are moved bit for bit (NaN payloads and signed zeros included).
+ * 16-byte aligned bases with rows, cols, lda and ldat all multiples of 4 take
+ * the TMA path; anything else (4-byte alignment is required) a plain tiled
+ * kernel.  rows == 0 or cols == 0: success, nothing written.
+ * Errors: INVALID_DIM (negative, or >= 2^31 - 1024), INVALID_LD, INVALID_POINTER,
+ * MISALIGNED, UNSUPPORTED_DEVICE, CUDA.
+ */
+int cudallm_transpose_f32(const float *A, float *AT, int64_t rows, int64_t cols, int64_t lda, int64_t ldat,
+                          void *stream);
+
+/*
+ * Task 14: *result = sum_{i<n} x[i].
+ *   x      : fp32, n elements (read only); result : one fp32 on the DEVICE.
+ * Every element is widened to double and added in double; the total is rounded
+ * to fp32 once, so |result - exact| <= 2^-24 |exact| + ~1e-13 sum|x_i|.  Equal
+ * inputs give bit-equal results.  n == 0 gives 0.  One kernel launch.
+ * Errors: INVALID_DIM (n < 0 or n > 2^40), INVALID_POINTER, MISALIGNED (4 bytes),
+ * UNSUPPORTED_DEVICE, CUDA.
+ */
+int cudallm_sum_f32(const float *x, int64_t n, float *result, void *stream);
+
+/*
+ * Task 15: *result = sum_{i<n} a[i] * b[i].
+ * Products are formed in double (exact) and added in double; one rounding to
+ * fp32 at the end.  Otherwise as cudallm_sum_f32.  a and b may be the same array.
+ */
+int cudallm_dot_f32(const float *a, const float *b, int64_t n, float *result, void *stream);
+
+/*
+ * Task 4: LayerNorm of `batch` samples of m elements each (the paper's input of
+ * shape (batch_size, features, dim1, dim2) has m = features * dim1 * dim2 and is
+ * passed as it lies in memory: sample s occupies x[s*m .. s*m + m)).
+ *     mean_s = (1/m) sum_i x[s][i]
+ *     var_s  = (1/m) sum_i (x[s][i] - mean_s)^2              (biased estimate)
+ *     y[s][i] = (x[s][i] - mean_s) / sqrt(var_s + eps) * gamma[i] + beta[i]
+ *   x, y        : fp32, batch * m elements; y may be x itself (in place), else
+ *                 must not overlap x
+ *   gamma, beta : fp32, m elements each (one per position of a sample), or NULL
+ *                 for "all ones" / "all zeros"
+ *   eps         : >= 0 (the usual value is 1e-5)
+ * Statistics are accumulated in double; (x - mean) / sqrt(var + eps) is formed
+ * in double and rounded to fp32, then one fp32 multiply-add applies gamma and
+ * beta.  batch == 0 or m == 0: success, nothing written.
+ * Errors: INVALID_DIM (negative, batch >= 2^31, m > 2^40, eps negative or not
+ * finite), INVALID_POINTER (x or y NULL), MISALIGNED (4 bytes), WORKSPACE (an
+ * external workspace is set and too small), UNSUPPORTED_DEVICE, CUDA.
+ */
+int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta, float *y, int64_t batch,
+                          int64_t m, float eps, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+
+#endif /* CUDALLM_TASKS_H */

@@ -38,7 +38,7 @@ _vp = ctypes.c_void_p
 _int = ctypes.c_int
 _sz = ctypes.c_size_t
 
-# name -> (restype, argtypes); mirrors include/cudallm_gemm.h
+# name -> (restype, argtypes); mirrors include/cudallm_gemm.h and include/cudallm_tasks.h
 SIGNATURES = {
     "cudallm_gemm_bf16": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp]),
     "cudallm_gemm_f32": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp]),
@@ -57,6 +57,10 @@ SIGNATURES = {
     "cudallm_device_status": (_int, [_vp, ctypes.POINTER(_int), ctypes.POINTER(_int)]),
     "cudallm_strerror": (ctypes.c_char_p, [_int]),
     "cudallm_version": (_int, []),
+    "cudallm_transpose_f32": (_int, [_vp, _vp] + [_i64] * 4 + [_vp]),
+    "cudallm_sum_f32": (_int, [_vp, _i64, _vp, _vp]),
+    "cudallm_dot_f32": (_int, [_vp, _vp, _i64, _vp, _vp]),
+    "cudallm_layernorm_f32": (_int, [_vp, _vp, _vp, _vp, _i64, _i64, ctypes.c_float, _vp]),
 }
 
 
@@ -126,6 +130,30 @@ def mhsa_bf16(Q, K, V, O, N, d_model, h, ldq, ldk, ldv, ldo, stream=None, check=
     """Multi-head self-attention (Task 6): bf16 Q, K, V (N x d_model), fp32 O."""
     st = lib().cudallm_mhsa_bf16(_p(Q), _p(K), _p(V), _p(O), N, d_model, h, ldq, ldk, ldv, ldo, _s(stream))
     return _check(st, "cudallm_mhsa_bf16", check)
+
+
+def transpose_f32(A, AT, rows, cols, lda, ldat, stream=None, check=True):
+    """Task 8: AT (cols x rows, pitch ldat) = transpose of A (rows x cols, pitch lda), fp32."""
+    st = lib().cudallm_transpose_f32(_p(A), _p(AT), rows, cols, lda, ldat, _s(stream))
+    return _check(st, "cudallm_transpose_f32", check)
+
+
+def sum_f32(x, n, result, stream=None, check=True):
+    """Task 14: result[0] (device fp32) = sum of the n fp32 elements of x."""
+    st = lib().cudallm_sum_f32(_p(x), n, _p(result), _s(stream))
+    return _check(st, "cudallm_sum_f32", check)
+
+
+def dot_f32(a, b, n, result, stream=None, check=True):
+    """Task 15: result[0] (device fp32) = a . b over n fp32 elements."""
+    st = lib().cudallm_dot_f32(_p(a), _p(b), n, _p(result), _s(stream))
+    return _check(st, "cudallm_dot_f32", check)
+
+
+def layernorm_f32(x, gamma, beta, y, batch, m, eps=1e-5, stream=None, check=True):
+    """Task 4: LayerNorm of ``batch`` samples of ``m`` fp32 elements; gamma / beta may be None."""
+    st = lib().cudallm_layernorm_f32(_p(x), _p(gamma), _p(beta), _p(y), batch, m, ctypes.c_float(eps), _s(stream))
+    return _check(st, "cudallm_layernorm_f32", check)
 
 
 def gemm_bf16_batched(A, B, C, M, N, K, lda, ldb, ldc, strideA, strideB, strideC, batch,

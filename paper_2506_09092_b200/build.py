@@ -12,7 +12,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libcudallm_gemm.so")
-HEADER = os.path.join(os.path.dirname(PKG), "include", "cudallm_gemm.h")
+HEADERS = sorted(glob.glob(os.path.join(os.path.dirname(PKG), "include", "*.h")))
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
@@ -27,7 +27,7 @@ def sources():
 
 
 def _deps():
-    return sources() + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + [HEADER]
+    return sources() + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + HEADERS
 
 
 def up_to_date() -> bool:

@@ -2,12 +2,14 @@
 // selection, workspace, tensor-map encoding and kernel launches.
 // See include/cudallm_gemm.h for the contract of every entry point.
 #include "../../include/cudallm_gemm.h"
+#include "../../include/cudallm_tasks.h"
 
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <algorithm>
 #include <cstring>
 #include <mutex>
 
@@ -15,6 +17,7 @@
 #include "umma_gemm.cuh"
 #include "umma_gemm_2cta.cuh"
 #include "mhsa.cuh"
+#include "hbm_tasks.cuh"
 
 using namespace cudallm;
 
@@ -398,7 +401,7 @@ struct MapKey {
     const void *base;
     int64_t inner, rows, batch, ld, stride;
     int box_inner, box_rows;
-    int kind;                              // 0 = bf16 operand, 1 = fp32 C, 2 = bf16 C
+    int kind;                              // 0 = bf16 operand, 1 = fp32 C, 2 = bf16 C, 3 = fp32 input
     bool operator==(const MapKey &o) const
     {
         return base == o.base && inner == o.inner && rows == o.rows && batch == o.batch && ld == o.ld
@@ -415,7 +418,8 @@ struct MapCache {
 MapCache g_map_cache[kMaxDevices];
 
 // kind 0: a bf16 operand read in 128-byte-swizzled boxes; kind 1 / 2: fp32 / bf16
-// C written in boxes of 32 columns x 32 rows (128- / 64-byte swizzle).
+// C written in boxes of 32 columns x 32 rows (128- / 64-byte swizzle); kind 3: an
+// fp32 matrix read in such boxes.
 int encode_map(int dev, CUtensorMap *tm, const void *base, int64_t inner, int64_t rows, int64_t batch,
                int64_t ld, int64_t stride, int box_inner, int box_rows, int kind)
 {
@@ -426,16 +430,16 @@ int encode_map(int dev, CUtensorMap *tm, const void *base, int64_t inner, int64_
             *tm = mc.map[i];
             return CUDALLM_OK;
         }
-    const cuuint64_t es = (kind == 1) ? 4 : 2;
+    const cuuint64_t es = (kind == 1 || kind == 3) ? 4 : 2;
     cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batch};
     cuuint64_t item_stride = (batch > 1) ? (cuuint64_t)stride * es : (cuuint64_t)rows * ld * es;
     cuuint64_t strides[2] = {(cuuint64_t)ld * es, item_stride};
     cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = g_encode(tm, kind == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+    CUresult r = g_encode(tm, (kind == 1 || kind == 3) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
                           const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                           kind == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
-                          kind == 0 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          (kind == 0 || kind == 3) ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -1201,3 +1205,5 @@ int cudallm_version(void)
 }
 
 }  // extern "C"
+
+#include "hbm_tasks_host.cuh"

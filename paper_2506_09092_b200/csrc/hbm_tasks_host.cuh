@@ -1,0 +1,168 @@
+// Host side of the entry points declared in include/cudallm_tasks.h.  This file
+// is included at the end of cudallm_gemm.cu and uses that file's device state,
+// workspace, tensor-map cache and error plumbing.
+#pragma once
+
+namespace {
+
+__device__ cudallm::ReduceScratch g_reduce_scratch;      // zero-initialised: the ticket starts at 0
+
+constexpr int64_t kTaskMaxElems = int64_t(1) << 40;
+
+int task_device(int *dev_out)
+{
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    *dev_out = dev;
+    return probe_device(dev);
+}
+
+int run_reduce(const float *a, const float *b, int64_t n, float *result, bool dot, void *stream_v)
+{
+    if (n < 0 || n > kTaskMaxElems) return CUDALLM_ERR_INVALID_DIM;
+    if (!result || (n > 0 && (!a || (dot && !b)))) return CUDALLM_ERR_INVALID_POINTER;
+    if ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(result)
+         | (dot ? reinterpret_cast<uintptr_t>(b) : 0)) & 3)
+        return CUDALLM_ERR_MISALIGNED;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int st = task_device(&dev);
+    if (st != CUDALLM_OK) return st;
+    ReduceScratch *scratch = nullptr;
+    CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void **>(&scratch), g_reduce_scratch));
+    // one block per 8192 elements, at most four blocks of 512 threads per SM
+    int64_t blocks = cdiv(n, int64_t(kRedThreads) * 16);
+    const int64_t cap = std::min<int64_t>(kRedMaxBlocks, int64_t(4) * g_dev[dev].sm_count);
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    const bool vec = !dot || ((reinterpret_cast<uintptr_t>(a) & 15) == (reinterpret_cast<uintptr_t>(b) & 15));
+    const unsigned g = (unsigned)blocks;
+    if (dot) {
+        if (vec) reduce_kernel<true, true><<<g, kRedThreads, 0, stream>>>(a, b, n, result, scratch);
+        else     reduce_kernel<true, false><<<g, kRedThreads, 0, stream>>>(a, b, n, result, scratch);
+    } else {
+        reduce_kernel<false, true><<<g, kRedThreads, 0, stream>>>(a, a, n, result, scratch);
+    }
+    CUDA_TRY(cudaGetLastError());
+    return CUDALLM_OK;
+}
+
+}  // namespace
+
+int cudallm_sum_f32(const float *x, int64_t n, float *result, void *stream)
+{
+    return run_reduce(x, nullptr, n, result, false, stream);
+}
+
+int cudallm_dot_f32(const float *a, const float *b, int64_t n, float *result, void *stream)
+{
+    return run_reduce(a, b, n, result, true, stream);
+}
+
+int cudallm_transpose_f32(const float *A, float *AT, int64_t rows, int64_t cols, int64_t lda, int64_t ldat,
+                          void *stream_v)
+{
+    if (rows < 0 || cols < 0 || rows > kMaxDim || cols > kMaxDim) return CUDALLM_ERR_INVALID_DIM;
+    if (rows == 0 || cols == 0) return CUDALLM_OK;
+    if (lda < cols || ldat < rows) return CUDALLM_ERR_INVALID_LD;
+    if (lda > kTaskMaxElems || ldat > kTaskMaxElems) return CUDALLM_ERR_INVALID_DIM;
+    if ((long double)rows * lda > (long double)kMaxElems || (long double)cols * ldat > (long double)kMaxElems)
+        return CUDALLM_ERR_INVALID_DIM;
+    if (!A || !AT) return CUDALLM_ERR_INVALID_POINTER;
+    if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(AT)) & 3) return CUDALLM_ERR_MISALIGNED;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int st = task_device(&dev);
+    if (st != CUDALLM_OK) return st;
+    DeviceState &d = g_dev[dev];
+
+    const bool tma = ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(AT)) & 15) == 0
+                  && rows % 4 == 0 && cols % 4 == 0 && lda % 4 == 0 && ldat % 4 == 0;
+    if (!tma) {
+        const int64_t tiles_c = cdiv(cols, 32);
+        const int64_t tiles = cdiv(rows, 32) * tiles_c;
+        const int64_t grid = std::min<int64_t>(tiles, int64_t(d.sm_count) * 16);
+        transpose_simple_kernel<<<(unsigned)grid, 256, 0, stream>>>(A, AT, (int)rows, (int)cols, lda, ldat,
+                                                                    (int)tiles_c, tiles);
+        CUDA_TRY(cudaGetLastError());
+        return CUDALLM_OK;
+    }
+    st = ensure_workspace(dev, kHeaderBytes, stream);          // for the status word
+    if (st != CUDALLM_OK) return st;
+    CUtensorMap tin, tout;
+    st = encode_map(dev, &tin, A, cols, rows, 1, lda, 0, 32, 32, 3);
+    if (st != CUDALLM_OK) return st;
+    st = encode_map(dev, &tout, AT, rows, cols, 1, ldat, 0, 32, 32, 1);
+    if (st != CUDALLM_OK) return st;
+    TransposeParams tp{};
+    tp.rows = (int)rows; tp.cols = (int)cols;
+    tp.patches_r = (int)cdiv(rows, kTrPatch);
+    tp.patches_c = (int)cdiv(cols, kTrPatch);
+    tp.status = static_cast<int *>(d.ws);
+    if (!d.smem_attr_set[9]) {
+        CUDA_TRY(cudaFuncSetAttribute(transpose_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      kTrSmemBytes));
+        d.smem_attr_set[9] = true;
+    }
+    const int64_t patches = int64_t(tp.patches_r) * tp.patches_c;
+    const int64_t grid = std::min<int64_t>(cdiv(patches, kTrWarps), d.sm_count);
+    transpose_tma_kernel<<<(unsigned)grid, kTrWarps * 32, kTrSmemBytes, stream>>>(tin, tout, tp);
+    CUDA_TRY(cudaGetLastError());
+    return CUDALLM_OK;
+}
+
+int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta, float *y, int64_t batch,
+                          int64_t m, float eps, void *stream_v)
+{
+    if (batch < 0 || m < 0 || batch > kMaxDim || m > kTaskMaxElems) return CUDALLM_ERR_INVALID_DIM;
+    if (!(eps >= 0.f) || !(eps <= 3.0e38f)) return CUDALLM_ERR_INVALID_DIM;
+    if ((long double)batch * m > (long double)kMaxElems) return CUDALLM_ERR_INVALID_DIM;
+    if (batch == 0 || m == 0) return CUDALLM_OK;
+    if (!x || !y) return CUDALLM_ERR_INVALID_POINTER;
+    const uintptr_t all = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)
+                        | reinterpret_cast<uintptr_t>(gamma) | reinterpret_cast<uintptr_t>(beta);
+    if (all & 3) return CUDALLM_ERR_MISALIGNED;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int st = task_device(&dev);
+    if (st != CUDALLM_OK) return st;
+    DeviceState &d = g_dev[dev];
+
+    // Groups that run side by side: at most one per sample, at most one per SM,
+    // and few enough that two samples per group (the one being normalised and
+    // the one whose sums are being taken) stay within 48 MB of L2.
+    const int64_t sample_bytes = m * 4;
+    int64_t groups = std::max<int64_t>(1, (int64_t(48) << 20) / (2 * sample_bytes));
+    groups = std::min<int64_t>(groups, std::min<int64_t>(batch, d.sm_count));
+    // CTAs per group: the SMs divided among the groups, but at least 4096 elements per CTA
+    int64_t G = std::max<int64_t>(1, std::min<int64_t>(d.sm_count / groups, cdiv(m, 4096)));
+    const int64_t slice = round_up(cdiv(m, G), 4);
+    G = cdiv(m, slice);                                        // no empty CTAs
+    const bool vec = (all & 15) == 0 && m % 4 == 0;
+
+    const size_t off_arrived = kHeaderBytes;
+    const size_t off_partials = (size_t)round_up((int64_t)(off_arrived + (size_t)batch * 4), 256);
+    const size_t total = off_partials + (size_t)batch * (size_t)G * 16;
+    st = ensure_workspace(dev, total, stream);
+    if (st != CUDALLM_OK) return st;
+    uint8_t *ws = static_cast<uint8_t *>(d.ws);
+    CUDA_TRY(cudaMemsetAsync(ws + off_arrived, 0, (size_t)batch * 4, stream));
+
+    LayerNormParams lp{};
+    lp.x = x; lp.gamma = gamma; lp.beta = beta; lp.y = y;
+    lp.m = m; lp.slice = slice;
+    lp.batch = (int)batch; lp.group_size = (int)G; lp.num_groups = (int)groups;
+    lp.eps = (double)eps;
+    lp.partials = reinterpret_cast<double *>(ws + off_partials);
+    lp.arrived = reinterpret_cast<unsigned int *>(ws + off_arrived);
+    lp.status = reinterpret_cast<int *>(ws);
+    const unsigned grid = (unsigned)(groups * G);              // <= SM count: all CTAs are resident
+    if (vec) layernorm_kernel<true><<<grid, kLnThreads, 0, stream>>>(lp);
+    else     layernorm_kernel<false><<<grid, kLnThreads, 0, stream>>>(lp);
+    CUDA_TRY(cudaGetLastError());
+    return CUDALLM_OK;
+}

@@ -236,3 +236,39 @@ def fnv1a64(a: np.ndarray) -> int:
         h = (h ^ acc) * prime
         h = (h ^ s) * prime
     return int(h)
+
+
+# Tasks 8, 14, 15, 4: float32 arrays -------------------------------------------
+# The paper's sizes (its table of input sizes): transpose N x N with N = 2^10 ..
+# 2^14; reduction N = 2^10 .. 2^18 (steps of 4x); dot product N = 2^16 .. 2^20;
+# LayerNorm (16, 4, d, d) with d = 2^6 .. 2^10.  Values are seeded float32 draws.
+
+TRANSPOSE_SIZES = [1 << k for k in range(10, 15)]
+REDUCTION_SIZES = [1 << k for k in range(10, 19, 2)]
+DOT_SIZES = [1 << k for k in range(16, 21)]
+LAYERNORM_SHAPES = [(16, 4, 1 << k, 1 << k) for k in range(6, 11)]
+
+
+def task_array(seed: int, which: int, n: int, dist: str = "normal", std: float = 1.0,
+               mean: float = 0.0) -> np.ndarray:
+    """``n`` float32 values from ``default_rng([seed, which])``: ``normal`` (times std, plus
+    mean) or ``uniform`` on [-1, 1) (plus mean)."""
+    rng = np.random.default_rng([int(seed), int(which)])
+    if dist == "uniform":
+        x = rng.uniform(-1.0, 1.0, n).astype(np.float32)
+    else:
+        x = rng.standard_normal(n, dtype=np.float32) * np.float32(std)
+    if mean:
+        x = x + np.float32(mean)
+    return np.ascontiguousarray(x, dtype=np.float32)
+
+
+def layernorm_inputs(seed: int, batch: int, m: int):
+    """(x [batch * m], gamma [m], beta [m]) as float32: samples with different means and
+    spreads (sample s: mean s - batch / 2, std 0.5 + s / 4), gamma around 1, beta around 0."""
+    x = task_array(seed, 0, batch * m).reshape(batch, m)
+    s = np.arange(batch, dtype=np.float32)[:, None]
+    x = x * (np.float32(0.5) + s / np.float32(4)) + (s - np.float32(batch / 2))
+    gamma = task_array(seed, 1, m, "uniform") * np.float32(0.5) + np.float32(1.0)
+    beta = task_array(seed, 2, m) * np.float32(0.1)
+    return np.ascontiguousarray(x.reshape(-1), dtype=np.float32), gamma, beta
