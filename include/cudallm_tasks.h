@@ -78,9 +78,10 @@ int cudallm_dot_f32(const float *a, const float *b, int64_t n, float *result, vo
  *   gamma, beta : fp32, m elements each (one per position of a sample), or NULL
  *                 for "all ones" / "all zeros"
  *   eps         : >= 0 (the usual value is 1e-5)
- * Statistics are accumulated in double; (x - mean) / sqrt(var + eps) is formed
- * in double and rounded to fp32, then one fp32 multiply-add applies gamma and
- * beta.  batch == 0 or m == 0: success, nothing written.
+ * Statistics are accumulated in double.  The output is formed in fp32 from the
+ * mean held as two floats (so a mean far larger than the spread costs no
+ * accuracy) and 1/sqrt(var + eps) rounded to fp32:
+ * |y - exact| <= 2^-22 (|x - mean| |gamma| / sqrt(var + eps) + |beta|).  batch == 0 or m == 0: success, nothing written.
  * Errors: INVALID_DIM (negative, batch >= 2^31, m > 2^40, eps negative or not
  * finite), INVALID_POINTER (x or y NULL), MISALIGNED (4 bytes), WORKSPACE (an
  * external workspace is set and too small), UNSUPPORTED_DEVICE, CUDA.

@@ -132,21 +132,42 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
     if (st != CUDALLM_OK) return st;
     DeviceState &d = g_dev[dev];
 
-    // Groups that run side by side: at most one per sample, at most one per SM,
-    // and few enough that two samples per group (the one being normalised and
-    // the one whose sums are being taken) stay within 48 MB of L2.
-    const int64_t sample_bytes = m * 4;
-    int64_t groups = std::max<int64_t>(1, (int64_t(48) << 20) / (2 * sample_bytes));
-    groups = std::min<int64_t>(groups, std::min<int64_t>(batch, d.sm_count));
-    // CTAs per group: the SMs divided among the groups, but at least 4096 elements per CTA
-    int64_t G = std::max<int64_t>(1, std::min<int64_t>(d.sm_count / groups, cdiv(m, 4096)));
-    const int64_t slice = round_up(cdiv(m, G), 4);
-    G = cdiv(m, slice);                                        // no empty CTAs
-    const bool vec = (all & 15) == 0 && m % 4 == 0;
+    const bool vec = (all & 31) == 0 && m % 8 == 0;            // 32-byte loads and stores
+    const int sms = d.sm_count;
+    // Aligned data is cut into 4 KiB blocks that the CTAs of a group take in turn.
+    const int64_t total_blocks = cdiv(m, (int64_t)kLnBlockPieces * 8);
+    // Shared-memory kernel: the blocks of a bundle of T samples per CTA, one CTA per SM.
+    constexpr int64_t kLnSmemBudget = 227 * 1024 - 2048;
+    const int64_t cap = kLnSmemBudget / 4;                     // elements of shared memory per CTA
+    int64_t groups = 1, T = 1;
+    int64_t G = std::max<int64_t>(1, std::min<int64_t>(sms, total_blocks));
+    const int64_t chunks = cdiv(cdiv(total_blocks, G), kLnChunkBlocks);
+    int64_t slice = cdiv(total_blocks, G) * (kLnBlockBytes / 4);   // shared memory per sample, in elements
+    bool use_smem = vec && slice <= cap && chunks <= kLnMaxChunks;
+    if (use_smem) {
+        const int64_t max_groups = std::max<int64_t>(1, sms / G);
+        // samples per bundle: what fits, but no more than needed to give every group one bundle
+        while (T * 2 <= kLnMaxBundle && T * 2 * slice <= cap && T * max_groups < batch) T *= 2;
+        groups = std::min<int64_t>(max_groups, cdiv(batch, T));
+        // More than two bundles per group: every bundle costs a meeting of the group with
+        // the memory system idle; streaming with fewer meetings is cheaper even though x
+        // is then read twice.
+        if (cdiv(cdiv(batch, T), groups) > 2) use_smem = false;
+    }
+    if (!use_smem) {
+        // Streaming kernel, one CTA per SM: blocks in turn (aligned data) or contiguous
+        // slices of at least 1024 elements (anything else).
+        G = std::max<int64_t>(1, std::min<int64_t>(sms, vec ? total_blocks : m / 1024));
+        slice = round_up(cdiv(m, G), 8);
+        if (!vec) G = cdiv(m, slice);                          // no empty CTAs
+        const int64_t max_groups = std::max<int64_t>(1, sms / G);
+        T = std::min<int64_t>(kLnMaxBundle, std::max<int64_t>(1, cdiv(batch, max_groups)));
+        groups = std::min<int64_t>(max_groups, cdiv(batch, T));
+    }
 
     const size_t off_arrived = kHeaderBytes;
     const size_t off_partials = (size_t)round_up((int64_t)(off_arrived + (size_t)batch * 4), 256);
-    const size_t total = off_partials + (size_t)batch * (size_t)G * 16;
+    const size_t total = off_partials + (size_t)batch * (size_t)G * 32;
     st = ensure_workspace(dev, total, stream);
     if (st != CUDALLM_OK) return st;
     uint8_t *ws = static_cast<uint8_t *>(d.ws);
@@ -155,14 +176,25 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
     LayerNormParams lp{};
     lp.x = x; lp.gamma = gamma; lp.beta = beta; lp.y = y;
     lp.m = m; lp.slice = slice;
-    lp.batch = (int)batch; lp.group_size = (int)G; lp.num_groups = (int)groups;
+    lp.batch = (int)batch; lp.group_size = (int)G; lp.num_groups = (int)groups; lp.bundle = (int)T;
     lp.eps = (double)eps;
     lp.partials = reinterpret_cast<double *>(ws + off_partials);
     lp.arrived = reinterpret_cast<unsigned int *>(ws + off_arrived);
     lp.status = reinterpret_cast<int *>(ws);
-    const unsigned grid = (unsigned)(groups * G);              // <= SM count: all CTAs are resident
-    if (vec) layernorm_kernel<true><<<grid, kLnThreads, 0, stream>>>(lp);
-    else     layernorm_kernel<false><<<grid, kLnThreads, 0, stream>>>(lp);
+    const unsigned grid = (unsigned)(groups * G);              // all CTAs are resident at once
+    if (use_smem) {
+        const size_t smem = (size_t)(T * slice * 4);
+        if (!d.smem_attr_set[10]) {
+            CUDA_TRY(cudaFuncSetAttribute(layernorm_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)kLnSmemBudget));
+            d.smem_attr_set[10] = true;
+        }
+        layernorm_smem_kernel<<<grid, kLnThreads, smem, stream>>>(lp);
+    } else if (vec) {
+        layernorm_stream_kernel<true><<<grid, kLnThreads, 0, stream>>>(lp);
+    } else {
+        layernorm_stream_kernel<false><<<grid, kLnThreads, 0, stream>>>(lp);
+    }
     CUDA_TRY(cudaGetLastError());
     return CUDALLM_OK;
 }

@@ -7,9 +7,12 @@ Bars
 * sum / dot: the kernels accumulate in double and round once, so
   |gpu - ref| <= 2^-24 |ref| + 2 n 2^-53 * sum|terms|  (the second term covers
   the different summation orders of the two double accumulations);
-* LayerNorm: |gpu - ref| <= 2^-23 * (|x - mean| rstd |gamma| + |beta|) + 1e-9 |gamma|
-  (one rounding of the normalised value to float32, one fused multiply-add; the
-  last term covers the statistics' summation order).
+* LayerNorm: |gpu - ref| <= 2^-20 * (|z| + 1) |gamma| + 2^-22 |beta|, z = (x - mean) rstd.
+  The kernels take the moments in float32 about a pilot value near the data
+  (7 + 3 roundings of 2^-24 per 32-byte piece, relative to the deviations, so the
+  mean is good to ~2^-21.5 of the spread and 1/sqrt(var + eps) to ~2^-22
+  relative) and form the output in float32 from a two-float mean (four roundings
+  of 2^-24); the bound leaves a factor of two.
 """
 import numpy as np
 import pytest
@@ -197,14 +200,15 @@ def check_layernorm(got, x, gamma, beta, batch, m, eps=1e-5):
     g = np.ones(m) if gamma is None else gamma.astype(np.float64)
     b = np.zeros(m) if beta is None else beta.astype(np.float64)
     z = np.abs(x.astype(np.float64).reshape(batch, m) - mean[:, None]) * rstd[:, None]
-    bound = 2.0 ** -23 * (z * np.abs(g) + np.abs(b)) + 1e-9 * np.abs(g)
+    bound = 2.0 ** -20 * (z + 1.0) * np.abs(g) + 2.0 ** -22 * np.abs(b)
     err = np.abs(got - ref)
     assert np.all(np.isfinite(got))
     assert np.all(err <= bound), (float((err / np.maximum(bound, 1e-300)).max()), np.unravel_index(np.argmax(err - bound), err.shape))
 
 
 @pytest.mark.parametrize("batch,m", [(1, 4), (3, 7), (16, 4 * 64 * 64), (16, 4 * 128 * 128), (5, 4096 * 3 + 4),
-                                     (2, 1 << 20), (200, 1000), (7, 100003), (16, 4 * 256 * 256)])
+                                     (2, 1 << 20), (200, 1000), (7, 100003), (16, 4 * 256 * 256),
+                                     (40, 200000), (33, 100024), (1, 8)])
 def test_layernorm_against_oracle(batch, m):
     x, gamma, beta = gi.layernorm_inputs(4, batch, m)
     check_layernorm(run_layernorm(x, gamma, beta, batch, m), x, gamma, beta, batch, m)
