@@ -317,6 +317,22 @@ def run_ours(args):
     a_total, a_avg = time_steps(lambda i: B.mhsa_bf16(aq, ak, av, ao, aN, aD, aH, aD, aD, aD, aD, stream),
                                 a_steps, 5, barrier)
 
+    # ---------- the bandwidth-bound float32 tasks (8, 14, 15, 4) at their largest paper size,
+    #            plus a 1 GiB stream for the two reductions (the paper's largest is 4 MB) ----------
+    hbm_tasks = []
+    for task, size, label in (("transpose", gi.TRANSPOSE_SIZES[-1], "Task 8"), ("layernorm", 1024, "Task 4"),
+                              ("sum", gi.REDUCTION_SIZES[-1], "Task 14"), ("dot", gi.DOT_SIZES[-1], "Task 15"),
+                              ("sum", 1 << 28, "Task 14 beyond the paper's sizes"),
+                              ("dot", 1 << 27, "Task 15 beyond the paper's sizes")):
+        launch_t, bytes_t, what = H.task_problem(task, size)
+        t_steps = max(args.steps, 20)
+        _, t_avg = time_steps(launch_t, t_steps, 3, barrier)
+        hbm_tasks.append({"task": label, "call": f"cudallm_{task}_f32", "input": what, "us_per_call": t_avg * 1e6,
+                          "steps": t_steps, "value": bytes_t / t_avg / 1e9, "unit": "GB/s (algorithmic bytes)",
+                          "frac_of_measured_hbm": bytes_t / t_avg / 1e9 / peaks["hbm_gbs"]})
+        del launch_t
+        torch.cuda.empty_cache()
+
     line = None
     if rank == 0:
         clocks = sampler.summary()
@@ -364,6 +380,7 @@ def run_ours(args):
             "call": "cudallm_mhsa_bf16 (one fused kernel, 64 CTAs)", "us_per_call": a_avg * 1e6,
             "steps": a_steps, "value": 4.0 * aN * aN * aD / a_avg / 1e12, "unit": "TFLOP/s (4 N^2 d_model)",
             "note": "2.6 MB of operands and output: L2-resident and launch-latency bound, no roofline claimed"}
+        line["hbm_tasks_f32"] = hbm_tasks
         if world == 1:
             line["cpu_baseline"] = cpu_baseline_sample(cfg, A, Bm)
     if use_dist:

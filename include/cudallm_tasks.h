@@ -78,10 +78,14 @@ int cudallm_dot_f32(const float *a, const float *b, int64_t n, float *result, vo
  *   gamma, beta : fp32, m elements each (one per position of a sample), or NULL
  *                 for "all ones" / "all zeros"
  *   eps         : >= 0 (the usual value is 1e-5)
- * Statistics are accumulated in double.  The output is formed in fp32 from the
- * mean held as two floats (so a mean far larger than the spread costs no
- * accuracy) and 1/sqrt(var + eps) rounded to fp32:
- * |y - exact| <= 2^-22 (|x - mean| |gamma| / sqrt(var + eps) + |beta|).  batch == 0 or m == 0: success, nothing written.
+ * Arithmetic: the moments are taken in fp32 about a pilot value close to the
+ * data (so a mean far larger than the spread costs no accuracy), combined in
+ * double; the output is formed in fp32 from the mean held as two floats and
+ * 1/sqrt(var + eps) rounded to fp32.  With z = (x - mean) / sqrt(var + eps):
+ * |y - exact| <= 2^-20 (|z| + 1) |gamma| + 2^-22 |beta| for data whose spread is
+ * not dominated by a few outliers; squared deviations must stay inside the fp32
+ * range (|x - mean| below about 1e19).  batch == 0 or m == 0: success, nothing
+ * written.
  * Errors: INVALID_DIM (negative, batch >= 2^31, m > 2^40, eps negative or not
  * finite), INVALID_POINTER (x or y NULL), MISALIGNED (4 bytes), WORKSPACE (an
  * external workspace is set and too small), UNSUPPORTED_DEVICE, CUDA.

@@ -37,15 +37,15 @@ __device__ __forceinline__ void tma_load_3d(const CUtensorMap *tm, uint32_t smem
 // wavefront per row) and writes it as row c of a staging block, again in the
 // swizzled layout -- and lane 0 stores the block with TMA to AT.  Both
 // directions move whole 128-byte lines, and the patches that run at the same
-// time are neighbours along a row of A, so DRAM sees 256 contiguous bytes per
-// row of a patch.  Out-of-range parts of a box are zero-filled on load and
+// time form compact squares (see the patch order in the kernel).  Out-of-range parts of a box are zero-filled on load and
 // clipped on store (rows and cols are multiples of 4 on this path, so the
 // 16-byte clipping granule is exact).
 constexpr int kTrWarps = 4;                      // warps per CTA
 constexpr int kTrStages = 2;                     // 64 x 64 patches in flight per warp
 constexpr int kTrPatch = 64;
 constexpr int kTrPatchBytes = kTrPatch * kTrPatch * 4;               // 16 KiB
-constexpr int kTrWarpBytes = kTrStages * kTrPatchBytes + 2 * 4096;   // ring + two staging blocks
+constexpr int kTrStaging = 4;                    // 4 KiB staging blocks per warp (TMA stores in flight)
+constexpr int kTrWarpBytes = kTrStages * kTrPatchBytes + kTrStaging * 4096;
 constexpr int kTrSmemBytes = kTrWarps * kTrWarpBytes + kTrWarps * kTrStages * 8 + 1024;
 
 struct TransposeParams {
@@ -78,13 +78,30 @@ transpose_tma_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_c
     }
     __syncthreads();
 
-    const long long total = static_cast<long long>(p.patches_r) * p.patches_c;
+    // Patch order: super-tiles of 8 x 8 patches (512 x 512 elements), row-major inside a
+    // super-tile.  The ~600 patches in flight on the GPU then cover a few compact squares,
+    // so that DRAM sees runs of 2 KB on the read side AND on the write side (in plain
+    // row-major order the writes of concurrent patches are 256-byte pieces 4 N bytes apart).
+    const int sc_count = (p.patches_c + 7) >> 3;
+    const long long total = static_cast<long long>((p.patches_r + 7) >> 3) * sc_count * 64;
     const long long step = static_cast<long long>(gridDim.x) * kTrWarps;
-    const long long first = static_cast<long long>(blockIdx.x) * kTrWarps + warp;
+    auto decode = [&](long long id, int &pr, int &pc) -> bool {
+        const long long sup = id >> 6;
+        const int within = static_cast<int>(id & 63);
+        const int sr = static_cast<int>(sup / sc_count), sc = static_cast<int>(sup - static_cast<long long>(sr) * sc_count);
+        pr = sr * 8 + (within >> 3);
+        pc = sc * 8 + (within & 7);
+        return pr < p.patches_r && pc < p.patches_c;
+    };
+    auto next_valid = [&](long long id) {                // first id >= `id` on this warp's stride that is a patch
+        int pr, pc;
+        while (id < total && !decode(id, pr, pc)) id += step;
+        return id;
+    };
 
-    auto issue = [&](long long patch, int s) {           // lane 0 only
-        const int pr = static_cast<int>(patch / p.patches_c);
-        const int pc = static_cast<int>(patch - static_cast<long long>(pr) * p.patches_c);
+    auto issue = [&](long long id, int s) {              // lane 0 only
+        int pr, pc;
+        decode(id, pr, pc);
         const uint32_t dst = ring + s * kTrPatchBytes;
         mbar_expect_tx(bars + 8 * s, kTrPatchBytes);
 #pragma unroll
@@ -94,22 +111,25 @@ transpose_tma_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_c
     };
 
     // prologue: fill the ring
-    if (lane == 0)
-        for (int s = 0; s < kTrStages; ++s)
-            if (first + s * step < total) issue(first + s * step, s);
+    long long id_cons = next_valid(static_cast<long long>(blockIdx.x) * kTrWarps + warp);
+    long long id_issue = id_cons;
+    for (int s = 0; s < kTrStages && id_issue < total; ++s) {
+        if (lane == 0) issue(id_issue, s);
+        id_issue = next_valid(id_issue + step);
+    }
 
     uint32_t sel = 0;
     int s = 0;
     uint32_t phase = 0;
-    for (long long patch = first; patch < total; patch += step) {
+    for (; id_cons < total; id_cons = next_valid(id_cons + step)) {
         bool ok = mbar_wait(bars + 8 * s, phase, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) {
             if (lane == 0) task_report_timeout(p.status, kRoleTranspose, s);
             break;
         }
-        const int pr = static_cast<int>(patch / p.patches_c);
-        const int pc = static_cast<int>(patch - static_cast<long long>(pr) * p.patches_c);
+        int pr, pc;
+        decode(id_cons, pr, pc);
         const uint32_t src = ring + s * kTrPatchBytes;
 #pragma unroll 1
         for (int b = 0; b < 4; ++b) {
@@ -123,8 +143,8 @@ transpose_tma_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_c
             for (int r = 0; r < 32; ++r)
                 v[r] = ld_shared_f32(box + r * 128 + ((((lane >> 2) ^ (r & 7))) << 4) + (lane & 3) * 4);
             const uint32_t blk = staging + sel * 4096u;
-            sel ^= 1u;
-            if (lane == 0) bulk_wait_group_read<1>();                 // the store before the last has read blk
+            sel = (sel + 1) % kTrStaging;
+            if (lane == 0) bulk_wait_group_read<kTrStaging - 1>();    // the store that used blk has read it
             __syncwarp();
 #pragma unroll
             for (int q = 0; q < 8; ++q)                               // row `lane` of the transposed box
@@ -133,12 +153,15 @@ transpose_tma_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_c
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                tma_store_3d(&tmap_out, blk, r0, c0, 0);                 // AT: x = row index of A, y = column of A
+                tma_store_3d(&tmap_out, blk, r0, c0, 0);              // AT: x = row index of A, y = column of A
                 bulk_commit_group();
             }
         }
         __syncwarp();                                                 // every lane has read the ring stage
-        if (lane == 0 && patch + kTrStages * step < total) issue(patch + kTrStages * step, s);
+        if (id_issue < total) {
+            if (lane == 0) issue(id_issue, s);
+            id_issue = next_valid(id_issue + step);
+        }
         if (++s == kTrStages) { s = 0; phase ^= 1; }
     }
     if (lane == 0) bulk_wait_group_read<0>();

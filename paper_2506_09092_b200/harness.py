@@ -394,7 +394,13 @@ def _main(argv=None):
     ap.add_argument("--search", action="store_true",
                     help="validate every variant on closed-form cases, time the valid ones, report the fastest")
     ap.add_argument("--table", default=None, help="with --search: JSON file to record the winner in")
+    ap.add_argument("--task", default=None, choices=["transpose", "sum", "dot", "layernorm"],
+                    help="time one of the float32 tasks (8, 14, 15, 4) instead of a GEMM configuration")
+    ap.add_argument("--size", type=int, default=None,
+                    help="with --task: N (transpose: N x N; sum, dot: N elements; layernorm: (16, 4, N, N))")
     args = ap.parse_args(argv)
+    if args.task:
+        return _task_main(args)
     if args.search:
         cfg = gi.CONFIGS[args.config]
         res = search_config(cfg, iters=args.iters)
@@ -432,6 +438,53 @@ def _main(argv=None):
                           "us_min": t["min_s"] * 1e6, "us_median": t["median_s"] * 1e6,
                           "tflops": cfg.flops / t["median_s"] / 1e12,
                           "gbs": cfg.algorithmic_bytes / t["median_s"] / 1e9}), flush=True)
+
+
+def task_problem(task: str, size: int, nsets: int | None = None):
+    """(launch(i), algorithmic bytes per call, description) for one float32 task on seeded
+    device inputs, with enough rotating buffer sets to exceed L2 (at most 8)."""
+    import torch
+    from . import binding as B
+    from . import inputs as gi
+
+    st = torch.cuda.current_stream()
+    if task == "transpose":
+        bytes_ = 8 * size * size
+        n = nsets or max(1, min(8, (600 << 20) // bytes_))
+        A = [torch.from_numpy(gi.task_array(8, i, size * size)).cuda() for i in range(n)]
+        T = [torch.empty(size * size, device="cuda") for _ in range(n)]
+        return (lambda i: B.transpose_f32(A[i % n], T[i % n], size, size, size, size, st)), bytes_, f"{size} x {size}"
+    if task in ("sum", "dot"):
+        per = 4 * size * (2 if task == "dot" else 1)
+        n = nsets or max(1, min(8, (600 << 20) // per))
+        X = [torch.from_numpy(gi.task_array(14, i, size)).cuda() for i in range(n)]
+        r = torch.zeros(1, device="cuda")
+        if task == "sum":
+            return (lambda i: B.sum_f32(X[i % n], size, r, st)), per, f"n = {size}"
+        Y = [torch.from_numpy(gi.task_array(15, i, size, "uniform")).cuda() for i in range(n)]
+        return (lambda i: B.dot_f32(X[i % n], Y[i % n], size, r, st)), per, f"n = {size}"
+    batch, m = 16, 4 * size * size
+    bytes_ = 8 * batch * m + 8 * m
+    n = nsets or max(1, min(8, (600 << 20) // bytes_))
+    x, gamma, beta = gi.layernorm_inputs(4, batch, m)
+    X = [torch.from_numpy(x).cuda() for _ in range(n)]
+    Y = [torch.empty(batch * m, device="cuda") for _ in range(n)]
+    g, b = torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda()
+    return (lambda i: B.layernorm_f32(X[i % n], g, b, Y[i % n], batch, m, 1e-5, st)), bytes_, f"(16, 4, {size}, {size})"
+
+
+def _task_main(args):
+    import json
+    import torch
+    from . import binding as B
+
+    default = {"transpose": 8192, "sum": 1 << 28, "dot": 1 << 27, "layernorm": 512}
+    size = args.size or default[args.task]
+    launch, bytes_, what = task_problem(args.task, size, args.sets)
+    t = performance_profiler(launch, iters=args.iters, warmup=args.warmup)
+    code, detail = B.device_status(torch.cuda.current_stream())
+    print(json.dumps({"task": args.task, "input": what, "status": code, "us_min": t["min_s"] * 1e6,
+                      "us_median": t["median_s"] * 1e6, "gbs": bytes_ / t["median_s"] / 1e9}), flush=True)
 
 
 if __name__ == "__main__":
