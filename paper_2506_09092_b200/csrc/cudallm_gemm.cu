@@ -87,10 +87,11 @@ struct Variant {
     Family family;
     int block_n;
     int split_k;                       // 1 = none, 2..16 = every tile along K, kTailSplit = see above
+    int per_sm;                        // CTAs per SM: 1, or 2 for the two-stage kernels for short K
 };
 constexpr int kBlockNs[3] = {64, 128, 256};
 constexpr int kSplits[6] = {1, 2, 4, 8, 16, kTailSplit};
-constexpr int kNumVariants = 1 + 3 * 6 + 6;
+constexpr int kNumVariants = 1 + 3 * 6 + 6 + 2;
 Variant g_variants[kNumVariants];
 std::once_flag g_variants_once;
 
@@ -125,6 +126,19 @@ void build_variants()
             g_variants[v].split_k = sk;
             ++v;
         }
+        // Two CTAs per SM, each with a two-stage ring and half of tensor memory: for
+        // batches of products with one or two k-blocks, where a CTA's time goes into the
+        // first load's latency and the epilogue, and a second CTA fills those gaps.
+        for (int bn : {64, 128}) {
+            snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma_n%d_x2", bn);
+            g_variants[v].family = kUmma;
+            g_variants[v].block_n = bn;
+            g_variants[v].split_k = 1;
+            g_variants[v].per_sm = 2;
+            ++v;
+        }
+        for (int i = 0; i < kNumVariants; ++i)
+            if (g_variants[i].per_sm == 0) g_variants[i].per_sm = 1;
     });
 }
 
@@ -177,7 +191,10 @@ Tiling tiling_for(const Variant &v, const Problem &p, int slots)
     t.partial_bytes = t.helper_tiles * int64_t(kBlockM) * v.block_n * 4;
     return t;
 }
-inline int default_slots(const Variant &v) { return v.family == kUmmaPair ? kNumSMs / 2 : kNumSMs; }
+inline int default_slots(const Variant &v)
+{
+    return v.family == kUmmaPair ? kNumSMs / 2 : kNumSMs * (v.per_sm == 2 ? 2 : 1);
+}
 
 bool variant_supports(const Variant &v, const Problem &p)
 {
@@ -209,7 +226,8 @@ double variant_cost(const Variant &v, const Problem &p)
     const bool pair = v.family == kUmmaPair;
     const int slots = default_slots(v);
     const Tiling t = tiling_for(v, p, slots);
-    const double per_kb = pair ? kPairClocksPerKBlock : 300.0 + 0.83 * v.block_n;
+    // (the two-stage ring of the two-per-SM kernels cannot hide load latency: measured 2x on C5a)
+    const double per_kb = pair ? kPairClocksPerKBlock : (300.0 + 0.83 * v.block_n) * (v.per_sm == 2 ? 2.2 : 1.0);
     const double rows = p.M < kBlockM ? (double)p.M : (double)kBlockM;
     const double out_b = (p.out_dtype == CUDALLM_F32) ? 4.0 : 2.0;
     const double epi = rows * v.block_n * out_b / 32.0 + 1500.0;
@@ -497,9 +515,12 @@ int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb,
 {
     using L = SmemLayout<BLOCK_N, STAGES>;
     static_assert(L::kDynamicBytes <= 232448, "shared memory budget");
-    // More than half of an SM's shared memory, so two CTAs (and their tensor
-    // memory allocations) can never share an SM.
-    static_assert(L::kDynamicBytes > 120 * 1024, "one CTA per SM");
+    // Either more than half of an SM's shared memory, so two CTAs (and their tensor
+    // memory allocations) can never share an SM, or small enough that exactly two fit,
+    // each with at most half of tensor memory.
+    constexpr bool kTwoPerSm = L::kDynamicBytes <= 112 * 1024;
+    static_assert(L::kDynamicBytes > 120 * 1024 || (kTwoPerSm && 3 * L::kDynamicBytes > 233472 && BLOCK_N <= 128),
+                  "one or exactly two CTAs per SM");
     auto kernel = umma_gemm_kernel<BLOCK_N, STAGES, OUT_BF16>;
     DeviceState &d = g_dev[dev];
     if (!d.smem_attr_set[slot]) {
@@ -507,7 +528,8 @@ int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb,
                                       L::kDynamicBytes));
         d.smem_attr_set[slot] = true;
     }
-    int grid = gp.num_units < d.sm_count ? gp.num_units : d.sm_count;
+    const int cap = kTwoPerSm ? 2 * d.sm_count : d.sm_count;
+    int grid = gp.num_units < cap ? gp.num_units : cap;
     return launch_overlapped(kernel, grid, L::kDynamicBytes, stream, ta, tb, tc, gp);
 }
 
@@ -596,6 +618,13 @@ int launch_variant(int dev, const Variant &v, bool bf, const CUtensorMap &ta, co
     if (v.family == kUmmaPair)
         return bf ? launch_umma_pair<3, 2, true>(dev, ta, tb, tc, gp, stream)
                   : launch_umma_pair<3, 2, false>(dev, ta, tb, tc, gp, stream);
+    if (v.per_sm == 2) {
+        if (v.block_n == 64)
+            return bf ? launch_umma<64, 2, true>(dev, 11, ta, tb, tc, gp, stream)
+                      : launch_umma<64, 2, false>(dev, 12, ta, tb, tc, gp, stream);
+        return bf ? launch_umma<128, 2, true>(dev, 13, ta, tb, tc, gp, stream)
+                  : launch_umma<128, 2, false>(dev, 14, ta, tb, tc, gp, stream);
+    }
     switch (v.block_n) {
     case 64:  return bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, tc, gp, stream)
                         : launch_umma<64, 8, false>(dev, 1, ta, tb, tc, gp, stream);
@@ -656,7 +685,7 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
         st = bf ? prepare_umma_pair<3, 2, true>(dev, 6) : prepare_umma_pair<3, 2, false>(dev, 7);
         if (st != CUDALLM_OK) return st;
     }
-    const int slots = pair ? d.max_pairs : d.sm_count;
+    const int slots = pair ? d.max_pairs : d.sm_count * (v.per_sm == 2 ? 2 : 1);
     const Tiling t = tiling_for(v, p, slots);
     if (t.helper_tiles > kMaxHelperTiles || t.partial_bytes > kMaxPartialBytes)
         return CUDALLM_ERR_UNSUPPORTED_SHAPE;

@@ -50,7 +50,7 @@ def test_shape_grid(M):
     tile width (plus a split-K one where K allows)."""
     rng = np.random.default_rng(1000 + M)
     names = ["simt", "umma_n64", "umma_n128", "umma_n256", "umma_n64_sk2", "umma_n256_sk4",
-             "umma2_n256", "umma2_n256_sk2", "umma_n256_ts", "umma2_n256_ts"]
+             "umma2_n256", "umma2_n256_sk2", "umma_n256_ts", "umma2_n256_ts", "umma_n64_x2", "umma_n128_x2"]
     for ni, N in enumerate(DIMS):
         for ki in range(3):
             K = KS[(ni * 3 + ki + M) % len(KS)]
@@ -111,7 +111,8 @@ def test_batched(batch, out_dtype):
         cfgB = gi.random_operand(batch * 7 + M, 1, K, N, ldb, batch=batch, stride=sB)
         Cref, S = oracle.gemm_batched(cfgA, cfgB, M, N, K, lda, ldb, sA, sB, batch)
         for v in [B.VARIANT_AUTO] + variant_ids("simt", "umma_n64", "umma_n128", "umma_n128_sk2", "umma2_n256",
-                                                "umma2_n256_sk2", "umma_n128_ts", "umma2_n256_ts"):
+                                                "umma2_n256_sk2", "umma_n128_ts", "umma2_n256_ts", "umma_n64_x2",
+                                                "umma_n128_x2"):
             if v >= 0 and B.variant_supports(v, M, N, K, lda, ldb, ldc, batch, out_dtype) != 1:
                 continue
             vals, raw, guards = G.run_gemm(cfgA, cfgB, M, N, K, lda, ldb, ldc, out_dtype, batch,
@@ -136,7 +137,8 @@ def test_aligned_c_with_ragged_edges(out_dtype):
         A = gi.random_operand(M + N, 0, M, K, K, batch=batch, stride=sA)
         Bm = gi.random_operand(M + N, 1, K, N, N, batch=batch, stride=sB)
         Cref, S = oracle.gemm_batched(A, Bm, M, N, K, K, N, sA, sB, batch)
-        names = ("umma_n64", "umma_n128", "umma_n256", "umma_n64_sk2", "umma2_n256", "umma2_n256_sk2", "umma2_n256_ts")
+        names = ("umma_n64", "umma_n128", "umma_n256", "umma_n64_sk2", "umma2_n256", "umma2_n256_sk2", "umma2_n256_ts",
+                 "umma_n64_x2", "umma_n128_x2")
         for v in [B.VARIANT_AUTO] + variant_ids(*names):
             if v >= 0 and B.variant_supports(v, M, N, K, K, N, ldc, batch, out_dtype) != 1:
                 continue
