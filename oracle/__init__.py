@@ -343,7 +343,7 @@ def layernorm_f32(x, gamma, beta, batch: int, m: int, eps: float = 1e-5):
 
 
 TOL_MHSA = 1e-2      # |O_gpu - O_ref| <= 1e-2 * T  (probabilities are rounded to bf16 on the GPU)
-TOL_F32_IN = 1e-5    # |C_gpu - C_ref| <= 1e-5 * S for the fp32-operand path
+TOL_F32_IN = 1e-5    # |C_gpu - C_ref| <= 1e-5 * S for the fp32-operand path (three bf16 pieces per operand: ~2^-24 per product)
 
 
 # --------------------------------------------------------------------------
