@@ -508,12 +508,12 @@ int launch_overlapped(Kernel kernel, int grid, int smem_bytes, cudaStream_t stre
     return CUDALLM_OK;
 }
 
-template <int BLOCK_N, int STAGES, bool OUT_BF16>
+template <int BLOCK_N, int STAGES, int KSUB, bool OUT_BF16>
 int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tc,
                 const GemmParams &gp,
                 cudaStream_t stream)
 {
-    using L = SmemLayout<BLOCK_N, STAGES>;
+    using L = SmemLayout<BLOCK_N, STAGES, KSUB>;
     static_assert(L::kDynamicBytes <= 232448, "shared memory budget");
     // Either more than half of an SM's shared memory, so two CTAs (and their tensor
     // memory allocations) can never share an SM, or small enough that exactly two fit,
@@ -521,7 +521,7 @@ int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb,
     constexpr bool kTwoPerSm = L::kDynamicBytes <= 112 * 1024;
     static_assert(L::kDynamicBytes > 120 * 1024 || (kTwoPerSm && 3 * L::kDynamicBytes > 233472 && BLOCK_N <= 128),
                   "one or exactly two CTAs per SM");
-    auto kernel = umma_gemm_kernel<BLOCK_N, STAGES, OUT_BF16>;
+    auto kernel = umma_gemm_kernel<BLOCK_N, STAGES, KSUB, OUT_BF16>;
     DeviceState &d = g_dev[dev];
     if (!d.smem_attr_set[slot]) {
         CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -620,18 +620,18 @@ int launch_variant(int dev, const Variant &v, bool bf, const CUtensorMap &ta, co
                   : launch_umma_pair<3, 2, false>(dev, ta, tb, tc, gp, stream);
     if (v.per_sm == 2) {
         if (v.block_n == 64)
-            return bf ? launch_umma<64, 2, true>(dev, 11, ta, tb, tc, gp, stream)
-                      : launch_umma<64, 2, false>(dev, 12, ta, tb, tc, gp, stream);
-        return bf ? launch_umma<128, 2, true>(dev, 13, ta, tb, tc, gp, stream)
-                  : launch_umma<128, 2, false>(dev, 14, ta, tb, tc, gp, stream);
+            return bf ? launch_umma<64, 2, 1, true>(dev, 11, ta, tb, tc, gp, stream)
+                      : launch_umma<64, 2, 1, false>(dev, 12, ta, tb, tc, gp, stream);
+        return bf ? launch_umma<128, 2, 1, true>(dev, 13, ta, tb, tc, gp, stream)
+                  : launch_umma<128, 2, 1, false>(dev, 14, ta, tb, tc, gp, stream);
     }
     switch (v.block_n) {
-    case 64:  return bf ? launch_umma<64, 8, true>(dev, 0, ta, tb, tc, gp, stream)
-                        : launch_umma<64, 8, false>(dev, 1, ta, tb, tc, gp, stream);
-    case 128: return bf ? launch_umma<128, 6, true>(dev, 2, ta, tb, tc, gp, stream)
-                        : launch_umma<128, 6, false>(dev, 3, ta, tb, tc, gp, stream);
-    default:  return bf ? launch_umma<256, 4, true>(dev, 4, ta, tb, tc, gp, stream)
-                        : launch_umma<256, 4, false>(dev, 5, ta, tb, tc, gp, stream);
+    case 64:  return bf ? launch_umma<64, 4, 2, true>(dev, 0, ta, tb, tc, gp, stream)
+                        : launch_umma<64, 4, 2, false>(dev, 1, ta, tb, tc, gp, stream);
+    case 128: return bf ? launch_umma<128, 3, 2, true>(dev, 2, ta, tb, tc, gp, stream)
+                        : launch_umma<128, 3, 2, false>(dev, 3, ta, tb, tc, gp, stream);
+    default:  return bf ? launch_umma<256, 4, 1, true>(dev, 4, ta, tb, tc, gp, stream)
+                        : launch_umma<256, 4, 1, false>(dev, 5, ta, tb, tc, gp, stream);
     }
 }
 
@@ -1108,8 +1108,8 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     // The array keeps the last call's contents.  The status word and the flags
     // must start at zero; partial tiles are written before they are read.
     CUDA_TRY(cudaMemsetAsync(scratch, 0, kNoallocHeaderBytes, stream));
-    st = (p.out_dtype == CUDALLM_BF16) ? launch_umma<64, 8, true>(dev, 0, ta, tb, tc, gp, stream)
-                                       : launch_umma<64, 8, false>(dev, 1, ta, tb, tc, gp, stream);
+    st = (p.out_dtype == CUDALLM_BF16) ? launch_umma<64, 4, 2, true>(dev, 0, ta, tb, tc, gp, stream)
+                                       : launch_umma<64, 4, 2, false>(dev, 1, ta, tb, tc, gp, stream);
     if (st != CUDALLM_OK) return st;
     int host_status[2] = {0, 0};
     CUDA_TRY(cudaMemcpyAsync(host_status, scratch, sizeof host_status, cudaMemcpyDeviceToHost, stream));

@@ -92,11 +92,14 @@ constexpr int kEpiWarpBytes = 8192;
 constexpr int kEpiStageBytes = 4 * kEpiWarpBytes;
 static_assert(32 * kEpiPitch * 4 <= kEpiWarpBytes, "element-wise staging block");
 
-template <int BLOCK_N, int STAGES>
+// A stage holds KSUB (1 or 2) 64-deep k-blocks, each [A 128 x 64 | B 64 x BLOCK_N]: with
+// two, the producer and the MMA thread pay one barrier round trip per 128 of K.
+template <int BLOCK_N, int STAGES, int KSUB = 1>
 struct SmemLayout {
     static constexpr int kABytes = kBlockM * kBlockK * 2;
     static constexpr int kBBytes = kBlockK * BLOCK_N * 2;
-    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kSubBytes = kABytes + kBBytes;
+    static constexpr int kStageBytes = KSUB * kSubBytes;
     static constexpr int kEpiOffset = STAGES * kStageBytes;          // 1024-byte aligned (swizzled staging)
     static constexpr int kBarOffset = kEpiOffset + kEpiStageBytes;
     // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
@@ -396,12 +399,13 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
     return ok;
 }
 
-template <int BLOCK_N, int STAGES, bool OUT_BF16>
+template <int BLOCK_N, int STAGES, int KSUB, bool OUT_BF16>
 __global__ void __launch_bounds__(kNumThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                  const __grid_constant__ CUtensorMap tmap_c, const GemmParams p)
 {
-    using L = SmemLayout<BLOCK_N, STAGES>;
+    using L = SmemLayout<BLOCK_N, STAGES, KSUB>;
+    static_assert(KSUB == 1 || KSUB == 2, "k-blocks per stage");
     static_assert(BLOCK_N % 64 == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
     constexpr uint32_t kTmemCols = 2 * BLOCK_N;          // 128, 256 or 512: power of two
 
@@ -457,22 +461,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             for (int u = blockIdx.x; ok && u < p.num_units; u += gridDim.x) {
                 const UnitCoord c = decode_unit(p, u);
                 constexpr int boxes = BLOCK_N / 64;
-                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
                     if (!tok && !mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) {
                         report_timeout(p.status, kRoleProducer, stage);
                         ok = false;
                         break;
                     }
-                    // probes the next stage, then issues this stage's loads (one asm block)
+                    // probes the next stage, then issues this stage's loads (one asm block);
+                    // a stage takes up to KSUB k-blocks, all from the same operand segment
                     const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
                     const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
                     const KBlockCoord kc = kblock_coord(p, kb, c.b);
+                    const int nsub = min(min(c.kb_end - kb, KSUB), kc.left_in_segment);
                     tok = tma_stage_step<false>(empty_bar(nstage), nphase ^ 1, full_bar(stage), 1,
-                                                p.a_box_bytes + boxes * (64 * kBlockK * 2), full_bar(stage),
+                                                nsub * (p.a_box_bytes + boxes * (64 * kBlockK * 2)), full_bar(stage),
                                                 &tmap_a, &tmap_b, sa, sa + L::kABytes, kc.k,
                                                 c.m_tile * kBlockM, c.n_tile * BLOCK_N, kc.batch_a,
-                                                kc.batch_b, boxes, 1, 0);
+                                                kc.batch_b, boxes, nsub, L::kSubBytes);
+                    kb += nsub - KSUB;                   // the loop adds KSUB
                     stage = nstage;
                     phase = nphase;
                 }
@@ -495,25 +502,29 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     break;
                 }
                 const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
-                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                bool first_of_unit = true;
+                for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
                     if (!tok && !mbar_wait(full_bar(stage), phase, abort_flag)) {
                         report_timeout(p.status, kRoleMma, stage);
                         ok = false;
                         break;
                     }
-                    // probes the next stage, then issues this stage's four MMAs and the
-                    // commit that frees the stage when they retire (one asm block).
+                    // probes the next stage, then issues this stage's MMAs (four per k-block) and
+                    // the commit that frees the stage when they retire (one asm block).
                     // A: K-major, 8-row groups 1024 B apart (SBO); 16 K-elements = 32 B.
                     // B: MN-major, 64-column chunks 8192 B apart (LBO), 8-k groups
                     //    1024 B apart (SBO); 16 k = 2048 B.
+                    const int nsub = min(min(c.kb_end - kb, KSUB), kblock_coord(p, kb, c.b).left_in_segment);
                     const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
                     const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
                     tok = umma_stage_step<false>(full_bar(nstage), nphase, d_tmem, idesc,
-                                                 kb > c.kb_begin ? 1u : 0u,
+                                                 first_of_unit ? 0u : 1u,
                                                  make_smem_desc_sw128(sa, 16, 1024),
                                                  make_smem_desc_sw128(sa + L::kABytes, 8192, 1024),
-                                                 0, 1, empty_bar(stage), 0);
+                                                 L::kSubBytes, nsub, empty_bar(stage), 0);
+                    first_of_unit = false;
+                    kb += nsub - KSUB;                   // the loop adds KSUB
                     stage = nstage;
                     phase = nphase;
                 }
