@@ -946,7 +946,7 @@ int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int6
         d.smem_attr_set[8] = true;
     }
     dim3 grid((unsigned)cdiv(N, kMhsaRows), (unsigned)h);
-    mhsa_kernel<<<grid, kMhsaRows, L.total, stream>>>(mp);
+    mhsa_kernel<<<grid, kMhsaThreads, L.total, stream>>>(mp);
     CUDA_TRY(cudaGetLastError());
     return CUDALLM_OK;
 }

@@ -11,13 +11,16 @@
 //      (8-row x 16-byte core matrices), zero-padding rows and d_k;
 //   2. one thread issues S = Q_i K_i^T with tcgen05.mma into tensor memory: all
 //      keys at once, 128 lanes x up to 512 fp32 columns -- the whole of TMEM;
-//   3. each thread owns one query row (one TMEM lane): two passes over its row
-//      of S (maximum; then p = exp2((s - max) * log2(e)/sqrt(d_k)), masked beyond
-//      N, summed, rounded to bf16 and written to shared memory as the K-major
-//      A operand of the second product);
+//   3. two threads share one query row (one TMEM lane; warps w and w + 4 read
+//      the same lanes), each taking half of the key chunks: two passes over
+//      the row of S (maximum, exchanged through shared memory; then
+//      p = exp2((s - max) * log2(e)/sqrt(d_k)), masked beyond N, summed, rounded
+//      to bf16 and written to shared memory as the K-major A operand of the
+//      second product);
 //   4. one thread issues O = P V_i (V_i is the MN-major B operand) into the TMEM
 //      columns that S no longer needs;
-//   5. each thread divides its row of O by its row sum and stores d_k floats.
+//   5. the row's two threads divide their halves of the row of O by the row sum
+//      and store them.
 //
 // The two waits on tensor-core completion are bounded like those of the GEMM
 // kernels.
@@ -29,6 +32,7 @@
 namespace cudallm {
 
 constexpr int kMhsaRows = 128;        // queries per CTA
+constexpr int kMhsaThreads = 256;     // two threads per query row
 constexpr int kMhsaMaxKeys = 512;     // = TMEM columns
 constexpr int kMhsaMaxDk = 32;
 
@@ -75,7 +79,7 @@ __device__ __forceinline__ float fast_exp2(float x)
 
 struct MhsaSmem {
     // byte offsets inside the dynamic shared memory block (all multiples of 128)
-    int q, k, v, p, bar, total;
+    int q, k, v, p, bar, xch, total;
 };
 __host__ __device__ inline MhsaSmem mhsa_smem_layout(int keys_pad, int dkp)
 {
@@ -85,11 +89,12 @@ __host__ __device__ inline MhsaSmem mhsa_smem_layout(int keys_pad, int dkp)
     s.v = s.k + (dkp / 8) * keys_pad * 16;            // (keys_pad/8) k groups x (dkp/8) column groups x 128 B
     s.p = s.v + (keys_pad / 8) * (dkp / 8) * 128;     // (keys_pad/8) chunks x 16 row groups x 128 B
     s.bar = s.p + (keys_pad / 8) * 2048;
-    s.total = s.bar + 64;
+    s.xch = s.bar + 64;                               // row maxima and row sums of the two halves
+    s.total = s.xch + 2 * kMhsaThreads * 4;
     return s;
 }
 
-__global__ void __launch_bounds__(kMhsaRows, 1)
+__global__ void __launch_bounds__(kMhsaThreads, 1)
 mhsa_kernel(const MhsaParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -100,6 +105,9 @@ mhsa_kernel(const MhsaParams p)
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L.bar + 20);
 
     const int tid = threadIdx.x, warp = tid >> 5;
+    const int row_in = tid & (kMhsaRows - 1);         // query row of this thread inside the block
+    const int half = tid >> 7;                        // which half of the key chunks it takes
+    float *xch = reinterpret_cast<float *>(smem + L.xch);
     const int head = blockIdx.y;
     const int q0 = blockIdx.x * kMhsaRows;
     const int col0 = head * p.dk;
@@ -116,17 +124,17 @@ mhsa_kernel(const MhsaParams p)
     }
 
     // ---- 1. operands -> shared memory, in core-matrix order -------------------
-    // Each thread keeps sixteen 16-byte loads in flight (the copies are latency-bound).
+    // Each thread keeps up to sixteen 16-byte loads in flight (the copies are latency-bound).
     const uint4 zero = make_uint4(0, 0, 0, 0);
     const int lbo_k = p.keys_pad * 16;                // bytes between d_k chunks of K
     const int lbo_v = kchunks * 128;                  // bytes between groups of 8 keys of V
     auto copy_operand = [&](int which, int total) {
-        for (int i0 = tid; i0 < total; i0 += 16 * kMhsaRows) {
+        for (int i0 = tid; i0 < total; i0 += 16 * kMhsaThreads) {
             uint4 x[16];
             int dst[16];
 #pragma unroll
             for (int u = 0; u < 16; ++u) {
-                const int i = i0 + u * kMhsaRows;
+                const int i = i0 + u * kMhsaThreads;
                 x[u] = zero;
                 dst[u] = -1;
                 if (i < total) {
@@ -182,23 +190,24 @@ mhsa_kernel(const MhsaParams p)
     ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
 
-    // ---- 3. softmax over this thread's row ------------------------------------
-    const uint32_t t_row = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    // ---- 3. softmax: this thread's half of its row ------------------------------
+    const uint32_t t_row = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     // Four 32-column loads are in flight per wait: a TMEM round trip costs far
     // more than the arithmetic on 32 values.
     float row_max = -INFINITY;
     const int nch = p.keys_pad / 32;
+    const int ch_lo = half ? (nch + 1) / 2 : 0, ch_hi = half ? nch : (nch + 1) / 2;
     if (ok) {
 #pragma unroll 1
-        for (int ch0 = 0; ch0 < nch; ch0 += 4) {
+        for (int ch0 = ch_lo; ch0 < ch_hi; ch0 += 4) {
             uint32_t r[4][32];
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                if (ch0 + u < nch) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
+                if (ch0 + u < ch_hi) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
             tmem_ld_wait();
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                if (ch0 + u < nch) {
+                if (ch0 + u < ch_hi) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
                         if ((ch0 + u) * 32 + j < p.N) row_max = fmaxf(row_max, __uint_as_float(r[u][j]));
@@ -206,21 +215,24 @@ mhsa_kernel(const MhsaParams p)
             }
         }
     }
+    xch[tid] = row_max;
+    __syncthreads();
+    row_max = fmaxf(xch[row_in], xch[row_in + kMhsaRows]);          // the first half always has a key < N
     float row_sum = 0.f;
     const float neg_max_scaled = -row_max * p.scale_log2;
     if (ok) {
-        const int r_off = (tid >> 3) * 128 + (tid & 7) * 16;                 // this row inside a chunk of P
+        const int r_off = (row_in >> 3) * 128 + (row_in & 7) * 16;           // this row inside a chunk of P
 #pragma unroll 1
-        for (int ch0 = 0; ch0 < nch; ch0 += 4) {
+        for (int ch0 = ch_lo; ch0 < ch_hi; ch0 += 4) {
             uint32_t r[4][32];
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                if (ch0 + u < nch) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
+                if (ch0 + u < ch_hi) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
             tmem_ld_wait();
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int ch = ch0 + u;
-                if (ch < nch) {
+                if (ch < ch_hi) {
                     uint32_t w[16];
 #pragma unroll
                     for (int j = 0; j < 32; j += 2) {
@@ -243,6 +255,7 @@ mhsa_kernel(const MhsaParams p)
             }
         }
     }
+    xch[kMhsaThreads + tid] = row_sum;
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();                                   // everyone is done reading S and writing P
@@ -264,18 +277,19 @@ mhsa_kernel(const MhsaParams p)
     }
     tc_fence_after();
 
-    // ---- 5. normalise and store -------------------------------------------------
+    // ---- 5. normalise and store (each of the row's two threads: half of d_k) -----
     if (ok) {
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_row, r);                  // d_k <= 32 columns are meaningful
         tmem_ld_wait();
-        const int row = q0 + tid;
+        const int row = q0 + row_in;
         if (row < p.N) {
-            const float inv = 1.f / row_sum;
+            // (the sums were exchanged before the barrier that precedes the second product)
+            const float inv = 1.f / (xch[kMhsaThreads + row_in] + xch[kMhsaThreads + row_in + kMhsaRows]);
             float *dst = p.O + row * p.ldo + col0;
 #pragma unroll
             for (int d = 0; d < kMhsaMaxDk; ++d)
-                if (d < p.dk) dst[d] = __uint_as_float(r[d]) * inv;
+                if (d < p.dk && (d >> 4) == half) dst[d] = __uint_as_float(r[d]) * inv;
         }
     } else if (tid == 0) {
         if (atomicCAS(p.status, 0, -9) == 0) p.status[1] = 0x600;
