@@ -124,45 +124,47 @@ mhsa_kernel(const MhsaParams p)
     }
 
     // ---- 1. operands -> shared memory, in core-matrix order -------------------
-    // Each thread keeps up to sixteen 16-byte loads in flight (the copies are latency-bound).
+    // One list of 16-byte pieces: Q's, then K's, then V's.  Each thread keeps up to
+    // eighteen loads in flight (the copies are latency-bound; at the largest size,
+    // N = 512 and d_k = 32, that is the thread's whole share, fetched in one go).
     const uint4 zero = make_uint4(0, 0, 0, 0);
     const int lbo_k = p.keys_pad * 16;                // bytes between d_k chunks of K
     const int lbo_v = kchunks * 128;                  // bytes between groups of 8 keys of V
-    auto copy_operand = [&](int which, int total) {
-        for (int i0 = tid; i0 < total; i0 += 16 * kMhsaThreads) {
-            uint4 x[16];
-            int dst[16];
+    const int n_q = kMhsaRows * kchunks, n_kv = p.keys_pad * kchunks;
+    const int total = n_q + 2 * n_kv;
+    constexpr int kInFlight = 18;
+    for (int i0 = tid; i0 < total; i0 += kInFlight * kMhsaThreads) {
+        uint4 x[kInFlight];
+        int dst[kInFlight];
 #pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                const int i = i0 + u * kMhsaThreads;
-                x[u] = zero;
-                dst[u] = -1;
-                if (i < total) {
-                    const __nv_bfloat16 *src = nullptr;
-                    if (which == 0) {                 // Q: chunk-major, row within the block
-                        const int c = i / kMhsaRows, r = i - c * kMhsaRows, row = q0 + r;
-                        dst[u] = L.q + c * 2048 + (r >> 3) * 128 + (r & 7) * 16;
-                        if (row < p.N && c * 8 < p.dk) src = p.Q + row * p.ldq + col0 + c * 8;
-                    } else if (which == 1) {          // K: chunk-major, key
-                        const int c = i / p.keys_pad, j = i - c * p.keys_pad;
-                        dst[u] = L.k + c * lbo_k + (j >> 3) * 128 + (j & 7) * 16;
-                        if (j < p.N && c * 8 < p.dk) src = p.K + j * p.ldk + col0 + c * 8;
-                    } else {                          // V: key-major, chunk of d_k
-                        const int j = i / kchunks, c = i - j * kchunks;
-                        dst[u] = L.v + (j >> 3) * lbo_v + c * 128 + (j & 7) * 16;
-                        if (j < p.N && c * 8 < p.dk) src = p.V + j * p.ldv + col0 + c * 8;
-                    }
-                    if (src) x[u] = *reinterpret_cast<const uint4 *>(src);
+        for (int u = 0; u < kInFlight; ++u) {
+            int i = i0 + u * kMhsaThreads;
+            x[u] = zero;
+            dst[u] = -1;
+            if (i < total) {
+                const __nv_bfloat16 *src = nullptr;
+                if (i < n_q) {                        // Q: chunk-major, row within the block
+                    const int c = i / kMhsaRows, r = i - c * kMhsaRows, row = q0 + r;
+                    dst[u] = L.q + c * 2048 + (r >> 3) * 128 + (r & 7) * 16;
+                    if (row < p.N && c * 8 < p.dk) src = p.Q + row * p.ldq + col0 + c * 8;
+                } else if (i < n_q + n_kv) {          // K: chunk-major, key
+                    i -= n_q;
+                    const int c = i / p.keys_pad, j = i - c * p.keys_pad;
+                    dst[u] = L.k + c * lbo_k + (j >> 3) * 128 + (j & 7) * 16;
+                    if (j < p.N && c * 8 < p.dk) src = p.K + j * p.ldk + col0 + c * 8;
+                } else {                              // V: key-major, chunk of d_k
+                    i -= n_q + n_kv;
+                    const int j = i / kchunks, c = i - j * kchunks;
+                    dst[u] = L.v + (j >> 3) * lbo_v + c * 128 + (j & 7) * 16;
+                    if (j < p.N && c * 8 < p.dk) src = p.V + j * p.ldv + col0 + c * 8;
                 }
+                if (src) x[u] = *reinterpret_cast<const uint4 *>(src);
             }
-#pragma unroll
-            for (int u = 0; u < 16; ++u)
-                if (dst[u] >= 0) *reinterpret_cast<uint4 *>(smem + dst[u]) = x[u];
         }
-    };
-    copy_operand(0, kMhsaRows * kchunks);
-    copy_operand(1, p.keys_pad * kchunks);
-    copy_operand(2, p.keys_pad * kchunks);
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u)
+            if (dst[u] >= 0) *reinterpret_cast<uint4 *>(smem + dst[u]) = x[u];
+    }
     fence_proxy_async_smem();                         // make the writes visible to the tensor core
     tc_fence_before();
     __syncthreads();
