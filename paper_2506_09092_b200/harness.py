@@ -373,6 +373,38 @@ class TunedTable:
         with open(path) as f:
             return cls(json.load(f))
 
+    @classmethod
+    def packaged(cls):
+        """The table recorded on a B200 with ``--search --config all --table ...`` and shipped with
+        the package (benchmark configurations and the paper's Task 2 sizes)."""
+        import os
+        return cls.load(os.path.join(os.path.dirname(os.path.abspath(__file__)), "tuned_b200.json"))
+
+
+def _search_one(cfg, iters, table_path):
+    """Validate and time every variant on one configuration; print one JSON line per variant
+    (validation outcome: ok / mismatch / launch error / device timeout) and the winner; record
+    the winner in the table file if one is given."""
+    import json
+    import os
+    from . import binding as B
+
+    res = search_config(cfg, iters=iters)
+    for v, rep in res.reports.items():
+        print(json.dumps({"config": cfg.name, "variant": B.variant_name(v), "validation": rep.status,
+                          "detail": rep.detail,
+                          "us": None if v not in res.latencies else res.latencies[v] * 1e6}), flush=True)
+    best = None if res.best is None else B.variant_name(res.best)
+    print(json.dumps({"config": cfg.name, "best": best,
+                      "us": None if res.best is None else res.best_latency * 1e6,
+                      "library_choice": B.variant_name(B.select_variant(
+                          cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype))}),
+          flush=True)
+    if table_path and res.best is not None:
+        table = TunedTable.load(table_path) if os.path.exists(table_path) else TunedTable()
+        table.record(cfg, best, res.best_latency)
+        table.save(table_path)
+
 
 def _main(argv=None):
     """``python -m paper_2506_09092_b200.harness --config C2``: run one benchmark
@@ -385,7 +417,10 @@ def _main(argv=None):
     from . import inputs as gi
 
     ap = argparse.ArgumentParser()
-    ap.add_argument("--config", default="C2", choices=sorted(gi.CONFIGS))
+    ladder = {f"T2-{k + 1}": gi.task2_ladder(k) for k in range(5)}     # the paper's Task 2 sizes
+    all_configs = dict(gi.CONFIGS, **ladder)
+    ap.add_argument("--config", default="C2", choices=sorted(all_configs) + ["all"],
+                    help="a benchmark configuration, a size of the paper's Task 2 ladder, or (with --search) all")
     ap.add_argument("--variant", default="auto")
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
@@ -402,25 +437,14 @@ def _main(argv=None):
     if args.task:
         return _task_main(args)
     if args.search:
-        cfg = gi.CONFIGS[args.config]
-        res = search_config(cfg, iters=args.iters)
-        for v, rep in res.reports.items():
-            print(json.dumps({"config": cfg.name, "variant": B.variant_name(v), "validation": rep.status,
-                              "detail": rep.detail,
-                              "us": None if v not in res.latencies else res.latencies[v] * 1e6}), flush=True)
-        best = None if res.best is None else B.variant_name(res.best)
-        print(json.dumps({"config": cfg.name, "best": best,
-                          "us": None if res.best is None else res.best_latency * 1e6,
-                          "library_choice": B.variant_name(B.select_variant(
-                              cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype))}),
-              flush=True)
-        if args.table and res.best is not None:
-            import os
-            table = TunedTable.load(args.table) if os.path.exists(args.table) else TunedTable()
-            table.record(cfg, best, res.best_latency)
-            table.save(args.table)
+        for name in (sorted(all_configs) if args.config == "all" else [args.config]):
+            if args.config == "all" and all_configs[name].flops > 2e12:
+                continue                                   # the largest ladder size: minutes of validation
+            _search_one(all_configs[name], args.iters, args.table)
         return
-    cfg = gi.CONFIGS[args.config]
+    if args.config == "all":
+        ap.error("--config all needs --search")
+    cfg = all_configs[args.config]
     names = {B.variant_name(v): v for v in range(B.num_variants())}
     prob = DeviceProblem(cfg, nsets=args.sets)
     if args.all_variants:

@@ -212,3 +212,17 @@ def test_closed_form_comparison_rules():
     assert H.compare_closed_form(bf, (rounded, exact, True))[0]
     trunc = exact.copy(); trunc[1, 1] = 254.0                   # more than half a spacing away
     assert not H.compare_closed_form(bf, (trunc, exact, True))[0]
+
+
+def test_packaged_tuned_table_names_existing_variants():
+    """The dispatch table recorded by the search on a B200 covers the benchmark configurations
+    and names only variants the library has and that support the shape."""
+    table = H.TunedTable.packaged()
+    names = {B.variant_name(v): v for v in range(B.num_variants())}
+    for cfg in gi.CONFIGS.values():
+        name = table.lookup(cfg.M, cfg.N, cfg.K, cfg.batch, cfg.out_dtype)
+        assert name in names, (cfg.name, name)
+        assert B.variant_supports(names[name], cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch,
+                                  cfg.out_dtype) == 1
+        assert table.variant_id(cfg.M, cfg.N, cfg.K, cfg.batch, cfg.out_dtype) == names[name]
+    assert table.lookup(7, 7, 7, 1, 0) is None and table.variant_id(7, 7, 7, 1, 0) == -1
