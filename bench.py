@@ -181,6 +181,34 @@ def cpu_baseline_sample(cfg, A, Bm, target_s=12.0):
                       f"C_ref and S in fp64, {dt:.2f} s"}
 
 
+def task_cpu_baselines():
+    """The task oracles as they stand (single-threaded C), timed on bounded samples of the
+    same seeded inputs; algorithmic GB/s like the GPU figures beside them."""
+    import numpy as np
+    import oracle
+    from paper_2506_09092_b200 import inputs as gi
+    out = {}
+    n = 4096
+    A = gi.task_array(8, 0, n * n)
+    t0 = time.perf_counter(); oracle.transpose_f32(A, n, n); dt = time.perf_counter() - t0
+    out["transpose"] = {"value": 8.0 * n * n / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+                        "sample": f"{n} x {n} fp32, {dt:.2f} s"}
+    x = gi.task_array(14, 0, 1 << 26)
+    t0 = time.perf_counter(); oracle.sum_f32(x); dt = time.perf_counter() - t0
+    out["sum"] = {"value": 4.0 * x.size / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+                  "sample": f"n = 2^26, {dt:.2f} s"}
+    y = gi.task_array(15, 1, 1 << 26, "uniform")
+    t0 = time.perf_counter(); oracle.dot_f32(x, y); dt = time.perf_counter() - t0
+    out["dot"] = {"value": 8.0 * x.size / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+                  "sample": f"n = 2^26, {dt:.2f} s"}
+    batch, m = 16, 4 * 256 * 256
+    xs, g, b = gi.layernorm_inputs(4, batch, m)
+    t0 = time.perf_counter(); oracle.layernorm_f32(xs, g, b, batch, m); dt = time.perf_counter() - t0
+    out["layernorm"] = {"value": (8.0 * batch * m + 8.0 * m) / dt / 1e9, "unit": "GB/s", "cores": 1,
+                        "kind": "oracle", "sample": f"(16, 4, 256, 256) fp32, y in fp64, {dt:.2f} s"}
+    return out
+
+
 # ------------------------------------------------------------ reference arm --
 def run_reference(args):
     rank, local, world = dist_env()
@@ -383,6 +411,9 @@ def run_ours(args):
         line["hbm_tasks_f32"] = hbm_tasks
         if world == 1:
             line["cpu_baseline"] = cpu_baseline_sample(cfg, A, Bm)
+            cpu_tasks = task_cpu_baselines()
+            for entry in hbm_tasks:
+                entry["cpu_baseline"] = cpu_tasks[entry["call"].split("_")[1]]
     if use_dist:
         dist.barrier()
         dist.destroy_process_group()

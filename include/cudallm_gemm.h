@@ -145,7 +145,7 @@ int cudallm_gemm_bf16_variant(int variant,
  * cudallm_host_staging_bytes(...) and 256-byte aligned.  The call copies
  * M*lda and K*ldb elements in, multiplies, copies M*ldc elements out, and
  * SYNCHRONISES `stream` before returning.  Internally B is copied first and A
- * in up to 8 row blocks on a second stream; each block is multiplied on
+ * in up to 4 row blocks on a second stream; each block is multiplied on
  * `stream` as soon as it has arrived and its rows of C return on a third
  * stream, so the two copy directions and the multiplication overlap.  The two
  * extra streams and their events are created on the first call per device.

@@ -304,7 +304,7 @@ DeviceState g_dev[kMaxDevices];
 std::mutex g_mutex;
 
 // Streams and events of the host-buffer entry point (created on first use).
-constexpr int kHostPipeChunks = 8;
+constexpr int kHostPipeChunks = 4;
 struct HostPipe {
     bool ready = false;
     cudaStream_t in = nullptr, out = nullptr;
