@@ -16,6 +16,11 @@
  * transpose or the LayerNorm kernel that runs out is reported through
  * cudallm_device_status().
  *
+ * The LayerNorm kernels make the CTAs of a launch wait for one another (with a
+ * time limit); like the split-K GEMM variants they assume that the launch has
+ * the GPU to itself.  If another kernel holds SMs for seconds, such a wait can
+ * run out and is reported as CUDALLM_ERR_DEVICE_TIMEOUT by cudallm_device_status().
+ *
  * cudallm_sum_f32 / cudallm_dot_f32 keep their per-block partial sums in one
  * fixed scratch area per device, and cudallm_layernorm_f32 keeps its per-sample
  * partial statistics in the library workspace: calls of these functions must
