@@ -374,6 +374,7 @@ struct LayerNormParams {
     int num_groups;          // groups that run side by side; grid = num_groups * G
     int bundle;              // T: samples per bundle, 1 .. 16 (a power of two for the shared-memory kernel)
     double eps;
+    double inv_m;            // 1 / m (the fp64 pipe is slow: no division on the device)
     double *partials;        // [batch][G][4]: A, B, mean and element count of the CTA's share
     unsigned int *arrived;   // [bundles], zero at launch
     int *status;
@@ -493,13 +494,13 @@ __device__ __forceinline__ float warp_sum_f32(float v)
 // of the entries' own B plus n_k (mean_k - mean)^2.  Only the sum of the A_k and
 // the differences of means need double.  Lane 0 writes (mean high, mean low,
 // 1 / sqrt(var + eps)) to out.
-__device__ __forceinline__ void ln_combine(const double *slots, int G, long long m, double eps, int lane,
+__device__ __forceinline__ void ln_combine(const double *slots, int G, double inv_m, double eps, int lane,
                                            float *out)
 {
     double a = 0.0;
     for (int k = lane; k < G; k += 32) a += __ldcg(slots + 4 * k);
     a = warp_sum(a);
-    const double mean = a / static_cast<double>(m);
+    const double mean = a * inv_m;
     float m2 = 0.f;
     for (int k = lane; k < G; k += 32) {
         const float dm = static_cast<float>(__ldcg(slots + 4 * k + 2) - mean);
@@ -507,7 +508,7 @@ __device__ __forceinline__ void ln_combine(const double *slots, int G, long long
     }
     m2 = warp_sum_f32(m2);
     if (lane == 0) {
-        const double var = static_cast<double>(m2) / static_cast<double>(m);
+        const double var = static_cast<double>(m2) * inv_m;
         const float mh = static_cast<float>(mean);
         out[0] = mh;
         out[1] = static_cast<float>(mean - static_cast<double>(mh));
@@ -709,7 +710,7 @@ layernorm_smem_kernel(const LayerNormParams p)
         if (abort_flag) return;
         // 3. warp t combines the group's entries of sample t
         if (warp < tb)
-            ln_combine(p.partials + static_cast<long long>(s0 + warp) * p.group_size * 4, p.group_size, p.m,
+            ln_combine(p.partials + static_cast<long long>(s0 + warp) * p.group_size * 4, p.group_size, p.inv_m,
                        p.eps, lane, stat[warp]);
         __syncthreads();
         // 4. pass 2, chunk position by chunk position: thread -> block 4 c + tid / 128, piece tid % 128
@@ -850,7 +851,7 @@ layernorm_stream_kernel(const LayerNormParams p)
         __syncthreads();
         if (abort_flag) return;
         if (warp < tb)
-            ln_combine(p.partials + static_cast<long long>(s0 + warp) * p.group_size * 4, p.group_size, p.m,
+            ln_combine(p.partials + static_cast<long long>(s0 + warp) * p.group_size * 4, p.group_size, p.inv_m,
                        p.eps, lane, stat[warp]);
         __syncthreads();
         // ---- pass 2, the sample read last first, two samples per sweep

@@ -30,8 +30,10 @@ int run_reduce(const float *a, const float *b, int64_t n, float *result, bool do
     std::lock_guard<std::mutex> lock(g_mutex);
     int st = task_device(&dev);
     if (st != CUDALLM_OK) return st;
-    ReduceScratch *scratch = nullptr;
-    CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void **>(&scratch), g_reduce_scratch));
+    static ReduceScratch *scratch_of[kMaxDevices] = {};        // looked up once per device (g_mutex is held)
+    if (!scratch_of[dev])
+        CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void **>(&scratch_of[dev]), g_reduce_scratch));
+    ReduceScratch *scratch = scratch_of[dev];
     // one block per 8192 elements, at most four blocks of 512 threads per SM
     int64_t blocks = cdiv(n, int64_t(kRedThreads) * 16);
     const int64_t cap = std::min<int64_t>(kRedMaxBlocks, int64_t(4) * g_dev[dev].sm_count);
@@ -178,6 +180,7 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
     lp.m = m; lp.slice = slice;
     lp.batch = (int)batch; lp.group_size = (int)G; lp.num_groups = (int)groups; lp.bundle = (int)T;
     lp.eps = (double)eps;
+    lp.inv_m = 1.0 / (double)m;
     lp.partials = reinterpret_cast<double *>(ws + off_partials);
     lp.arrived = reinterpret_cast<unsigned int *>(ws + off_arrived);
     lp.status = reinterpret_cast<int *>(ws);
