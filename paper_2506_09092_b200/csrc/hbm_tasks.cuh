@@ -29,22 +29,25 @@ __device__ __forceinline__ void tma_load_3d(const CUtensorMap *tm, uint32_t smem
 }
 
 // ============================================================== Task 8 ====
-// AT[j][i] = A[i][j].  Every warp runs its own pipeline over 64 x 64 patches of
-// A: lane 0 asks TMA for the patch as four 32 x 32 boxes (128-byte swizzle, so
-// that rows AND columns of a box can be read without bank conflicts) into one
-// of the warp's ring stages; when the bytes have landed the warp turns each
-// box around -- lane c reads column c of the box (one conflict-free 128-byte
-// wavefront per row) and writes it as row c of a staging block, again in the
-// swizzled layout -- and lane 0 stores the block with TMA to AT.  Both
-// directions move whole 128-byte lines, and the patches that run at the same
-// time form compact squares (see the patch order in the kernel).  Out-of-range parts of a box are zero-filled on load and
-// clipped on store (rows and cols are multiples of 4 on this path, so the
-// 16-byte clipping granule is exact).
-constexpr int kTrWarps = 4;                      // warps per CTA
-constexpr int kTrStages = 2;                     // 64 x 64 patches in flight per warp
-constexpr int kTrPatch = 64;
-constexpr int kTrPatchBytes = kTrPatch * kTrPatch * 4;               // 16 KiB
-constexpr int kTrStaging = 4;                    // 4 KiB staging blocks per warp (TMA stores in flight)
+// AT[j][i] = A[i][j].  Every warp runs its own pipeline over patches of 32 rows x
+// 64 columns of A: lane 0 asks TMA for the patch as one unswizzled box (256-byte
+// rows) into one of the warp's ring stages; when the bytes have landed the warp
+// turns each 32 x 32 half around -- lane c reads column c (for a fixed row the
+// lanes read 128 consecutive bytes: conflict-free) and writes it as row c of a
+// staging block in the 128-byte-swizzled layout of AT's tensor map -- and lane
+// 0 stores the block with TMA to AT.  Both directions move whole 128-byte
+// lines, and the patches that run at the same time form compact rectangles
+// (see the patch order in the kernel).  Eight warps per SM: a warp spends most
+// of its time waiting (TMA completion, the proxy fence before each store), so
+// two warps per scheduler overlap their waits.  Out-of-range parts of a box are
+// zero-filled on load and clipped on store (rows and cols are multiples of 4 on
+// this path, so the 16-byte clipping granule is exact).
+constexpr int kTrWarps = 8;                      // warps per CTA
+constexpr int kTrStages = 2;                     // patches in flight per warp
+constexpr int kTrPatchRows = 32, kTrPatchCols = 64;
+constexpr int kTrBoxes = kTrPatchCols / 32;      // 32 x 32 boxes per patch
+constexpr int kTrPatchBytes = kTrPatchRows * kTrPatchCols * 4;       // 8 KiB
+constexpr int kTrStaging = 2;                    // 4 KiB staging blocks per warp (TMA stores in flight)
 constexpr int kTrWarpBytes = kTrStages * kTrPatchBytes + kTrStaging * 4096;
 constexpr int kTrSmemBytes = kTrWarps * kTrWarpBytes + kTrWarps * kTrStages * 8 + 1024;
 
@@ -78,10 +81,10 @@ transpose_tma_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_c
     }
     __syncthreads();
 
-    // Patch order: super-tiles of 8 x 8 patches (512 x 512 elements), row-major inside a
-    // super-tile.  The ~600 patches in flight on the GPU then cover a few compact squares,
-    // so that DRAM sees runs of 2 KB on the read side AND on the write side (in plain
-    // row-major order the writes of concurrent patches are 256-byte pieces 4 N bytes apart).
+    // Patch order: super-tiles of 8 x 8 patches (256 rows x 512 columns), row-major inside a
+    // super-tile.  The patches in flight on the GPU then cover a few compact rectangles,
+    // so that DRAM sees runs of 1-2 KB on the read side AND on the write side (in plain
+    // row-major order the writes of concurrent patches are 128-byte pieces 4 N bytes apart).
     const int sc_count = (p.patches_c + 7) >> 3;
     const long long total = static_cast<long long>((p.patches_r + 7) >> 3) * sc_count * 64;
     const long long step = static_cast<long long>(gridDim.x) * kTrWarps;
@@ -104,10 +107,8 @@ transpose_tma_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_c
         decode(id, pr, pc);
         const uint32_t dst = ring + s * kTrPatchBytes;
         mbar_expect_tx(bars + 8 * s, kTrPatchBytes);
-#pragma unroll
-        for (int b = 0; b < 4; ++b)                      // box b: rows 32 (b / 2).., columns 32 (b % 2)..
-            tma_load_3d(&tmap_in, dst + b * 4096, bars + 8 * s, pc * kTrPatch + 32 * (b & 1),
-                        pr * kTrPatch + 32 * (b >> 1), 0);
+        // one unswizzled box: row r of the patch lies at r * 256 bytes
+        tma_load_3d(&tmap_in, dst, bars + 8 * s, pc * kTrPatchCols, pr * kTrPatchRows, 0);
     };
 
     // prologue: fill the ring
@@ -132,16 +133,16 @@ transpose_tma_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_c
         decode(id_cons, pr, pc);
         const uint32_t src = ring + s * kTrPatchBytes;
 #pragma unroll 1
-        for (int b = 0; b < 4; ++b) {
-            const int r0 = pr * kTrPatch + 32 * (b >> 1);            // first row / column of the box in A
-            const int c0 = pc * kTrPatch + 32 * (b & 1);
+        for (int b = 0; b < kTrBoxes; ++b) {
+            const int r0 = pr * kTrPatchRows;                        // first row / column of the box in A
+            const int c0 = pc * kTrPatchCols + 32 * b;
             if (r0 >= p.rows || c0 >= p.cols) continue;               // warp-uniform: nothing to store
-            const uint32_t box = src + b * 4096;
-            // lane = column c of the box: element (r, c) lies at r * 128 + ((c / 4) ^ (r % 8)) * 16 + (c % 4) * 4
+            // lane = column c of the 32 x 32 box: for a fixed row the 32 lanes read 128
+            // consecutive bytes, so the patch needs no swizzle on the way in
+            const uint32_t box = src + (32 * b + lane) * 4;
             float v[32];
 #pragma unroll
-            for (int r = 0; r < 32; ++r)
-                v[r] = ld_shared_f32(box + r * 128 + ((((lane >> 2) ^ (r & 7))) << 4) + (lane & 3) * 4);
+            for (int r = 0; r < 32; ++r) v[r] = ld_shared_f32(box + r * (kTrPatchCols * 4));
             const uint32_t blk = staging + sel * 4096u;
             sel = (sel + 1) % kTrStaging;
             if (lane == 0) bulk_wait_group_read<kTrStaging - 1>();    // the store that used blk has read it

@@ -95,14 +95,14 @@ int cudallm_transpose_f32(const float *A, float *AT, int64_t rows, int64_t cols,
     st = ensure_workspace(dev, kHeaderBytes, stream);          // for the status word
     if (st != CUDALLM_OK) return st;
     CUtensorMap tin, tout;
-    st = encode_map(dev, &tin, A, cols, rows, 1, lda, 0, 32, 32, 3);
+    st = encode_map(dev, &tin, A, cols, rows, 1, lda, 0, kTrPatchCols, kTrPatchRows, 3);
     if (st != CUDALLM_OK) return st;
     st = encode_map(dev, &tout, AT, rows, cols, 1, ldat, 0, 32, 32, 1);
     if (st != CUDALLM_OK) return st;
     TransposeParams tp{};
     tp.rows = (int)rows; tp.cols = (int)cols;
-    tp.patches_r = (int)cdiv(rows, kTrPatch);
-    tp.patches_c = (int)cdiv(cols, kTrPatch);
+    tp.patches_r = (int)cdiv(rows, kTrPatchRows);
+    tp.patches_c = (int)cdiv(cols, kTrPatchCols);
     tp.status = static_cast<int *>(d.ws);
     if (!d.smem_attr_set[9]) {
         CUDA_TRY(cudaFuncSetAttribute(transpose_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
