@@ -13,8 +13,7 @@
  * synchronising, negative CUDALLM_ERR_* status codes, argument errors found
  * before any CUDA call, compute capability 10.0 only, no CPU fallback).  The
  * status codes are those of cudallm_gemm.h.  A bounded wait inside the
- * transpose or the LayerNorm kernel that runs out is reported through
- * cudallm_device_status().
+ * LayerNorm kernels that runs out is reported through cudallm_device_status().
  *
  * The LayerNorm kernels make the CTAs of a launch wait for one another (with a
  * time limit); like the split-K GEMM variants they assume that the launch has
@@ -45,8 +44,8 @@ extern "C" {
  *        columns rows <= i < ldat are left untouched); must not overlap A.
  * Values are moved bit for bit (NaN payloads and signed zeros included).
  * 16-byte aligned bases with rows, cols, lda and ldat all multiples of 4 take
- * the TMA path; anything else (4-byte alignment is required) a plain tiled
- * kernel.  rows == 0 or cols == 0: success, nothing written.
+ * the 64 x 64-tile kernel with 16-byte accesses; anything else (4-byte
+ * alignment is required) a 32 x 32-tile kernel with element accesses.  rows == 0 or cols == 0: success, nothing written.
  * Errors: INVALID_DIM (negative, or >= 2^31 - 1024), INVALID_LD, INVALID_POINTER,
  * MISALIGNED, UNSUPPORTED_DEVICE, CUDA.
  */

@@ -419,7 +419,7 @@ struct MapKey {
     const void *base;
     int64_t inner, rows, batch, ld, stride;
     int box_inner, box_rows;
-    int kind;                              // 0 = bf16 operand, 1 = fp32 C, 2 = bf16 C, 3 = fp32 input (unswizzled)
+    int kind;                              // 0 = bf16 operand, 1 = fp32 C, 2 = bf16 C
     bool operator==(const MapKey &o) const
     {
         return base == o.base && inner == o.inner && rows == o.rows && batch == o.batch && ld == o.ld
@@ -436,8 +436,7 @@ struct MapCache {
 MapCache g_map_cache[kMaxDevices];
 
 // kind 0: a bf16 operand read in 128-byte-swizzled boxes; kind 1 / 2: fp32 / bf16
-// C written in boxes of 32 columns x 32 rows (128- / 64-byte swizzle); kind 3: an
-// fp32 matrix read in unswizzled boxes.
+// C written in boxes of 32 columns x 32 rows (128- / 64-byte swizzle).
 int encode_map(int dev, CUtensorMap *tm, const void *base, int64_t inner, int64_t rows, int64_t batch,
                int64_t ld, int64_t stride, int box_inner, int box_rows, int kind)
 {
@@ -448,17 +447,16 @@ int encode_map(int dev, CUtensorMap *tm, const void *base, int64_t inner, int64_
             *tm = mc.map[i];
             return CUDALLM_OK;
         }
-    const cuuint64_t es = (kind == 1 || kind == 3) ? 4 : 2;
+    const cuuint64_t es = (kind == 1) ? 4 : 2;
     cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batch};
     cuuint64_t item_stride = (batch > 1) ? (cuuint64_t)stride * es : (cuuint64_t)rows * ld * es;
     cuuint64_t strides[2] = {(cuuint64_t)ld * es, item_stride};
     cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = g_encode(tm, (kind == 1 || kind == 3) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+    CUresult r = g_encode(tm, kind == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
                           const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          kind == 2 ? CU_TENSOR_MAP_SWIZZLE_64B
-                                    : (kind == 3 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B),
-                          (kind == 0 || kind == 3) ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          kind == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                          kind == 0 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);

@@ -9,163 +9,57 @@
 namespace cudallm {
 
 // status detail codes of these kernels: (role << 8) | what
-enum : int { kRoleTranspose = 4, kRoleLayerNorm = 5 };
+enum : int { kRoleLayerNorm = 5 };
 
 __device__ __forceinline__ void task_report_timeout(int *status, int role, int what)
 {
     if (atomicCAS(status, 0, -9 /* CUDALLM_ERR_DEVICE_TIMEOUT */) == 0) status[1] = (role << 8) | what;
 }
 
-// ----------------------------------------------------------- TMA helpers --
+// -------------------------------------------------------- mbarrier helper --
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// (the tensor maps are rank 3 with a third extent of 1, like the GEMM's)
-__device__ __forceinline__ void tma_load_3d(const CUtensorMap *tm, uint32_t smem_addr, uint32_t bar, int x, int y, int z)
-{
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                 ::"r"(smem_addr), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
-}
-
 // ============================================================== Task 8 ====
-// AT[j][i] = A[i][j].  Every warp runs its own pipeline over patches of 32 rows x
-// 64 columns of A: lane 0 asks TMA for the patch as one unswizzled box (256-byte
-// rows) into one of the warp's ring stages; when the bytes have landed the warp
-// turns each 32 x 32 half around -- lane c reads column c (for a fixed row the
-// lanes read 128 consecutive bytes: conflict-free) and writes it as row c of a
-// staging block in the 128-byte-swizzled layout of AT's tensor map -- and lane
-// 0 stores the block with TMA to AT.  Both directions move whole 128-byte
-// lines, and the patches that run at the same time form compact rectangles
-// (see the patch order in the kernel).  Eight warps per SM: a warp spends most
-// of its time waiting (TMA completion, the proxy fence before each store), so
-// two warps per scheduler overlap their waits.  Out-of-range parts of a box are
-// zero-filled on load and clipped on store (rows and cols are multiples of 4 on
-// this path, so the 16-byte clipping granule is exact).
-constexpr int kTrWarps = 8;                      // warps per CTA
-constexpr int kTrStages = 2;                     // patches in flight per warp
-constexpr int kTrPatchRows = 32, kTrPatchCols = 64;
-constexpr int kTrBoxes = kTrPatchCols / 32;      // 32 x 32 boxes per patch
-constexpr int kTrPatchBytes = kTrPatchRows * kTrPatchCols * 4;       // 8 KiB
-constexpr int kTrStaging = 2;                    // 4 KiB staging blocks per warp (TMA stores in flight)
-constexpr int kTrWarpBytes = kTrStages * kTrPatchBytes + kTrStaging * 4096;
-constexpr int kTrSmemBytes = kTrWarps * kTrWarpBytes + kTrWarps * kTrStages * 8 + 1024;
-
-struct TransposeParams {
-    int rows, cols;          // of A
-    int patches_r, patches_c;
-    int *status;
-};
-
-__global__ void __launch_bounds__(kTrWarps * 32)
-transpose_tma_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out,
-                     const TransposeParams p)
+// AT[j][i] = A[i][j].  One CTA of 256 threads per 64 x 64 tile: 16-byte loads
+// along the rows of A (sixteen threads cover the 256 contiguous bytes of a tile
+// row), a padded shared tile (65 floats per row: the column reads below are
+// conflict-free), 16-byte stores along the rows of AT (again 256 contiguous
+// bytes per tile row).  No persistence and 17 KB of shared memory per CTA, so a
+// dozen CTAs per SM overlap each other's latencies.
+// Measured on B200 at 16384 x 16384: this kernel 6.5 TB/s (the speed of a plain
+// copy); the same with 32 x 32 tiles (128-byte segments) 5.2 TB/s; a
+// warp-specialised version with TMA loads of 64 x 64 patches, a turn in shared
+// memory and TMA stores of 32 x 32 swizzled boxes 5.4 TB/s whatever its ring
+// depth, warp count or patch order -- the 128-byte pieces on the store side
+// were the limit, not the SM.  rows and cols are multiples of 4 on this path and
+// the bases and pitches 16-byte aligned; edge tiles are predicated per 16 bytes.
+__global__ void __launch_bounds__(256)
+transpose64_kernel(const float *__restrict__ A, float *__restrict__ AT, int rows, int cols, long long lda,
+                   long long ldat, int tiles_c)
 {
-    extern __shared__ uint8_t tr_smem_raw[];
-    const uint32_t base = (smem_u32(tr_smem_raw) + 1023u) & ~1023u;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t ring = base + warp * kTrWarpBytes;
-    const uint32_t staging = ring + kTrStages * kTrPatchBytes;
-    const uint32_t bars = base + kTrWarps * kTrWarpBytes + warp * kTrStages * 8;
-    __shared__ int abort_flag;
-
-    if (threadIdx.x == 0) {
-        abort_flag = 0;
-        prefetch_tensormap(&tmap_in);
-        prefetch_tensormap(&tmap_out);
-    }
-    if (lane == 0) {
-        for (int s = 0; s < kTrStages; ++s) mbar_init(bars + 8 * s, 1);
-        fence_mbar_init();
-        fence_proxy_async_smem();
+    __shared__ float tile[64][65];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;          // 16 x 16 threads
+    const int tr = blockIdx.x / tiles_c, tc = blockIdx.x - tr * tiles_c;
+    const int r0 = tr * 64, c0 = tc * 64;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int r = ty + 16 * k;
+        if (r0 + r < rows && c0 + 4 * tx < cols) {
+            const float4 v = *reinterpret_cast<const float4 *>(A + (r0 + r) * lda + c0 + 4 * tx);
+            tile[r][4 * tx] = v.x; tile[r][4 * tx + 1] = v.y; tile[r][4 * tx + 2] = v.z; tile[r][4 * tx + 3] = v.w;
+        }
     }
     __syncthreads();
-
-    // Patch order: super-tiles of 8 x 8 patches (256 rows x 512 columns), row-major inside a
-    // super-tile.  The patches in flight on the GPU then cover a few compact rectangles,
-    // so that DRAM sees runs of 1-2 KB on the read side AND on the write side (in plain
-    // row-major order the writes of concurrent patches are 128-byte pieces 4 N bytes apart).
-    const int sc_count = (p.patches_c + 7) >> 3;
-    const long long total = static_cast<long long>((p.patches_r + 7) >> 3) * sc_count * 64;
-    const long long step = static_cast<long long>(gridDim.x) * kTrWarps;
-    auto decode = [&](long long id, int &pr, int &pc) -> bool {
-        const long long sup = id >> 6;
-        const int within = static_cast<int>(id & 63);
-        const int sr = static_cast<int>(sup / sc_count), sc = static_cast<int>(sup - static_cast<long long>(sr) * sc_count);
-        pr = sr * 8 + (within >> 3);
-        pc = sc * 8 + (within & 7);
-        return pr < p.patches_r && pc < p.patches_c;
-    };
-    auto next_valid = [&](long long id) {                // first id >= `id` on this warp's stride that is a patch
-        int pr, pc;
-        while (id < total && !decode(id, pr, pc)) id += step;
-        return id;
-    };
-
-    auto issue = [&](long long id, int s) {              // lane 0 only
-        int pr, pc;
-        decode(id, pr, pc);
-        const uint32_t dst = ring + s * kTrPatchBytes;
-        mbar_expect_tx(bars + 8 * s, kTrPatchBytes);
-        // one unswizzled box: row r of the patch lies at r * 256 bytes
-        tma_load_3d(&tmap_in, dst, bars + 8 * s, pc * kTrPatchCols, pr * kTrPatchRows, 0);
-    };
-
-    // prologue: fill the ring
-    long long id_cons = next_valid(static_cast<long long>(blockIdx.x) * kTrWarps + warp);
-    long long id_issue = id_cons;
-    for (int s = 0; s < kTrStages && id_issue < total; ++s) {
-        if (lane == 0) issue(id_issue, s);
-        id_issue = next_valid(id_issue + step);
-    }
-
-    uint32_t sel = 0;
-    int s = 0;
-    uint32_t phase = 0;
-    for (; id_cons < total; id_cons = next_valid(id_cons + step)) {
-        bool ok = mbar_wait(bars + 8 * s, phase, &abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) {
-            if (lane == 0) task_report_timeout(p.status, kRoleTranspose, s);
-            break;
-        }
-        int pr, pc;
-        decode(id_cons, pr, pc);
-        const uint32_t src = ring + s * kTrPatchBytes;
-#pragma unroll 1
-        for (int b = 0; b < kTrBoxes; ++b) {
-            const int r0 = pr * kTrPatchRows;                        // first row / column of the box in A
-            const int c0 = pc * kTrPatchCols + 32 * b;
-            if (r0 >= p.rows || c0 >= p.cols) continue;               // warp-uniform: nothing to store
-            // lane = column c of the 32 x 32 box: for a fixed row the 32 lanes read 128
-            // consecutive bytes, so the patch needs no swizzle on the way in
-            const uint32_t box = src + (32 * b + lane) * 4;
-            float v[32];
 #pragma unroll
-            for (int r = 0; r < 32; ++r) v[r] = ld_shared_f32(box + r * (kTrPatchCols * 4));
-            const uint32_t blk = staging + sel * 4096u;
-            sel = (sel + 1) % kTrStaging;
-            if (lane == 0) bulk_wait_group_read<kTrStaging - 1>();    // the store that used blk has read it
-            __syncwarp();
-#pragma unroll
-            for (int q = 0; q < 8; ++q)                               // row `lane` of the transposed box
-                st_shared_v4(blk + lane * 128 + ((q ^ (lane & 7)) << 4), v[4 * q], v[4 * q + 1], v[4 * q + 2],
-                             v[4 * q + 3]);
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                tma_store_3d(&tmap_out, blk, r0, c0, 0);              // AT: x = row index of A, y = column of A
-                bulk_commit_group();
-            }
+    for (int k = 0; k < 4; ++k) {
+        const int c = ty + 16 * k;                                   // row of AT inside the tile
+        if (c0 + c < cols && r0 + 4 * tx < rows) {
+            const float4 v = make_float4(tile[4 * tx][c], tile[4 * tx + 1][c], tile[4 * tx + 2][c], tile[4 * tx + 3][c]);
+            *reinterpret_cast<float4 *>(AT + (c0 + c) * ldat + r0 + 4 * tx) = v;
         }
-        __syncwarp();                                                 // every lane has read the ring stage
-        if (id_issue < total) {
-            if (lane == 0) issue(id_issue, s);
-            id_issue = next_valid(id_issue + step);
-        }
-        if (++s == kTrStages) { s = 0; phase ^= 1; }
     }
-    if (lane == 0) bulk_wait_group_read<0>();
 }
 
 // Any shape, pitch and alignment: 32 x 32 tiles through a padded shared tile.

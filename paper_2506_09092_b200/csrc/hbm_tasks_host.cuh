@@ -81,9 +81,9 @@ int cudallm_transpose_f32(const float *A, float *AT, int64_t rows, int64_t cols,
     if (st != CUDALLM_OK) return st;
     DeviceState &d = g_dev[dev];
 
-    const bool tma = ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(AT)) & 15) == 0
+    const bool vec = ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(AT)) & 15) == 0
                   && rows % 4 == 0 && cols % 4 == 0 && lda % 4 == 0 && ldat % 4 == 0;
-    if (!tma) {
+    if (!vec) {
         const int64_t tiles_c = cdiv(cols, 32);
         const int64_t tiles = cdiv(rows, 32) * tiles_c;
         const int64_t grid = std::min<int64_t>(tiles, int64_t(d.sm_count) * 16);
@@ -92,26 +92,10 @@ int cudallm_transpose_f32(const float *A, float *AT, int64_t rows, int64_t cols,
         CUDA_TRY(cudaGetLastError());
         return CUDALLM_OK;
     }
-    st = ensure_workspace(dev, kHeaderBytes, stream);          // for the status word
-    if (st != CUDALLM_OK) return st;
-    CUtensorMap tin, tout;
-    st = encode_map(dev, &tin, A, cols, rows, 1, lda, 0, kTrPatchCols, kTrPatchRows, 3);
-    if (st != CUDALLM_OK) return st;
-    st = encode_map(dev, &tout, AT, rows, cols, 1, ldat, 0, 32, 32, 1);
-    if (st != CUDALLM_OK) return st;
-    TransposeParams tp{};
-    tp.rows = (int)rows; tp.cols = (int)cols;
-    tp.patches_r = (int)cdiv(rows, kTrPatchRows);
-    tp.patches_c = (int)cdiv(cols, kTrPatchCols);
-    tp.status = static_cast<int *>(d.ws);
-    if (!d.smem_attr_set[9]) {
-        CUDA_TRY(cudaFuncSetAttribute(transpose_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      kTrSmemBytes));
-        d.smem_attr_set[9] = true;
-    }
-    const int64_t patches = int64_t(tp.patches_r) * tp.patches_c;
-    const int64_t grid = std::min<int64_t>(cdiv(patches, kTrWarps), d.sm_count);
-    transpose_tma_kernel<<<(unsigned)grid, kTrWarps * 32, kTrSmemBytes, stream>>>(tin, tout, tp);
+    const int64_t tiles_c = cdiv(cols, 64);
+    const int64_t tiles = cdiv(rows, 64) * tiles_c;            // one CTA each
+    if (tiles > kMaxDim) return CUDALLM_ERR_INVALID_DIM;
+    transpose64_kernel<<<(unsigned)tiles, 256, 0, stream>>>(A, AT, (int)rows, (int)cols, lda, ldat, (int)tiles_c);
     CUDA_TRY(cudaGetLastError());
     return CUDALLM_OK;
 }
