@@ -12,13 +12,8 @@
  * caller, pitches in elements, calls enqueue on `stream` and return without
  * synchronising, negative CUDALLM_ERR_* status codes, argument errors found
  * before any CUDA call, compute capability 10.0 only, no CPU fallback).  The
- * status codes are those of cudallm_gemm.h.  A bounded wait inside the
- * LayerNorm kernels that runs out is reported through cudallm_device_status().
- *
- * The LayerNorm kernels make the CTAs of a launch wait for one another (with a
- * time limit); like the split-K GEMM variants they assume that the launch has
- * the GPU to itself.  If another kernel holds SMs for seconds, such a wait can
- * run out and is reported as CUDALLM_ERR_DEVICE_TIMEOUT by cudallm_device_status().
+ * status codes are those of cudallm_gemm.h.  None of these kernels waits for
+ * another CTA.
  *
  * cudallm_sum_f32 / cudallm_dot_f32 keep their per-block partial sums in one
  * fixed scratch area per device, and cudallm_layernorm_f32 keeps its per-sample

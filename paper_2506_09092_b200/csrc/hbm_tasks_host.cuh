@@ -9,6 +9,25 @@ __device__ cudallm::ReduceScratch g_reduce_scratch;      // zero-initialised: th
 
 constexpr int64_t kTaskMaxElems = int64_t(1) << 40;
 
+// Launch with programmatic stream serialisation (the kernels call griddepcontrol.wait before
+// they touch global memory): the launch latency hides behind the previous kernel of the stream.
+template <typename... KArgs, typename... Args>
+int launch_task(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+    return CUDALLM_OK;
+}
+
 int task_device(int *dev_out)
 {
     int dev = 0;
@@ -41,14 +60,9 @@ int run_reduce(const float *a, const float *b, int64_t n, float *result, bool do
     if (blocks < 1) blocks = 1;
     const bool vec = !dot || ((reinterpret_cast<uintptr_t>(a) & 15) == (reinterpret_cast<uintptr_t>(b) & 15));
     const unsigned g = (unsigned)blocks;
-    if (dot) {
-        if (vec) reduce_kernel<true, true><<<g, kRedThreads, 0, stream>>>(a, b, n, result, scratch);
-        else     reduce_kernel<true, false><<<g, kRedThreads, 0, stream>>>(a, b, n, result, scratch);
-    } else {
-        reduce_kernel<false, true><<<g, kRedThreads, 0, stream>>>(a, a, n, result, scratch);
-    }
-    CUDA_TRY(cudaGetLastError());
-    return CUDALLM_OK;
+    if (dot) return vec ? launch_task(reduce_kernel<true, true>, g, kRedThreads, stream, a, b, (long long)n, result, scratch)
+                        : launch_task(reduce_kernel<true, false>, g, kRedThreads, stream, a, b, (long long)n, result, scratch);
+    return launch_task(reduce_kernel<false, true>, g, kRedThreads, stream, a, a, (long long)n, result, scratch);
 }
 
 }  // namespace
@@ -87,17 +101,14 @@ int cudallm_transpose_f32(const float *A, float *AT, int64_t rows, int64_t cols,
         const int64_t tiles_c = cdiv(cols, 32);
         const int64_t tiles = cdiv(rows, 32) * tiles_c;
         const int64_t grid = std::min<int64_t>(tiles, int64_t(d.sm_count) * 16);
-        transpose_simple_kernel<<<(unsigned)grid, 256, 0, stream>>>(A, AT, (int)rows, (int)cols, lda, ldat,
-                                                                    (int)tiles_c, tiles);
-        CUDA_TRY(cudaGetLastError());
-        return CUDALLM_OK;
+        return launch_task(transpose_simple_kernel, (unsigned)grid, 256, stream, A, AT, (int)rows, (int)cols,
+                           (long long)lda, (long long)ldat, (int)tiles_c, (long long)tiles);
     }
     const int64_t tiles_c = cdiv(cols, 64);
     const int64_t tiles = cdiv(rows, 64) * tiles_c;            // one CTA each
     if (tiles > kMaxDim) return CUDALLM_ERR_INVALID_DIM;
-    transpose64_kernel<<<(unsigned)tiles, 256, 0, stream>>>(A, AT, (int)rows, (int)cols, lda, ldat, (int)tiles_c);
-    CUDA_TRY(cudaGetLastError());
-    return CUDALLM_OK;
+    return launch_task(transpose64_kernel, (unsigned)tiles, 256, stream, A, AT, (int)rows, (int)cols,
+                       (long long)lda, (long long)ldat, (int)tiles_c);
 }
 
 int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta, float *y, int64_t batch,
@@ -120,68 +131,33 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
 
     const bool vec = (all & 31) == 0 && m % 8 == 0;            // 32-byte loads and stores
     const int sms = d.sm_count;
-    // Aligned data is cut into 4 KiB blocks that the CTAs of a group take in turn.
-    const int64_t total_blocks = cdiv(m, (int64_t)kLnBlockPieces * 8);
-    // Shared-memory kernel: the blocks of a bundle of T samples per CTA, one CTA per SM.
-    constexpr int64_t kLnSmemBudget = 227 * 1024 - 2048;
-    const int64_t cap = kLnSmemBudget / 4;                     // elements of shared memory per CTA
-    int64_t groups = 1, T = 1;
-    int64_t G = std::max<int64_t>(1, std::min<int64_t>(sms, total_blocks));
-    const int64_t chunks = cdiv(cdiv(total_blocks, G), kLnChunkBlocks);
-    int64_t slice = cdiv(total_blocks, G) * (kLnBlockBytes / 4);   // shared memory per sample, in elements
-    bool use_smem = vec && slice <= cap && chunks <= kLnMaxChunks;
-    if (use_smem) {
-        const int64_t max_groups = std::max<int64_t>(1, sms / G);
-        // samples per bundle: what fits, but no more than needed to give every group one bundle
-        while (T * 2 <= kLnMaxBundle && T * 2 * slice <= cap && T * max_groups < batch) T *= 2;
-        groups = std::min<int64_t>(max_groups, cdiv(batch, T));
-        // More than two bundles per group: every bundle costs a meeting of the group with
-        // the memory system idle; streaming with fewer meetings is cheaper even though x
-        // is then read twice.
-        if (cdiv(cdiv(batch, T), groups) > 2) use_smem = false;
-    }
-    if (!use_smem) {
-        // Streaming kernel, one CTA per SM: blocks in turn (aligned data) or contiguous
-        // slices of at least 1024 elements (anything else).
-        G = std::max<int64_t>(1, std::min<int64_t>(sms, vec ? total_blocks : m / 1024));
-        slice = round_up(cdiv(m, G), 8);
-        if (!vec) G = cdiv(m, slice);                          // no empty CTAs
-        const int64_t max_groups = std::max<int64_t>(1, sms / G);
-        T = std::min<int64_t>(kLnMaxBundle, std::max<int64_t>(1, cdiv(batch, max_groups)));
-        groups = std::min<int64_t>(max_groups, cdiv(batch, T));
-    }
+    // first kernel: about eight CTAs per SM in total, at least 4096 elements each, at most 256 parts
+    int64_t parts = std::max<int64_t>(1, std::min<int64_t>(cdiv(int64_t(8) * sms, batch), m / 4096));
+    parts = std::min<int64_t>(parts, 256);
+    const int64_t part_len = round_up(cdiv(m, parts), 8);
+    parts = cdiv(m, part_len);
+    // second kernel: 8192 elements of each sample of a pair per CTA
+    const int64_t chunk_len = 8192;
+    const int64_t chunks = cdiv(m, chunk_len);
+    const int64_t npairs = (batch + 1) / 2;
+    if (batch * parts > kMaxDim || npairs * chunks > kMaxDim) return CUDALLM_ERR_INVALID_DIM;
 
-    const size_t off_arrived = kHeaderBytes;
-    const size_t off_partials = (size_t)round_up((int64_t)(off_arrived + (size_t)batch * 4), 256);
-    const size_t total = off_partials + (size_t)batch * (size_t)G * 32;
+    const size_t off_partials = kHeaderBytes;
+    const size_t total = off_partials + (size_t)batch * (size_t)parts * 32;
     st = ensure_workspace(dev, total, stream);
     if (st != CUDALLM_OK) return st;
     uint8_t *ws = static_cast<uint8_t *>(d.ws);
-    CUDA_TRY(cudaMemsetAsync(ws + off_arrived, 0, (size_t)batch * 4, stream));
 
-    LayerNormParams lp{};
+    LayerNorm2Params lp{};
     lp.x = x; lp.gamma = gamma; lp.beta = beta; lp.y = y;
-    lp.m = m; lp.slice = slice;
-    lp.batch = (int)batch; lp.group_size = (int)G; lp.num_groups = (int)groups; lp.bundle = (int)T;
+    lp.m = m; lp.part_len = part_len; lp.chunk_len = chunk_len;
+    lp.batch = (int)batch; lp.parts = (int)parts; lp.chunks = (int)chunks;
     lp.eps = (double)eps;
     lp.inv_m = 1.0 / (double)m;
     lp.partials = reinterpret_cast<double *>(ws + off_partials);
-    lp.arrived = reinterpret_cast<unsigned int *>(ws + off_arrived);
-    lp.status = reinterpret_cast<int *>(ws);
-    const unsigned grid = (unsigned)(groups * G);              // all CTAs are resident at once
-    if (use_smem) {
-        const size_t smem = (size_t)(T * slice * 4);
-        if (!d.smem_attr_set[10]) {
-            CUDA_TRY(cudaFuncSetAttribute(layernorm_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)kLnSmemBudget));
-            d.smem_attr_set[10] = true;
-        }
-        layernorm_smem_kernel<<<grid, kLnThreads, smem, stream>>>(lp);
-    } else if (vec) {
-        layernorm_stream_kernel<true><<<grid, kLnThreads, 0, stream>>>(lp);
-    } else {
-        layernorm_stream_kernel<false><<<grid, kLnThreads, 0, stream>>>(lp);
-    }
-    CUDA_TRY(cudaGetLastError());
-    return CUDALLM_OK;
+    st = vec ? launch_task(layernorm_moments_kernel<true>, (unsigned)(batch * parts), kLn2Threads, stream, lp)
+             : launch_task(layernorm_moments_kernel<false>, (unsigned)(batch * parts), kLn2Threads, stream, lp);
+    if (st != CUDALLM_OK) return st;
+    return vec ? launch_task(layernorm_apply_kernel<true>, (unsigned)(npairs * chunks), kLn2Threads, stream, lp)
+               : launch_task(layernorm_apply_kernel<false>, (unsigned)(npairs * chunks), kLn2Threads, stream, lp);
 }
