@@ -250,14 +250,17 @@ reduce_kernel(const float *__restrict__ a, const float *__restrict__ b, long lon
 // 32-byte loads (sm_100 has 256-bit global accesses; half as many instructions
 // per byte in flight) with an L2 eviction priority: plain for the first read of
 // x, "evict last" for gamma and beta, which are read again for every sample, and
-// "evict first" for the second and last read of x.
+// "evict first" for the second and last read of x.  The first read must NOT
+// carry L1::no_allocate: measured with ncu, lines fetched that way are not kept
+// in L2 either (the second kernel then re-read all of a 17 MB x from DRAM; with
+// the plain load it reads 3 KB).
 struct Float8 {
     float v[8];
 };
 __device__ __forceinline__ Float8 ld8(const float *p)
 {
     Float8 r;
-    asm volatile("ld.global.L1::no_allocate.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+    asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                  : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]),
                    "=f"(r.v[6]), "=f"(r.v[7]) : "l"(p) : "memory");
     return r;
