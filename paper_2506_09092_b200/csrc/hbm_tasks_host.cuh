@@ -131,8 +131,9 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
 
     const bool vec = (all & 31) == 0 && m % 8 == 0;            // 32-byte loads and stores
     const int sms = d.sm_count;
-    // first kernel: about eight CTAs per SM in total, at least 4096 elements each, at most 256 parts
-    int64_t parts = std::max<int64_t>(1, std::min<int64_t>(cdiv(int64_t(8) * sms, batch), m / 4096));
+    // first kernel: about four CTAs per SM in total (what is resident at once: one wave), at
+    // least 4096 elements each, at most 256 parts
+    int64_t parts = std::max<int64_t>(1, std::min<int64_t>(cdiv(int64_t(4) * sms, batch), m / 4096));
     parts = std::min<int64_t>(parts, 256);
     const int64_t part_len = round_up(cdiv(m, parts), 8);
     parts = cdiv(m, part_len);
