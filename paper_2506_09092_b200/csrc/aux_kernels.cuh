@@ -8,6 +8,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "ptx.cuh"
+
 namespace cudallm {
 
 // One thread per element of C; fp32 FMA accumulation in ascending k
@@ -42,6 +44,8 @@ pack_rows_kernel(const uint16_t *__restrict__ src, uint16_t *__restrict__ dst,
                  int rows, int cols, long long ld_src, long long ld_dst,
                  long long stride_src, long long stride_dst, int batch)
 {
+    grid_launch_dependents();
+    grid_dependency_wait();                              // the workspace may still be read by the previous kernel
     const int chunks = (cols + 7) >> 3;
     const long long per_item = static_cast<long long>(rows) * chunks;
     const long long total = per_item * batch;
@@ -74,6 +78,8 @@ __global__ void __launch_bounds__(256)
 split3_rows_kernel(const float *__restrict__ src, uint16_t *__restrict__ dst, int rows, int cols,
                    long long ld_src, long long ld_dst, long long piece_stride)
 {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int chunks = (cols + 7) >> 3;
     const long long total = static_cast<long long>(rows) * chunks;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;

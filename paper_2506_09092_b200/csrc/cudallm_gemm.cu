@@ -486,6 +486,26 @@ int encode_c_map(int dev, CUtensorMap *tm, const Problem &p, bool c_tma)
 }
 
 // ---------------------------------------------------------------- launches --
+// Launch of a plain kernel with programmatic stream serialisation (the kernel calls
+// griddepcontrol.wait before it touches global memory): its launch latency hides behind the
+// previous kernel of the stream.
+template <typename... KArgs, typename... Args>
+int launch_serialised(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+    return CUDALLM_OK;
+}
+
 // Launch with programmatic stream serialisation: the kernel may begin while the
 // previous kernel of the stream drains; it waits (griddepcontrol.wait) before it
 // touches global memory.
@@ -602,12 +622,9 @@ int launch_pack(const void *src, void *dst, int64_t rows, int64_t cols, int64_t 
     const int64_t total = rows * cdiv(cols, 8) * batch;
     int64_t blocks = cdiv(total, 256);
     if (blocks > 148 * 16) blocks = 148 * 16;
-    pack_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const uint16_t *>(src),
-                                                           static_cast<uint16_t *>(dst), (int)rows,
-                                                           (int)cols, ld_src, ld_dst, s_src, s_dst,
-                                                           (int)batch);
-    CUDA_TRY(cudaGetLastError());
-    return CUDALLM_OK;
+    return launch_serialised(pack_rows_kernel, (unsigned)blocks, 256, stream, static_cast<const uint16_t *>(src),
+                             static_cast<uint16_t *>(dst), (int)rows, (int)cols, (long long)ld_src,
+                             (long long)ld_dst, (long long)s_src, (long long)s_dst, (int)batch);
 }
 
 // Launches the tcgen05 kernel of variant `v` (lone CTAs or CTA pairs).
@@ -869,13 +886,14 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
         const int64_t total = rows * cdiv(cols, 8);
         int64_t blocks = cdiv(total, 256);
         if (blocks > kNumSMs * 16) blocks = kNumSMs * 16;
-        split3_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const float *>(src),
-                                                                 static_cast<uint16_t *>(dst), (int)rows,
-                                                                 (int)cols, ld_src, ld_dst, rows * ld_dst);
+        return launch_serialised(split3_rows_kernel, (unsigned)blocks, 256, stream, static_cast<const float *>(src),
+                                 static_cast<uint16_t *>(dst), (int)rows, (int)cols, (long long)ld_src,
+                                 (long long)ld_dst, (long long)(rows * ld_dst));
     };
-    split(A, ws + off_a, M, K, lda, ldap);
-    CUDA_TRY(cudaGetLastError());
-    split(B, ws + off_b, K, N, ldb, ldbp);
+    st = split(A, ws + off_a, M, K, lda, ldap);
+    if (st != CUDALLM_OK) return st;
+    st = split(B, ws + off_b, K, N, ldb, ldbp);
+    if (st != CUDALLM_OK) return st;
     CUDA_TRY(cudaGetLastError());
 
     CUtensorMap ta, tb;

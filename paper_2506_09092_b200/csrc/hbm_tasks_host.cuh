@@ -9,25 +9,6 @@ __device__ cudallm::ReduceScratch g_reduce_scratch;      // zero-initialised: th
 
 constexpr int64_t kTaskMaxElems = int64_t(1) << 40;
 
-// Launch with programmatic stream serialisation (the kernels call griddepcontrol.wait before
-// they touch global memory): the launch latency hides behind the previous kernel of the stream.
-template <typename... KArgs, typename... Args>
-int launch_task(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream, Args... args)
-{
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
-    return CUDALLM_OK;
-}
-
 int task_device(int *dev_out)
 {
     int dev = 0;
@@ -60,9 +41,9 @@ int run_reduce(const float *a, const float *b, int64_t n, float *result, bool do
     if (blocks < 1) blocks = 1;
     const bool vec = !dot || ((reinterpret_cast<uintptr_t>(a) & 15) == (reinterpret_cast<uintptr_t>(b) & 15));
     const unsigned g = (unsigned)blocks;
-    if (dot) return vec ? launch_task(reduce_kernel<true, true>, g, kRedThreads, stream, a, b, (long long)n, result, scratch)
-                        : launch_task(reduce_kernel<true, false>, g, kRedThreads, stream, a, b, (long long)n, result, scratch);
-    return launch_task(reduce_kernel<false, true>, g, kRedThreads, stream, a, a, (long long)n, result, scratch);
+    if (dot) return vec ? launch_serialised(reduce_kernel<true, true>, g, kRedThreads, stream, a, b, (long long)n, result, scratch)
+                        : launch_serialised(reduce_kernel<true, false>, g, kRedThreads, stream, a, b, (long long)n, result, scratch);
+    return launch_serialised(reduce_kernel<false, true>, g, kRedThreads, stream, a, a, (long long)n, result, scratch);
 }
 
 }  // namespace
@@ -101,13 +82,13 @@ int cudallm_transpose_f32(const float *A, float *AT, int64_t rows, int64_t cols,
         const int64_t tiles_c = cdiv(cols, 32);
         const int64_t tiles = cdiv(rows, 32) * tiles_c;
         const int64_t grid = std::min<int64_t>(tiles, int64_t(d.sm_count) * 16);
-        return launch_task(transpose_simple_kernel, (unsigned)grid, 256, stream, A, AT, (int)rows, (int)cols,
+        return launch_serialised(transpose_simple_kernel, (unsigned)grid, 256, stream, A, AT, (int)rows, (int)cols,
                            (long long)lda, (long long)ldat, (int)tiles_c, (long long)tiles);
     }
     const int64_t tiles_c = cdiv(cols, 64);
     const int64_t tiles = cdiv(rows, 64) * tiles_c;            // one CTA each
     if (tiles > kMaxDim) return CUDALLM_ERR_INVALID_DIM;
-    return launch_task(transpose64_kernel, (unsigned)tiles, 256, stream, A, AT, (int)rows, (int)cols,
+    return launch_serialised(transpose64_kernel, (unsigned)tiles, 256, stream, A, AT, (int)rows, (int)cols,
                        (long long)lda, (long long)ldat, (int)tiles_c);
 }
 
@@ -156,9 +137,9 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
     lp.eps = (double)eps;
     lp.inv_m = 1.0 / (double)m;
     lp.partials = reinterpret_cast<double *>(ws + off_partials);
-    st = vec ? launch_task(layernorm_moments_kernel<true>, (unsigned)(batch * parts), kLn2Threads, stream, lp)
-             : launch_task(layernorm_moments_kernel<false>, (unsigned)(batch * parts), kLn2Threads, stream, lp);
+    st = vec ? launch_serialised(layernorm_moments_kernel<true>, (unsigned)(batch * parts), kLn2Threads, stream, lp)
+             : launch_serialised(layernorm_moments_kernel<false>, (unsigned)(batch * parts), kLn2Threads, stream, lp);
     if (st != CUDALLM_OK) return st;
-    return vec ? launch_task(layernorm_apply_kernel<true>, (unsigned)(npairs * chunks), kLn2Threads, stream, lp)
-               : launch_task(layernorm_apply_kernel<false>, (unsigned)(npairs * chunks), kLn2Threads, stream, lp);
+    return vec ? launch_serialised(layernorm_apply_kernel<true>, (unsigned)(npairs * chunks), kLn2Threads, stream, lp)
+               : launch_serialised(layernorm_apply_kernel<false>, (unsigned)(npairs * chunks), kLn2Threads, stream, lp);
 }
