@@ -299,3 +299,23 @@ def test_host_buffer_entry_point():
         assert oracle.check(got, Cref, S, G.tol_for(out_dtype)).ok
         if pad:
             assert np.all(raw[:, N:] == -1)           # host padding untouched
+
+
+@pytest.mark.parametrize("out_dtype", [gi.F32, gi.BF16])
+def test_short_wide_products(out_dtype):
+    """One or two tile rows and 100 to 280 tile columns (more tiles than the
+    grid has CTAs, a thin last round), N a multiple of 16 or not, C with
+    padding columns, B's pitch aligned for TMA or not."""
+    cases = [(16, 16384, 128, 16384), (16, 16381, 96, 16384), (40, 7104, 64, 7104), (16, 11840, 70, 11848),
+             (130, 17760, 64, 17760), (16, 35520, 64, 35520)]
+    for (M, N, K, ldc) in cases:
+        A = gi.random_operand(M + N, 0, M, K, K)
+        Bm = gi.random_operand(M + N, 1, K, N, N)
+        Cref, S = oracle.gemm_batched(A, Bm, M, N, K, K, N, M * K, K * N, 1)
+        for v in [B.VARIANT_AUTO] + variant_ids("umma_n128", "umma_n256_ts", "umma2_n256_ts", "umma_n64_x2"):
+            if v >= 0 and B.variant_supports(v, M, N, K, K, N, ldc, 1, out_dtype) != 1:
+                continue
+            vals, raw, guards = G.run_gemm(A, Bm, M, N, K, K, N, ldc, out_dtype, 1, M * K, K * N, M * ldc, variant=v)
+            r = oracle.check(vals, Cref, S, G.tol_for(out_dtype))
+            assert guards, f"padding or guard band overwritten ({B.variant_name(v)}, {(M, N, K, ldc)})"
+            assert r.ok, (B.variant_name(v), M, N, K, ldc, r)
