@@ -296,7 +296,7 @@ struct DeviceState {
     bool ws_external = false;
     void *ws_internal = nullptr; // owned allocation (kept when an external one is set)
     size_t ws_internal_bytes = 0;
-    bool smem_attr_set[16] = {};
+    bool smem_attr_set[24] = {};
     int max_pairs = 0;           // co-resident 2-CTA clusters of the pair kernel (0 = not asked yet)
     int epoch = 0;               // last split-K flag value used on this device
 };
@@ -527,12 +527,12 @@ int launch_overlapped(Kernel kernel, int grid, int smem_bytes, cudaStream_t stre
     return CUDALLM_OK;
 }
 
-template <int BLOCK_N, int STAGES, int KSUB, bool OUT_BF16>
+template <int BLOCK_N, int STAGES, int KSUB, bool OUT_BF16, int A_ROWS = kBlockM>
 int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tc,
                 const GemmParams &gp,
                 cudaStream_t stream)
 {
-    using L = SmemLayout<BLOCK_N, STAGES, KSUB>;
+    using L = SmemLayout<BLOCK_N, STAGES, KSUB, A_ROWS>;
     static_assert(L::kDynamicBytes <= 232448, "shared memory budget");
     // Either more than half of an SM's shared memory, so two CTAs (and their tensor
     // memory allocations) can never share an SM, or small enough that exactly two fit,
@@ -540,7 +540,7 @@ int launch_umma(int dev, int slot, const CUtensorMap &ta, const CUtensorMap &tb,
     constexpr bool kTwoPerSm = L::kDynamicBytes <= 112 * 1024;
     static_assert(L::kDynamicBytes > 120 * 1024 || (kTwoPerSm && 3 * L::kDynamicBytes > 233472 && BLOCK_N <= 128),
                   "one or exactly two CTAs per SM");
-    auto kernel = umma_gemm_kernel<BLOCK_N, STAGES, KSUB, OUT_BF16>;
+    auto kernel = umma_gemm_kernel<BLOCK_N, STAGES, KSUB, OUT_BF16, A_ROWS>;
     DeviceState &d = g_dev[dev];
     if (!d.smem_attr_set[slot]) {
         CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -644,8 +644,17 @@ int launch_variant(int dev, const Variant &v, bool bf, const CUtensorMap &ta, co
     switch (v.block_n) {
     case 64:  return bf ? launch_umma<64, 4, 2, true>(dev, 0, ta, tb, tc, gp, stream)
                         : launch_umma<64, 4, 2, false>(dev, 1, ta, tb, tc, gp, stream);
-    case 128: return bf ? launch_umma<128, 3, 2, true>(dev, 2, ta, tb, tc, gp, stream)
-                        : launch_umma<128, 3, 2, false>(dev, 3, ta, tb, tc, gp, stream);
+    case 128:
+        // short A (M <= 16 / M <= 64): its rows take 2 / 8 KiB of a k-block's shared memory
+        // instead of 16, and the ring holds 10 / 8 k-blocks instead of 6
+        if (gp.M <= 16)
+            return bf ? launch_umma<128, 5, 2, true, 16>(dev, 16, ta, tb, tc, gp, stream)
+                      : launch_umma<128, 5, 2, false, 16>(dev, 17, ta, tb, tc, gp, stream);
+        if (gp.M <= 64)
+            return bf ? launch_umma<128, 4, 2, true, 64>(dev, 18, ta, tb, tc, gp, stream)
+                      : launch_umma<128, 4, 2, false, 64>(dev, 19, ta, tb, tc, gp, stream);
+        return bf ? launch_umma<128, 3, 2, true>(dev, 2, ta, tb, tc, gp, stream)
+                  : launch_umma<128, 3, 2, false>(dev, 3, ta, tb, tc, gp, stream);
     default:  return bf ? launch_umma<256, 4, 1, true>(dev, 4, ta, tb, tc, gp, stream)
                         : launch_umma<256, 4, 1, false>(dev, 5, ta, tb, tc, gp, stream);
     }

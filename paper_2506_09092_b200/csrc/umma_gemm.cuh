@@ -92,11 +92,19 @@ constexpr int kEpiWarpBytes = 8192;
 constexpr int kEpiStageBytes = 4 * kEpiWarpBytes;
 static_assert(32 * kEpiPitch * 4 <= kEpiWarpBytes, "element-wise staging block");
 
-// A stage holds KSUB (1 or 2) 64-deep k-blocks, each [A 128 x 64 | B 64 x BLOCK_N]: with
+// A stage holds KSUB (1 or 2) 64-deep k-blocks, each [A A_ROWS x 64 | B 64 x BLOCK_N]: with
 // two, the producer and the MMA thread pay one barrier round trip per 128 of K.
-template <int BLOCK_N, int STAGES, int KSUB = 1>
+// A_ROWS < 128 is for products with M <= A_ROWS: the TMA box of A then has at most
+// A_ROWS rows, and the shared memory saved buys more stages, i.e. more bytes of B in
+// flight per SM, which is what bounds a short, wide product.  The MMA still reads
+// 128 rows: rows >= A_ROWS are whatever follows in the stage (B's data), and the rows of
+// the accumulator they produce are never stored.
+template <int BLOCK_N, int STAGES, int KSUB = 1, int A_ROWS = kBlockM>
 struct SmemLayout {
-    static constexpr int kABytes = kBlockM * kBlockK * 2;
+    static_assert(A_ROWS % 8 == 0 && A_ROWS >= 8 && A_ROWS <= kBlockM, "rows of A per stage");
+    static_assert(A_ROWS * kBlockK * 2 + kBlockK * BLOCK_N * 2 >= kBlockM * kBlockK * 2,
+                  "the 128 rows the MMA reads must lie inside the k-block's own bytes");
+    static constexpr int kABytes = A_ROWS * kBlockK * 2;
     static constexpr int kBBytes = kBlockK * BLOCK_N * 2;
     static constexpr int kSubBytes = kABytes + kBBytes;
     static constexpr int kStageBytes = KSUB * kSubBytes;
@@ -399,12 +407,12 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
     return ok;
 }
 
-template <int BLOCK_N, int STAGES, int KSUB, bool OUT_BF16>
+template <int BLOCK_N, int STAGES, int KSUB, bool OUT_BF16, int A_ROWS = kBlockM>
 __global__ void __launch_bounds__(kNumThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                  const __grid_constant__ CUtensorMap tmap_c, const GemmParams p)
 {
-    using L = SmemLayout<BLOCK_N, STAGES, KSUB>;
+    using L = SmemLayout<BLOCK_N, STAGES, KSUB, A_ROWS>;
     static_assert(KSUB == 1 || KSUB == 2, "k-blocks per stage");
     static_assert(BLOCK_N % 64 == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
     constexpr uint32_t kTmemCols = 2 * BLOCK_N;          // 128, 256 or 512: power of two
