@@ -231,6 +231,28 @@ __device__ __forceinline__ bool wait_flag(const int *flag, int epoch, volatile i
     }
 }
 
+// One thread's row of a 32-column block -> staging block `blk`, in the swizzled layout
+// that store_block_staged describes.
+template <bool OUT_BF16>
+__device__ __forceinline__ void stage_row_swizzled(uint32_t blk, int lane, const float (&v)[32])
+{
+    if (OUT_BF16) {
+        const uint32_t row = blk + lane * 64;
+        const uint32_t x = (lane >> 1) & 3;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            st_shared_v4_b32(row + ((q ^ x) << 4), pack_bf16x2(v[8 * q], v[8 * q + 1]),
+                             pack_bf16x2(v[8 * q + 2], v[8 * q + 3]), pack_bf16x2(v[8 * q + 4], v[8 * q + 5]),
+                             pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+    } else {
+        const uint32_t row = blk + lane * 128;
+        const uint32_t x = lane & 7;
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            st_shared_v4(row + ((q ^ x) << 4), v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    }
+}
+
 // Stores one 32 x 32 block of the accumulator (this warp's 32 rows, 32
 // consecutive columns from col0) to C.  Each thread arrives with the 32 values
 // of ITS row (v); writing them as they are would make every store instruction
@@ -259,21 +281,7 @@ __device__ __forceinline__ void store_block_staged(const GemmParams &p, const CU
         sel ^= 1u;
         if (lane == 0) bulk_wait_group_read<1>();        // the store before the last one has read `blk`
         __syncwarp();
-        if (OUT_BF16) {
-            const uint32_t row = blk + lane * 64;
-            const uint32_t x = (lane >> 1) & 3;
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                st_shared_v4_b32(row + ((q ^ x) << 4), pack_bf16x2(v[8 * q], v[8 * q + 1]),
-                                 pack_bf16x2(v[8 * q + 2], v[8 * q + 3]), pack_bf16x2(v[8 * q + 4], v[8 * q + 5]),
-                                 pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
-        } else {
-            const uint32_t row = blk + lane * 128;
-            const uint32_t x = lane & 7;
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                st_shared_v4(row + ((q ^ x) << 4), v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-        }
+        stage_row_swizzled<OUT_BF16>(blk, lane, v);
         fence_proxy_async_smem();                        // generic-proxy writes -> visible to the TMA unit
         __syncwarp();
         if (lane == 0) {
@@ -308,6 +316,30 @@ __device__ __forceinline__ void store_block_staged(const GemmParams &p, const CU
         }
     }
     __syncwarp();                                        // the block is reused for the next chunk
+}
+
+// Two adjacent 32-column blocks (columns col0 .. col0 + 63) at once, both by TMA: the
+// same steps as two calls of store_block_staged, but with one wait for the staging
+// blocks, one proxy fence and one warp barrier, whose latencies (about 600 clocks per
+// block in all) are what an epilogue that is not hidden behind a main loop consists of.
+template <bool OUT_BF16>
+__device__ __forceinline__ void store_two_blocks_staged(const CUtensorMap *tmap_c, uint32_t stage, uint32_t sel,
+                                                        const float (&va)[32], const float (&vb)[32], int b,
+                                                        int row0, int col0, int lane)
+{
+    const uint32_t blk_a = stage + sel * 4096u, blk_b = stage + (sel ^ 1u) * 4096u;
+    if (lane == 0) bulk_wait_group_read<0>();            // both staging blocks have been read
+    __syncwarp();
+    stage_row_swizzled<OUT_BF16>(blk_a, lane, va);
+    stage_row_swizzled<OUT_BF16>(blk_b, lane, vb);
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        tma_store_3d(tmap_c, blk_a, col0, row0, b);
+        bulk_commit_group();                             // a group each, as store_block_staged counts them
+        tma_store_3d(tmap_c, blk_b, col0 + 32, row0, b);
+        bulk_commit_group();
+    }
 }
 
 // Epilogue of one unit, called by the four epilogue warps.  `row` is this
@@ -373,6 +405,21 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
     for (int ch = (S > 1 ? c.split : 0); ch < kChunks; ch += S) {
         const int col0 = c.n_tile * BLOCK_N + ch * 32;
         if (col0 >= p.N) break;                          // warp-uniform: nothing further to store
+        if (S == 1 && p.c_tma && (ch & 1) == 0 && (col0 + 64 <= p.N || (p.n_edge_tma && col0 + 32 < p.N))) {
+            uint32_t ra[32], rb[32];
+            tmem_ld_32x32b_x32(t_addr + ch * 32, ra);
+            tmem_ld_32x32b_x32(t_addr + ch * 32 + 32, rb);
+            tmem_ld_wait();
+            float va[32], vb[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                va[j] = __uint_as_float(ra[j]);
+                vb[j] = __uint_as_float(rb[j]);
+            }
+            store_two_blocks_staged<OUT_BF16>(tmap_c, stage, sel, va, vb, c.b, row0, col0, lane);
+            ++ch;                                        // (the loop adds S == 1)
+            continue;
+        }
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_addr + ch * 32, r);
         tmem_ld_wait();
