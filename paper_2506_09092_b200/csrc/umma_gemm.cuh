@@ -499,12 +499,23 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
         tmem_relinquish();
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    // The producer needs the barriers, which its own thread 0 has just initialised, but
+    // not tensor memory: warp 0 announces its arrival and goes on (the first loads are
+    // on their way while the allocation completes); the other warps wait for everything.
+    uint32_t tmem_base = 0;
+    if (warp_idx == 0) {
+        __syncwarp();
+        named_bar_arrive(1, kNumThreads);
+    } else {
+        tc_fence_before();
+        named_bar_sync(1, kNumThreads);
+        tc_fence_after();
+        tmem_base = *tmem_slot;
+    }
     grid_launch_dependents();
-    grid_dependency_wait();          // from here on global memory may be read and written
+    // Each role waits for the previous kernel of the stream where it first touches global
+    // memory: the producer just before its first load (the first unit's coordinates are
+    // worked out before), the epilogue warps before their loop; the MMA thread never does.
 
     if (warp_idx == 0) {
         // ------------------------------------------------ TMA producer ----
@@ -513,6 +524,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             uint32_t phase = 0;
             bool ok = true;
             uint32_t tok = 1;                            // the first STAGES stages start out free
+            bool waited = false;
             for (int u = blockIdx.x; ok && u < p.num_units; u += gridDim.x) {
                 const UnitCoord c = decode_unit(p, u);
                 constexpr int boxes = BLOCK_N / 64;
@@ -529,6 +541,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
                     const KBlockCoord kc = kblock_coord(p, kb, c.b);
                     const int nsub = min(min(c.kb_end - kb, KSUB), kc.left_in_segment);
+                    if (!waited) {
+                        grid_dependency_wait();
+                        waited = true;
+                    }
                     tok = tma_stage_step<false>(empty_bar(nstage), nphase ^ 1, full_bar(stage), 1,
                                                 nsub * (p.a_box_bytes + boxes * (64 * kBlockK * 2)), full_bar(stage),
                                                 &tmap_a, &tmap_b, sa, sa + L::kABytes, kc.k,
@@ -596,6 +612,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         uint32_t acc_phase = 0;
         uint32_t sel = 0;                                // staging block of the next TMA store
         const uint32_t stage_addr = smem_base + L::kEpiOffset + quad * kEpiWarpBytes;
+        grid_dependency_wait();
         for (int u = blockIdx.x; u < p.num_units; u += gridDim.x) {
             const UnitCoord c = decode_unit(p, u);
             bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
