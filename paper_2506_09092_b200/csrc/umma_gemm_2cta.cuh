@@ -123,7 +123,8 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     grid_launch_dependents();
-    grid_dependency_wait();          // from here on global memory may be read and written
+    // Each role waits for the previous kernel of the stream where it first touches global
+    // memory (the producer just before its first load, the epilogue warps before their loop).
 
     if (warp_idx == 0) {
         // ------------------------------------------------ TMA producer ----
@@ -132,6 +133,7 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             uint32_t phase = 0;
             bool ok = true;
             uint32_t tok = 1;                            // the first STAGES stages start out free
+            bool waited = false;
             const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
             for (int u = pair; ok && u < p.num_units; u += num_pairs) {
                 const UnitCoord c = decode_unit(p, u);
@@ -149,6 +151,10 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
                     const uint32_t nphase = (stage + 1 == STAGES) ? phase ^ 1 : phase;
                     const uint32_t sa = smem_base + stage * L::kStageBytes;
+                    if (!waited) {
+                        grid_dependency_wait();
+                        waited = true;
+                    }
                     tok = tma_stage_step<true>(empty_bar(nstage), nphase ^ 1, full_bar(stage),
                                                rank == 0 ? 1u : 0u,
                                                2 * nsub * (L::kABytes + boxes * (64 * kBlockK * 2)),
@@ -221,6 +227,7 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         uint32_t acc_phase = 0;
         uint32_t sel = 0;
         const uint32_t stage_addr = smem_base + L::kEpiOffset + quad * kEpiWarpBytes;
+        grid_dependency_wait();
         for (int u = pair; u < p.num_units; u += num_pairs) {
             const UnitCoord c = decode_unit(p, u);
             bool ok = mbar_wait<true>(tfull_bar(acc), acc_phase, abort_flag);
