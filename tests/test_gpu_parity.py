@@ -319,3 +319,21 @@ def test_short_wide_products(out_dtype):
             r = oracle.check(vals, Cref, S, G.tol_for(out_dtype))
             assert guards, f"padding or guard band overwritten ({B.variant_name(v)}, {(M, N, K, ldc)})"
             assert r.ok, (B.variant_name(v), M, N, K, ldc, r)
+
+
+@pytest.mark.parametrize("out_dtype", [gi.F32, gi.BF16])
+def test_short_a_boundaries(out_dtype):
+    """The 128-column kernel has instantiations for M <= 16 and M <= 64 whose
+    stages hold fewer rows of A and whose rings are deeper (10 and 8 k-blocks):
+    M on both sides of each boundary, K short and long enough to wrap the ring
+    several times, plain, split-K and tail-split variants."""
+    rng = np.random.default_rng(77)
+    for M in (8, 16, 17, 33, 63, 64, 65):
+        for (N, K) in ((300, 64), (300, 200), (520, 1000), (129, 2500)):
+            A = bits(rng.standard_normal((M, K)))
+            Bm = bits(rng.uniform(-1, 1, (K, N)))
+            ref = oracle.gemm(A, Bm, M, N, K)
+            for v in variant_ids("umma_n128", "umma_n128_sk2", "umma_n128_ts", "umma_n128_sk4"):
+                if B.variant_supports(v, M, N, K, K, N, N, 1, out_dtype) != 1:
+                    continue
+                check_case(A.ravel(), Bm.ravel(), M, N, K, out_dtype, v, ref=ref)
