@@ -616,15 +616,26 @@ int launch_simt(const Problem &p, cudaStream_t stream)
     return CUDALLM_OK;
 }
 
-int launch_pack(const void *src, void *dst, int64_t rows, int64_t cols, int64_t ld_src, int64_t ld_dst,
-                int64_t s_src, int64_t s_dst, int64_t batch, cudaStream_t stream)
+PackJob pack_job(const void *src, void *dst, int64_t rows, int64_t cols, int64_t ld_src, int64_t ld_dst,
+                 int64_t s_src, int64_t s_dst, int64_t batch)
 {
-    const int64_t total = rows * cdiv(cols, 8) * batch;
-    int64_t blocks = cdiv(total, 256);
+    PackJob j{};
+    j.src = static_cast<const uint16_t *>(src);
+    j.dst = static_cast<uint16_t *>(dst);
+    j.rows = (int)rows; j.cols = (int)cols; j.batch = (int)batch;
+    j.ld_src = ld_src; j.ld_dst = ld_dst; j.stride_src = s_src; j.stride_dst = s_dst;
+    j.total_rows = rows * batch;
+    return j;
+}
+
+// One launch repacks both jobs (either may be empty: total_rows == 0).
+int launch_pack(const PackJob &a, const PackJob &b, cudaStream_t stream)
+{
+    const int64_t total = a.total_rows * cdiv(a.cols, 8) + b.total_rows * cdiv(b.cols, 8);
+    if (total == 0) return CUDALLM_OK;
+    int64_t blocks = cdiv(total, 256);                   // one thread per 16-byte piece, grid-stride
     if (blocks > 148 * 16) blocks = 148 * 16;
-    return launch_serialised(pack_rows_kernel, (unsigned)blocks, 256, stream, static_cast<const uint16_t *>(src),
-                             static_cast<uint16_t *>(dst), (int)rows, (int)cols, (long long)ld_src,
-                             (long long)ld_dst, (long long)s_src, (long long)s_dst, (int)batch);
+    return launch_serialised(pack_rows_kernel, (unsigned)blocks, 256, stream, a, b);
 }
 
 // Launches the tcgen05 kernel of variant `v` (lone CTAs or CTA pairs).
@@ -724,16 +735,17 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
 
     const void *A = p.A, *B = p.B;
     int64_t lda = p.lda, ldb = p.ldb, sA = p.sA, sB = p.sB;
+    PackJob ja{}, jb{};
     if (pack_a) {
-        st = launch_pack(p.A, ws + pl.off_pack_a, p.M, p.K, p.lda, pl.ldap, p.sA, pl.sAp, p.batch, stream);
-        if (st != CUDALLM_OK) return st;
+        ja = pack_job(p.A, ws + pl.off_pack_a, p.M, p.K, p.lda, pl.ldap, p.sA, pl.sAp, p.batch);
         A = ws + pl.off_pack_a; lda = pl.ldap; sA = pl.sAp;
     }
     if (pack_b) {
-        st = launch_pack(p.B, ws + pl.off_pack_b, p.K, p.N, p.ldb, pl.ldbp, p.sB, pl.sBp, p.batch, stream);
-        if (st != CUDALLM_OK) return st;
+        jb = pack_job(p.B, ws + pl.off_pack_b, p.K, p.N, p.ldb, pl.ldbp, p.sB, pl.sBp, p.batch);
         B = ws + pl.off_pack_b; ldb = pl.ldbp; sB = pl.sBp;
     }
+    st = launch_pack(ja, jb, stream);
+    if (st != CUDALLM_OK) return st;
 
     CUtensorMap ta, tb;
     // Rows of A beyond M only feed rows of C that are never stored, so the box
