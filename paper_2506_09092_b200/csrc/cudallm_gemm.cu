@@ -506,6 +506,25 @@ int launch_serialised(void (*kernel)(KArgs...), unsigned grid, unsigned block, c
     return CUDALLM_OK;
 }
 
+// The same for a kernel with a two-dimensional grid and dynamic shared memory.
+template <typename... KArgs, typename... Args>
+int launch_serialised_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem_bytes, cudaStream_t stream,
+                           Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+    return CUDALLM_OK;
+}
+
 // Launch with programmatic stream serialisation: the kernel may begin while the
 // previous kernel of the stream drains; it waits (griddepcontrol.wait) before it
 // touches global memory.
@@ -984,9 +1003,7 @@ int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int6
         d.smem_attr_set[8] = true;
     }
     dim3 grid((unsigned)cdiv(N, kMhsaRows), (unsigned)h);
-    mhsa_kernel<<<grid, kMhsaThreads, L.total, stream>>>(mp);
-    CUDA_TRY(cudaGetLastError());
-    return CUDALLM_OK;
+    return launch_serialised_smem(mhsa_kernel, grid, dim3(kMhsaThreads), (size_t)L.total, stream, mp);
 }
 
 size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,

@@ -8,7 +8,11 @@
 //
 //   1. all threads copy Q_i (128 x d_k), K_i (N x d_k) and V_i (N x d_k) into
 //      shared memory, directly in the tensor core's unswizzled operand layouts
-//      (8-row x 16-byte core matrices), zero-padding rows and d_k;
+//      (8-row x 16-byte core matrices), zero-padding rows and d_k; the 16-byte
+//      pieces of one row go to neighbouring lanes (a warp's load touches 8 rows,
+//      not 32: the copy is bound by the number of 128-byte lines per
+//      instruction), and the strides between d_k chunks carry 32 bytes of
+//      padding so that those lanes' stores fall on distinct banks;
 //   2. one thread issues S = Q_i K_i^T with tcgen05.mma into tensor memory: all
 //      keys at once, 128 lanes x up to 512 fp32 columns -- the whole of TMEM;
 //   3. two threads share one query row (one TMEM lane; warps w and w + 4 read
@@ -19,8 +23,9 @@
 //      second product);
 //   4. one thread issues O = P V_i (V_i is the MN-major B operand) into the TMEM
 //      columns that S no longer needs;
-//   5. the row's two threads divide their halves of the row of O by the row sum
-//      and store them.
+//   5. the row's two threads divide their halves of the row of O by the row sum;
+//      the block goes through shared memory so that a warp's store covers whole
+//      rows of the head's columns.
 //
 // The two waits on tensor-core completion are bounded like those of the GEMM
 // kernels.
@@ -78,17 +83,28 @@ __device__ __forceinline__ float fast_exp2(float x)
 }
 
 struct MhsaSmem {
-    // byte offsets inside the dynamic shared memory block (all multiples of 128)
+    // byte offsets inside the dynamic shared memory block (multiples of 32) and strides
     int q, k, v, p, bar, xch, total;
+    int lbo_q, lbo_k;       // bytes between the d_k chunks (8 elements wide) of Q and of K
+    int lbo_v, sbo_v;       // V: bytes between groups of 8 keys, and between d_k chunks inside a group
 };
+constexpr int kMhsaOutPitch = 36;     // floats per row of the output staging block (conflict-free 16-byte stores)
 __host__ __device__ inline MhsaSmem mhsa_smem_layout(int keys_pad, int dkp)
 {
     MhsaSmem s;
-    s.q = 0;                                          // (dkp/8) chunks x 16 row groups x 128 B
-    s.k = s.q + (dkp / 8) * 2048;                     // (dkp/8) chunks x (keys_pad/8) row groups x 128 B
-    s.v = s.k + (dkp / 8) * keys_pad * 16;            // (keys_pad/8) k groups x (dkp/8) column groups x 128 B
-    s.p = s.v + (keys_pad / 8) * (dkp / 8) * 128;     // (keys_pad/8) chunks x 16 row groups x 128 B
-    s.bar = s.p + (keys_pad / 8) * 2048;
+    const int kchunks = dkp / 8;
+    s.lbo_q = kMhsaRows * 16 + 32;                    // [chunk][row][16 B] + padding
+    s.lbo_k = keys_pad * 16 + 32;                     // [chunk][key][16 B] + padding
+    s.sbo_v = 128 + 32;                               // [key group][chunk][key in group][16 B] + padding
+    s.lbo_v = kchunks * s.sbo_v;
+    s.q = 0;
+    s.k = s.q + kchunks * s.lbo_q;
+    s.v = s.k + kchunks * s.lbo_k;
+    s.p = s.v + (keys_pad / 8) * s.lbo_v;             // (keys_pad/8) chunks x 16 row groups x 128 B
+    s.p = (s.p + 127) & ~127;
+    int p_bytes = (keys_pad / 8) * 2048;
+    if (p_bytes < kMhsaRows * kMhsaOutPitch * 4) p_bytes = kMhsaRows * kMhsaOutPitch * 4;   // reused for the output block
+    s.bar = s.p + p_bytes;
     s.xch = s.bar + 64;                               // row maxima and row sums of the two halves
     s.total = s.xch + 2 * kMhsaThreads * 4;
     return s;
@@ -111,7 +127,7 @@ mhsa_kernel(const MhsaParams p)
     const int head = blockIdx.y;
     const int q0 = blockIdx.x * kMhsaRows;
     const int col0 = head * p.dk;
-    const int kchunks = p.dkp / 8;                    // 16-byte chunks along d_k
+    const int kchunks = p.dkp / 8;                    // 16-byte chunks along d_k: 2 or 4
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -123,40 +139,42 @@ mhsa_kernel(const MhsaParams p)
         tmem_relinquish();
     }
 
+    grid_launch_dependents();
+    grid_dependency_wait();                           // (launched with programmatic stream serialisation)
+
     // ---- 1. operands -> shared memory, in core-matrix order -------------------
-    // One list of 16-byte pieces: Q's, then K's, then V's.  Each thread keeps up to
-    // eighteen loads in flight (the copies are latency-bound; at the largest size,
-    // N = 512 and d_k = 32, that is the thread's whole share, fetched in one go).
+    // One list of 16-byte pieces: the rows of Q, then K's, then V's, the d_k chunks of a
+    // row on neighbouring lanes.  Each thread keeps up to eighteen loads in flight (at the
+    // largest size, N = 512 and d_k = 32, that is its whole share, fetched in one go).
     const uint4 zero = make_uint4(0, 0, 0, 0);
-    const int lbo_k = p.keys_pad * 16;                // bytes between d_k chunks of K
-    const int lbo_v = kchunks * 128;                  // bytes between groups of 8 keys of V
-    const int n_q = kMhsaRows * kchunks, n_kv = p.keys_pad * kchunks;
-    const int total = n_q + 2 * n_kv;
+    const int kshift = kchunks == 4 ? 2 : 1;          // kchunks is 2 or 4
+    const int total = (kMhsaRows + 2 * p.keys_pad) << kshift;
     constexpr int kInFlight = 18;
     for (int i0 = tid; i0 < total; i0 += kInFlight * kMhsaThreads) {
         uint4 x[kInFlight];
         int dst[kInFlight];
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u) {
-            int i = i0 + u * kMhsaThreads;
+            const int i = i0 + u * kMhsaThreads;
             x[u] = zero;
             dst[u] = -1;
             if (i < total) {
                 const __nv_bfloat16 *src = nullptr;
-                if (i < n_q) {                        // Q: chunk-major, row within the block
-                    const int c = i / kMhsaRows, r = i - c * kMhsaRows, row = q0 + r;
-                    dst[u] = L.q + c * 2048 + (r >> 3) * 128 + (r & 7) * 16;
-                    if (row < p.N && c * 8 < p.dk) src = p.Q + row * p.ldq + col0 + c * 8;
-                } else if (i < n_q + n_kv) {          // K: chunk-major, key
-                    i -= n_q;
-                    const int c = i / p.keys_pad, j = i - c * p.keys_pad;
-                    dst[u] = L.k + c * lbo_k + (j >> 3) * 128 + (j & 7) * 16;
-                    if (j < p.N && c * 8 < p.dk) src = p.K + j * p.ldk + col0 + c * 8;
-                } else {                              // V: key-major, chunk of d_k
-                    i -= n_q + n_kv;
-                    const int j = i / kchunks, c = i - j * kchunks;
-                    dst[u] = L.v + (j >> 3) * lbo_v + c * 128 + (j & 7) * 16;
-                    if (j < p.N && c * 8 < p.dk) src = p.V + j * p.ldv + col0 + c * 8;
+                const int c = i & (kchunks - 1);
+                int r = i >> kshift;
+                const bool live = c * 8 < p.dk;
+                if (r < kMhsaRows) {                  // Q: row within the block
+                    const int row = q0 + r;
+                    dst[u] = L.q + c * L.lbo_q + r * 16;
+                    if (row < p.N && live) src = p.Q + row * p.ldq + col0 + c * 8;
+                } else if (r < kMhsaRows + p.keys_pad) {
+                    r -= kMhsaRows;                   // K: key
+                    dst[u] = L.k + c * L.lbo_k + r * 16;
+                    if (r < p.N && live) src = p.K + r * p.ldk + col0 + c * 8;
+                } else {
+                    r -= kMhsaRows + p.keys_pad;      // V: key
+                    dst[u] = L.v + (r >> 3) * L.lbo_v + c * L.sbo_v + (r & 7) * 16;
+                    if (r < p.N && live) src = p.V + r * p.ldv + col0 + c * 8;
                 }
                 if (src) x[u] = *reinterpret_cast<const uint4 *>(src);
             }
@@ -180,9 +198,9 @@ mhsa_kernel(const MhsaParams p)
             if (n == 0) break;
             const uint32_t idesc = make_idesc_bf16(kMhsaRows, n, 0, 0);      // both operands K-major
             for (int ks = 0; ks < p.dkp / 16; ++ks) {
-                const uint64_t da = make_smem_desc_plain(sbase + L.q + ks * 2 * 2048, 2048, 128);
-                const uint64_t db = make_smem_desc_plain(sbase + L.k + ks * 2 * lbo_k + part * (256 / 8) * 128,
-                                                         lbo_k, 128);
+                const uint64_t da = make_smem_desc_plain(sbase + L.q + ks * 2 * L.lbo_q, L.lbo_q, 128);
+                const uint64_t db = make_smem_desc_plain(sbase + L.k + ks * 2 * L.lbo_k + part * (256 / 8) * 128,
+                                                         L.lbo_k, 128);
                 umma_bf16_1cta(tmem + part * 256, da, db, idesc, ks > 0 ? 1u : 0u);
             }
         }
@@ -210,9 +228,14 @@ mhsa_kernel(const MhsaParams p)
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 if (ch0 + u < ch_hi) {
+                    if ((ch0 + u) * 32 + 32 <= p.N) {                        // all 32 keys exist
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if ((ch0 + u) * 32 + j < p.N) row_max = fmaxf(row_max, __uint_as_float(r[u][j]));
+                        for (int j = 0; j < 32; ++j) row_max = fmaxf(row_max, __uint_as_float(r[u][j]));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if ((ch0 + u) * 32 + j < p.N) row_max = fmaxf(row_max, __uint_as_float(r[u][j]));
+                    }
                 }
             }
         }
@@ -236,13 +259,14 @@ mhsa_kernel(const MhsaParams p)
                 const int ch = ch0 + u;
                 if (ch < ch_hi) {
                     uint32_t w[16];
+                    const bool full = ch * 32 + 32 <= p.N;                   // all 32 keys exist
 #pragma unroll
                     for (int j = 0; j < 32; j += 2) {
                         // exp2(s * c - max * c): one FMA and one ex2.approx per element
                         float e0 = 0.f, e1 = 0.f;
-                        if (ch * 32 + j < p.N)
+                        if (full || ch * 32 + j < p.N)
                             e0 = fast_exp2(fmaf(__uint_as_float(r[u][j]), p.scale_log2, neg_max_scaled));
-                        if (ch * 32 + j + 1 < p.N)
+                        if (full || ch * 32 + j + 1 < p.N)
                             e1 = fast_exp2(fmaf(__uint_as_float(r[u][j + 1]), p.scale_log2, neg_max_scaled));
                         const uint32_t packed = pack_bf16x2(e0, e1);
                         // the row sum uses the rounded probabilities: exactly what the second product sees
@@ -268,7 +292,7 @@ mhsa_kernel(const MhsaParams p)
         const uint32_t idesc = make_idesc_bf16(kMhsaRows, p.dkp, 0, 1);      // V: MN-major
         for (int ks = 0; ks < p.keys_pad / 16; ++ks) {
             const uint64_t da = make_smem_desc_plain(sbase + L.p + ks * 2 * 2048, 2048, 128);
-            const uint64_t db = make_smem_desc_plain(sbase + L.v + ks * 2 * lbo_v, lbo_v, 128);
+            const uint64_t db = make_smem_desc_plain(sbase + L.v + ks * 2 * L.lbo_v, L.lbo_v, L.sbo_v);
             umma_bf16_1cta(tmem, da, db, idesc, ks > 0 ? 1u : 0u);
         }
         umma_commit(bar);
@@ -280,14 +304,28 @@ mhsa_kernel(const MhsaParams p)
     tc_fence_after();
 
     // ---- 5. normalise and store (each of the row's two threads: half of d_k) -----
+    // P's shared memory is free now and takes the 128 x d_k block of O, rows 36 floats
+    // apart; then every 16-byte store instruction of a warp covers whole rows of the
+    // head's columns instead of 32 different rows.
+    const bool vec_out = ((reinterpret_cast<uintptr_t>(p.O) & 15) == 0) && (p.ldo % 4 == 0);
+    float *stage = reinterpret_cast<float *>(smem + L.p);
     if (ok) {
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_row, r);                  // d_k <= 32 columns are meaningful
         tmem_ld_wait();
         const int row = q0 + row_in;
-        if (row < p.N) {
-            // (the sums were exchanged before the barrier that precedes the second product)
-            const float inv = 1.f / (xch[kMhsaThreads + row_in] + xch[kMhsaThreads + row_in + kMhsaRows]);
+        // (the sums were exchanged before the barrier that precedes the second product)
+        const float inv = 1.f / (xch[kMhsaThreads + row_in] + xch[kMhsaThreads + row_in + kMhsaRows]);
+        if (vec_out) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const int d = half * 16 + g * 4;
+                if (d < p.dk)
+                    *reinterpret_cast<float4 *>(stage + row_in * kMhsaOutPitch + d) =
+                        make_float4(__uint_as_float(r[d]) * inv, __uint_as_float(r[d + 1]) * inv,
+                                    __uint_as_float(r[d + 2]) * inv, __uint_as_float(r[d + 3]) * inv);
+            }
+        } else if (row < p.N) {
             float *dst = p.O + row * p.ldo + col0;
 #pragma unroll
             for (int d = 0; d < kMhsaMaxDk; ++d)
@@ -298,6 +336,15 @@ mhsa_kernel(const MhsaParams p)
     }
     tc_fence_before();
     __syncthreads();
+    if (ok && vec_out) {
+        const int per_row = p.dk / 4;                  // 16-byte pieces per row: 2, 4, 6 or 8
+        const int rows = min(kMhsaRows, p.N - q0);
+        for (int i = tid; i < rows * per_row; i += kMhsaThreads) {
+            const int r = i / per_row, c = i - r * per_row;
+            *reinterpret_cast<float4 *>(p.O + (q0 + r) * p.ldo + col0 + c * 4) =
+                *reinterpret_cast<const float4 *>(stage + r * kMhsaOutPitch + c * 4);
+        }
+    }
     if (warp == 0) {
         __syncwarp();
         tc_fence_after();
