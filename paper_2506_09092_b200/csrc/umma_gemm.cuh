@@ -383,7 +383,9 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
             }
             __syncwarp();                                // tcgen05.ld needs the whole warp
         }
-        __threadfence();
+        // The warp barrier orders every lane's partial sums before lane 0's release store,
+        // whose fence is cumulative over them (the order a grid-wide barrier relies on too):
+        // one fence per warp instead of one per lane plus the store's own.
         __syncwarp();
         if (lane == 0) st_release_gpu(p.flags + my_slot * 4 + quad, p.epoch);
         if (c.split >= kChunks) return true;             // this unit owns no chunk
@@ -393,8 +395,7 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
             const long long slot = static_cast<long long>(c.slot0 + s) * ctas_per_tile + cta_slot;
             ok = wait_flag(p.flags + slot * 4 + quad, p.epoch, abort_flag) && ok;
         }
-        ok = __all_sync(0xffffffffu, ok);
-        __threadfence();
+        ok = __all_sync(0xffffffffu, ok);          // (every lane polled with acquire loads itself)
     }
 
     const int row0 = row - lane;                         // global row of this warp's lane 0
