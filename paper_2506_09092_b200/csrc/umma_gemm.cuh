@@ -13,7 +13,8 @@
 // first dp_tiles tiles are one unit each.  Every later tile is cut along K into
 // split_k units with consecutive indices (these units come first in the unit
 // order, so their epilogues overlap later main loops), and its 32-column chunks are dealt
-// round-robin to those units: unit j owns chunk c iff c mod split_k == j.  In
+// round-robin to those units, two adjacent chunks at a time where the tile has at least two
+// chunks per unit: unit j owns group q iff q mod split_k == j.  In
 // its epilogue a unit first writes the chunks it does not own (its fp32 partial
 // sums) to the workspace and raises a flag; then, for each chunk it owns, it
 // waits for the other units' flags, adds the partial chunks in split order
@@ -365,12 +366,16 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
     bool ok = true;
 
     if (S > 1) {
+        // Ownership goes by groups of two adjacent chunks where the tile has at least two
+        // chunks per unit (unit j owns group q iff q mod S == j), else by single chunks: an
+        // owner then fetches both chunks' partial sums in one round trip and stores 64 columns.
+        const int g = (kChunks >= 2 * S) ? 2 : 1;
         // 1. hand the chunks other units own to them
         const long long my_slot = static_cast<long long>(c.slot0 + c.split) * ctas_per_tile + cta_slot;
         float4 *mine = reinterpret_cast<float4 *>(p.partials) + my_slot * kTileF4;
 #pragma unroll 1
         for (int ch = 0; ch < kChunks; ++ch) {
-            if (ch % S == c.split) continue;
+            if ((ch / g) % S == c.split) continue;
             uint32_t r[32];
             tmem_ld_32x32b_x32(t_addr + ch * 32, r);
             tmem_ld_wait();
@@ -388,7 +393,7 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
         // one fence per warp instead of one per lane plus the store's own.
         __syncwarp();
         if (lane == 0) st_release_gpu(p.flags + my_slot * 4 + quad, p.epoch);
-        if (c.split >= kChunks) return true;             // this unit owns no chunk
+        if (c.split * g >= kChunks) return true;         // this unit owns no chunk
         // 2. the same epilogue warp of every other unit wrote the rows this warp needs
         for (int s = 0; s < S; ++s) {
             if (s == c.split) continue;
@@ -396,17 +401,74 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
             ok = wait_flag(p.flags + slot * 4 + quad, p.epoch, abort_flag) && ok;
         }
         ok = __all_sync(0xffffffffu, ok);          // (every lane polled with acquire loads itself)
+
+        const int row0 = row - lane;                     // global row of this warp's lane 0
+        if (row0 >= p.M) return ok;                      // the whole warp is below the matrix
+        const float4 *tile0 = reinterpret_cast<const float4 *>(p.partials)
+                            + (static_cast<long long>(c.slot0) * ctas_per_tile + cta_slot) * kTileF4;
+        // 3. the groups this unit owns: sum over the units in index order (this unit's own
+        //    term comes from TMEM), round once, store
+#pragma unroll 1
+        for (int grp = c.split; grp * g < kChunks; grp += S) {
+            const int ch = grp * g;
+            const int col0 = c.n_tile * BLOCK_N + ch * 32;
+            if (col0 >= p.N) break;                      // warp-uniform: nothing further to store
+            const bool two = g == 2 && col0 + 32 < p.N;
+            uint32_t ra[32], rb[32];
+            tmem_ld_32x32b_x32(t_addr + ch * 32, ra);
+            if (two) tmem_ld_32x32b_x32(t_addr + ch * 32 + 32, rb);
+            tmem_ld_wait();
+            float va[32], vb[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) va[j] = vb[j] = 0.f;
+            for (int s = 0; s < S; ++s) {
+                if (s == c.split) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        va[j] += __uint_as_float(ra[j]);
+                        if (two) vb[j] += __uint_as_float(rb[j]);
+                    }
+                } else if (row_ok) {
+                    const float4 *part = tile0 + static_cast<long long>(s) * ctas_per_tile * kTileF4
+                                       + (ch * 8) * kBlockM + row_in_tile;
+                    float4 ta[8], tb[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) ta[q] = __ldcg(part + q * kBlockM);
+                    if (two) {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) tb[q] = __ldcg(part + (8 + q) * kBlockM);
+                    }
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        va[4 * q] += ta[q].x; va[4 * q + 1] += ta[q].y;
+                        va[4 * q + 2] += ta[q].z; va[4 * q + 3] += ta[q].w;
+                    }
+                    if (two) {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            vb[4 * q] += tb[q].x; vb[4 * q + 1] += tb[q].y;
+                            vb[4 * q + 2] += tb[q].z; vb[4 * q + 3] += tb[q].w;
+                        }
+                    }
+                }
+            }
+            if (two && p.c_tma && (col0 + 64 <= p.N || p.n_edge_tma)) {
+                store_two_blocks_staged<OUT_BF16>(tmap_c, stage, sel, va, vb, c.b, row0, col0, lane);
+            } else {
+                store_block_staged<OUT_BF16>(p, tmap_c, stage, sel, va, c.b, row0, col0, lane);
+                if (two) store_block_staged<OUT_BF16>(p, tmap_c, stage, sel, vb, c.b, row0, col0 + 32, lane);
+            }
+        }
+        return ok;
     }
 
     const int row0 = row - lane;                         // global row of this warp's lane 0
     if (row0 >= p.M) return ok;                          // the whole warp is below the matrix
-    const float4 *tile0 = reinterpret_cast<const float4 *>(p.partials)
-                        + (static_cast<long long>(c.slot0) * ctas_per_tile + cta_slot) * kTileF4;
 #pragma unroll 1
-    for (int ch = (S > 1 ? c.split : 0); ch < kChunks; ch += S) {
+    for (int ch = 0; ch < kChunks; ++ch) {
         const int col0 = c.n_tile * BLOCK_N + ch * 32;
         if (col0 >= p.N) break;                          // warp-uniform: nothing further to store
-        if (S == 1 && p.c_tma && (ch & 1) == 0 && (col0 + 64 <= p.N || (p.n_edge_tma && col0 + 32 < p.N))) {
+        if (p.c_tma && (ch & 1) == 0 && (col0 + 64 <= p.N || (p.n_edge_tma && col0 + 32 < p.N))) {
             uint32_t ra[32], rb[32];
             tmem_ld_32x32b_x32(t_addr + ch * 32, ra);
             tmem_ld_32x32b_x32(t_addr + ch * 32 + 32, rb);
@@ -418,45 +480,25 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
                 vb[j] = __uint_as_float(rb[j]);
             }
             store_two_blocks_staged<OUT_BF16>(tmap_c, stage, sel, va, vb, c.b, row0, col0, lane);
-            ++ch;                                        // (the loop adds S == 1)
+            ++ch;
             continue;
         }
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_addr + ch * 32, r);
         tmem_ld_wait();
         float v[32];
-        if (S == 1) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-        } else {
-            // sum over the splits in index order; this unit's own term comes from TMEM
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = 0.f;
-            for (int s = 0; s < S; ++s) {
-                if (s == c.split) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(r[j]);
-                } else if (row_ok) {
-                    const float4 *part = tile0 + static_cast<long long>(s) * ctas_per_tile * kTileF4
-                                       + (ch * 8) * kBlockM + row_in_tile;
-                    float4 t[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) t[q] = __ldcg(part + q * kBlockM);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        v[4 * q] += t[q].x; v[4 * q + 1] += t[q].y;
-                        v[4 * q + 2] += t[q].z; v[4 * q + 3] += t[q].w;
-                    }
-                }
-            }
-        }
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
         store_block_staged<OUT_BF16>(p, tmap_c, stage, sel, v, c.b, row0, col0, lane);
     }
     return ok;
 }
 
+// (Instantiations whose shared memory lets two CTAs share an SM must also fit two CTAs'
+// registers: 65536 / (2 x 192) = 170 per thread.)
 template <int BLOCK_N, int STAGES, int KSUB, bool OUT_BF16, int A_ROWS = kBlockM>
-__global__ void __launch_bounds__(kNumThreads, 1)
+__global__ void __launch_bounds__(kNumThreads,
+                                  SmemLayout<BLOCK_N, STAGES, KSUB, A_ROWS>::kDynamicBytes <= 112 * 1024 ? 2 : 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                  const __grid_constant__ CUtensorMap tmap_c, const GemmParams p)
 {
