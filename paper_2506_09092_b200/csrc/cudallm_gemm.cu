@@ -239,9 +239,9 @@ double variant_cost(const Variant &v, const Problem &p)
         const double rounds = (double)cdiv((int64_t)split_units, slots);
         const double part_main = (double)cdiv(t.kblocks, t.split) * per_kb;
         // exchange of partial chunks between the units of a tile: each unit writes
-        // and reads (S-1)/S of a tile through L2; measured a few microseconds per
-        // unit, growing with the number of partners
-        const double fix = 2500.0 + (t.split - 1) * 3500.0;
+        // and reads (S-1)/S of a tile through L2; measured ~2.4 us for two units of a
+        // 128 x 128 tile, growing with the number of partners and the size of the tile
+        const double fix = 2000.0 + (t.split - 1) * (1500.0 + rows * v.block_n * 4.0 / 64.0);
         compute += rounds * (part_main + fix);
     }
     compute += epi;
