@@ -240,6 +240,29 @@ int cudallm_select_variant(int64_t M, int64_t N, int64_t K,
                            int64_t batch, int out_dtype);
 
 /*
+ * Dispatch table: the persisted outcome of the search (Algorithm 1's arg-min
+ * over the valid candidates, one entry per problem shape).  An entry says that
+ * `variant` is the fastest valid kernel for products of shape (M, N, K, batch,
+ * out_dtype).  cudallm_gemm_bf16, cudallm_gemm_bf16_batched,
+ * cudallm_gemm_bf16_host and cudallm_select_variant look the shape up first and
+ * use the entry if that variant can run the problem; otherwise, and for every
+ * shape without an entry, the cost model decides.
+ * The table is process-wide, starts empty and holds at most 65536 entries.
+ *   cudallm_dispatch_set    adds or replaces an entry; variant == -1 removes it.
+ *                           Errors: INVALID_DIM (a negative size), INVALID_DTYPE,
+ *                           INVALID_VARIANT (not -1 and not a variant id),
+ *                           TOO_LARGE (table full).
+ *   cudallm_dispatch_get    *variant = the entry's variant, or -1 if there is none.
+ *                           Errors: as above, INVALID_POINTER (variant == NULL).
+ *   cudallm_dispatch_clear  empties the table; returns the number of entries it held.
+ * Host-side only: no CUDA call.  Safe to call from several threads; a change is
+ * seen by calls that start after it returns.
+ */
+int cudallm_dispatch_set(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int variant);
+int cudallm_dispatch_get(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int *variant);
+int cudallm_dispatch_clear(void);
+
+/*
  * Workspace.  Upper bound of the scratch bytes any variant may need for the
  * problem (repacked operands, split-K partial tiles and their flags).  Without
  * cudallm_set_workspace the library allocates (and grows) one workspace per

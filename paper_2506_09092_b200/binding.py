@@ -49,6 +49,9 @@ SIGNATURES = {
     "cudallm_host_staging_bytes": (_sz, [_i64] * 6 + [_int]),
     "cudallm_gemm_bf16_splitk_noalloc": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _int, _vp]),
     "cudallm_num_variants": (_int, []),
+    "cudallm_dispatch_set": (_int, [_i64, _i64, _i64, _i64, _int, _int]),
+    "cudallm_dispatch_get": (_int, [_i64, _i64, _i64, _i64, _int, ctypes.POINTER(ctypes.c_int)]),
+    "cudallm_dispatch_clear": (_int, []),
     "cudallm_variant_name": (ctypes.c_char_p, [_int]),
     "cudallm_variant_supports": (_int, [_int] + [_i64] * 7 + [_int]),
     "cudallm_select_variant": (_int, [_i64] * 7 + [_int]),
@@ -190,6 +193,24 @@ def gemm_bf16_splitk_noalloc(A, B, C, M, N, K, lda, ldb, ldc, out_dtype, split_k
 
 def host_staging_bytes(M, N, K, lda, ldb, ldc, out_dtype) -> int:
     return int(lib().cudallm_host_staging_bytes(M, N, K, lda, ldb, ldc, out_dtype))
+
+
+def dispatch_set(M, N, K, batch, out_dtype, variant, check=True) -> int:
+    """Record ``variant`` as the kernel for products of this shape (-1 removes the entry):
+    the library's automatic choice uses it before its cost model."""
+    return _check(lib().cudallm_dispatch_set(M, N, K, batch, out_dtype, variant), "cudallm_dispatch_set", check)
+
+
+def dispatch_get(M, N, K, batch, out_dtype) -> int:
+    """The recorded variant for the shape, or -1."""
+    v = ctypes.c_int(-1)
+    _check(lib().cudallm_dispatch_get(M, N, K, batch, out_dtype, ctypes.byref(v)), "cudallm_dispatch_get", True)
+    return int(v.value)
+
+
+def dispatch_clear() -> int:
+    """Empty the dispatch table; returns how many entries it held."""
+    return int(lib().cudallm_dispatch_clear())
 
 
 def num_variants() -> int:

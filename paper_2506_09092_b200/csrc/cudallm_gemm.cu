@@ -11,7 +11,9 @@
 #include <cstdio>
 #include <algorithm>
 #include <cstring>
+#include <atomic>
 #include <mutex>
+#include <unordered_map>
 
 #include "aux_kernels.cuh"
 #include "umma_gemm.cuh"
@@ -253,10 +255,38 @@ double variant_cost(const Variant &v, const Problem &p)
     return (compute > memory ? compute : memory) + 4000.0;
 }
 
+// Dispatch table: shape -> variant recorded by a search (cudallm_dispatch_set).
+struct DispatchKey {
+    int64_t M, N, K, batch;
+    int out_dtype;
+    bool operator==(const DispatchKey &o) const
+    {
+        return M == o.M && N == o.N && K == o.K && batch == o.batch && out_dtype == o.out_dtype;
+    }
+};
+struct DispatchHash {
+    size_t operator()(const DispatchKey &k) const
+    {
+        uint64_t h = 0x9E3779B97F4A7C15ull;
+        for (uint64_t x : {(uint64_t)k.M, (uint64_t)k.N, (uint64_t)k.K, (uint64_t)k.batch, (uint64_t)k.out_dtype})
+            h = (h ^ x) * 0x100000001B3ull + (h >> 29);
+        return (size_t)h;
+    }
+};
+constexpr size_t kMaxDispatchEntries = 65536;
+std::unordered_map<DispatchKey, int, DispatchHash> g_dispatch;
+std::mutex g_dispatch_mutex;
+std::atomic<uint64_t> g_dispatch_generation{0};      // bumped by every change of the table
+
 int select_variant_uncached(const Problem &p)
 {
     build_variants();
     if (is_empty(p) || p.K == 0) return 0;
+    {
+        std::lock_guard<std::mutex> lock(g_dispatch_mutex);
+        const auto it = g_dispatch.find(DispatchKey{p.M, p.N, p.K, p.batch, p.out_dtype});
+        if (it != g_dispatch.end() && variant_supports(g_variants[it->second], p)) return it->second;
+    }
     int best = -1;
     double best_cost = 0;
     for (int v = 1; v < kNumVariants; ++v) {
@@ -267,17 +297,18 @@ int select_variant_uncached(const Problem &p)
     return best < 0 ? 0 : best;
 }
 
-// The choice depends only on the shape; repeated calls with the same shape (the
-// common case) reuse the previous answer.
+// The choice depends only on the shape (and the dispatch table); repeated calls with
+// the same shape (the common case) reuse the previous answer.
 int select_variant(const Problem &p)
 {
-    struct Last { int64_t M, N, K, batch; int out_dtype, variant; };
-    static thread_local Last last = {-1, -1, -1, -1, -1, 0};
+    struct Last { int64_t M, N, K, batch; int out_dtype, variant; uint64_t generation; };
+    static thread_local Last last = {-1, -1, -1, -1, -1, 0, 0};
+    const uint64_t gen = g_dispatch_generation.load(std::memory_order_acquire);
     if (last.M == p.M && last.N == p.N && last.K == p.K && last.batch == p.batch
-        && last.out_dtype == p.out_dtype)
+        && last.out_dtype == p.out_dtype && last.generation == gen)
         return last.variant;
     const int v = select_variant_uncached(p);
-    last = Last{p.M, p.N, p.K, p.batch, p.out_dtype, v};
+    last = Last{p.M, p.N, p.K, p.batch, p.out_dtype, v, gen};
     return v;
 }
 
@@ -1202,6 +1233,52 @@ int cudallm_select_variant(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t
     int st = validate(p);
     if (st != CUDALLM_OK) return st;
     return select_variant(p);
+}
+
+static int dispatch_key_status(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype)
+{
+    if (M < 0 || N < 0 || K < 0 || batch < 0) return CUDALLM_ERR_INVALID_DIM;
+    if (out_dtype != CUDALLM_F32 && out_dtype != CUDALLM_BF16) return CUDALLM_ERR_INVALID_DTYPE;
+    return CUDALLM_OK;
+}
+
+int cudallm_dispatch_set(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int variant)
+{
+    build_variants();
+    const int st = dispatch_key_status(M, N, K, batch, out_dtype);
+    if (st != CUDALLM_OK) return st;
+    if (variant < -1 || variant >= kNumVariants) return CUDALLM_ERR_INVALID_VARIANT;
+    const DispatchKey key{M, N, K, batch, out_dtype};
+    std::lock_guard<std::mutex> lock(g_dispatch_mutex);
+    if (variant < 0) {
+        g_dispatch.erase(key);
+    } else {
+        if (g_dispatch.size() >= kMaxDispatchEntries && g_dispatch.find(key) == g_dispatch.end())
+            return CUDALLM_ERR_TOO_LARGE;
+        g_dispatch[key] = variant;
+    }
+    g_dispatch_generation.fetch_add(1, std::memory_order_release);
+    return CUDALLM_OK;
+}
+
+int cudallm_dispatch_get(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int *variant)
+{
+    const int st = dispatch_key_status(M, N, K, batch, out_dtype);
+    if (st != CUDALLM_OK) return st;
+    if (!variant) return CUDALLM_ERR_INVALID_POINTER;
+    std::lock_guard<std::mutex> lock(g_dispatch_mutex);
+    const auto it = g_dispatch.find(DispatchKey{M, N, K, batch, out_dtype});
+    *variant = it == g_dispatch.end() ? -1 : it->second;
+    return CUDALLM_OK;
+}
+
+int cudallm_dispatch_clear(void)
+{
+    std::lock_guard<std::mutex> lock(g_dispatch_mutex);
+    const int n = (int)g_dispatch.size();
+    g_dispatch.clear();
+    g_dispatch_generation.fetch_add(1, std::memory_order_release);
+    return n;
 }
 
 size_t cudallm_workspace_bytes(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,

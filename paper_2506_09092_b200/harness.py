@@ -373,6 +373,23 @@ class TunedTable:
         with open(path) as f:
             return cls(json.load(f))
 
+    def install(self) -> int:
+        """Enter every record into the library's dispatch table (``cudallm_dispatch_set``), so
+        that its automatic choice uses the searched winners; returns how many were entered
+        (records that name a variant this build does not have are skipped)."""
+        from . import binding as B
+        names = {B.variant_name(v): v for v in range(B.num_variants())}
+        n = 0
+        for key, rec in self.entries.items():
+            shape, dtype = key.split(":")
+            M, N, K, batch = (int(x) for x in shape.split("x"))
+            v = names.get(rec["variant"])
+            if v is None:
+                continue
+            B.dispatch_set(M, N, K, batch, B.BF16 if dtype == "bf16" else B.F32, v)
+            n += 1
+        return n
+
     @classmethod
     def packaged(cls):
         """The table recorded on a B200 with ``--search --config all --table ...`` and shipped with
@@ -429,6 +446,8 @@ def _main(argv=None):
     ap.add_argument("--search", action="store_true",
                     help="validate every variant on closed-form cases, time the valid ones, report the fastest")
     ap.add_argument("--table", default=None, help="with --search: JSON file to record the winner in")
+    ap.add_argument("--dispatch", default=None,
+                    help="a table file, or 'packaged': enter its records into the library's dispatch table first")
     ap.add_argument("--task", default=None, choices=["transpose", "sum", "dot", "layernorm"],
                     help="time one of the float32 tasks (8, 14, 15, 4) instead of a GEMM configuration")
     ap.add_argument("--size", type=int, default=None,
@@ -436,6 +455,9 @@ def _main(argv=None):
     args = ap.parse_args(argv)
     if args.task:
         return _task_main(args)
+    if args.dispatch:
+        table = TunedTable.packaged() if args.dispatch == "packaged" else TunedTable.load(args.dispatch)
+        table.install()
     if args.search:
         for name in (sorted(all_configs) if args.config == "all" else [args.config]):
             if args.config == "all" and all_configs[name].flops > 2e12:

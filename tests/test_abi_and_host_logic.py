@@ -226,3 +226,55 @@ def test_packaged_tuned_table_names_existing_variants():
                                   cfg.out_dtype) == 1
         assert table.variant_id(cfg.M, cfg.N, cfg.K, cfg.batch, cfg.out_dtype) == names[name]
     assert table.lookup(7, 7, 7, 1, 0) is None and table.variant_id(7, 7, 7, 1, 0) == -1
+
+
+def test_dispatch_table_overrides_the_cost_model_for_its_shapes():
+    """An entry of the dispatch table is what the automatic choice returns for that shape
+    (and only that shape); an entry whose variant cannot run the shape is ignored; removing
+    or clearing restores the cost model's answer.  Host logic only: no GPU needed."""
+    names = {B.variant_name(v): v for v in range(B.num_variants())}
+    shape = (4096, 4096, 4096)
+    args = shape + (4096, 4096, 4096, 1, B.BF16)           # M, N, K, lda, ldb, ldc, batch, dtype
+    assert B.dispatch_clear() >= 0
+    try:
+        model = B.select_variant(*args)
+        other = names["umma_n128"] if model != names["umma_n128"] else names["umma_n256"]
+        assert B.dispatch_get(*shape, 1, B.BF16) == -1
+        B.dispatch_set(*shape, 1, B.BF16, other)
+        assert B.dispatch_get(*shape, 1, B.BF16) == other
+        assert B.select_variant(*args) == other
+        f32_model = B.select_variant(*shape, 4096, 4096, 4096, 1, B.F32)
+        B.dispatch_set(*shape, 1, B.BF16, other)                 # (again: replaces)
+        assert B.select_variant(*shape, 4096, 4096, 4096, 1, B.F32) == f32_model      # another key: the model
+        B.dispatch_set(*shape, 1, B.BF16, -1)
+        assert B.select_variant(*args) == model
+        # a variant that cannot run the shape (16 K-parts of a single k-block) is not used
+        small = (256, 256, 64)
+        small_model = B.select_variant(*small, 64, 256, 256, 1, B.F32)
+        B.dispatch_set(*small, 1, B.F32, names["umma_n64_sk16"])
+        assert B.variant_supports(names["umma_n64_sk16"], *small, 64, 256, 256, 1, B.F32) == 0
+        assert B.select_variant(*small, 64, 256, 256, 1, B.F32) == small_model
+        assert B.dispatch_clear() == 1
+        # argument errors
+        assert B.dispatch_set(-1, 1, 1, 1, B.F32, 1, check=False) == B.ERR_INVALID_DIM
+        assert B.dispatch_set(1, 1, 1, 1, 7, 1, check=False) == B.ERR_INVALID_DTYPE
+        assert B.dispatch_set(1, 1, 1, 1, B.F32, B.num_variants(), check=False) == B.ERR_INVALID_VARIANT
+        assert B.dispatch_set(1, 1, 1, 1, B.F32, -2, check=False) == B.ERR_INVALID_VARIANT
+    finally:
+        B.dispatch_clear()
+
+
+def test_packaged_table_installs_into_the_dispatch_table():
+    table = H.TunedTable.packaged()
+    names = {B.variant_name(v): v for v in range(B.num_variants())}
+    try:
+        B.dispatch_clear()
+        assert table.install() == len(table.entries)
+        for key, rec in table.entries.items():
+            shape, dtype = key.split(":")
+            M, N, K, batch = (int(x) for x in shape.split("x"))
+            dt = B.BF16 if dtype == "bf16" else B.F32
+            assert B.dispatch_get(M, N, K, batch, dt) == names[rec["variant"]]
+            assert B.select_variant(M, N, K, K, N, N, batch, dt) == names[rec["variant"]]
+    finally:
+        B.dispatch_clear()
