@@ -100,3 +100,27 @@ def test_paper_task2_ladder_larger_sizes_closed_form(step):
     want = torch.outer(torch.from_numpy(u.astype(np.float32)).cuda(),
                        torch.from_numpy(v_.astype(np.float32)).cuda()) * scale      # exact in fp32
     assert torch.equal(dC.view(cfg.M, cfg.N), want)
+
+
+def test_automatic_choice_follows_the_dispatch_table():
+    """With an entry in the dispatch table the plain entry point runs that variant
+    (here split-K kernels the cost model would not pick for the shape) and the
+    result still agrees with the oracle; other shapes are untouched."""
+    names = _names()
+    rng = np.random.default_rng(5)
+    M, N, K = 200, 330, 1030
+    A = bits(rng.standard_normal((M, K))); Bm = bits(rng.standard_normal((K, N)))
+    Cref, S = oracle.gemm(A, Bm, M, N, K)
+    try:
+        B.dispatch_clear()
+        model = B.select_variant(M, N, K, K, N, N, 1, gi.F32)
+        for forced in ("umma_n64_sk4", "umma2_n256_sk2", "umma_n128_sk2"):
+            assert names[forced] != model
+            B.dispatch_set(M, N, K, 1, gi.F32, names[forced])
+            assert B.select_variant(M, N, K, K, N, N, 1, gi.F32) == names[forced]
+            vals, raw, guards = G.run_gemm(A.ravel(), Bm.ravel(), M, N, K, K, N, N, gi.F32)      # automatic choice
+            r = oracle.check(vals[0], Cref, S, G.tol_for(gi.F32))
+            assert guards and r.ok, (forced, r)
+        assert B.select_variant(M, N, K + 1, K + 1, N, N, 1, gi.F32) != -1
+    finally:
+        B.dispatch_clear()
