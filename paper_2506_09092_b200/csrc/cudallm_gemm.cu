@@ -1023,7 +1023,7 @@ int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int6
     mp.N = (int)N; mp.h = (int)h; mp.dk = (int)dk;
     mp.keys_pad = (int)round_up(N, 32);
     mp.dkp = (int)round_up(dk, 16);
-    mp.tmem_cols = 32;
+    mp.tmem_cols = 64;                                  // the second product writes dkp + 16 <= 48 columns
     while (mp.tmem_cols < mp.keys_pad) mp.tmem_cols *= 2;
     mp.ldq = ldq; mp.ldk = ldk; mp.ldv = ldv; mp.ldo = ldo;
     mp.scale_log2 = 1.4426950408889634f / sqrtf((float)dk);

@@ -21,8 +21,10 @@
 //      p = exp2((s - max) * log2(e)/sqrt(d_k)), masked beyond N, summed, rounded
 //      to bf16 and written to shared memory as the K-major A operand of the
 //      second product);
-//   4. one thread issues O = P V_i (V_i is the MN-major B operand) into the TMEM
-//      columns that S no longer needs;
+//   4. one thread issues O = P [V_i | 1] (V_i is the MN-major B operand, with a
+//      column of ones behind its d_k columns) into the TMEM columns that S no
+//      longer needs: column d_k of O is the row sum of the rounded probabilities,
+//      exactly what the product saw, at no cost to the softmax threads;
 //   5. the row's two threads divide their halves of the row of O by the row sum;
 //      the block goes through shared memory so that a warp's store covers whole
 //      rows of the head's columns.
@@ -47,7 +49,7 @@ struct MhsaParams {
     int N, h, dk;
     int keys_pad;           // N rounded up to 32
     int dkp;                // d_k rounded up to 16 (K of the first product, N of the second)
-    int tmem_cols;          // power of two >= max(keys_pad, 32): tensor-memory columns to allocate
+    int tmem_cols;          // power of two >= max(keys_pad, 64): tensor-memory columns to allocate
     long long ldq, ldk, ldv, ldo;
     float scale_log2;       // log2(e) / sqrt(d_k)
     int *status;
@@ -96,7 +98,10 @@ __host__ __device__ inline MhsaSmem mhsa_smem_layout(int keys_pad, int dkp)
     s.lbo_q = kMhsaRows * 16 + 32;                    // [chunk][row][16 B] + padding
     s.lbo_k = keys_pad * 16 + 32;                     // [chunk][key][16 B] + padding
     s.sbo_v = 128 + 32;                               // [key group][chunk][key in group][16 B] + padding
-    s.lbo_v = kchunks * s.sbo_v;
+    // one more chunk per key group: the column of ones.  (The second product has N = dkp + 16
+    // columns, so it also reads the chunk after that one -- the next group's first chunk, or
+    // the bytes behind V for the last group -- into output columns that nobody looks at.)
+    s.lbo_v = (kchunks + 1) * s.sbo_v;
     s.q = 0;
     s.k = s.q + kchunks * s.lbo_q;
     s.v = s.k + kchunks * s.lbo_k;
@@ -108,6 +113,25 @@ __host__ __device__ inline MhsaSmem mhsa_smem_layout(int keys_pad, int dkp)
     s.xch = s.bar + 64;                               // row maxima and row sums of the two halves
     s.total = s.xch + 2 * kMhsaThreads * 4;
     return s;
+}
+
+// 32 scores of one row -> 32 probabilities exp2(s * c - max * c), rounded to bf16 and packed
+// in pairs: one FMA and one ex2.approx per element.  MASKED: keys from `valid` on do not
+// exist (the ragged last chunk) and get probability 0.
+template <bool MASKED>
+__device__ __forceinline__ void mhsa_exp_chunk(const uint32_t (&r)[32], float scale, float neg_max_scaled,
+                                               int valid, uint32_t (&w)[16])
+{
+#pragma unroll
+    for (int j = 0; j < 32; j += 2) {
+        float e0 = fast_exp2(fmaf(__uint_as_float(r[j]), scale, neg_max_scaled));
+        float e1 = fast_exp2(fmaf(__uint_as_float(r[j + 1]), scale, neg_max_scaled));
+        if (MASKED) {
+            if (j >= valid) e0 = 0.f;
+            if (j + 1 >= valid) e1 = 0.f;
+        }
+        w[j >> 1] = pack_bf16x2(e0, e1);
+    }
 }
 
 __global__ void __launch_bounds__(kMhsaThreads, 1)
@@ -183,6 +207,10 @@ mhsa_kernel(const MhsaParams p)
         for (int u = 0; u < kInFlight; ++u)
             if (dst[u] >= 0) *reinterpret_cast<uint4 *>(smem + dst[u]) = x[u];
     }
+    // behind V's d_k chunks: a column of ones (bf16 1.0 in element 0 of the chunk)
+    for (int j = tid; j < p.keys_pad; j += kMhsaThreads)
+        *reinterpret_cast<uint4 *>(smem + L.v + (j >> 3) * L.lbo_v + kchunks * L.sbo_v + (j & 7) * 16) =
+            make_uint4(0x3F80u, 0, 0, 0);
     fence_proxy_async_smem();                         // make the writes visible to the tensor core
     tc_fence_before();
     __syncthreads();
@@ -243,7 +271,6 @@ mhsa_kernel(const MhsaParams p)
     xch[tid] = row_max;
     __syncthreads();
     row_max = fmaxf(xch[row_in], xch[row_in + kMhsaRows]);          // the first half always has a key < N
-    float row_sum = 0.f;
     const float neg_max_scaled = -row_max * p.scale_log2;
     if (ok) {
         const int r_off = (row_in >> 3) * 128 + (row_in & 7) * 16;           // this row inside a chunk of P
@@ -259,20 +286,8 @@ mhsa_kernel(const MhsaParams p)
                 const int ch = ch0 + u;
                 if (ch < ch_hi) {
                     uint32_t w[16];
-                    const bool full = ch * 32 + 32 <= p.N;                   // all 32 keys exist
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        // exp2(s * c - max * c): one FMA and one ex2.approx per element
-                        float e0 = 0.f, e1 = 0.f;
-                        if (full || ch * 32 + j < p.N)
-                            e0 = fast_exp2(fmaf(__uint_as_float(r[u][j]), p.scale_log2, neg_max_scaled));
-                        if (full || ch * 32 + j + 1 < p.N)
-                            e1 = fast_exp2(fmaf(__uint_as_float(r[u][j + 1]), p.scale_log2, neg_max_scaled));
-                        const uint32_t packed = pack_bf16x2(e0, e1);
-                        // the row sum uses the rounded probabilities: exactly what the second product sees
-                        row_sum += __uint_as_float(packed << 16) + __uint_as_float(packed & 0xFFFF0000u);
-                        w[j >> 1] = packed;
-                    }
+                    if (ch * 32 + 32 <= p.N) mhsa_exp_chunk<false>(r[u], p.scale_log2, neg_max_scaled, 32, w);
+                    else                     mhsa_exp_chunk<true>(r[u], p.scale_log2, neg_max_scaled, p.N - ch * 32, w);
 #pragma unroll
                     for (int g = 0; g < 4; ++g)                              // 8 keys = one 16-byte chunk
                         *reinterpret_cast<uint4 *>(smem + L.p + (ch * 4 + g) * 2048 + r_off) =
@@ -281,7 +296,6 @@ mhsa_kernel(const MhsaParams p)
             }
         }
     }
-    xch[kMhsaThreads + tid] = row_sum;
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();                                   // everyone is done reading S and writing P
@@ -289,7 +303,7 @@ mhsa_kernel(const MhsaParams p)
 
     // ---- 4. O = P V -------------------------------------------------------------
     if (tid == 0 && ok) {
-        const uint32_t idesc = make_idesc_bf16(kMhsaRows, p.dkp, 0, 1);      // V: MN-major
+        const uint32_t idesc = make_idesc_bf16(kMhsaRows, p.dkp + 16, 0, 1); // [V | 1 | unused]: MN-major
         for (int ks = 0; ks < p.keys_pad / 16; ++ks) {
             const uint64_t da = make_smem_desc_plain(sbase + L.p + ks * 2 * 2048, 2048, 128);
             const uint64_t db = make_smem_desc_plain(sbase + L.v + ks * 2 * L.lbo_v, L.lbo_v, L.sbo_v);
@@ -310,26 +324,28 @@ mhsa_kernel(const MhsaParams p)
     const bool vec_out = ((reinterpret_cast<uintptr_t>(p.O) & 15) == 0) && (p.ldo % 4 == 0);
     float *stage = reinterpret_cast<float *>(smem + L.p);
     if (ok) {
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(t_row, r);                  // d_k <= 32 columns are meaningful
+        uint32_t r[32], r2[32];
+        tmem_ld_32x32b_x32(t_row, r);                  // d_k <= 32 columns of O ...
+        if (p.dkp == 32) tmem_ld_32x32b_x32(t_row + 32, r2);                 // ... and the row sum in column dkp
         tmem_ld_wait();
         const int row = q0 + row_in;
-        // (the sums were exchanged before the barrier that precedes the second product)
-        const float inv = 1.f / (xch[kMhsaThreads + row_in] + xch[kMhsaThreads + row_in + kMhsaRows]);
+        const float inv = 1.f / __uint_as_float(p.dkp == 32 ? r2[0] : r[16]);
+        float o[16];                                   // this thread's half of the row
+#pragma unroll
+        for (int k = 0; k < 16; ++k) o[k] = __uint_as_float(half ? r[16 + k] : r[k]) * inv;
         if (vec_out) {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 const int d = half * 16 + g * 4;
                 if (d < p.dk)
                     *reinterpret_cast<float4 *>(stage + row_in * kMhsaOutPitch + d) =
-                        make_float4(__uint_as_float(r[d]) * inv, __uint_as_float(r[d + 1]) * inv,
-                                    __uint_as_float(r[d + 2]) * inv, __uint_as_float(r[d + 3]) * inv);
+                        make_float4(o[4 * g], o[4 * g + 1], o[4 * g + 2], o[4 * g + 3]);
             }
         } else if (row < p.N) {
-            float *dst = p.O + row * p.ldo + col0;
+            float *dst = p.O + row * p.ldo + col0 + half * 16;
 #pragma unroll
-            for (int d = 0; d < kMhsaMaxDk; ++d)
-                if (d < p.dk && (d >> 4) == half) dst[d] = __uint_as_float(r[d]) * inv;
+            for (int k = 0; k < 16; ++k)
+                if (half * 16 + k < p.dk) dst[k] = o[k];
         }
     } else if (tid == 0) {
         if (atomicCAS(p.status, 0, -9) == 0) p.status[1] = 0x600;
