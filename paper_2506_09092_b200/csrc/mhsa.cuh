@@ -168,45 +168,34 @@ mhsa_kernel(const MhsaParams p)
 
     // ---- 1. operands -> shared memory, in core-matrix order -------------------
     // One list of 16-byte pieces: the rows of Q, then K's, then V's, the d_k chunks of a
-    // row on neighbouring lanes.  Each thread keeps up to eighteen loads in flight (at the
-    // largest size, N = 512 and d_k = 32, that is its whole share, fetched in one go).
-    const uint4 zero = make_uint4(0, 0, 0, 0);
+    // row on neighbouring lanes (at the largest size, N = 512 and d_k = 32, eighteen per thread).
     const int kshift = kchunks == 4 ? 2 : 1;          // kchunks is 2 or 4
     const int total = (kMhsaRows + 2 * p.keys_pad) << kshift;
-    constexpr int kInFlight = 18;
-    for (int i0 = tid; i0 < total; i0 += kInFlight * kMhsaThreads) {
-        uint4 x[kInFlight];
-        int dst[kInFlight];
-#pragma unroll
-        for (int u = 0; u < kInFlight; ++u) {
-            const int i = i0 + u * kMhsaThreads;
-            x[u] = zero;
-            dst[u] = -1;
-            if (i < total) {
-                const __nv_bfloat16 *src = nullptr;
-                const int c = i & (kchunks - 1);
-                int r = i >> kshift;
-                const bool live = c * 8 < p.dk;
-                if (r < kMhsaRows) {                  // Q: row within the block
-                    const int row = q0 + r;
-                    dst[u] = L.q + c * L.lbo_q + r * 16;
-                    if (row < p.N && live) src = p.Q + row * p.ldq + col0 + c * 8;
-                } else if (r < kMhsaRows + p.keys_pad) {
-                    r -= kMhsaRows;                   // K: key
-                    dst[u] = L.k + c * L.lbo_k + r * 16;
-                    if (r < p.N && live) src = p.K + r * p.ldk + col0 + c * 8;
-                } else {
-                    r -= kMhsaRows + p.keys_pad;      // V: key
-                    dst[u] = L.v + (r >> 3) * L.lbo_v + c * L.sbo_v + (r & 7) * 16;
-                    if (r < p.N && live) src = p.V + r * p.ldv + col0 + c * 8;
-                }
-                if (src) x[u] = *reinterpret_cast<const uint4 *>(src);
-            }
+    // Asynchronous 16-byte copies straight into shared memory (a piece outside the
+    // operand -- a padding row or d_k chunk -- copies zero source bytes: it is zero-filled).
+    for (int i = tid; i < total; i += kMhsaThreads) {
+        const __nv_bfloat16 *src = p.Q;               // (any valid address: no byte of it is read)
+        uint32_t bytes = 0;
+        int dst;
+        const int c = i & (kchunks - 1);
+        int r = i >> kshift;
+        const bool live = c * 8 < p.dk;
+        if (r < kMhsaRows) {                          // Q: row within the block
+            const int row = q0 + r;
+            dst = L.q + c * L.lbo_q + r * 16;
+            if (row < p.N && live) { src = p.Q + row * p.ldq + col0 + c * 8; bytes = 16; }
+        } else if (r < kMhsaRows + p.keys_pad) {
+            r -= kMhsaRows;                           // K: key
+            dst = L.k + c * L.lbo_k + r * 16;
+            if (r < p.N && live) { src = p.K + r * p.ldk + col0 + c * 8; bytes = 16; }
+        } else {
+            r -= kMhsaRows + p.keys_pad;              // V: key
+            dst = L.v + (r >> 3) * L.lbo_v + c * L.sbo_v + (r & 7) * 16;
+            if (r < p.N && live) { src = p.V + r * p.ldv + col0 + c * 8; bytes = 16; }
         }
-#pragma unroll
-        for (int u = 0; u < kInFlight; ++u)
-            if (dst[u] >= 0) *reinterpret_cast<uint4 *>(smem + dst[u]) = x[u];
+        cp_async_16(sbase + dst, src, bytes);
     }
+    cp_async_wait_all();
     // behind V's d_k chunks: a column of ones (bf16 1.0 in element 0 of the chunk)
     for (int j = tid; j < p.keys_pad; j += kMhsaThreads)
         *reinterpret_cast<uint4 *>(smem + L.v + (j >> 3) * L.lbo_v + kchunks * L.sbo_v + (j & 7) * 16) =

@@ -37,6 +37,19 @@ __device__ __forceinline__ void grid_launch_dependents()
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// ------------------------------------------------- asynchronous copies --
+// 16 bytes global -> shared without passing through registers; only the first `src_bytes`
+// (0 or 16) are read from global memory, the rest of the 16 is zero-filled.
+__device__ __forceinline__ void cp_async_16(uint32_t smem_addr, const void *gptr, uint32_t src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gptr), "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
+
 // ------------------------------------------------------- named barriers --
 // Barrier `id` (1..15; 0 is __syncthreads) over `threads` threads of the CTA: whole
 // warps either wait for all of them or only announce their arrival and go on.
