@@ -36,7 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 L2_BYTES = 126e6
 # DRAM traffic of one launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).
-NCU_TRAFFIC_BYTES = {"C2": 120.6e6, "C5a": 274.6e6}
+NCU_TRAFFIC_BYTES = {"C2": 119.4e6, "C5a": 273.1e6}
 
 
 def load_peaks():
