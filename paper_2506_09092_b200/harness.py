@@ -448,10 +448,11 @@ def _main(argv=None):
     ap.add_argument("--table", default=None, help="with --search: JSON file to record the winner in")
     ap.add_argument("--dispatch", default=None,
                     help="a table file, or 'packaged': enter its records into the library's dispatch table first")
-    ap.add_argument("--task", default=None, choices=["transpose", "sum", "dot", "layernorm"],
-                    help="time one of the float32 tasks (8, 14, 15, 4) instead of a GEMM configuration")
+    ap.add_argument("--task", default=None, choices=["transpose", "sum", "dot", "layernorm", "attention"],
+                    help="time one of the other tasks (8, 14, 15, 4, 6) instead of a GEMM configuration")
     ap.add_argument("--size", type=int, default=None,
-                    help="with --task: N (transpose: N x N; sum, dot: N elements; layernorm: (16, 4, N, N))")
+                    help="with --task: N (transpose: N x N; sum, dot: N elements; layernorm: (16, 4, N, N); "
+                         "attention: N queries and keys)")
     args = ap.parse_args(argv)
     if args.task:
         return _task_main(args)
@@ -487,13 +488,25 @@ def _main(argv=None):
 
 
 def task_problem(task: str, size: int, nsets: int | None = None):
-    """(launch(i), algorithmic bytes per call, description) for one float32 task on seeded
-    device inputs, with enough rotating buffer sets to exceed L2 (at most 8)."""
+    """(launch(i), algorithmic bytes per call, description) for one task on seeded device
+    inputs, with enough rotating buffer sets to exceed L2 (at most 8)."""
     import torch
     from . import binding as B
     from . import inputs as gi
 
     st = torch.cuda.current_stream()
+    if task == "attention":
+        # Task 6: the paper's (N, d_model, h) with this N, else d_model = N and 32 columns per head
+        paper = {64: (32, 4), 128: (64, 8), 256: (128, 8), 384: (256, 16), 512: (512, 16)}
+        dm, h = paper.get(size, (size, max(1, size // 32)))
+        bytes_ = 3 * 2 * size * dm + 4 * size * dm
+        n = nsets or 8
+        rng = [torch.Generator(device="cuda").manual_seed(600 + i) for i in range(n)]
+        Q, K, V = ([torch.randn(size, dm, device="cuda", generator=rng[i]).bfloat16() for i in range(n)]
+                   for _ in range(3))
+        O = [torch.empty(size, dm, device="cuda") for _ in range(n)]
+        return (lambda i: B.mhsa_bf16(Q[i % n], K[i % n], V[i % n], O[i % n], size, dm, h, dm, dm, dm, dm, st)), \
+            bytes_, f"N = {size}, d_model = {dm}, h = {h}"
     if task == "transpose":
         bytes_ = 8 * size * size
         n = nsets or max(1, min(8, (600 << 20) // bytes_))
@@ -524,7 +537,7 @@ def _task_main(args):
     import torch
     from . import binding as B
 
-    default = {"transpose": 8192, "sum": 1 << 28, "dot": 1 << 27, "layernorm": 512}
+    default = {"transpose": 8192, "sum": 1 << 28, "dot": 1 << 27, "layernorm": 512, "attention": 512}
     size = args.size or default[args.task]
     launch, bytes_, what = task_problem(args.task, size, args.sets)
     t = performance_profiler(launch, iters=args.iters, warmup=args.warmup)
