@@ -496,9 +496,10 @@ def task_problem(task: str, size: int, nsets: int | None = None):
 
     st = torch.cuda.current_stream()
     if task == "attention":
-        # Task 6: the paper's (N, d_model, h) with this N, else d_model = N and 32 columns per head
+        # Task 6: the paper's (N, d_model, h) with this N, else about N columns, 32 per head
         paper = {64: (32, 4), 128: (64, 8), 256: (128, 8), 384: (256, 16), 512: (512, 16)}
-        dm, h = paper.get(size, (size, max(1, size // 32)))
+        heads = max(1, size // 32)
+        dm, h = paper.get(size, (32 * heads, heads))
         bytes_ = 3 * 2 * size * dm + 4 * size * dm
         n = nsets or 8
         rng = [torch.Generator(device="cuda").manual_seed(600 + i) for i in range(n)]

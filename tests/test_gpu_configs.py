@@ -124,3 +124,15 @@ def test_search_finds_a_valid_fastest_variant_and_rejects_a_broken_one():
     broken = got.copy(); broken[-1, -1] += 1.0                       # last row / column of an edge tile
     rep = H.function_validator(0, [case], lambda v, c: (0, (broken, exact, pad_ok)), H.compare_closed_form)
     assert rep.status == H.MISMATCH
+
+
+@pytest.mark.parametrize("task,size", [("transpose", 256), ("sum", 1 << 12), ("dot", 1 << 12), ("layernorm", 64),
+                                       ("attention", 64), ("attention", 200)])
+def test_harness_task_commands_run(task, size, capsys):
+    """The command line that the task profiles cite (`--task ... --size ...`) runs, reports a
+    clean device status and a positive time."""
+    import json
+    from paper_2506_09092_b200 import harness as H
+    H._main(["--task", task, "--size", str(size), "--iters", "2", "--warmup", "1"])
+    line = json.loads(capsys.readouterr().out.strip().splitlines()[-1])
+    assert line["task"] == task and line["status"] == 0 and line["us_median"] > 0
