@@ -9,12 +9,15 @@ on seeded synthetic operands that are already resident in HBM.  The line
 printed by rank 0 carries the device-timed TFLOP/s (``value``), the same
 metric through the host-buffer entry point with the copies inside the timed
 region (``e2e``), the roofline fraction of the GEMM kernel against the measured
-cuBLAS bf16 peak of this pool (``roofline``), the skinny HBM-bound workload C5a
-in GB/s against the measured copy bandwidth (``skinny``), and the CPU oracle
-timed on the host cores on a bounded sample (``cpu_baseline``).
+cuBLAS bf16 burst peak of this pool (``roofline``), the same kernel run back to
+back for two seconds against the measured sustained peak (``sustained``, with
+the SM clocks seen), the skinny HBM-bound workload C5a in GB/s against the
+measured copy bandwidth (``roofline_hbm``), and the CPU oracle timed on the
+host cores on a bounded sample (``cpu_baseline``).
 
-With N > 1 (launched by torchrun, one rank per GPU) every rank multiplies its
-own row shard of the same size: weak scaling, no data-path collective.
+With N > 1 every rank multiplies its own row shard of the same size: weak
+scaling, no data-path collective.  Under torchrun the ranks are taken from the
+environment; a plain ``python bench.py --gpus N`` starts the N ranks itself.
 
 ``--impl reference`` times the CPU oracle as it stands (no GPU work).
 """
@@ -34,9 +37,28 @@ sys.path.insert(0, ROOT)
 METRIC = "GEMM TFLOP/s & % of dense-bf16 peak at 4096^3; HBM GB/s & % on skinny M=16"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 L2_BYTES = 126e6
-# DRAM traffic of one launch of the dominant kernel, from the ncu capture
-# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).
-NCU_TRAFFIC_BYTES = {"C2": 119.4e6, "C5a": 273.1e6}
+# Where the DRAM traffic of one launch of the dominant kernel is recorded: the committed
+# summaries of the ncu captures (dram__bytes_read.sum and dram__bytes_write.sum rows).
+NCU_SUMMARY = {"C2": "profiles/umma_gemm_2cta_C2_4096cubed.md", "C5a": "profiles/umma_gemm_n128_C5a_skinny.md"}
+
+
+def ncu_traffic_bytes(name):
+    """dram read + write bytes per launch from the committed ncu summary, or None."""
+    import re
+    try:
+        text = open(os.path.join(ROOT, NCU_SUMMARY[name])).read()
+    except (OSError, KeyError):
+        return None
+    total = 0.0
+    for key in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+        m = re.search(re.escape(key) + r"[^|\n]*\|\s*([0-9.]+)\s*MB", text)
+        if not m:
+            m2 = re.search(r"dram__bytes_read\.sum / write\s*\|\s*([0-9.]+)\s*MB\s*/\s*([0-9.]+)\s*MB", text)
+            if not m2:
+                return None
+            return (float(m2.group(1)) + float(m2.group(2))) * 1e6
+        total += float(m.group(1)) * 1e6
+    return total
 
 
 def load_peaks():
@@ -89,9 +111,8 @@ class ClockSampler:
             pass
 
     def _run(self):
-        while not self._stop.is_set():
+        while not self._stop.is_set():       # an NVML query takes a fraction of a millisecond: no pause
             self._poll_once()
-            time.sleep(0.001)
 
     def start(self):
         if self.nv is None:
@@ -107,7 +128,7 @@ class ClockSampler:
     def summary(self):
         s = sorted(self.samples)
         return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(s)}
+                "sm_mhz_min": s[0] if s else None, "reasons": sorted(self.reasons), "samples": len(s)}
 
 
 # ------------------------------------------------------------------ helpers --
@@ -147,15 +168,46 @@ def time_steps(launch, steps, warmup, barrier, sampler=None):
     return total, total / steps
 
 
-def launches_per_call(B, cfg, variant_name):
-    n = 1
-    if "_sk" in variant_name:
-        n += 1                                   # split-K reduction kernel
-    if cfg.lda_ % 8 or (cfg.batch > 1 and cfg.strideA % 8):
-        n += 1                                   # repack A
-    if cfg.ldb_ % 8 or (cfg.batch > 1 and cfg.strideB % 8):
-        n += 1                                   # repack B
-    return n
+def launches_per_call(cfg):
+    """Kernels of the library per call: the GEMM kernel (split tiles are summed inside it), plus
+    one repacking launch if an operand cannot be addressed by TMA."""
+    unaligned = (cfg.lda_ % 8 or cfg.ldb_ % 8
+                 or (cfg.batch > 1 and (cfg.strideA % 8 or cfg.strideB % 8)))
+    return 2 if unaligned else 1
+
+
+def kernel_name(variant_name):
+    """The __global__ function a variant runs."""
+    if variant_name == "simt":
+        return "simt_gemm_kernel"
+    return "umma_gemm_2cta_kernel" if variant_name.startswith("umma2_") else "umma_gemm_kernel"
+
+
+def sustained_run(launch, flops_per_call, est_s_per_call, seconds, peak_sustained, local, barrier):
+    """Back-to-back calls for about `seconds` between two CUDA events, NVML clocks sampled
+    throughout (sampling only).  Returns the record for the JSON line."""
+    import torch
+    n = max(10, int(seconds / max(est_s_per_call, 1e-7)) + 1)
+    sampler = ClockSampler(local)
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record()
+    for i in range(n):
+        launch(i)
+    e1.record()
+    torch.cuda.synchronize()
+    sampler.stop()
+    barrier()
+    t = e0.elapsed_time(e1) * 1e-3
+    clocks = sampler.summary()
+    tfl = flops_per_call * n / t / 1e12
+    us = t / n * 1e6
+    return {"value": tfl, "unit": "TFLOP/s", "seconds": t, "calls": n, "us_per_call": us,
+            "peak": peak_sustained, "frac": tfl / peak_sustained, "frac_of_nominal_2250": tfl / 2250.0,
+            "clocks": clocks,
+            "us_x_mhz": us * clocks["sm_mhz"] if clocks["sm_mhz"] else None}
 
 
 def cpu_baseline_sample(cfg, A, Bm, target_s=12.0):
@@ -181,31 +233,37 @@ def cpu_baseline_sample(cfg, A, Bm, target_s=12.0):
                       f"C_ref and S in fp64, {dt:.2f} s"}
 
 
-def task_cpu_baselines():
-    """The task oracles as they stand (single-threaded C), timed on bounded samples of the
-    same seeded inputs; algorithmic GB/s like the GPU figures beside them."""
+def task_cpu_baselines(workloads):
+    """The task oracles as they stand (single-threaded C), timed on the same seeded inputs and
+    sizes as the GPU figures beside them (`workloads`: (task, size) pairs); algorithmic GB/s."""
     import numpy as np
     import oracle
     from paper_2506_09092_b200 import inputs as gi
     out = {}
-    n = 4096
-    A = gi.task_array(8, 0, n * n)
-    t0 = time.perf_counter(); oracle.transpose_f32(A, n, n); dt = time.perf_counter() - t0
-    out["transpose"] = {"value": 8.0 * n * n / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
-                        "sample": f"{n} x {n} fp32, {dt:.2f} s"}
-    x = gi.task_array(14, 0, 1 << 26)
-    t0 = time.perf_counter(); oracle.sum_f32(x); dt = time.perf_counter() - t0
-    out["sum"] = {"value": 4.0 * x.size / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
-                  "sample": f"n = 2^26, {dt:.2f} s"}
-    y = gi.task_array(15, 1, 1 << 26, "uniform")
-    t0 = time.perf_counter(); oracle.dot_f32(x, y); dt = time.perf_counter() - t0
-    out["dot"] = {"value": 8.0 * x.size / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
-                  "sample": f"n = 2^26, {dt:.2f} s"}
-    batch, m = 16, 4 * 256 * 256
-    xs, g, b = gi.layernorm_inputs(4, batch, m)
-    t0 = time.perf_counter(); oracle.layernorm_f32(xs, g, b, batch, m); dt = time.perf_counter() - t0
-    out["layernorm"] = {"value": (8.0 * batch * m + 8.0 * m) / dt / 1e9, "unit": "GB/s", "cores": 1,
-                        "kind": "oracle", "sample": f"(16, 4, 256, 256) fp32, y in fp64, {dt:.2f} s"}
+    for task, size in workloads:
+        if task == "transpose":
+            A = gi.task_array(8, 0, size * size)
+            t0 = time.perf_counter(); oracle.transpose_f32(A, size, size); dt = time.perf_counter() - t0
+            rec = {"value": 8.0 * size * size / dt / 1e9, "sample": f"{size} x {size} fp32, {dt:.2f} s"}
+            del A
+        elif task == "sum":
+            x = gi.task_array(14, 0, size)
+            t0 = time.perf_counter(); oracle.sum_f32(x); dt = time.perf_counter() - t0
+            rec = {"value": 4.0 * size / dt / 1e9, "sample": f"n = {size}, {dt:.3f} s"}
+        elif task == "dot":
+            x = gi.task_array(14, 0, size)
+            y = gi.task_array(15, 0, size, "uniform")
+            t0 = time.perf_counter(); oracle.dot_f32(x, y); dt = time.perf_counter() - t0
+            rec = {"value": 8.0 * size / dt / 1e9, "sample": f"n = {size}, {dt:.3f} s"}
+        else:
+            batch, m = 16, 4 * size * size
+            xs, g, b = gi.layernorm_inputs(4, batch, m)
+            t0 = time.perf_counter(); oracle.layernorm_f32(xs, g, b, batch, m); dt = time.perf_counter() - t0
+            rec = {"value": (8.0 * batch * m + 8.0 * m) / dt / 1e9,
+                   "sample": f"(16, 4, {size}, {size}) fp32, y in fp64, {dt:.2f} s"}
+            del xs
+        rec.update({"unit": "GB/s", "cores": 1, "kind": "oracle"})
+        out[(task, size)] = rec
     return out
 
 
@@ -298,7 +356,28 @@ def run_ours(args):
     total_max = sharding.max_over_ranks(total, device="cuda")
     value = sharding.aggregate_throughput(cfg.flops * args.steps, world, total_max) / 1e12
     achieved = cfg.flops / kern_avg / 1e12             # one kernel per step: step time = launch duration
-    n_launch = launches_per_call(B, cfg, vname)
+    n_launch = launches_per_call(cfg)
+
+    # ---------------- the same kernel back to back for seconds (clock sag), C2 and C3 --
+    sustained = {}
+    if not args.no_sustained:
+        sustained["C2"] = sustained_run(lambda i: prob.launch(i, stream=stream), cfg.flops, kern_avg,
+                                        args.sustained_seconds, peaks["bf16_tflops_sustained"], local, barrier)
+        c3 = gi.CONFIGS["C3"]
+        c3p = H.DeviceProblem(c3, nsets=1)             # one set is 338 MB > L2
+        c3_name = B.variant_name(B.select_variant(c3.M, c3.N, c3.K, c3.lda_, c3.ldb_, c3.ldc_, c3.batch, c3.out_dtype))
+        _, c3_avg = time_steps(lambda i: c3p.launch(i, stream=stream), 20, 3, barrier)
+        sustained["C3"] = sustained_run(lambda i: c3p.launch(i, stream=stream), c3.flops, c3_avg,
+                                        args.sustained_seconds, peaks["bf16_tflops_sustained"], local, barrier)
+        sustained["C3"].update({"workload": workload_name(c3), "variant": c3_name,
+                                "burst": {"us_per_call": c3_avg * 1e6, "value": c3.flops / c3_avg / 1e12,
+                                          "frac_of_burst_peak": c3.flops / c3_avg / 1e12 / peaks["bf16_tflops"]}})
+        sustained["C2"].update({"workload": workload_name(cfg), "variant": vname})
+        del c3p
+        torch.cuda.empty_cache()
+        code, detail = B.device_status(stream)
+        if code != 0:
+            raise RuntimeError(f"device status {code} detail {detail:#x}")
 
     # -------------------------------------------- e2e: host buffers, copies --
     hA = torch.from_numpy(A.view(np.int16)).pin_memory()
@@ -348,11 +427,13 @@ def run_ours(args):
     # ---------- the bandwidth-bound float32 tasks (8, 14, 15, 4) at their largest paper size,
     #            plus a 1 GiB stream for the two reductions (the paper's largest is 4 MB) ----------
     hbm_tasks = []
+    task_workloads = []
     for task, size, label in (("transpose", gi.TRANSPOSE_SIZES[-1], "Task 8"), ("layernorm", 1024, "Task 4"),
                               ("sum", gi.REDUCTION_SIZES[-1], "Task 14"), ("dot", gi.DOT_SIZES[-1], "Task 15"),
                               ("sum", 1 << 28, "Task 14 beyond the paper's sizes"),
                               ("dot", 1 << 27, "Task 15 beyond the paper's sizes")):
         launch_t, bytes_t, what = H.task_problem(task, size)
+        task_workloads.append((task, size))
         t_steps = max(args.steps, 20)
         _, t_avg = time_steps(launch_t, t_steps, 3, barrier)
         hbm_tasks.append({"task": label, "call": f"cudallm_{task}_f32", "input": what, "us_per_call": t_avg * 1e6,
@@ -385,16 +466,18 @@ def run_ours(args):
             "gpu_launches": n_launch * args.steps,
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
                          "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                         "traffic": NCU_TRAFFIC_BYTES["C2"], "peak_source": f"of {peak_src} (burst)",
-                         "kernel": f"umma_gemm_kernel ({vname})",
+                         "traffic": ncu_traffic_bytes("C2"), "traffic_source": NCU_SUMMARY["C2"],
+                         "peak_source": f"of {peak_src} (burst: the timed region is milliseconds long)",
+                         "kernel": f"{kernel_name(vname)} ({vname})",
                          "frac_of_nominal_2250": achieved / 2250.0},
-            "skinny": {"workload": workload_name(sk), "variant": sk_name, "value": sk_gbs, "unit": "GB/s",
-                       "us_per_call": sk_avg * 1e6, "steps": sk_steps,
-                       "roofline": {"bound": "hbm", "achieved": sk_gbs, "peak": peaks["hbm_gbs"],
-                                    "unit": "GB/s", "frac": sk_gbs / peaks["hbm_gbs"],
-                                    "traffic": NCU_TRAFFIC_BYTES["C5a"],
-                                    "peak_source": f"of {peak_src}",
-                                    "frac_of_nominal_8000": sk_gbs / 8000.0}},
+            # the second half of the metric: the skinny M = 16 product against the copy bandwidth
+            "roofline_hbm": {"workload": workload_name(sk), "variant": sk_name, "kernel": f"{kernel_name(sk_name)} ({sk_name})",
+                             "bound": "hbm", "achieved": sk_gbs, "value": sk_gbs, "peak": peaks["hbm_gbs"],
+                             "unit": "GB/s", "frac": sk_gbs / peaks["hbm_gbs"],
+                             "traffic": ncu_traffic_bytes("C5a"), "traffic_source": NCU_SUMMARY["C5a"],
+                             "peak_source": f"of {peak_src}", "us_per_call": sk_avg * 1e6, "steps": sk_steps,
+                             "frac_of_nominal_8000": sk_gbs / 8000.0},
+            "sustained": sustained,
         }
         line["task2_fp32"] = {
             "workload": f"paper Task 2, size 2^14: A ({t2.M} x {t2.K}) x B ({t2.K} x {t2.N}), fp32 in and out, N(0,1)",
@@ -411,9 +494,10 @@ def run_ours(args):
         line["hbm_tasks_f32"] = hbm_tasks
         if world == 1:
             line["cpu_baseline"] = cpu_baseline_sample(cfg, A, Bm)
-            cpu_tasks = task_cpu_baselines()
-            for entry in hbm_tasks:
-                entry["cpu_baseline"] = cpu_tasks[entry["call"].split("_")[1]]
+            if not args.no_task_baselines:
+                cpu_tasks = task_cpu_baselines(task_workloads)
+                for entry, key in zip(hbm_tasks, task_workloads):
+                    entry["cpu_baseline"] = cpu_tasks[key]
     if use_dist:
         dist.barrier()
         dist.destroy_process_group()
@@ -422,16 +506,38 @@ def run_ours(args):
     return 0
 
 
+def self_launch(args):
+    """`python bench.py --gpus N` outside torchrun: start the N ranks here, one per GPU."""
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--sustained-seconds", type=float, default=2.2,
+                    help="length of the back-to-back runs of C2 and C3 behind the `sustained` record")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the seconds-long runs")
+    ap.add_argument("--no-task-baselines", action="store_true",
+                    help="skip timing the CPU oracles of the float32 tasks")
     args = ap.parse_args()
     if args.steps < 1:
         ap.error("--steps must be >= 1")
+    if args.gpus < 1:
+        ap.error("--gpus must be >= 1")
     args.warmup = max(args.warmup, 3)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return self_launch(args)
+    if "WORLD_SIZE" in os.environ and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        ap.error(f"--gpus {args.gpus} but WORLD_SIZE={os.environ['WORLD_SIZE']}")
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

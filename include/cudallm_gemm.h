@@ -37,11 +37,15 @@
  *  - The library is for compute capability 10.0 devices only and has no CPU
  *    fallback.
  *  - Calls that need the workspace (repacking, split-K) share one workspace
- *    per device; such calls must not run concurrently on different streams.
+ *    per device; such calls must not run concurrently on different streams,
+ *    unless each of those streams has a workspace of its own
+ *    (cudallm_set_workspace_for_stream).
  *  - Split-K variants make some CTAs wait (with a time limit) for partial
  *    results of other CTAs of the same launch; they assume that the launch has
  *    the GPU to itself.  If another kernel holds SMs for seconds, such a wait
- *    can run out and is reported as CUDALLM_ERR_DEVICE_TIMEOUT.
+ *    can run out and is reported as CUDALLM_ERR_DEVICE_TIMEOUT.  On a stream
+ *    with a workspace of its own the library's automatic choice therefore keeps
+ *    to variants without such waits.
  */
 #ifndef CUDALLM_GEMM_H
 #define CUDALLM_GEMM_H
@@ -87,9 +91,8 @@ int cudallm_gemm_bf16(const void *A, const void *B, void *C,
                       int out_dtype, void *stream);
 
 /*
- * C = A x B with 32-bit floating point operands and result: Task 2 exactly as
- * the paper states it ("multiplies two matrices of 32-bit floating point
- * numbers").
+ * C = A x B with 32-bit floating point operands and result: the element type
+ * the paper's Task 2 description gives for both factors and the product.
  *   A : fp32, M x K, row stride lda >= K      (read only)
  *   B : fp32, K x N, row stride ldb >= N      (read only)
  *   C : fp32, M x N, row stride ldc >= N
@@ -187,11 +190,13 @@ size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K,
  *    behind the header: CUDALLM_NOALLOC_HEADER_BYTES + P * 32 KiB <=
  *    CUDALLM_NOALLOC_SCRATCH_BYTES, i.e. P <= 254; else the call returns
  *    CUDALLM_ERR_TOO_LARGE and nothing runs.
- *  - The call SYNCHRONISES `stream` before it returns and reports a kernel
- *    whose bounded wait ran out as CUDALLM_ERR_DEVICE_TIMEOUT.
- *  - The first call on each device looks up the array's device address (and,
- *    like any first launch, lets the driver load the kernels).  Make that
- *    first call outside any stream capture.
+ *  - The call SYNCHRONISES `stream` before it returns (it reads the kernel's
+ *    status word back) and reports a kernel whose bounded wait ran out as
+ *    CUDALLM_ERR_DEVICE_TIMEOUT.  A synchronisation is not allowed on a stream
+ *    that is being captured: never make this call, first or later, inside a
+ *    stream capture.
+ *  - The first call on each device also looks up the array's device address
+ *    (and, like any first launch, lets the driver load the kernels).
  *  - All calls on a device share the one array, which keeps whatever the last
  *    call left in it; each call clears the words that must start at zero (the
  *    status word and the helper flags).  Two calls that overlap on the GPU
@@ -275,6 +280,56 @@ size_t cudallm_workspace_bytes(int64_t M, int64_t N, int64_t K,
                                int64_t lda, int64_t ldb, int64_t ldc,
                                int64_t batch, int out_dtype);
 int cudallm_set_workspace(void *dev_ptr, size_t bytes);
+
+/*
+ * A workspace of its own for the calls made on `stream` (current device), so
+ * that calls which need scratch (repacking, split-K, LayerNorm, the fp32
+ * product) can run on several streams at once: flags, partial sums, repacked
+ * operands and the status word of that stream's calls then live in `dev_ptr`.
+ * Same requirements as cudallm_set_workspace: 256-byte aligned, at least
+ * cudallm_workspace_bytes(...) for the products to come, zero-filled once,
+ * valid until replaced or removed with (stream, NULL, 0); it may not overlap
+ * another stream's workspace (CUDALLM_ERR_WORKSPACE).  A call whose needs
+ * exceed it returns CUDALLM_ERR_WORKSPACE; it is never grown.
+ * cudallm_device_status(stream, ...) reads this workspace's status word.
+ * Attaching a workspace to a stream also tells the library that launches may
+ * share the GPU: cudallm_gemm_bf16 / _batched on that stream choose only among
+ * variants whose CTAs do not wait for one another (a forced split variant still
+ * runs, with the caveat stated at the top of this file).
+ */
+int cudallm_set_workspace_for_stream(void *stream, void *dev_ptr, size_t bytes);
+
+/*
+ * Sizes the library's own workspace of the current device to at least `bytes`
+ * now (cudaMalloc; synchronises the device if an older, smaller one has to be
+ * replaced), so that later calls up to that need allocate nothing.  Returns
+ * CUDALLM_ERR_WORKSPACE while a caller-provided workspace is set.
+ */
+int cudallm_reserve_workspace(size_t bytes);
+
+/*
+ * Releases what the library holds on every device: its own workspaces, the
+ * streams and events of cudallm_gemm_bf16_host, and the stream-workspace table
+ * (caller-provided buffers are only forgotten).  Synchronises those devices.
+ * The library can be used again afterwards.
+ */
+int cudallm_shutdown(void);
+
+/*
+ * Test hooks for the bounded waits inside the kernels (host side; they change
+ * how later launches are parameterised, nothing that has been enqueued).
+ *   CUDALLM_DEBUG_WAIT_LIMIT_NS          value = the wall-clock limit of every
+ *       in-kernel wait in nanoseconds (0 restores the default of 2 s).
+ *   CUDALLM_DEBUG_MISS_NEXT_SPLIT_FLAGS  value != 0: the next launch that splits
+ *       tiles along K raises its hand-over flags to a value that no unit waits
+ *       for, so every such wait runs out after the limit; the kernel then
+ *       returns normally, C is unspecified, and cudallm_device_status reports
+ *       CUDALLM_ERR_DEVICE_TIMEOUT.  One launch only.
+ * Returns CUDALLM_ERR_INVALID_VARIANT for an unknown `what`.
+ */
+#define CUDALLM_DEBUG_WAIT_LIMIT_NS          1
+#define CUDALLM_DEBUG_MISS_NEXT_SPLIT_FLAGS  2
+int cudallm_debug_set(int what, unsigned long long value);
 
 /*
  * Synchronises `stream`, then reads and clears the device status word that

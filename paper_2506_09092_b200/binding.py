@@ -57,6 +57,10 @@ SIGNATURES = {
     "cudallm_select_variant": (_int, [_i64] * 7 + [_int]),
     "cudallm_workspace_bytes": (_sz, [_i64] * 7 + [_int]),
     "cudallm_set_workspace": (_int, [_vp, _sz]),
+    "cudallm_set_workspace_for_stream": (_int, [_vp, _vp, _sz]),
+    "cudallm_reserve_workspace": (_int, [_sz]),
+    "cudallm_shutdown": (_int, []),
+    "cudallm_debug_set": (_int, [_int, ctypes.c_ulonglong]),
     "cudallm_device_status": (_int, [_vp, ctypes.POINTER(_int), ctypes.POINTER(_int)]),
     "cudallm_strerror": (ctypes.c_char_p, [_int]),
     "cudallm_version": (_int, []),
@@ -236,6 +240,30 @@ def workspace_bytes(M, N, K, lda, ldb, ldc, batch, out_dtype) -> int:
 
 def set_workspace(dev_ptr, nbytes: int, check=True):
     return _check(lib().cudallm_set_workspace(_p(dev_ptr), nbytes), "cudallm_set_workspace", check)
+
+
+def set_workspace_for_stream(stream, dev_ptr, nbytes: int, check=True):
+    """Attach a caller-owned workspace to ``stream`` (``dev_ptr=None`` removes it)."""
+    return _check(lib().cudallm_set_workspace_for_stream(_s(stream), _p(dev_ptr), nbytes),
+                  "cudallm_set_workspace_for_stream", check)
+
+
+def reserve_workspace(nbytes: int, check=True):
+    """Size the library's own workspace of the current device now."""
+    return _check(lib().cudallm_reserve_workspace(nbytes), "cudallm_reserve_workspace", check)
+
+
+def shutdown(check=True):
+    """Release the library's workspaces, streams and events on every device."""
+    return _check(lib().cudallm_shutdown(), "cudallm_shutdown", check)
+
+
+DEBUG_WAIT_LIMIT_NS, DEBUG_MISS_NEXT_SPLIT_FLAGS = 1, 2
+
+
+def debug_set(what: int, value: int, check=True):
+    """Test hooks of the kernels' bounded waits (see the header)."""
+    return _check(lib().cudallm_debug_set(what, value), "cudallm_debug_set", check)
 
 
 def device_status(stream=None):

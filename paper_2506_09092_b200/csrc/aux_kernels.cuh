@@ -2,13 +2,16 @@
 //  * simt_gemm_kernel  -- fully predicated CUDA-core GEMM for any shape and
 //    alignment (bring-up cross-check on the device; also serves K == 0).
 //  * pack_rows_kernel  -- copies operands whose leading dimension or base
-//    is not 16-byte aligned into an aligned workspace so that TMA can read them.
+//    is not 16-byte aligned into an aligned workspace so that TMA can read them
+//    (small or batched products; large single products repack inside the GEMM
+//    kernel, see row_copy.cuh).
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 #include "ptx.cuh"
+#include "row_copy.cuh"
 
 namespace cudallm {
 
@@ -37,66 +40,69 @@ simt_gemm_kernel(const __nv_bfloat16 *__restrict__ A, const __nv_bfloat16 *__res
     }
 }
 
-// One operand to repack: dst[b][r][0..cols) = src[b][r][0..cols), columns up to the next
-// multiple of 8 zero; dst is 16-byte aligned and its row pitch ld_dst and batch stride are
-// multiples of 8 elements; src needs 2-byte alignment only.
-struct PackJob {
-    const uint16_t *src;
-    uint16_t *dst;
-    int rows, cols, batch;
-    long long ld_src, ld_dst, stride_src, stride_dst;
-    long long total_rows;                                // rows * batch (0 = nothing to do)
-};
-
-// Repacks up to two operands in one launch: one thread per 16-byte piece of the
-// destination, the pieces of job a first, then those of job b.  A piece whose source lies
-// strictly inside its row is read as five 4-byte words from the 4-byte boundary at or
-// below it and shifted into place (the source of a row with an odd pitch is 2 bytes past
-// such a boundary every other row); the first and the last piece of a row are read element
-// by element, so that nothing outside [src, src + cols) of the row is touched.
-__global__ void __launch_bounds__(256)
+// Repacks up to two operands in one launch.  The unit of work is up to 512 consecutive
+// elements of one row, copied by one warp with 16-byte loads and stores (row_copy.cuh); the
+// units of job a come first, then those of job b, and the warps of the grid take them in
+// turn.  Eight warps per CTA and as many CTAs as fit: the copy then runs at about 80 % of
+// what a plain device-to-device copy of the same bytes reaches.
+constexpr int kPackThreads = 256;
+// The units of one job, taken in turn by the warps of the grid starting with warp `first_warp`
+// (so that job b's units continue where job a's ended).  Index = uint32_t where the unit
+// count allows it: its divisions are several times cheaper.
+template <typename Index>
+__device__ __forceinline__ void pack_job_units(const PackJob &j, Index first_warp, Index nwarps, int lane)
+{
+    const Index groups = static_cast<Index>((j.cols + 511) >> 9);
+    const Index total = static_cast<Index>(j.total_rows) * groups;
+    const Index rows = static_cast<Index>(j.rows);
+    const int cols = j.cols;
+    const long long ld_src = j.ld_src, ld_dst = j.ld_dst, s_src = j.stride_src, s_dst = j.stride_dst;
+    const bool batched = j.batch > 1;
+    for (Index u = first_warp; u < total; u += nwarps) {
+        const Index row = groups == 1 ? u : u / groups;
+        const int c0 = static_cast<int>(u - row * groups) * 512;
+        long long off_src, off_dst;
+        if (batched) {
+            const Index item = row / rows, r = row - item * rows;
+            off_src = item * s_src + r * ld_src + c0;
+            off_dst = item * s_dst + r * ld_dst + c0;
+        } else {
+            off_src = row * ld_src + c0;
+            off_dst = row * ld_dst + c0;
+        }
+        const uint16_t *src = j.src + off_src;
+        uint16_t *dst = j.dst + off_dst;
+        if (cols - c0 >= 514) {                          // warp-uniform: not the last unit of its row
+            row_copy_interior(src, dst, lane);
+        } else {
+            RowCopy rc;
+            row_copy_load(rc, src, cols - c0, lane);
+            row_copy_store(rc, src, dst, cols - c0, lane);
+        }
+    }
+}
+template <typename Index>
+__device__ __forceinline__ void pack_rows_loop(const PackJob &a, const PackJob &b)
+{
+    const int lane = threadIdx.x & 31;
+    const Index nwarps = static_cast<Index>(gridDim.x) * (kPackThreads / 32);
+    const Index gwarp = static_cast<Index>(blockIdx.x) * (kPackThreads / 32) + (threadIdx.x >> 5);
+    pack_job_units<Index>(a, gwarp, nwarps, lane);
+    // job b starts with the warp after the one that took job a's last unit
+    const Index units_a = static_cast<Index>(a.total_rows) * static_cast<Index>((a.cols + 511) >> 9);
+    const Index shift = units_a % nwarps;
+    pack_job_units<Index>(b, gwarp >= shift ? gwarp - shift : gwarp + nwarps - shift, nwarps, lane);
+}
+__global__ void __launch_bounds__(kPackThreads)
 pack_rows_kernel(const PackJob a, const PackJob b)
 {
     grid_launch_dependents();
     grid_dependency_wait();                              // the workspace may still be read by the previous kernel
-    const long long pieces_a = a.total_rows * ((a.cols + 7) >> 3);
-    const long long total = pieces_a + b.total_rows * ((b.cols + 7) >> 3);
-    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
-         i += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const bool first = i < pieces_a;
-        const long long k = first ? i : i - pieces_a;
-        const int rows = first ? a.rows : b.rows;
-        const int cols = first ? a.cols : b.cols;
-        const int chunks = (cols + 7) >> 3;
-        const long long row = k / chunks;
-        const int c0 = static_cast<int>(k - row * chunks) * 8;
-        const long long item = row / rows;
-        const long long r = row - item * rows;
-        const uint16_t *s = (first ? a.src : b.src) + item * (first ? a.stride_src : b.stride_src)
-                          + r * (first ? a.ld_src : b.ld_src) + c0;
-        uint16_t *d = (first ? a.dst : b.dst) + item * (first ? a.stride_dst : b.stride_dst)
-                    + r * (first ? a.ld_dst : b.ld_dst) + c0;
-        uint4 w;
-        if (c0 > 0 && c0 + 10 <= cols) {
-            const uint32_t odd = (reinterpret_cast<uintptr_t>(s) >> 1) & 1;
-            const uint32_t *q = reinterpret_cast<const uint32_t *>(s - odd);
-            const uint32_t w0 = q[0], w1 = q[1], w2 = q[2], w3 = q[3], w4 = q[4];
-            const uint32_t sh = odd * 16;
-            w.x = __funnelshift_r(w0, w1, sh);
-            w.y = __funnelshift_r(w1, w2, sh);
-            w.z = __funnelshift_r(w2, w3, sh);
-            w.w = __funnelshift_r(w3, w4, sh);
-        } else {
-            uint16_t v[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = (c0 + j < cols) ? s[j] : static_cast<uint16_t>(0);
-            w.x = v[0] | (static_cast<uint32_t>(v[1]) << 16);
-            w.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
-            w.z = v[4] | (static_cast<uint32_t>(v[5]) << 16);
-            w.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
-        }
-        *reinterpret_cast<uint4 *>(d) = w;
-    }
+    const unsigned long long total = static_cast<unsigned long long>(a.total_rows) * ((a.cols + 511) >> 9)
+                                   + static_cast<unsigned long long>(b.total_rows) * ((b.cols + 511) >> 9);
+    const unsigned long long reach = total + static_cast<unsigned long long>(gridDim.x) * (kPackThreads / 32);
+    if (reach < (1ull << 32)) pack_rows_loop<uint32_t>(a, b);
+    else                      pack_rows_loop<unsigned long long>(a, b);
 }
 
 // Cuts fp32 values into three bf16 pieces: x = p0 + p1 + p2 exactly for normal

@@ -278,18 +278,23 @@ std::unordered_map<DispatchKey, int, DispatchHash> g_dispatch;
 std::mutex g_dispatch_mutex;
 std::atomic<uint64_t> g_dispatch_generation{0};      // bumped by every change of the table
 
-int select_variant_uncached(const Problem &p)
+// `no_waits`: only variants whose CTAs never wait for one another (no split tiles), for
+// calls that may share the GPU with other launches of this library.
+int select_variant_uncached(const Problem &p, bool no_waits)
 {
     build_variants();
     if (is_empty(p) || p.K == 0) return 0;
     {
         std::lock_guard<std::mutex> lock(g_dispatch_mutex);
         const auto it = g_dispatch.find(DispatchKey{p.M, p.N, p.K, p.batch, p.out_dtype});
-        if (it != g_dispatch.end() && variant_supports(g_variants[it->second], p)) return it->second;
+        if (it != g_dispatch.end() && variant_supports(g_variants[it->second], p)
+            && !(no_waits && g_variants[it->second].split_k != 1))
+            return it->second;
     }
     int best = -1;
     double best_cost = 0;
     for (int v = 1; v < kNumVariants; ++v) {
+        if (no_waits && g_variants[v].split_k != 1) continue;
         if (!variant_supports(g_variants[v], p)) continue;
         const double c = variant_cost(g_variants[v], p);
         if (best < 0 || c < best_cost) { best = v; best_cost = c; }
@@ -299,16 +304,16 @@ int select_variant_uncached(const Problem &p)
 
 // The choice depends only on the shape (and the dispatch table); repeated calls with
 // the same shape (the common case) reuse the previous answer.
-int select_variant(const Problem &p)
+int select_variant(const Problem &p, bool no_waits = false)
 {
-    struct Last { int64_t M, N, K, batch; int out_dtype, variant; uint64_t generation; };
-    static thread_local Last last = {-1, -1, -1, -1, -1, 0, 0};
+    struct Last { int64_t M, N, K, batch; int out_dtype, variant; uint64_t generation; bool no_waits; };
+    static thread_local Last last = {-1, -1, -1, -1, -1, 0, 0, false};
     const uint64_t gen = g_dispatch_generation.load(std::memory_order_acquire);
     if (last.M == p.M && last.N == p.N && last.K == p.K && last.batch == p.batch
-        && last.out_dtype == p.out_dtype && last.generation == gen)
+        && last.out_dtype == p.out_dtype && last.generation == gen && last.no_waits == no_waits)
         return last.variant;
-    const int v = select_variant_uncached(p);
-    last = Last{p.M, p.N, p.K, p.batch, p.out_dtype, v, gen};
+    const int v = select_variant_uncached(p, no_waits);
+    last = Last{p.M, p.N, p.K, p.batch, p.out_dtype, v, gen, no_waits};
     return v;
 }
 
@@ -318,21 +323,48 @@ constexpr size_t kFlagBytes = kMaxHelperTiles * 4 * sizeof(int);
 constexpr size_t kHeaderBytes = 256 + kFlagBytes;    // zeroed when a workspace is created
 constexpr int kMaxDevices = 64;
 
+// A workspace: the device's default one (allocated and grown by the library unless the
+// caller set one) or one that the caller attached to a stream.
+struct Workspace {
+    void *ptr = nullptr;         // active buffer
+    size_t bytes = 0;
+    bool external = false;       // the caller's: never grown or freed here
+    void *internal = nullptr;    // owned allocation (kept while an external one is set)
+    size_t internal_bytes = 0;
+};
+
 struct DeviceState {
     bool probed = false;
     bool supported = false;
     int sm_count = 0;
-    void *ws = nullptr;          // active workspace
-    size_t ws_bytes = 0;
-    bool ws_external = false;
-    void *ws_internal = nullptr; // owned allocation (kept when an external one is set)
-    size_t ws_internal_bytes = 0;
+    Workspace ws;                // the device's default workspace
+    std::unordered_map<cudaStream_t, Workspace> stream_ws;   // cudallm_set_workspace_for_stream
     bool smem_attr_set[24] = {};
     int max_pairs = 0;           // co-resident 2-CTA clusters of the pair kernel (0 = not asked yet)
     int epoch = 0;               // last split-K flag value used on this device
 };
 DeviceState g_dev[kMaxDevices];
 std::mutex g_mutex;
+
+// Host-side knobs of the kernels' bounded waits (cudallm_debug_set): the limit itself, and a
+// one-shot request to raise the split-K flags of the next split launch to a value nobody
+// waits for, so that every such wait runs out (the self-test of the timeout path).
+std::atomic<unsigned long long> g_wait_limit_ns{kWaitLimitNs};
+std::atomic<int> g_skew_next_flags{0};
+
+// The workspace calls on `stream` use: the one attached to the stream, else the device's.
+Workspace &workspace_for(DeviceState &d, cudaStream_t stream)
+{
+    if (!d.stream_ws.empty()) {
+        const auto it = d.stream_ws.find(stream);
+        if (it != d.stream_ws.end()) return it->second;
+    }
+    return d.ws;
+}
+bool stream_has_workspace(DeviceState &d, cudaStream_t stream)
+{
+    return !d.stream_ws.empty() && d.stream_ws.find(stream) != d.stream_ws.end();
+}
 
 // Streams and events of the host-buffer entry point (created on first use).
 constexpr int kHostPipeChunks = 4;
@@ -358,10 +390,12 @@ int probe_device(int dev)
     CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
     CUDA_TRY(cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev));
     CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    d.probed = true;
     d.supported = (major == 10 && minor == 0);
     d.sm_count = sms;
-    if (!d.supported) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    if (!d.supported) {
+        d.probed = true;
+        return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    }
     if (!g_encode) {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -372,34 +406,35 @@ int probe_device(int dev)
         }
         g_encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
+    d.probed = true;                 // only now: a failed look-up above is retried by the next call
     return CUDALLM_OK;
 }
 
-// Make sure the active workspace of `dev` holds `bytes`; allocates or grows the
-// internal one (never an external one).
-int ensure_workspace(int dev, size_t bytes, cudaStream_t stream)
+// Make sure workspace `w` holds `bytes`; allocates or grows an internal one (never a
+// caller-provided one).  `exact`: allocate just `bytes` (cudallm_reserve_workspace).
+int ensure_workspace(Workspace &w, size_t bytes, cudaStream_t stream, bool exact = false)
 {
-    DeviceState &d = g_dev[dev];
-    if (d.ws && d.ws_bytes >= bytes) return CUDALLM_OK;
-    if (d.ws_external) return CUDALLM_ERR_WORKSPACE;
-    size_t want = bytes < (size_t(8) << 20) ? (size_t(8) << 20) : bytes + bytes / 4;
-    if (d.ws_internal) {
+    if (w.ptr && w.bytes >= bytes) return CUDALLM_OK;
+    if (w.external) return CUDALLM_ERR_WORKSPACE;
+    size_t want = exact ? bytes : (bytes < (size_t(8) << 20) ? (size_t(8) << 20) : bytes + bytes / 4);
+    if (want < kHeaderBytes) want = kHeaderBytes;
+    if (w.internal) {
         CUDA_TRY(cudaDeviceSynchronize());            // earlier launches may still use it
-        CUDA_TRY(cudaFree(d.ws_internal));
-        d.ws_internal = nullptr;
-        d.ws_internal_bytes = 0;
-        d.ws = nullptr;
-        d.ws_bytes = 0;
+        CUDA_TRY(cudaFree(w.internal));
+        w.internal = nullptr;
+        w.internal_bytes = 0;
+        w.ptr = nullptr;
+        w.bytes = 0;
     }
     void *ptr = nullptr;
     CUDA_TRY(cudaMalloc(&ptr, want));
     CUDA_TRY(cudaMemsetAsync(ptr, 0, kHeaderBytes, stream));
     // later launches on other streams must see the cleared header
     CUDA_TRY(cudaStreamSynchronize(stream));
-    d.ws_internal = ptr;
-    d.ws_internal_bytes = want;
-    d.ws = ptr;
-    d.ws_bytes = want;
+    w.internal = ptr;
+    w.internal_bytes = want;
+    w.ptr = ptr;
+    w.bytes = want;
     return CUDALLM_OK;
 }
 
@@ -681,11 +716,11 @@ PackJob pack_job(const void *src, void *dst, int64_t rows, int64_t cols, int64_t
 // One launch repacks both jobs (either may be empty: total_rows == 0).
 int launch_pack(const PackJob &a, const PackJob &b, cudaStream_t stream)
 {
-    const int64_t total = a.total_rows * cdiv(a.cols, 8) + b.total_rows * cdiv(b.cols, 8);
-    if (total == 0) return CUDALLM_OK;
-    int64_t blocks = cdiv(total, 256);                   // one thread per 16-byte piece, grid-stride
-    if (blocks > 148 * 16) blocks = 148 * 16;
-    return launch_serialised(pack_rows_kernel, (unsigned)blocks, 256, stream, a, b);
+    const int64_t units = a.total_rows * cdiv(a.cols, 512) + b.total_rows * cdiv(b.cols, 512);
+    if (units == 0) return CUDALLM_OK;
+    int64_t blocks = cdiv(units, kPackThreads / 32);     // one warp per 512 elements of a row, grid-stride
+    if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
+    return launch_serialised(pack_rows_kernel, (unsigned)blocks, kPackThreads, stream, a, b);
 }
 
 // Launches the tcgen05 kernel of variant `v` (lone CTAs or CTA pairs).
@@ -752,13 +787,24 @@ GemmParams make_params(const Problem &p, const Tiling &t, int a_box_rows)
     gp.div_gm = make_fast_div((uint32_t)gp.group_m);
     const int last_gm = gp.tiles_m % gp.group_m;
     gp.div_gm_last = make_fast_div((uint32_t)(last_gm ? last_gm : gp.group_m));
+    gp.wait_limit_ns = g_wait_limit_ns.load(std::memory_order_relaxed);
     return gp;
 }
+
+// The launch's flag value for split tiles (0 when nothing is split); normally the units also
+// raise their flags to it.
+void set_split_epoch(GemmParams &gp, DeviceState &d, bool split);
 
 int next_epoch(DeviceState &d)
 {
     d.epoch = (d.epoch == 0x7fffffff) ? 1 : d.epoch + 1;
     return d.epoch;
+}
+void set_split_epoch(GemmParams &gp, DeviceState &d, bool split)
+{
+    gp.epoch = split ? next_epoch(d) : 0;
+    gp.flag_post = gp.epoch;
+    if (split && g_skew_next_flags.exchange(0)) gp.flag_post = gp.epoch ^ 0x40000000;
 }
 
 int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
@@ -779,9 +825,10 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     const bool pack_a = !a_operand_aligned(p);
     const bool pack_b = !b_operand_aligned(p);
     const Plan pl = make_plan(t, p, pack_a, pack_b);
-    st = ensure_workspace(dev, pl.total, stream);
+    Workspace &w = workspace_for(d, stream);
+    st = ensure_workspace(w, pl.total, stream);
     if (st != CUDALLM_OK) return st;
-    uint8_t *ws = static_cast<uint8_t *>(d.ws);
+    uint8_t *ws = static_cast<uint8_t *>(w.ptr);
 
     const void *A = p.A, *B = p.B;
     int64_t lda = p.lda, ldb = p.ldb, sA = p.sA, sB = p.sB;
@@ -810,11 +857,10 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     CUtensorMap tc;
     st = encode_c_map(dev, &tc, p, gp.c_tma != 0);
     if (st != CUDALLM_OK) return st;
-    gp.epoch = t.split > 1 ? next_epoch(d) : 0;
+    set_split_epoch(gp, d, t.split > 1);
     gp.partials = reinterpret_cast<float *>(ws + pl.off_partials);
     gp.flags = reinterpret_cast<int *>(ws + 256);
     gp.status = reinterpret_cast<int *>(ws);
-
     return launch_variant(dev, v, bf, ta, tb, tc, gp, stream);
 }
 
@@ -826,9 +872,8 @@ int run(int variant, const Problem &p, void *stream_v)
     if (variant != CUDALLM_VARIANT_AUTO && (variant < 0 || variant >= kNumVariants))
         return CUDALLM_ERR_INVALID_VARIANT;
     if (is_empty(p)) return CUDALLM_OK;
-    if (variant == CUDALLM_VARIANT_AUTO) variant = select_variant(p);
-    const Variant &v = g_variants[variant];
-    if (!variant_supports(v, p)) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+    if (variant != CUDALLM_VARIANT_AUTO && !variant_supports(g_variants[variant], p))
+        return CUDALLM_ERR_UNSUPPORTED_SHAPE;
 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     int dev = 0;
@@ -837,6 +882,11 @@ int run(int variant, const Problem &p, void *stream_v)
     std::lock_guard<std::mutex> lock(g_mutex);
     st = probe_device(dev);
     if (st != CUDALLM_OK) return st;
+    // A stream with a workspace of its own declares that other launches may share the GPU:
+    // the automatic choice then keeps to variants whose CTAs never wait for one another.
+    if (variant == CUDALLM_VARIANT_AUTO) variant = select_variant(p, stream_has_workspace(g_dev[dev], stream));
+    const Variant &v = g_variants[variant];
+    if (!variant_supports(v, p)) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
     if (v.family == kSimt) return launch_simt(p, stream);
     return run_umma(dev, v, p, stream);       // both tcgen05 families
 }
@@ -949,9 +999,10 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
     off = (size_t)round_up((int64_t)off + 3 * M * ldap * 2, 256);
     const size_t off_b = off;
     off = (size_t)round_up((int64_t)off + 3 * K * ldbp * 2, 256);
-    st = ensure_workspace(dev, off, stream);
+    Workspace &w = workspace_for(d, stream);
+    st = ensure_workspace(w, off, stream);
     if (st != CUDALLM_OK) return st;
-    uint8_t *ws = static_cast<uint8_t *>(d.ws);
+    uint8_t *ws = static_cast<uint8_t *>(w.ptr);
 
     auto split = [&](const void *src, void *dst, int64_t rows, int64_t cols, int64_t ld_src, int64_t ld_dst) {
         const int64_t total = rows * cdiv(cols, 8);
@@ -980,7 +1031,7 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
     if (st != CUDALLM_OK) return st;
     gp.K = (int)q.K;
     gp.piece_kblocks = (int)cdiv(K, kBlockK);
-    gp.epoch = t.split > 1 ? next_epoch(d) : 0;
+    set_split_epoch(gp, d, t.split > 1);
     gp.partials = reinterpret_cast<float *>(ws + off_partials);
     gp.flags = reinterpret_cast<int *>(ws + 256);
     gp.status = reinterpret_cast<int *>(ws);
@@ -1011,9 +1062,10 @@ int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int6
     std::lock_guard<std::mutex> lock(g_mutex);
     int st = probe_device(dev);
     if (st != CUDALLM_OK) return st;
-    st = ensure_workspace(dev, kHeaderBytes, stream);          // for the status word
-    if (st != CUDALLM_OK) return st;
     DeviceState &d = g_dev[dev];
+    Workspace &w = workspace_for(d, stream);
+    st = ensure_workspace(w, kHeaderBytes, stream);            // for the status word
+    if (st != CUDALLM_OK) return st;
 
     MhsaParams mp{};
     mp.Q = static_cast<const __nv_bfloat16 *>(Q);
@@ -1027,7 +1079,7 @@ int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int6
     while (mp.tmem_cols < mp.keys_pad) mp.tmem_cols *= 2;
     mp.ldq = ldq; mp.ldk = ldk; mp.ldv = ldv; mp.ldo = ldo;
     mp.scale_log2 = 1.4426950408889634f / sqrtf((float)dk);
-    mp.status = static_cast<int *>(d.ws);
+    mp.status = static_cast<int *>(w.ptr);
     const MhsaSmem L = mhsa_smem_layout(mp.keys_pad, mp.dkp);
     if (!d.smem_attr_set[8]) {
         CUDA_TRY(cudaFuncSetAttribute(mhsa_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
@@ -1148,7 +1200,7 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     if (cdiv(K, kBlockK) < split_k) return CUDALLM_ERR_UNSUPPORTED_SHAPE;   // also covers K == 0
     if (!a_operand_aligned(p) || !b_operand_aligned(p)) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
 
-    // always 128 x 64 tiles, every tile split: split_k - 1 partial tiles of 32 KiB each
+    // always 128 x 64 tiles, every tile split: split_k slots of 32 KiB per tile
     Variant v{};
     v.family = kUmma;
     v.block_n = 64;
@@ -1163,7 +1215,7 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     int dev = 0;
     CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
-    std::lock_guard<std::mutex> lock(g_mutex);
+    std::unique_lock<std::mutex> lock(g_mutex);
     st = probe_device(dev);
     if (st != CUDALLM_OK) return st;
     if (!g_noalloc_scratch_addr[dev]) {
@@ -1187,6 +1239,7 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     if (st != CUDALLM_OK) return st;
     g_noalloc_epoch[dev] = (g_noalloc_epoch[dev] == 0x7fffffff) ? 1 : g_noalloc_epoch[dev] + 1;
     gp.epoch = g_noalloc_epoch[dev];
+    gp.flag_post = gp.epoch;
     gp.status = reinterpret_cast<int *>(scratch);
     gp.flags = reinterpret_cast<int *>(scratch + 256);
     gp.partials = reinterpret_cast<float *>(scratch + kNoallocHeaderBytes);
@@ -1197,6 +1250,7 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C, int6
     st = (p.out_dtype == CUDALLM_BF16) ? launch_umma<64, 4, 2, true>(dev, 0, ta, tb, tc, gp, stream)
                                        : launch_umma<64, 4, 2, false>(dev, 1, ta, tb, tc, gp, stream);
     if (st != CUDALLM_OK) return st;
+    lock.unlock();                   // other library calls need not wait for this kernel
     int host_status[2] = {0, 0};
     CUDA_TRY(cudaMemcpyAsync(host_status, scratch, sizeof host_status, cudaMemcpyDeviceToHost, stream));
     CUDA_TRY(cudaStreamSynchronize(stream));
@@ -1303,18 +1357,108 @@ int cudallm_set_workspace(void *dev_ptr, size_t bytes)
     CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
     std::lock_guard<std::mutex> lock(g_mutex);
-    DeviceState &d = g_dev[dev];
+    Workspace &w = g_dev[dev].ws;
     if (!dev_ptr) {
-        d.ws = d.ws_internal;
-        d.ws_bytes = d.ws_internal_bytes;
-        d.ws_external = false;
+        w.ptr = w.internal;
+        w.bytes = w.internal_bytes;
+        w.external = false;
         return CUDALLM_OK;
     }
     if (bytes < kHeaderBytes || (reinterpret_cast<uintptr_t>(dev_ptr) % 256)) return CUDALLM_ERR_WORKSPACE;
-    d.ws = dev_ptr;
-    d.ws_bytes = bytes;
-    d.ws_external = true;
+    w.ptr = dev_ptr;
+    w.bytes = bytes;
+    w.external = true;
     return CUDALLM_OK;
+}
+
+int cudallm_set_workspace_for_stream(void *stream_v, void *dev_ptr, size_t bytes)
+{
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState &d = g_dev[dev];
+    if (!dev_ptr) {
+        d.stream_ws.erase(stream);
+        return CUDALLM_OK;
+    }
+    if (bytes < kHeaderBytes || (reinterpret_cast<uintptr_t>(dev_ptr) % 256)) return CUDALLM_ERR_WORKSPACE;
+    for (const auto &kv : d.stream_ws)           // two streams must not share scratch
+        if (kv.first != stream) {
+            const uint8_t *a = static_cast<const uint8_t *>(kv.second.ptr), *b = static_cast<const uint8_t *>(dev_ptr);
+            if (a < b + bytes && b < a + kv.second.bytes) return CUDALLM_ERR_WORKSPACE;
+        }
+    Workspace w;
+    w.ptr = dev_ptr;
+    w.bytes = bytes;
+    w.external = true;
+    d.stream_ws[stream] = w;
+    return CUDALLM_OK;
+}
+
+int cudallm_reserve_workspace(size_t bytes)
+{
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    Workspace &w = g_dev[dev].ws;
+    if (w.external) return CUDALLM_ERR_WORKSPACE;
+    return ensure_workspace(w, bytes < kHeaderBytes ? kHeaderBytes : bytes, nullptr, true);
+}
+
+int cudallm_shutdown(void)
+{
+    int cur = 0;
+    const bool have_dev = cudaGetDevice(&cur) == cudaSuccess;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int first_error = CUDALLM_OK;
+    for (int dev = 0; dev < kMaxDevices; ++dev) {
+        DeviceState &d = g_dev[dev];
+        HostPipe &hp = g_host_pipe[dev];
+        if (!d.ws.internal && !hp.ready) {
+            d.stream_ws.clear();
+            continue;
+        }
+        if (cudaSetDevice(dev) != cudaSuccess) continue;
+        cudaError_t e = cudaDeviceSynchronize();
+        if (d.ws.internal) {
+            if (e == cudaSuccess) e = cudaFree(d.ws.internal);
+            if (!d.ws.external) { d.ws.ptr = nullptr; d.ws.bytes = 0; }
+            d.ws.internal = nullptr;
+            d.ws.internal_bytes = 0;
+        }
+        if (hp.ready) {
+            cudaStreamDestroy(hp.in);
+            cudaStreamDestroy(hp.out);
+            for (int i = 0; i < kHostPipeChunks; ++i) {
+                cudaEventDestroy(hp.arrived[i]);
+                cudaEventDestroy(hp.computed[i]);
+            }
+            cudaEventDestroy(hp.start);
+            cudaEventDestroy(hp.done);
+            hp = HostPipe{};
+        }
+        d.stream_ws.clear();
+        if (e != cudaSuccess && first_error == CUDALLM_OK) first_error = cuda_fail(e, "cudallm_shutdown");
+    }
+    if (have_dev) cudaSetDevice(cur);
+    return first_error;
+}
+
+int cudallm_debug_set(int what, unsigned long long value)
+{
+    switch (what) {
+    case CUDALLM_DEBUG_WAIT_LIMIT_NS:
+        g_wait_limit_ns.store(value ? value : kWaitLimitNs);
+        return CUDALLM_OK;
+    case CUDALLM_DEBUG_MISS_NEXT_SPLIT_FLAGS:
+        g_skew_next_flags.store(value ? 1 : 0);
+        return CUDALLM_OK;
+    default:
+        return CUDALLM_ERR_INVALID_VARIANT;
+    }
 }
 
 int cudallm_device_status(void *stream_v, int *code, int *detail)
@@ -1328,12 +1472,13 @@ int cudallm_device_status(void *stream_v, int *code, int *detail)
     CUDA_TRY(cudaStreamSynchronize(stream));
     std::lock_guard<std::mutex> lock(g_mutex);
     DeviceState &d = g_dev[dev];
-    if (!d.ws) return CUDALLM_OK;                      // no kernel of ours has run yet
+    Workspace &w = workspace_for(d, stream);
+    if (!w.ptr) return CUDALLM_OK;                     // no kernel of ours has run yet
     int host[2] = {0, 0};
-    CUDA_TRY(cudaMemcpy(host, d.ws, sizeof host, cudaMemcpyDeviceToHost));
+    CUDA_TRY(cudaMemcpy(host, w.ptr, sizeof host, cudaMemcpyDeviceToHost));
     if (host[0] != 0) {
-        // a kernel gave up: its tile counters may be stale; clear the whole header
-        CUDA_TRY(cudaMemset(d.ws, 0, kHeaderBytes));
+        // a kernel gave up: flags and counters may be stale; clear the whole header
+        CUDA_TRY(cudaMemset(w.ptr, 0, kHeaderBytes));
     }
     if (code) *code = host[0];
     if (detail) *detail = host[1];

@@ -126,9 +126,10 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
 
     const size_t off_partials = kHeaderBytes;
     const size_t total = off_partials + (size_t)batch * (size_t)parts * 32;
-    st = ensure_workspace(dev, total, stream);
+    Workspace &w = workspace_for(d, stream);
+    st = ensure_workspace(w, total, stream);
     if (st != CUDALLM_OK) return st;
-    uint8_t *ws = static_cast<uint8_t *>(d.ws);
+    uint8_t *ws = static_cast<uint8_t *>(w.ptr);
 
     LayerNorm2Params lp{};
     lp.x = x; lp.gamma = gamma; lp.beta = beta; lp.y = y;

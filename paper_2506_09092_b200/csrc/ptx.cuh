@@ -98,15 +98,17 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     return ok != 0;
 }
 
-// Wall-clock limit of every in-kernel wait.  Far above any legitimate wait
-// (a whole GEMM takes well under a second), short enough that a logic error
-// ends the kernel instead of hanging the device.
+// Default wall-clock limit of every in-kernel wait.  Far above any legitimate
+// wait (a whole GEMM takes well under a second), short enough that a logic
+// error ends the kernel instead of hanging the device.  The GEMM kernels take
+// their limit from a kernel parameter (this value unless the host changed it).
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 // Wait for phase `parity` of `bar`.  Returns false if `*abort_flag` becomes
-// non-zero or the limit expires (then it also sets `*abort_flag`).
+// non-zero or `limit_ns` expires (then it also sets `*abort_flag`).
 template <bool kCluster = false>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          uint64_t limit_ns = kWaitLimitNs)
 {
     for (int i = 0; i < 128; ++i) {
         if (kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
@@ -118,7 +120,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                 return true;
         }
         if (*abort_flag) return false;
-        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        if (globaltimer_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             return false;
         }

@@ -77,6 +77,9 @@ struct GemmParams {
     int n_edge_tma;         // ... including the box that straddles column N (N * element size % 16 == 0)
     int a_box_bytes;        // bytes one TMA box of A delivers (box rows * 128)
     int epoch;              // value that marks a flag as raised in this launch (never 0)
+    int flag_post;          // value a unit raises its flags to: epoch (anything else only in the host's
+                            // self-test of the timeout path, where no wait may ever be satisfied)
+    unsigned long long wait_limit_ns;   // wall-clock limit of every bounded wait in the kernel
     float *partials;        // partial tiles of split units (workspace), 128 x BLOCK_N fp32 each
     int *flags;             // one per (partial tile, epilogue warp) (workspace)
     int *status;            // [0] = code, [1] = detail
@@ -115,7 +118,7 @@ struct SmemLayout {
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
     static constexpr int kBytes = kMiscOffset + 64;
-    static constexpr int kDynamicBytes = kBytes + 1024;  // slack for 1024-byte alignment
+    static constexpr int kDynamicBytes = kBytes;         // the base is declared 1024-byte aligned
 };
 
 __device__ __forceinline__ void report_timeout(int *status, int role, int what)
@@ -215,7 +218,8 @@ __device__ __forceinline__ void st_release_gpu(int *p, int v)
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 // Bounded wait until *flag == epoch.
-__device__ __forceinline__ bool wait_flag(const int *flag, int epoch, volatile int *abort_flag)
+__device__ __forceinline__ bool wait_flag(const int *flag, int epoch, volatile int *abort_flag,
+                                          uint64_t limit_ns)
 {
     if (ld_acquire_gpu(flag) == epoch) return true;
     const uint64_t t0 = globaltimer_ns();
@@ -225,7 +229,7 @@ __device__ __forceinline__ bool wait_flag(const int *flag, int epoch, volatile i
             __nanosleep(100);
         }
         if (*abort_flag) return false;
-        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        if (globaltimer_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             return false;
         }
@@ -392,13 +396,13 @@ __device__ __forceinline__ bool epilogue_tile(const GemmParams &p, const UnitCoo
         // whose fence is cumulative over them (the order a grid-wide barrier relies on too):
         // one fence per warp instead of one per lane plus the store's own.
         __syncwarp();
-        if (lane == 0) st_release_gpu(p.flags + my_slot * 4 + quad, p.epoch);
+        if (lane == 0) st_release_gpu(p.flags + my_slot * 4 + quad, p.flag_post);
         if (c.split * g >= kChunks) return true;         // this unit owns no chunk
         // 2. the same epilogue warp of every other unit wrote the rows this warp needs
         for (int s = 0; s < S; ++s) {
             if (s == c.split) continue;
             const long long slot = static_cast<long long>(c.slot0 + s) * ctas_per_tile + cta_slot;
-            ok = wait_flag(p.flags + slot * 4 + quad, p.epoch, abort_flag) && ok;
+            ok = wait_flag(p.flags + slot * 4 + quad, p.epoch, abort_flag, p.wait_limit_ns) && ok;
         }
         ok = __all_sync(0xffffffffu, ok);          // (every lane polled with acquire loads itself)
 
@@ -507,10 +511,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     static_assert(BLOCK_N % 64 == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
     constexpr uint32_t kTmemCols = 2 * BLOCK_N;          // 128, 256 or 512: power of two
 
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    // The swizzled stages need 1024-byte alignment in the shared window; the declaration asks
+    // for it (no slack is reserved) and the kernel refuses to run without it.
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *smem = smem_raw;
     const uint32_t smem_base = smem_u32(smem);
+    if (smem_base & 1023u) {
+        if (threadIdx.x == 0) report_timeout(p.status, 0, 0x7F);
+        return;
+    }
     const uint32_t bar_base = smem_base + L::kBarOffset;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
@@ -572,7 +581,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 const UnitCoord c = decode_unit(p, u);
                 constexpr int boxes = BLOCK_N / 64;
                 for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
-                    if (!tok && !mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) {
+                    if (!tok && !mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, p.wait_limit_ns)) {
                         report_timeout(p.status, kRoleProducer, stage);
                         ok = false;
                         break;
@@ -611,14 +620,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             for (int u = blockIdx.x; ok && u < p.num_units; u += gridDim.x) {
                 const UnitCoord c = decode_unit(p, u);
                 constexpr uint32_t idesc = make_idesc_bf16(kBlockM, BLOCK_N, 0, 1);
-                if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag)) {
+                if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, p.wait_limit_ns)) {
                     report_timeout(p.status, kRoleMma, 0x40 + acc);
                     break;
                 }
                 const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
                 bool first_of_unit = true;
                 for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
-                    if (!tok && !mbar_wait(full_bar(stage), phase, abort_flag)) {
+                    if (!tok && !mbar_wait(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) {
                         report_timeout(p.status, kRoleMma, stage);
                         ok = false;
                         break;
@@ -658,7 +667,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         grid_dependency_wait();
         for (int u = blockIdx.x; u < p.num_units; u += gridDim.x) {
             const UnitCoord c = decode_unit(p, u);
-            bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
+            bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.wait_limit_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
                 if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0x80 + acc);

@@ -68,7 +68,7 @@ struct PairSmemLayout {
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
     static constexpr int kBytes = kMiscOffset + 64;
-    static constexpr int kDynamicBytes = kBytes + 1024;
+    static constexpr int kDynamicBytes = kBytes;         // the base is declared 1024-byte aligned
 };
 
 template <int STAGES, int KSUB, bool OUT_BF16>
@@ -79,10 +79,15 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     using L = PairSmemLayout<STAGES, KSUB>;
     constexpr uint32_t kTmemCols = 2 * kPairN;                       // 512: two accumulators
 
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    // The swizzled stages need 1024-byte alignment in the shared window; the declaration asks
+    // for it (no slack is reserved) and the kernel refuses to run without it.
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *smem = smem_raw;
     const uint32_t smem_base = smem_u32(smem);
+    if (smem_base & 1023u) {
+        if (threadIdx.x == 0) report_timeout(p.status, 0, 0x7F);
+        return;
+    }
     const uint32_t bar_base = smem_base + L::kBarOffset;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
@@ -140,7 +145,7 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 constexpr int half = kPairN / 2;         // columns of B this CTA stages
                 constexpr int boxes = half / 64;
                 for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
-                    if (!tok && !mbar_wait<true>(empty_bar(stage), phase ^ 1, abort_flag)) {
+                    if (!tok && !mbar_wait<true>(empty_bar(stage), phase ^ 1, abort_flag, p.wait_limit_ns)) {
                         report_timeout(p.status, kRoleProducer, stage);
                         ok = false;
                         break;
@@ -186,14 +191,14 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             for (int u = pair; ok && u < p.num_units; u += num_pairs) {
                 const UnitCoord c = decode_unit(p, u);
                 constexpr uint32_t idesc = make_idesc_bf16(kPairM, kPairN, 0, 1);
-                if (!mbar_wait<true>(tempty_bar(acc), acc_phase ^ 1, abort_flag)) {
+                if (!mbar_wait<true>(tempty_bar(acc), acc_phase ^ 1, abort_flag, p.wait_limit_ns)) {
                     report_timeout(p.status, kRoleMma, 0x40 + acc);
                     break;
                 }
                 const uint32_t d_tmem = tmem_base + acc * kPairN;
                 bool first_of_unit = true;
                 for (int kb = c.kb_begin; kb < c.kb_end; kb += KSUB) {
-                    if (!tok && !mbar_wait<true>(full_bar(stage), phase, abort_flag)) {
+                    if (!tok && !mbar_wait<true>(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) {
                         report_timeout(p.status, kRoleMma, stage);
                         ok = false;
                         break;
@@ -230,7 +235,7 @@ umma_gemm_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         grid_dependency_wait();
         for (int u = pair; u < p.num_units; u += num_pairs) {
             const UnitCoord c = decode_unit(p, u);
-            bool ok = mbar_wait<true>(tfull_bar(acc), acc_phase, abort_flag);
+            bool ok = mbar_wait<true>(tfull_bar(acc), acc_phase, abort_flag, p.wait_limit_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
                 if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0x80 + acc);

@@ -95,6 +95,25 @@ def run_config(cfg: gi.GemmConfig, variant=B.VARIANT_AUTO, operands=None):
                     cfg.batch, cfg.strideA, cfg.strideB, cfg.strideC, variant)
 
 
+def log_observed_error(family: str, case: str, observed: float, bound: float, what: str, **extra):
+    """Append the largest error a parity test observed (in the units of its tolerance) to
+    ``observed_errors.jsonl`` in the directory the environment variable CUDALLM_ERROR_LOG_DIR
+    names (default: ``gpurun_out`` at the repository root, created on demand), so that the
+    share of each tolerance that is actually used can be read off."""
+    import json
+    import os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out_dir = os.environ.get("CUDALLM_ERROR_LOG_DIR", os.path.join(root, "gpurun_out"))
+    try:
+        os.makedirs(out_dir, exist_ok=True)
+        rec = dict(family=family, case=case, observed=float(observed), bound=float(bound),
+                   share=float(observed) / float(bound) if bound else None, what=what, **extra)
+        with open(os.path.join(out_dir, "observed_errors.jsonl"), "a") as f:
+            f.write(json.dumps(rec) + "\n")
+    except OSError:
+        pass
+
+
 def tol_for(out_dtype):
     return oracle.TOL_F32_OUT if out_dtype == gi.F32 else oracle.TOL_BF16_OUT
 

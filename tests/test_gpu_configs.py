@@ -1,10 +1,12 @@
 """The benchmark configurations at full size, in the launch configuration the
 benchmark times (automatic variant choice, device-resident operands).
 
-C1, C4, C5a and C5b are compared with the oracle on every element.  C2 and C3
-are compared on a seeded sample of full rows (the oracle needs tens of seconds
-for the whole product) and, on every element, against the integer rank-1
-closed form, which holds at any size."""
+Every configuration, C2 and C3 included, is compared with the oracle on every
+element (the oracle needs a few seconds for C2 and some tens of seconds for C3
+on the host cores), and against the integer rank-1 closed form, which holds at
+any size.  The largest scaled error each comparison observed is appended to a
+JSON-lines file beside the tests' other output, so that the margin under each
+tolerance can be read off."""
 import numpy as np
 import pytest
 import torch
@@ -23,11 +25,17 @@ def _run(cfg, A, Bm, variant=B.VARIANT_AUTO):
     return vals, raw
 
 
-@pytest.mark.parametrize("name", ["C1", "C4", "C5a", "C5b"])
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5a", "C5b"])
 def test_config_every_element(name):
+    """Every element of every benchmark configuration against the oracle; the product is run
+    twice and must come out bit for bit the same (fixed summation order, also where tiles
+    are split along K)."""
     cfg = gi.CONFIGS[name]
     A, Bm = cfg.make()
-    vals, _ = _run(cfg, A, Bm)
+    vals, raw = _run(cfg, A, Bm)
+    _, raw2 = _run(cfg, A, Bm)
+    assert np.array_equal(raw, raw2), f"{name}: two runs differ"
+    del raw2
     if cfg.batch > 1:
         Cref, S = oracle.gemm_batched(A, Bm, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_,
                                       cfg.strideA, cfg.strideB, cfg.batch)
@@ -35,22 +43,11 @@ def test_config_every_element(name):
     else:
         Cref, S = oracle.gemm(A, Bm, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_)
         r = oracle.check(vals[0], Cref, S, G.tol_for(cfg.out_dtype))
+    G.log_observed_error("gemm_bf16", name, r.max_scaled_err, G.tol_for(cfg.out_dtype),
+                         "max |C - C_ref| / sum|a||b|", variant=B.variant_name(
+                             B.select_variant(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype)))
     assert r.ok, (name, r)
-
-
-@pytest.mark.parametrize("name,nrows", [("C2", 384), ("C3", 96)])
-def test_config_sampled_rows(name, nrows):
-    cfg = gi.CONFIGS[name]
-    A, Bm = cfg.make()
-    vals, _ = _run(cfg, A, Bm)
-    rng = np.random.default_rng([cfg.seed, 99])
-    rows = np.sort(rng.choice(cfg.M, size=nrows, replace=False))
-    rows[0], rows[-1] = 0, cfg.M - 1                      # always include the edges
-    rows[1] = 127; rows[2] = 128                          # and a tile boundary
-    Cref, S = oracle.gemm_rows(A, Bm, rows, cfg.N, cfg.K, cfg.lda_, cfg.ldb_)
-    r = oracle.check(vals[0][rows], Cref, S, G.tol_for(cfg.out_dtype))
-    assert r.ok, (name, r)
-    assert np.isfinite(vals[0]).all()
+    assert np.isfinite(vals).all()
 
 
 @pytest.mark.parametrize("name", ["C2", "C3", "C5a", "C5b"])
@@ -68,6 +65,22 @@ def test_config_size_integer_closed_form(name):
     else:
         want = oracle.f64_to_bf16_bits(exact)
         assert ((raw[0] == want) | ((exact == 0) & (vals[0] == 0))).all()
+
+
+@pytest.mark.parametrize("name,variants", [
+    ("C2", ["umma2_n256", "umma_n256_ts"]),
+    ("C5a", ["umma_n128_sk2", "umma_n64_sk4"]),
+    ("C5b", ["umma2_n256_sk2", "umma_n128_ts"]),
+])
+def test_config_size_runs_are_bitwise_repeatable(name, variants):
+    """Split-K and tail-split variants at full size: two runs, identical bits."""
+    cfg = gi.CONFIGS[name]
+    A, Bm = cfg.make()
+    table = {B.variant_name(v): v for v in range(B.num_variants())}
+    for vn in variants:
+        _, raw = _run(cfg, A, Bm, table[vn])
+        _, raw2 = _run(cfg, A, Bm, table[vn])
+        assert np.array_equal(raw, raw2), (name, vn)
 
 
 def test_paper_task2_ladder_first_two_sizes():

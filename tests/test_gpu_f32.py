@@ -14,6 +14,7 @@ import pytest
 import torch
 
 import oracle
+import gpu_util as G
 from paper_2506_09092_b200 import binding as B
 from paper_2506_09092_b200 import inputs as gi
 
@@ -55,6 +56,7 @@ def run_f32(Af, Bf, M, N, K, pad=0, variant=-1, lead=0, expect=B.OK):
 def check(got, Af, Bf, M, N, K):
     Cref, S = oracle.gemm_f32(Af, Bf, M, N, K)
     r = oracle.check(got, Cref, S, TOL)
+    G.log_observed_error("gemm_f32", f"{M}x{N}x{K}", r.max_scaled_err, TOL, "max |C - C_ref| / sum|a||b|")
     assert r.ok, r
     return r.max_scaled_err
 

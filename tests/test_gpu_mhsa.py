@@ -9,6 +9,7 @@ import pytest
 import torch
 
 import oracle
+import gpu_util as G
 from paper_2506_09092_b200 import binding as B
 from paper_2506_09092_b200 import inputs as gi
 
@@ -46,6 +47,8 @@ def test_paper_sizes(N, dm, h):
     got = run(Q, K, V, N, dm, h)
     ref, T = oracle.mhsa(Q, K, V, N, dm, h)
     r = oracle.check(got, ref, T, oracle.TOL_MHSA)
+    G.log_observed_error("mhsa_bf16", f"N={N} d_model={dm} h={h}", r.max_scaled_err, oracle.TOL_MHSA,
+                         "max |O - O_ref| / sum_j p_ij |v_jc|")
     assert r.ok, r
     # sharper score distributions too (larger queries)
     Q2 = bits(3.0 * rng.standard_normal((N, dm)))

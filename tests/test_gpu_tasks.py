@@ -19,6 +19,7 @@ import pytest
 import torch
 
 import oracle
+import gpu_util as G
 from paper_2506_09092_b200 import binding as B
 from paper_2506_09092_b200 import inputs as gi
 
@@ -203,6 +204,8 @@ def check_layernorm(got, x, gamma, beta, batch, m, eps=1e-5):
     bound = 2.0 ** -20 * (z + 1.0) * np.abs(g) + 2.0 ** -22 * np.abs(b)
     err = np.abs(got - ref)
     assert np.all(np.isfinite(got))
+    G.log_observed_error("layernorm_f32", f"batch={batch} m={m}", float((err / np.maximum(bound, 1e-300)).max()), 1.0,
+                         "max |y - y_ref| / (2^-20 (|z| + 1)|gamma| + 2^-22 |beta|)")
     assert np.all(err <= bound), (float((err / np.maximum(bound, 1e-300)).max()), np.unravel_index(np.argmax(err - bound), err.shape))
 
 
