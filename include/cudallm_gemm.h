@@ -229,9 +229,20 @@ int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O,
                       int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
                       void *stream);
 
-/* Kernel variants (the candidate set of Algorithm 1's search). */
+/*
+ * Kernel variants (the candidate set of Algorithm 1's search).  A variant id is a number below
+ * cudallm_num_variants().  Wherever a call takes a `variant`, it also takes a variant CODE: the
+ * id plus two knobs that the search varies as well (cudallm_variant_code composes one):
+ *   group_rows  0 = the library's rule, else a power of two <= 16384: the tiles are visited in
+ *               raster groups of that many tile rows (what stays in L2 while B streams by);
+ *   tail_parts  0 = the library's rule, else 2..7, for the tail-splitting ("_ts") variants only:
+ *               the tiles of the ragged last wave are cut into up to that many parts along K.
+ * cudallm_variant_code returns the code, or CUDALLM_ERR_INVALID_VARIANT.
+ * cudallm_variant_name gives the variant's name for an id or a code (NULL if invalid).
+ */
 int cudallm_num_variants(void);
-const char *cudallm_variant_name(int variant);            /* NULL if out of range */
+const char *cudallm_variant_name(int variant);
+int cudallm_variant_code(int variant, int group_rows, int tail_parts);
 /* 1 if `variant` can run the problem, 0 if not, negative status on bad args. */
 int cudallm_variant_supports(int variant,
                              int64_t M, int64_t N, int64_t K,
@@ -246,26 +257,41 @@ int cudallm_select_variant(int64_t M, int64_t N, int64_t K,
 
 /*
  * Dispatch table: the persisted outcome of the search (Algorithm 1's arg-min
- * over the valid candidates, one entry per problem shape).  An entry says that
- * `variant` is the fastest valid kernel for products of shape (M, N, K, batch,
- * out_dtype).  cudallm_gemm_bf16, cudallm_gemm_bf16_batched,
- * cudallm_gemm_bf16_host and cudallm_select_variant look the shape up first and
- * use the entry if that variant can run the problem; otherwise, and for every
- * shape without an entry, the cost model decides.
- * The table is process-wide, starts empty and holds at most 65536 entries.
- *   cudallm_dispatch_set    adds or replaces an entry; variant == -1 removes it.
+ * over the valid candidates).  An entry says that `variant` (an id or a code) is
+ * the fastest valid kernel for a shape (M, N, K, batch, out_dtype), or for a
+ * shape CLASS: all shapes with the same ceil(M/128), ceil(N/64), ceil(K/64),
+ * batch and out_dtype, on the same side of M <= 16 and M <= 64, whose operands
+ * TMA can (tma_addressable != 0: 16-byte aligned bases, leading dimensions
+ * multiples of 8) or cannot address -- every variant cuts all of them into the
+ * same tiles and k-blocks.  cudallm_gemm_bf16, cudallm_gemm_bf16_batched,
+ * cudallm_gemm_bf16_host and cudallm_select_variant look up the exact shape,
+ * then its class, and use the entry if that variant can run the problem;
+ * otherwise the cost model decides.
+ * The tables are process-wide and hold at most 65536 entries each.  When the
+ * library is first used the class table receives the winners of the search
+ * recorded on a B200 and compiled into the library (the benchmark
+ * configurations, the paper's Task 2 sizes and a grid of other shapes);
+ * cudallm_dispatch_clear removes them too, cudallm_dispatch_load_packaged
+ * enters them again.
+ *   cudallm_dispatch_set / _set_class   add or replace an entry; variant == -1 removes it.
  *                           Errors: INVALID_DIM (a negative size), INVALID_DTYPE,
- *                           INVALID_VARIANT (not -1 and not a variant id),
+ *                           INVALID_VARIANT (not -1 and not a valid id or code),
  *                           TOO_LARGE (table full).
- *   cudallm_dispatch_get    *variant = the entry's variant, or -1 if there is none.
+ *   cudallm_dispatch_get / _get_class   *variant = the entry's variant, or -1 if there is none.
  *                           Errors: as above, INVALID_POINTER (variant == NULL).
- *   cudallm_dispatch_clear  empties the table; returns the number of entries it held.
+ *   cudallm_dispatch_clear  empties both tables; returns the number of entries they held.
+ *   cudallm_dispatch_load_packaged      returns the number of entries entered.
  * Host-side only: no CUDA call.  Safe to call from several threads; a change is
  * seen by calls that start after it returns.
  */
 int cudallm_dispatch_set(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int variant);
 int cudallm_dispatch_get(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int *variant);
+int cudallm_dispatch_set_class(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype,
+                               int tma_addressable, int variant);
+int cudallm_dispatch_get_class(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype,
+                               int tma_addressable, int *variant);
 int cudallm_dispatch_clear(void);
+int cudallm_dispatch_load_packaged(void);
 
 /*
  * Workspace.  Upper bound of the scratch bytes any variant may need for the

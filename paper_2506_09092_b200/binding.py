@@ -51,7 +51,11 @@ SIGNATURES = {
     "cudallm_num_variants": (_int, []),
     "cudallm_dispatch_set": (_int, [_i64, _i64, _i64, _i64, _int, _int]),
     "cudallm_dispatch_get": (_int, [_i64, _i64, _i64, _i64, _int, ctypes.POINTER(ctypes.c_int)]),
+    "cudallm_dispatch_set_class": (_int, [_i64, _i64, _i64, _i64, _int, _int, _int]),
+    "cudallm_dispatch_get_class": (_int, [_i64, _i64, _i64, _i64, _int, _int, ctypes.POINTER(ctypes.c_int)]),
     "cudallm_dispatch_clear": (_int, []),
+    "cudallm_dispatch_load_packaged": (_int, []),
+    "cudallm_variant_code": (_int, [_int, _int, _int]),
     "cudallm_variant_name": (ctypes.c_char_p, [_int]),
     "cudallm_variant_supports": (_int, [_int] + [_i64] * 7 + [_int]),
     "cudallm_select_variant": (_int, [_i64] * 7 + [_int]),
@@ -210,6 +214,39 @@ def dispatch_get(M, N, K, batch, out_dtype) -> int:
     v = ctypes.c_int(-1)
     _check(lib().cudallm_dispatch_get(M, N, K, batch, out_dtype, ctypes.byref(v)), "cudallm_dispatch_get", True)
     return int(v.value)
+
+
+def dispatch_set_class(M, N, K, batch, out_dtype, tma_addressable, variant, check=True) -> int:
+    """Record ``variant`` for the whole class of shapes that are tiled like this one."""
+    return _check(lib().cudallm_dispatch_set_class(M, N, K, batch, out_dtype, int(bool(tma_addressable)), variant),
+                  "cudallm_dispatch_set_class", check)
+
+
+def dispatch_get_class(M, N, K, batch, out_dtype, tma_addressable) -> int:
+    v = ctypes.c_int(-1)
+    _check(lib().cudallm_dispatch_get_class(M, N, K, batch, out_dtype, int(bool(tma_addressable)), ctypes.byref(v)),
+           "cudallm_dispatch_get_class", True)
+    return int(v.value)
+
+
+def dispatch_load_packaged() -> int:
+    """Enter the packaged search results into the class table; returns how many."""
+    return int(lib().cudallm_dispatch_load_packaged())
+
+
+def variant_code(variant: int, group_rows: int = 0, tail_parts: int = 0, check=True) -> int:
+    """Variant id plus the two knobs the search varies -> the code the entry points take."""
+    code = int(lib().cudallm_variant_code(variant, group_rows, tail_parts))
+    if check and code < 0:
+        raise CudallmError(code, "cudallm_variant_code")
+    return code
+
+
+def describe_code(code: int) -> str:
+    """Human-readable form of a variant code: name, and the knobs that are set."""
+    name = variant_name(code)
+    g, t = (code >> 8) & 0xF, (code >> 12) & 0x7
+    return name + (f"+g{1 << (g - 1)}" if g else "") + (f"+t{t}" if t else "")
 
 
 def dispatch_clear() -> int:

@@ -90,11 +90,25 @@ struct Variant {
     int block_n;
     int split_k;                       // 1 = none, 2..16 = every tile along K, kTailSplit = see above
     int per_sm;                        // CTAs per SM: 1, or 2 for the two-stage kernels for short K
+    int alt_ring;                      // 1: the other arrangement of the shared-memory ring (see build_variants)
 };
 constexpr int kBlockNs[3] = {64, 128, 256};
 constexpr int kSplits[6] = {1, 2, 4, 8, 16, kTailSplit};
-constexpr int kNumVariants = 1 + 3 * 6 + 6 + 2;
+constexpr int kNumVariants = 1 + 3 * 6 + 6 + 2 + 6;
 Variant g_variants[kNumVariants];
+
+// A variant code as the entry points take it: the variant id in the low 8 bits; above it two
+// knobs that the search varies and the dispatch table records, 0 meaning "the library's rule":
+//   bits 8..11  raster group height: g > 0 asks for groups of 2^(g-1) tile rows
+//   bits 12..14 tail split: t >= 2 cuts the tiles of the ragged last wave into up to t parts
+//               (at least 4 k-blocks each) instead of up to 4 parts of at least 8
+inline int code_base(int code) { return code & 0xFF; }
+inline int code_group(int code) { return (code >> 8) & 0xF; }
+inline int code_tail(int code) { return (code >> 12) & 0x7; }
+inline bool code_valid(int code)
+{
+    return code >= 0 && (code >> 15) == 0 && code_base(code) < kNumVariants && code_tail(code) != 1;
+}
 std::once_flag g_variants_once;
 
 void name_variant(Variant &v, const char *stem, int bn, int sk)
@@ -104,6 +118,8 @@ void name_variant(Variant &v, const char *stem, int bn, int sk)
     else snprintf(v.name, sizeof v.name, "%s_n%d_sk%d", stem, bn, sk);
 }
 
+int load_packaged_entries();
+std::once_flag g_packaged_once;
 void build_variants()
 {
     std::call_once(g_variants_once, [] {
@@ -139,9 +155,33 @@ void build_variants()
             g_variants[v].per_sm = 2;
             ++v;
         }
+        // The other arrangement of the same shared memory: one barrier round trip per two
+        // k-blocks where the standard kernel has one per k-block (256-column tiles), or per
+        // k-block where it has one per two (128-column tiles, CTA pairs).  Which one is faster
+        // depends on whether the MMA thread or the load latency bounds the shape: the search decides.
+        for (int bn : {128, 256})
+            for (int sk : {1, kTailSplit}) {
+                snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma_n%d_%s%s", bn, bn == 256 ? "k2" : "k1",
+                         sk == kTailSplit ? "_ts" : "");
+                g_variants[v].family = kUmma;
+                g_variants[v].block_n = bn;
+                g_variants[v].split_k = sk;
+                g_variants[v].alt_ring = 1;
+                ++v;
+            }
+        for (int sk : {1, kTailSplit}) {
+            snprintf(g_variants[v].name, sizeof g_variants[v].name, "umma2_n256_k1%s", sk == kTailSplit ? "_ts" : "");
+            g_variants[v].family = kUmmaPair;
+            g_variants[v].block_n = 256;
+            g_variants[v].split_k = sk;
+            g_variants[v].alt_ring = 1;
+            ++v;
+        }
         for (int i = 0; i < kNumVariants; ++i)
             if (g_variants[i].per_sm == 0) g_variants[i].per_sm = 1;
     });
+    // the dispatch table starts out with the packaged winners of the search
+    std::call_once(g_packaged_once, [] { load_packaged_entries(); });
 }
 
 constexpr int kNumSMs = 148;
@@ -161,8 +201,9 @@ struct Tiling {
     int64_t partial_bytes;
 };
 
-// `slots` = units that run at once (CTAs, or CTA pairs, of the persistent grid).
-Tiling tiling_for(const Variant &v, const Problem &p, int slots)
+// `slots` = units that run at once (CTAs, or CTA pairs, of the persistent grid); `tail` = the
+// tail-split knob of the variant code (0 = the default rule).
+Tiling tiling_for(const Variant &v, const Problem &p, int slots, int tail = 0)
 {
     const bool pair = v.family == kUmmaPair;
     Tiling t{};
@@ -176,13 +217,14 @@ Tiling tiling_for(const Variant &v, const Problem &p, int slots)
     if (v.split_k == kTailSplit) {
         // Split the tiles of the ragged last wave along K so that they fill the
         // grid about once: up to 4 parts, each at least 8 k-blocks deep.
-        const int64_t tail = t.tiles % slots;
-        int64_t parts = tail > 0 ? slots / tail : 1;
-        if (parts > 4) parts = 4;
-        while (parts > 1 && t.kblocks / parts < 8) --parts;
+        const int64_t left = t.tiles % slots;
+        int64_t parts = left > 0 ? slots / left : 1;
+        const int64_t max_parts = tail >= 2 ? tail : 4, min_depth = tail >= 2 ? 4 : 8;
+        if (parts > max_parts) parts = max_parts;
+        while (parts > 1 && t.kblocks / parts < min_depth) --parts;
         if (parts > 1) {
             t.split = (int)parts;
-            t.dp_tiles = t.tiles - tail;
+            t.dp_tiles = t.tiles - left;
         }
     } else if (v.split_k > 1) {
         t.split = v.split_k;
@@ -255,7 +297,11 @@ double variant_cost(const Variant &v, const Problem &p)
     return (compute > memory ? compute : memory) + 4000.0;
 }
 
-// Dispatch table: shape -> variant recorded by a search (cudallm_dispatch_set).
+// Dispatch table: what a search recorded (cudallm_dispatch_set / _set_class).  Two levels: an
+// entry for the exact shape, and an entry for the shape's class -- all shapes that every
+// variant cuts into the same tiles and k-blocks (same ceil(M / 128), ceil(N / 64), ceil(K / 64),
+// batch and output type, same side of the short-A limits M <= 16 and M <= 64, operands
+// addressable by TMA or not): the kernels do the same work on all of them.
 struct DispatchKey {
     int64_t M, N, K, batch;
     int out_dtype;
@@ -273,27 +319,47 @@ struct DispatchHash {
         return (size_t)h;
     }
 };
+// The class of a shape, written as a key of the same type: tile counts in place of sizes; the
+// short-A bucket and the alignment flag are folded into the M and out_dtype fields.
+DispatchKey class_key(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, bool aligned)
+{
+    const int64_t mt = (M + 127) / 128;
+    const int64_t bucket = M <= 16 ? 0 : M <= 64 ? 1 : 2;
+    return DispatchKey{mt * 4 + (mt == 1 ? bucket : 3), (N + 63) / 64, (K + 63) / 64, batch,
+                       out_dtype + (aligned ? 0 : 2)};
+}
 constexpr size_t kMaxDispatchEntries = 65536;
-std::unordered_map<DispatchKey, int, DispatchHash> g_dispatch;
+std::unordered_map<DispatchKey, int, DispatchHash> g_dispatch, g_dispatch_class;
 std::mutex g_dispatch_mutex;
-std::atomic<uint64_t> g_dispatch_generation{0};      // bumped by every change of the table
+std::atomic<uint64_t> g_dispatch_generation{0};      // bumped by every change of the tables
+
+inline bool a_operand_aligned(const Problem &p);
+inline bool b_operand_aligned(const Problem &p);
 
 // `no_waits`: only variants whose CTAs never wait for one another (no split tiles), for
-// calls that may share the GPU with other launches of this library.
+// calls that may share the GPU with other launches of this library.  Returns a variant code.
 int select_variant_uncached(const Problem &p, bool no_waits)
 {
     build_variants();
     if (is_empty(p) || p.K == 0) return 0;
     {
         std::lock_guard<std::mutex> lock(g_dispatch_mutex);
+        auto usable = [&](int code) {
+            const Variant &v = g_variants[code_base(code)];
+            return variant_supports(v, p) && !(no_waits && v.split_k != 1);
+        };
         const auto it = g_dispatch.find(DispatchKey{p.M, p.N, p.K, p.batch, p.out_dtype});
-        if (it != g_dispatch.end() && variant_supports(g_variants[it->second], p)
-            && !(no_waits && g_variants[it->second].split_k != 1))
-            return it->second;
+        if (it != g_dispatch.end() && usable(it->second)) return it->second;
+        if (!g_dispatch_class.empty()) {
+            const bool aligned = a_operand_aligned(p) && b_operand_aligned(p);
+            const auto ic = g_dispatch_class.find(class_key(p.M, p.N, p.K, p.batch, p.out_dtype, aligned));
+            if (ic != g_dispatch_class.end() && usable(ic->second)) return ic->second;
+        }
     }
     int best = -1;
     double best_cost = 0;
     for (int v = 1; v < kNumVariants; ++v) {
+        if (g_variants[v].alt_ring) continue;          // the model does not tell the rings apart: the search does
         if (no_waits && g_variants[v].split_k != 1) continue;
         if (!variant_supports(g_variants[v], p)) continue;
         const double c = variant_cost(g_variants[v], p);
@@ -302,18 +368,20 @@ int select_variant_uncached(const Problem &p, bool no_waits)
     return best < 0 ? 0 : best;
 }
 
-// The choice depends only on the shape (and the dispatch table); repeated calls with
-// the same shape (the common case) reuse the previous answer.
+// The choice depends only on the shape, the operands' alignment class and the dispatch
+// tables; repeated calls with the same shape (the common case) reuse the previous answer.
 int select_variant(const Problem &p, bool no_waits = false)
 {
-    struct Last { int64_t M, N, K, batch; int out_dtype, variant; uint64_t generation; bool no_waits; };
-    static thread_local Last last = {-1, -1, -1, -1, -1, 0, 0, false};
+    struct Last { int64_t M, N, K, batch; int out_dtype, variant; uint64_t generation; bool no_waits, aligned; };
+    static thread_local Last last = {-1, -1, -1, -1, -1, 0, 0, false, false};
     const uint64_t gen = g_dispatch_generation.load(std::memory_order_acquire);
+    const bool aligned = a_operand_aligned(p) && b_operand_aligned(p);
     if (last.M == p.M && last.N == p.N && last.K == p.K && last.batch == p.batch
-        && last.out_dtype == p.out_dtype && last.generation == gen && last.no_waits == no_waits)
+        && last.out_dtype == p.out_dtype && last.generation == gen && last.no_waits == no_waits
+        && last.aligned == aligned)
         return last.variant;
     const int v = select_variant_uncached(p, no_waits);
-    last = Last{p.M, p.N, p.K, p.batch, p.out_dtype, v, gen, no_waits};
+    last = Last{p.M, p.N, p.K, p.batch, p.out_dtype, v, gen, no_waits, aligned};
     return v;
 }
 
@@ -339,7 +407,7 @@ struct DeviceState {
     int sm_count = 0;
     Workspace ws;                // the device's default workspace
     std::unordered_map<cudaStream_t, Workspace> stream_ws;   // cudallm_set_workspace_for_stream
-    bool smem_attr_set[24] = {};
+    bool smem_attr_set[40] = {};
     int max_pairs = 0;           // co-resident 2-CTA clusters of the pair kernel (0 = not asked yet)
     int epoch = 0;               // last split-K flag value used on this device
 };
@@ -727,15 +795,26 @@ int launch_pack(const PackJob &a, const PackJob &b, cudaStream_t stream)
 int launch_variant(int dev, const Variant &v, bool bf, const CUtensorMap &ta, const CUtensorMap &tb,
                    const CUtensorMap &tc, const GemmParams &gp, cudaStream_t stream)
 {
-    if (v.family == kUmmaPair)
+    if (v.family == kUmmaPair) {
+        if (v.alt_ring)
+            return bf ? launch_umma_pair<6, 1, true>(dev, ta, tb, tc, gp, stream)
+                      : launch_umma_pair<6, 1, false>(dev, ta, tb, tc, gp, stream);
         return bf ? launch_umma_pair<3, 2, true>(dev, ta, tb, tc, gp, stream)
                   : launch_umma_pair<3, 2, false>(dev, ta, tb, tc, gp, stream);
+    }
     if (v.per_sm == 2) {
         if (v.block_n == 64)
             return bf ? launch_umma<64, 2, 1, true>(dev, 11, ta, tb, tc, gp, stream)
                       : launch_umma<64, 2, 1, false>(dev, 12, ta, tb, tc, gp, stream);
         return bf ? launch_umma<128, 2, 1, true>(dev, 13, ta, tb, tc, gp, stream)
                   : launch_umma<128, 2, 1, false>(dev, 14, ta, tb, tc, gp, stream);
+    }
+    if (v.alt_ring) {
+        if (v.block_n == 128)
+            return bf ? launch_umma<128, 6, 1, true>(dev, 24, ta, tb, tc, gp, stream)
+                      : launch_umma<128, 6, 1, false>(dev, 25, ta, tb, tc, gp, stream);
+        return bf ? launch_umma<256, 2, 2, true>(dev, 26, ta, tb, tc, gp, stream)
+                  : launch_umma<256, 2, 2, false>(dev, 27, ta, tb, tc, gp, stream);
     }
     switch (v.block_n) {
     case 64:  return bf ? launch_umma<64, 4, 2, true>(dev, 0, ta, tb, tc, gp, stream)
@@ -755,9 +834,15 @@ int launch_variant(int dev, const Variant &v, bool bf, const CUtensorMap &ta, co
                         : launch_umma<256, 4, 1, false>(dev, 5, ta, tb, tc, gp, stream);
     }
 }
+int prepare_pair(int dev, const Variant &v, bool bf)
+{
+    if (v.alt_ring) return bf ? prepare_umma_pair<6, 1, true>(dev, 28) : prepare_umma_pair<6, 1, false>(dev, 29);
+    return bf ? prepare_umma_pair<3, 2, true>(dev, 6) : prepare_umma_pair<3, 2, false>(dev, 7);
+}
 
-// Fills the kernel parameters that depend only on the problem and the tiling.
-GemmParams make_params(const Problem &p, const Tiling &t, int a_box_rows)
+// Fills the kernel parameters that depend only on the problem and the tiling.  `group` = the
+// raster-group knob of the variant code (0 = the rule below).
+GemmParams make_params(const Problem &p, const Tiling &t, int a_box_rows, int group_knob = 0)
 {
     GemmParams gp{};
     gp.C = p.C;
@@ -769,6 +854,7 @@ GemmParams make_params(const Problem &p, const Tiling &t, int a_box_rows)
     // (half of what one L2 partition holds), so that it stays resident while B streams by
     const int64_t tile_rows = cdiv(p.M, t.tiles_m);
     int64_t group = (int64_t(32) << 20) / (tile_rows * p.K * 2 + 1);
+    if (group_knob > 0) group = int64_t(1) << (group_knob - 1);
     if (group < 1) group = 1;
     if (group > t.tiles_m) group = t.tiles_m;
     gp.group_m = (int)group;
@@ -807,18 +893,19 @@ void set_split_epoch(GemmParams &gp, DeviceState &d, bool split)
     if (split && g_skew_next_flags.exchange(0)) gp.flag_post = gp.epoch ^ 0x40000000;
 }
 
-int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
+int run_umma(int dev, int code, const Problem &p, cudaStream_t stream)
 {
     DeviceState &d = g_dev[dev];
+    const Variant &v = g_variants[code_base(code)];
     const bool pair = v.family == kUmmaPair;
     const bool bf = p.out_dtype == CUDALLM_BF16;
     int st;
     if (pair) {
-        st = bf ? prepare_umma_pair<3, 2, true>(dev, 6) : prepare_umma_pair<3, 2, false>(dev, 7);
+        st = prepare_pair(dev, v, bf);
         if (st != CUDALLM_OK) return st;
     }
     const int slots = pair ? d.max_pairs : d.sm_count * (v.per_sm == 2 ? 2 : 1);
-    const Tiling t = tiling_for(v, p, slots);
+    const Tiling t = tiling_for(v, p, slots, code_tail(code));
     if (t.helper_tiles > kMaxHelperTiles || t.partial_bytes > kMaxPartialBytes)
         return CUDALLM_ERR_UNSUPPORTED_SHAPE;
 
@@ -853,7 +940,7 @@ int run_umma(int dev, const Variant &v, const Problem &p, cudaStream_t stream)
     st = encode_operand_map(dev, &tb, B, p.N, p.K, p.batch, ldb, sB, 64, kBlockK);
     if (st != CUDALLM_OK) return st;
 
-    GemmParams gp = make_params(p, t, a_box_rows);
+    GemmParams gp = make_params(p, t, a_box_rows, code_group(code));
     CUtensorMap tc;
     st = encode_c_map(dev, &tc, p, gp.c_tma != 0);
     if (st != CUDALLM_OK) return st;
@@ -869,10 +956,9 @@ int run(int variant, const Problem &p, void *stream_v)
     build_variants();
     int st = validate(p);
     if (st != CUDALLM_OK) return st;
-    if (variant != CUDALLM_VARIANT_AUTO && (variant < 0 || variant >= kNumVariants))
-        return CUDALLM_ERR_INVALID_VARIANT;
+    if (variant != CUDALLM_VARIANT_AUTO && !code_valid(variant)) return CUDALLM_ERR_INVALID_VARIANT;
     if (is_empty(p)) return CUDALLM_OK;
-    if (variant != CUDALLM_VARIANT_AUTO && !variant_supports(g_variants[variant], p))
+    if (variant != CUDALLM_VARIANT_AUTO && !variant_supports(g_variants[code_base(variant)], p))
         return CUDALLM_ERR_UNSUPPORTED_SHAPE;
 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
@@ -885,10 +971,10 @@ int run(int variant, const Problem &p, void *stream_v)
     // A stream with a workspace of its own declares that other launches may share the GPU:
     // the automatic choice then keeps to variants whose CTAs never wait for one another.
     if (variant == CUDALLM_VARIANT_AUTO) variant = select_variant(p, stream_has_workspace(g_dev[dev], stream));
-    const Variant &v = g_variants[variant];
+    const Variant &v = g_variants[code_base(variant)];
     if (!variant_supports(v, p)) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
     if (v.family == kSimt) return launch_simt(p, stream);
-    return run_umma(dev, v, p, stream);       // both tcgen05 families
+    return run_umma(dev, variant, p, stream);  // both tcgen05 families
 }
 
 Problem make_problem(const void *A, const void *B, void *C, int64_t M, int64_t N, int64_t K, int64_t lda,
@@ -952,7 +1038,7 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
     const Problem p = make_problem(A, B, C, M, N, K, lda, ldb, ldc, 0, 0, 0, 1, CUDALLM_F32);
     int st = validate(p);
     if (st != CUDALLM_OK) return st;
-    if (variant != CUDALLM_VARIANT_AUTO && (variant < 1 || variant >= kNumVariants))
+    if (variant != CUDALLM_VARIANT_AUTO && (!code_valid(variant) || code_base(variant) < 1))
         return CUDALLM_ERR_INVALID_VARIANT;
     if (is_empty(p)) return CUDALLM_OK;
     if (K > 0 && ((reinterpret_cast<uintptr_t>(A) & 3) || (reinterpret_cast<uintptr_t>(B) & 3)))
@@ -964,7 +1050,7 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
     q.K = 6 * round_up(K > 0 ? K : 1, kBlockK);
     q.lda = q.K;
     if (variant == CUDALLM_VARIANT_AUTO) variant = select_variant(q);
-    const Variant &v = g_variants[variant];
+    const Variant &v = g_variants[code_base(variant)];
     if (v.family == kSimt || !variant_supports(v, q)) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
@@ -977,7 +1063,7 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
     DeviceState &d = g_dev[dev];
     const bool pair = v.family == kUmmaPair;
     if (pair) {
-        st = prepare_umma_pair<3, 2, false>(dev, 7);
+        st = prepare_pair(dev, v, false);
         if (st != CUDALLM_OK) return st;
     }
     if (K == 0) {
@@ -986,7 +1072,7 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
         z.A = z.B = C;
         return launch_simt(z, stream);
     }
-    const Tiling t = tiling_for(v, q, pair ? d.max_pairs : d.sm_count);
+    const Tiling t = tiling_for(v, q, pair ? d.max_pairs : d.sm_count * (v.per_sm == 2 ? 2 : 1), code_tail(variant));
     if (t.helper_tiles > kMaxHelperTiles || t.partial_bytes > kMaxPartialBytes)
         return CUDALLM_ERR_UNSUPPORTED_SHAPE;
 
@@ -1025,7 +1111,7 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
     st = encode_operand_map(dev, &tb, ws + off_b, N, K, 3, ldbp, K * ldbp, 64, kBlockK);
     if (st != CUDALLM_OK) return st;
 
-    GemmParams gp = make_params(p, t, a_box_rows);
+    GemmParams gp = make_params(p, t, a_box_rows, code_group(variant));
     CUtensorMap tc;
     st = encode_c_map(dev, &tc, p, gp.c_tma != 0);
     if (st != CUDALLM_OK) return st;
@@ -1265,19 +1351,39 @@ int cudallm_num_variants(void)
 const char *cudallm_variant_name(int variant)
 {
     build_variants();
-    if (variant < 0 || variant >= kNumVariants) return nullptr;
-    return g_variants[variant].name;
+    if (!code_valid(variant)) return nullptr;
+    return g_variants[code_base(variant)].name;
+}
+
+static int compose_code(int variant, int group_rows, int tail_parts)
+{
+    if (variant < 0 || variant >= kNumVariants) return CUDALLM_ERR_INVALID_VARIANT;
+    int g = 0;
+    if (group_rows != 0) {
+        if (group_rows < 0 || group_rows > 16384 || (group_rows & (group_rows - 1))) return CUDALLM_ERR_INVALID_VARIANT;
+        while ((1 << g) < group_rows) ++g;
+        ++g;
+    }
+    if (tail_parts != 0 && (tail_parts < 2 || tail_parts > 7)) return CUDALLM_ERR_INVALID_VARIANT;
+    if (tail_parts != 0 && g_variants[variant].split_k != kTailSplit) return CUDALLM_ERR_INVALID_VARIANT;
+    return variant | (g << 8) | (tail_parts << 12);
+}
+
+int cudallm_variant_code(int variant, int group_rows, int tail_parts)
+{
+    build_variants();
+    return compose_code(variant, group_rows, tail_parts);
 }
 
 int cudallm_variant_supports(int variant, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
                              int64_t ldc, int64_t batch, int out_dtype)
 {
     build_variants();
-    if (variant < 0 || variant >= kNumVariants) return CUDALLM_ERR_INVALID_VARIANT;
+    if (!code_valid(variant)) return CUDALLM_ERR_INVALID_VARIANT;
     Problem p = shape_problem(M, N, K, lda, ldb, ldc, batch, out_dtype);
     int st = validate(p);
     if (st != CUDALLM_OK) return st;
-    return variant_supports(g_variants[variant], p) ? 1 : 0;
+    return variant_supports(g_variants[code_base(variant)], p) ? 1 : 0;
 }
 
 int cudallm_select_variant(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,
@@ -1296,23 +1402,35 @@ static int dispatch_key_status(int64_t M, int64_t N, int64_t K, int64_t batch, i
     return CUDALLM_OK;
 }
 
+static int dispatch_store(std::unordered_map<DispatchKey, int, DispatchHash> &table, const DispatchKey &key, int variant)
+{
+    if (variant != -1 && !code_valid(variant)) return CUDALLM_ERR_INVALID_VARIANT;
+    std::lock_guard<std::mutex> lock(g_dispatch_mutex);
+    if (variant < 0) {
+        table.erase(key);
+    } else {
+        if (table.size() >= kMaxDispatchEntries && table.find(key) == table.end()) return CUDALLM_ERR_TOO_LARGE;
+        table[key] = variant;
+    }
+    g_dispatch_generation.fetch_add(1, std::memory_order_release);
+    return CUDALLM_OK;
+}
+
 int cudallm_dispatch_set(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int variant)
 {
     build_variants();
     const int st = dispatch_key_status(M, N, K, batch, out_dtype);
     if (st != CUDALLM_OK) return st;
-    if (variant < -1 || variant >= kNumVariants) return CUDALLM_ERR_INVALID_VARIANT;
-    const DispatchKey key{M, N, K, batch, out_dtype};
-    std::lock_guard<std::mutex> lock(g_dispatch_mutex);
-    if (variant < 0) {
-        g_dispatch.erase(key);
-    } else {
-        if (g_dispatch.size() >= kMaxDispatchEntries && g_dispatch.find(key) == g_dispatch.end())
-            return CUDALLM_ERR_TOO_LARGE;
-        g_dispatch[key] = variant;
-    }
-    g_dispatch_generation.fetch_add(1, std::memory_order_release);
-    return CUDALLM_OK;
+    return dispatch_store(g_dispatch, DispatchKey{M, N, K, batch, out_dtype}, variant);
+}
+
+int cudallm_dispatch_set_class(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int tma_addressable,
+                               int variant)
+{
+    build_variants();
+    const int st = dispatch_key_status(M, N, K, batch, out_dtype);
+    if (st != CUDALLM_OK) return st;
+    return dispatch_store(g_dispatch_class, class_key(M, N, K, batch, out_dtype, tma_addressable != 0), variant);
 }
 
 int cudallm_dispatch_get(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int *variant)
@@ -1326,13 +1444,65 @@ int cudallm_dispatch_get(int64_t M, int64_t N, int64_t K, int64_t batch, int out
     return CUDALLM_OK;
 }
 
+int cudallm_dispatch_get_class(int64_t M, int64_t N, int64_t K, int64_t batch, int out_dtype, int tma_addressable,
+                               int *variant)
+{
+    const int st = dispatch_key_status(M, N, K, batch, out_dtype);
+    if (st != CUDALLM_OK) return st;
+    if (!variant) return CUDALLM_ERR_INVALID_POINTER;
+    std::lock_guard<std::mutex> lock(g_dispatch_mutex);
+    const auto it = g_dispatch_class.find(class_key(M, N, K, batch, out_dtype, tma_addressable != 0));
+    *variant = it == g_dispatch_class.end() ? -1 : it->second;
+    return CUDALLM_OK;
+}
+
 int cudallm_dispatch_clear(void)
 {
     std::lock_guard<std::mutex> lock(g_dispatch_mutex);
-    const int n = (int)g_dispatch.size();
+    const int n = (int)(g_dispatch.size() + g_dispatch_class.size());
     g_dispatch.clear();
+    g_dispatch_class.clear();
     g_dispatch_generation.fetch_add(1, std::memory_order_release);
     return n;
+}
+
+// The winners of the search as recorded on a B200 (generated from the package's table file
+// when the library is built): entered as class entries when the library is first used.
+struct PackagedEntry {
+    long long M, N, K, batch;
+    int out_dtype, tma_addressable;
+    const char *variant;
+    int group_rows, tail_parts;
+};
+static const PackagedEntry kPackaged[] = {
+#include "tuned_table.inc"
+    {0, 0, 0, 0, 0, 0, nullptr, 0, 0}
+};
+
+}  // extern "C"
+namespace {
+int load_packaged_entries()
+{
+    int n = 0;
+    for (const PackagedEntry *e = kPackaged; e->variant; ++e) {
+        int base = -1;
+        for (int v = 0; v < kNumVariants; ++v)
+            if (!strcmp(g_variants[v].name, e->variant)) base = v;
+        const int code = compose_code(base, e->group_rows, e->tail_parts);
+        if (code < 0 || dispatch_key_status(e->M, e->N, e->K, e->batch, e->out_dtype) != CUDALLM_OK) continue;
+        if (dispatch_store(g_dispatch_class, class_key(e->M, e->N, e->K, e->batch, e->out_dtype, e->tma_addressable != 0),
+                           code) == CUDALLM_OK)
+            ++n;
+    }
+    return n;
+}
+}  // namespace
+extern "C" {
+
+int cudallm_dispatch_load_packaged(void)
+{
+    build_variants();
+    return load_packaged_entries();
 }
 
 size_t cudallm_workspace_bytes(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,

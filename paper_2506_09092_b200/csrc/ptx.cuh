@@ -303,8 +303,7 @@ __device__ __forceinline__ uint32_t umma_stage_step(uint32_t next_bar, uint32_t 
 
 // Producer step for one stage of `nsub` (1 or 2) k-blocks: arm `full_bar` with
 // `tx_bytes` (if arm != 0); per k-block load one box of A and `boxes` boxes of
-// B (64 columns wide, 8 KB apart in shared memory; up to 4 for the first
-// k-block, up to 2 for the second).  The second k-block's tiles lie
+// B (64 columns wide, 8 KB apart in shared memory; up to 4 per k-block).  The second k-block's tiles lie
 // `sub_bytes` after the first's.  Returns 1 if `next_bar` has completed phase
 // `next_parity`.  `signal_bar` is where the loads complete their bytes (the
 // leader's barrier for CTA pairs).
@@ -321,8 +320,8 @@ __device__ __forceinline__ uint32_t tma_stage_step(uint32_t next_bar, uint32_t n
 #define CUDALLM_TMA_STEP(TESTW, TRYW, LOAD)                                                        \
     asm volatile(                                                                                  \
         "{\n\t"                                                                                    \
-        ".reg .pred pn, pa, p1, p2, p3, q0, q1;\n\t"                                               \
-        ".reg .b32 c1, c2, c3, s1, s2, s3, k1, ta1, tb1, tb2;\n\t"                                 \
+        ".reg .pred pn, pa, p1, p2, p3, q0, q1, q2, q3;\n\t"                                       \
+        ".reg .b32 c1, c2, c3, s1, s2, s3, k1, ta1, tb1, tb2, tb3, tb4;\n\t"                       \
         TESTW " pn, [%1], %2;\n\t"                                                                 \
         "setp.ne.b32 pa, %4, 0;\n\t"                                                               \
         "setp.gt.s32 p1, %15, 1;\n\t"                                                              \
@@ -330,9 +329,12 @@ __device__ __forceinline__ uint32_t tma_stage_step(uint32_t next_bar, uint32_t n
         "setp.gt.s32 p3, %15, 3;\n\t"                                                              \
         "setp.gt.s32 q0, %16, 1;\n\t"                                                              \
         "and.pred q1, q0, p1;\n\t"                                                                 \
+        "and.pred q2, q0, p2;\n\t"                                                                 \
+        "and.pred q3, q0, p3;\n\t"                                                                 \
         "add.s32 c1, %13, 64;\n\t add.s32 c2, %13, 128;\n\t add.s32 c3, %13, 192;\n\t"           \
         "add.u32 s1, %10, 8192;\n\t add.u32 s2, %10, 16384;\n\t add.u32 s3, %10, 24576;\n\t"     \
         "add.s32 k1, %11, 64;\n\t add.u32 ta1, %9, %17;\n\t add.u32 tb1, %10, %17;\n\t add.u32 tb2, s1, %17;\n\t" \
+        "add.u32 tb3, s2, %17;\n\t add.u32 tb4, s3, %17;\n\t"                                    \
         "@pa mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %5;\n\t"                           \
         LOAD " [%9], [%7, {%11, %12, %14}], [%6];\n\t"                                             \
         LOAD " [%10], [%8, {%13, %11, %18}], [%6];\n\t"                                            \
@@ -342,6 +344,8 @@ __device__ __forceinline__ uint32_t tma_stage_step(uint32_t next_bar, uint32_t n
         "@q0 " LOAD " [ta1], [%7, {k1, %12, %14}], [%6];\n\t"                                      \
         "@q0 " LOAD " [tb1], [%8, {%13, k1, %18}], [%6];\n\t"                                      \
         "@q1 " LOAD " [tb2], [%8, {c1, k1, %18}], [%6];\n\t"                                       \
+        "@q2 " LOAD " [tb3], [%8, {c2, k1, %18}], [%6];\n\t"                                       \
+        "@q3 " LOAD " [tb4], [%8, {c3, k1, %18}], [%6];\n\t"                                       \
         "@pn bra LDONE;\n\t"                                                                       \
         TRYW " pn, [%1], %2;\n\t"                                                                  \
         "LDONE:\n\t"                                                                               \

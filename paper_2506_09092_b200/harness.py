@@ -289,10 +289,30 @@ def compare_closed_form(case: ClosedFormCase, out):
     return True, 0.0, ""
 
 
-def search_config(cfg, candidates=None, iters: int = 10, passes: int = 3, cases=None) -> SearchResult:
+def knob_candidates(base: int, tiles_m: int):
+    """Variant codes that add the two search knobs to ``base``: raster groups of 1, 2, 4, ... tile
+    rows (while a group is smaller than the matrix), and for the tail-splitting variants the
+    number of parts."""
+    from . import binding as B
+    out = []
+    g = 1
+    while g < max(2, tiles_m) and g <= 64:
+        out.append(B.variant_code(base, g, 0))
+        g *= 2
+    if B.variant_name(base).endswith("_ts"):
+        out += [B.variant_code(base, 0, t) for t in (2, 3, 6)]
+    return out
+
+
+def search_config(cfg, candidates=None, iters: int = 10, passes: int = 3, cases=None, knobs: bool = False,
+                  top: int = 3) -> SearchResult:
     """Algorithm 1's round over the library's variants for one configuration:
     validate every candidate on seeded closed-form cases, time the valid ones
-    (interleaved passes, median), keep the fastest."""
+    (interleaved passes, median), keep the fastest.  With ``knobs`` a second round
+    widens the candidate set around the ``top`` fastest variants: the same kernels
+    with other raster-group heights and tail-split depths (variant codes), which
+    are validated and timed the same way; a code replaces its plain variant only
+    if it is more than 1 % faster (timing noise)."""
     import statistics
     from . import binding as B
     if candidates is None:
@@ -312,23 +332,36 @@ def search_config(cfg, candidates=None, iters: int = 10, passes: int = 3, cases=
     prob = DeviceProblem(cfg)
     samples = {}
 
-    def profile(v):
-        return samples[v]
+    def time_round(todo):
+        for v in todo:
+            samples[v] = []
+        for _ in range(passes):
+            for v in todo:
+                t = performance_profiler(lambda i: prob.launch(i, v), iters=iters, warmup=2)
+                samples[v].append(t["median_s"])
+        for v in todo:
+            samples[v] = statistics.median(samples[v])
 
     res = SearchResult(best=None, best_latency=float("inf"))
     for v in candidates:
         res.reports[v] = function_validator(v, cases, run, compare)
         if res.reports[v].ok:
             res.valid.append(v)
-    for v in res.valid:
-        samples[v] = []
-    for _ in range(passes):
-        for v in res.valid:
-            t = performance_profiler(lambda i: prob.launch(i, v), iters=iters, warmup=2)
-            samples[v].append(t["median_s"])
-    for v in res.valid:
-        samples[v] = statistics.median(samples[v])
-    timed = search(res.valid, lambda v: res.reports[v], profile)
+    time_round(res.valid)
+    if knobs and res.valid:
+        leaders = sorted(res.valid, key=lambda v: samples[v])[:top]
+        tiles_m = -(-cfg.M // 128)
+        extra = [c for v in leaders for c in knob_candidates(v, tiles_m)]
+        ok_extra = []
+        for c in extra:
+            res.reports[c] = function_validator(c, cases, run, compare)
+            if res.reports[c].ok:
+                ok_extra.append(c)
+        time_round(ok_extra + leaders)                  # the leaders again, in the same round
+        for c in ok_extra:
+            if samples[c] < 0.99 * samples[c & 0xFF]:
+                res.valid.append(c)
+    timed = search(res.valid, lambda v: res.reports[v], lambda v: samples[v])
     timed.reports = res.reports
     return timed
 
@@ -344,9 +377,17 @@ class TunedTable:
     def key(M, N, K, batch, out_dtype):
         return f"{M}x{N}x{K}x{batch}:{'bf16' if out_dtype == 1 else 'f32'}"
 
-    def record(self, cfg, variant_name, latency_s):
-        self.entries[self.key(cfg.M, cfg.N, cfg.K, cfg.batch, cfg.out_dtype)] = {
-            "variant": variant_name, "us": round(latency_s * 1e6, 2)}
+    def record(self, cfg, code, latency_s):
+        """Enter the winner (a variant id or code) for the configuration's shape."""
+        from . import binding as B
+        g, t = (code >> 8) & 0xF, (code >> 12) & 0x7
+        tma = cfg.lda_ % 8 == 0 and cfg.ldb_ % 8 == 0 and (cfg.batch == 1 or (cfg.strideA % 8 == 0 and cfg.strideB % 8 == 0))
+        rec = {"variant": B.variant_name(code), "us": round(latency_s * 1e6, 2), "tma": bool(tma)}
+        if g:
+            rec["group"] = 1 << (g - 1)
+        if t:
+            rec["tail"] = t
+        self.entries[self.key(cfg.M, cfg.N, cfg.K, cfg.batch, cfg.out_dtype)] = rec
 
     def lookup(self, M, N, K, batch, out_dtype):
         e = self.entries.get(self.key(M, N, K, batch, out_dtype))
@@ -374,9 +415,10 @@ class TunedTable:
             return cls(json.load(f))
 
     def install(self) -> int:
-        """Enter every record into the library's dispatch table (``cudallm_dispatch_set``), so
-        that its automatic choice uses the searched winners; returns how many were entered
-        (records that name a variant this build does not have are skipped)."""
+        """Enter every record into the library's dispatch tables (``cudallm_dispatch_set_class``: the
+        record's shape stands for all shapes that are tiled like it), so that its automatic
+        choice uses the searched winners; returns how many were entered (records that name a
+        variant this build does not have are skipped)."""
         from . import binding as B
         names = {B.variant_name(v): v for v in range(B.num_variants())}
         n = 0
@@ -386,7 +428,8 @@ class TunedTable:
             v = names.get(rec["variant"])
             if v is None:
                 continue
-            B.dispatch_set(M, N, K, batch, B.BF16 if dtype == "bf16" else B.F32, v)
+            code = B.variant_code(v, rec.get("group", 0), rec.get("tail", 0))
+            B.dispatch_set_class(M, N, K, batch, B.BF16 if dtype == "bf16" else B.F32, rec.get("tma", True), code)
             n += 1
         return n
 
@@ -398,28 +441,43 @@ class TunedTable:
         return cls.load(os.path.join(os.path.dirname(os.path.abspath(__file__)), "tuned_b200.json"))
 
 
-def _search_one(cfg, iters, table_path):
-    """Validate and time every variant on one configuration; print one JSON line per variant
+def search_grid():
+    """Shapes beyond the benchmark configurations that the packaged table covers: M from 16 to
+    8192 against eight N x K pairs (bf16 output), plus a few irregular ones."""
+    from . import inputs as gi
+    shapes = []
+    for (N, K) in [(4096, 4096), (11008, 4096), (4096, 11008), (8192, 8192), (18944, 4096), (1024, 8192),
+                   (2048, 2048), (6144, 3072)]:
+        for M in (16, 128, 256, 512, 1024, 2048, 4096, 8192):
+            if M * N * K <= 6e11:
+                shapes.append((M, N, K))
+    shapes += [(777, 3333, 1111), (1000, 1000, 1000), (5000, 5000, 512), (300, 20000, 256), (20000, 300, 2048)]
+    return [gi.GemmConfig(f"G{M}x{N}x{K}", M, N, K, gi.BF16, seed=900 + i) for i, (M, N, K) in enumerate(shapes)]
+
+
+def _search_one(cfg, iters, table_path, knobs=True, cases=None, passes=3):
+    """Validate and time every variant on one configuration; print one JSON line per candidate
     (validation outcome: ok / mismatch / launch error / device timeout) and the winner; record
     the winner in the table file if one is given."""
     import json
     import os
     from . import binding as B
 
-    res = search_config(cfg, iters=iters)
+    res = search_config(cfg, iters=iters, knobs=knobs, cases=cases, passes=passes)
     for v, rep in res.reports.items():
-        print(json.dumps({"config": cfg.name, "variant": B.variant_name(v), "validation": rep.status,
+        print(json.dumps({"config": cfg.name, "candidate": B.describe_code(v), "validation": rep.status,
                           "detail": rep.detail,
-                          "us": None if v not in res.latencies else res.latencies[v] * 1e6}), flush=True)
-    best = None if res.best is None else B.variant_name(res.best)
-    print(json.dumps({"config": cfg.name, "best": best,
-                      "us": None if res.best is None else res.best_latency * 1e6,
-                      "library_choice": B.variant_name(B.select_variant(
-                          cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype))}),
+                          "us": None if v not in res.latencies else round(res.latencies[v] * 1e6, 2)}), flush=True)
+    best = None if res.best is None else B.describe_code(res.best)
+    choice = B.select_variant(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype)
+    print(json.dumps({"config": cfg.name, "shape": [cfg.M, cfg.N, cfg.K, cfg.batch], "best": best,
+                      "us": None if res.best is None else round(res.best_latency * 1e6, 2),
+                      "library_choice": B.describe_code(choice),
+                      "library_choice_us": None if choice not in res.latencies else round(res.latencies[choice] * 1e6, 2)}),
           flush=True)
     if table_path and res.best is not None:
         table = TunedTable.load(table_path) if os.path.exists(table_path) else TunedTable()
-        table.record(cfg, best, res.best_latency)
+        table.record(cfg, res.best, res.best_latency)
         table.save(table_path)
 
 
@@ -436,8 +494,12 @@ def _main(argv=None):
     ap = argparse.ArgumentParser()
     ladder = {f"T2-{k + 1}": gi.task2_ladder(k) for k in range(5)}     # the paper's Task 2 sizes
     all_configs = dict(gi.CONFIGS, **ladder)
-    ap.add_argument("--config", default="C2", choices=sorted(all_configs) + ["all"],
-                    help="a benchmark configuration, a size of the paper's Task 2 ladder, or (with --search) all")
+    ap.add_argument("--config", default="C2", choices=sorted(all_configs) + ["all", "grid"],
+                    help="a benchmark configuration, a size of the paper's Task 2 ladder, or (with --search) all of "
+                         "those / the grid of other shapes that the packaged table covers")
+    ap.add_argument("--no-knobs", action="store_true", help="with --search: plain variants only")
+    ap.add_argument("--model-only", action="store_true",
+                    help="empty the dispatch tables first, so that the cost model alone chooses")
     ap.add_argument("--variant", default="auto")
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
@@ -456,17 +518,27 @@ def _main(argv=None):
     args = ap.parse_args(argv)
     if args.task:
         return _task_main(args)
+    if args.model_only:
+        B.dispatch_clear()
     if args.dispatch:
         table = TunedTable.packaged() if args.dispatch == "packaged" else TunedTable.load(args.dispatch)
         table.install()
     if args.search:
+        if args.config == "grid":
+            # the candidates' arithmetic does not depend on the shape: two ragged cases and the shape itself
+            for cfg in search_grid():
+                cases = default_cases()[:2] + [ClosedFormCase(f"{cfg.name}-shape", cfg.M, cfg.N, cfg.K, cfg.out_dtype, 7)]
+                _search_one(cfg, args.iters, args.table, not args.no_knobs, cases=cases, passes=2)
+            return
         for name in (sorted(all_configs) if args.config == "all" else [args.config]):
-            if args.config == "all" and all_configs[name].flops > 2e12:
-                continue                                   # the largest ladder size: minutes of validation
-            _search_one(all_configs[name], args.iters, args.table)
+            cfg = all_configs[name]
+            cases = None
+            if cfg.flops > 2e12:                           # the largest ladder size: skip the shape-sized case
+                cases = default_cases()
+            _search_one(cfg, args.iters, args.table, not args.no_knobs, cases=cases)
         return
-    if args.config == "all":
-        ap.error("--config all needs --search")
+    if args.config in ("all", "grid"):
+        ap.error("--config all / grid needs --search")
     cfg = all_configs[args.config]
     names = {B.variant_name(v): v for v in range(B.num_variants())}
     prob = DeviceProblem(cfg, nsets=args.sets)
@@ -481,7 +553,7 @@ def _main(argv=None):
     for v in todo:
         t = performance_profiler(lambda i: prob.launch(i, v), iters=args.iters, warmup=args.warmup)
         code, detail = B.device_status(torch.cuda.current_stream())
-        print(json.dumps({"config": cfg.name, "variant": B.variant_name(v), "status": code,
+        print(json.dumps({"config": cfg.name, "variant": B.describe_code(v), "status": code,
                           "us_min": t["min_s"] * 1e6, "us_median": t["median_s"] * 1e6,
                           "tflops": cfg.flops / t["median_s"] / 1e12,
                           "gbs": cfg.algorithmic_bytes / t["median_s"] / 1e9}), flush=True)

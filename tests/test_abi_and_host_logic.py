@@ -184,15 +184,19 @@ def test_function_validator_failure_classes():
 
 
 def test_tuned_table_roundtrip(tmp_path):
+    names = {B.variant_name(v): v for v in range(B.num_variants())}
     t = H.TunedTable()
-    t.record(gi.CONFIGS["C2"], "umma2_n256_ts", 98.7e-6)
-    t.record(gi.CONFIGS["C4"], "umma_n128", 14.4e-6)
+    t.record(gi.CONFIGS["C2"], B.variant_code(names["umma2_n256_ts"], 4, 3), 98.7e-6)
+    t.record(gi.CONFIGS["C4"], names["umma_n128"], 14.4e-6)
+    t.record(gi.CONFIGS["C5b"], names["umma2_n256"], 70e-6)
     path = tmp_path / "tuned.json"
     t.save(path)
     u = H.TunedTable.load(path)
+    assert u.entries[H.TunedTable.key(4096, 4096, 4096, 1, 1)] == {"variant": "umma2_n256_ts", "us": 98.7, "tma": True,
+                                                                  "group": 4, "tail": 3}
+    assert u.entries[H.TunedTable.key(3001, 1999, 5003, 1, 0)]["tma"] is False     # odd pitches
     assert u.lookup(4096, 4096, 4096, 1, 1) == "umma2_n256_ts"
     assert u.lookup(4096, 4096, 4096, 1, 0) is None            # other output type: not tuned
-    names = {B.variant_name(v): v for v in range(B.num_variants())}
     assert u.variant_id(128, 128, 64, 512, 0, names) == names["umma_n128"]
     assert u.variant_id(1, 2, 3, 1, 0, names) == -1            # miss: the library chooses
     u.entries[H.TunedTable.key(5, 5, 5, 1, 0)] = {"variant": "no_such_kernel", "us": 1.0}
@@ -262,19 +266,82 @@ def test_dispatch_table_overrides_the_cost_model_for_its_shapes():
         assert B.dispatch_set(1, 1, 1, 1, B.F32, -2, check=False) == B.ERR_INVALID_VARIANT
     finally:
         B.dispatch_clear()
+        B.dispatch_load_packaged()
 
 
-def test_packaged_table_installs_into_the_dispatch_table():
+def test_variant_codes_carry_the_search_knobs():
+    names = {B.variant_name(v): v for v in range(B.num_variants())}
+    ts, plain = names["umma2_n256_ts"], names["umma_n128"]
+    assert B.variant_code(ts) == ts and B.describe_code(ts) == "umma2_n256_ts"
+    code = B.variant_code(ts, 8, 3)
+    assert code != ts and code & 0xFF == ts and B.variant_name(code) == "umma2_n256_ts"
+    assert B.describe_code(code) == "umma2_n256_ts+g8+t3"
+    assert B.variant_supports(code, 4096, 4096, 4096, 4096, 4096, 4096, 1, B.BF16) == 1
+    assert B.variant_code(plain, 0, 3, check=False) == B.ERR_INVALID_VARIANT      # not a tail-splitting variant
+    assert B.variant_code(plain, 3, 0, check=False) == B.ERR_INVALID_VARIANT      # not a power of two
+    assert B.variant_code(ts, 0, 8, check=False) == B.ERR_INVALID_VARIANT
+    assert B.variant_code(99, 0, 0, check=False) == B.ERR_INVALID_VARIANT
+    assert B.variant_name(1 << 20) is None
+    p = 4096
+    assert B.gemm_bf16_variant(1 << 20, p, p, p, 4, 4, 4, 4, 4, 4, 16, 16, 16, 1, 0, check=False) == B.ERR_INVALID_VARIANT
+    # the two arrangements of the shared-memory ring are separate candidates
+    for n in ("umma_n128_k1", "umma_n256_k2", "umma2_n256_k1", "umma2_n256_k1_ts"):
+        assert n in names
+
+
+def test_class_entries_cover_every_shape_that_is_tiled_alike():
+    """A class entry recorded for one shape is used for every shape with the same tile and
+    k-block counts (and only those); the exact-shape table wins over it; shapes whose operands
+    TMA cannot address form classes of their own."""
+    names = {B.variant_name(v): v for v in range(B.num_variants())}
+    try:
+        B.dispatch_clear()
+        model = B.select_variant(4000, 4090, 4050, 4056, 4096, 4096, 1, B.BF16)
+        code = B.variant_code(names["umma_n128_ts"] if model != names["umma_n128_ts"] else names["umma_n256_ts"], 2, 3)
+        B.dispatch_set_class(4096, 4096, 4096, 1, B.BF16, True, code)
+        assert B.dispatch_get_class(3969, 4033, 4090, 1, B.BF16, True) == code       # same ceilings
+        assert B.select_variant(4096, 4096, 4096, 4096, 4096, 4096, 1, B.BF16) == code
+        assert B.select_variant(4000, 4090, 4050, 4056, 4096, 4096, 1, B.BF16) == code
+        assert B.select_variant(4000, 4090, 4050, 4051, 4096, 4096, 1, B.BF16) != code    # lda odd: another class
+        assert B.select_variant(4096, 4096, 4097, 4104, 4096, 4096, 1, B.BF16) != code    # one more k-block
+        assert B.select_variant(4096, 4096, 4096, 4096, 4096, 4096, 1, B.F32) != code     # other output type
+        exact = names["umma2_n256"]
+        B.dispatch_set(4000, 4090, 4050, 1, B.BF16, exact)
+        assert B.select_variant(4000, 4090, 4050, 4056, 4096, 4096, 1, B.BF16) == exact
+        assert B.select_variant(4096, 4096, 4096, 4096, 4096, 4096, 1, B.BF16) == code
+        # short-A buckets are classes of their own
+        B.dispatch_set_class(16, 4096, 4096, 1, B.F32, True, names["umma_n128_sk2"])
+        assert B.dispatch_get_class(9, 4096, 4096, 1, B.F32, True) == names["umma_n128_sk2"]
+        assert B.dispatch_get_class(17, 4096, 4096, 1, B.F32, True) == -1
+        assert B.dispatch_set_class(16, 4096, 4096, 1, B.F32, True, -1) == B.OK
+        assert B.dispatch_get_class(9, 4096, 4096, 1, B.F32, True) == -1
+        assert B.dispatch_clear() == 2
+    finally:
+        B.dispatch_clear()
+        B.dispatch_load_packaged()
+
+
+def test_library_starts_with_the_packaged_winners():
+    """The packaged table is compiled into the library and entered at first use; clearing
+    removes it, cudallm_dispatch_load_packaged brings it back."""
     table = H.TunedTable.packaged()
     names = {B.variant_name(v): v for v in range(B.num_variants())}
     try:
         B.dispatch_clear()
-        assert table.install() == len(table.entries)
+        assert B.dispatch_load_packaged() == len(table.entries)
         for key, rec in table.entries.items():
             shape, dtype = key.split(":")
             M, N, K, batch = (int(x) for x in shape.split("x"))
             dt = B.BF16 if dtype == "bf16" else B.F32
-            assert B.dispatch_get(M, N, K, batch, dt) == names[rec["variant"]]
-            assert B.select_variant(M, N, K, K, N, N, batch, dt) == names[rec["variant"]]
+            code = B.variant_code(names[rec["variant"]], rec.get("group", 0), rec.get("tail", 0))
+            assert B.dispatch_get_class(M, N, K, batch, dt, rec.get("tma", True)) == code, key
+        B.dispatch_clear()
+        assert table.install() == len(table.entries)                     # the same through the Python table
+        for key, rec in table.entries.items():
+            shape, dtype = key.split(":")
+            M, N, K, batch = (int(x) for x in shape.split("x"))
+            dt = B.BF16 if dtype == "bf16" else B.F32
+            assert B.variant_name(B.dispatch_get_class(M, N, K, batch, dt, rec.get("tma", True))) == rec["variant"]
     finally:
         B.dispatch_clear()
+        B.dispatch_load_packaged()

@@ -50,7 +50,8 @@ def test_shape_grid(M):
     tile width (plus a split-K one where K allows)."""
     rng = np.random.default_rng(1000 + M)
     names = ["simt", "umma_n64", "umma_n128", "umma_n256", "umma_n64_sk2", "umma_n256_sk4",
-             "umma2_n256", "umma2_n256_sk2", "umma_n256_ts", "umma2_n256_ts", "umma_n64_x2", "umma_n128_x2"]
+             "umma2_n256", "umma2_n256_sk2", "umma_n256_ts", "umma2_n256_ts", "umma_n64_x2", "umma_n128_x2",
+             "umma_n128_k1", "umma_n256_k2_ts", "umma2_n256_k1", "umma2_n256_k1_ts"]
     for ni, N in enumerate(DIMS):
         for ki in range(3):
             K = KS[(ni * 3 + ki + M) % len(KS)]
@@ -74,7 +75,13 @@ def test_padded_leading_dimensions_and_offset_bases(pad, out_dtype):
         ref = oracle.gemm(A, Bm, M, N, K)
         lda, ldb, ldc = K + pad, N + pad, N + pad
         Ap, Bp = gi.embed(A, lda), gi.embed(Bm, ldb)       # NaN padding: reading it poisons C
-        for v in [B.VARIANT_AUTO] + variant_ids("simt", "umma_n128", "umma_n256_sk2", "umma2_n256", "umma2_n256_ts"):
+        ids = variant_ids("simt", "umma_n128", "umma_n256_sk2", "umma2_n256", "umma2_n256_ts", "umma_n256_k2",
+                          "umma2_n256_k1_ts")
+        # the same kernels with the search's knobs set: raster groups of one or two tile rows,
+        # the ragged last wave cut into up to two or six parts
+        ts = variant_ids("umma2_n256_ts", "umma_n128_ts")
+        codes = [B.variant_code(ts[0], 1, 2), B.variant_code(ts[1], 2, 6), B.variant_code(ids[1], 1, 0)]
+        for v in [B.VARIANT_AUTO] + ids + codes:
             if v >= 0 and B.variant_supports(v, M, N, K, lda, ldb, ldc, 1, out_dtype) != 1:
                 continue
             check_case(Ap, Bp, M, N, K, out_dtype, v, lda, ldb, ldc, ref=ref)
@@ -246,7 +253,7 @@ def test_power_of_two_scaling_bitwise_and_run_to_run_identical():
     A = bits(rng.standard_normal((M, K))); Bm = bits(rng.standard_normal((K, N)))
     for out_dtype in (gi.F32, gi.BF16):
         for v in [B.VARIANT_AUTO] + variant_ids("umma_n128", "umma_n256_sk4", "umma_n64_sk8", "umma2_n256_sk4",
-                                                "umma2_n256_ts"):
+                                                "umma2_n256_ts", "umma2_n256_k1_ts", "umma_n128_k1"):
             _, raw0, _ = G.run_gemm(A.ravel(), Bm.ravel(), M, N, K, K, N, N, out_dtype, variant=v)
             _, raw1, _ = G.run_gemm(A.ravel(), Bm.ravel(), M, N, K, K, N, N, out_dtype, variant=v)
             assert np.array_equal(raw0, raw1)                       # deterministic

@@ -122,8 +122,21 @@ def test_automatic_choice_follows_the_dispatch_table():
             r = oracle.check(vals[0], Cref, S, G.tol_for(gi.F32))
             assert guards and r.ok, (forced, r)
         assert B.select_variant(M, N, K + 1, K + 1, N, N, 1, gi.F32) != -1
+        # a class entry with knobs set: used for another shape of the same class, result still right
+        B.dispatch_clear()
+        code = B.variant_code(names["umma_n128_ts"], 1, 3)
+        B.dispatch_set_class(M, N, K, 1, gi.F32, True, code)
+        M2, N2, K2 = M - 3, N - 5, K - 5                              # same tile and k-block counts
+        A2 = bits(rng.standard_normal((M2, K2))); B2 = bits(rng.standard_normal((K2, N2)))
+        A2p, B2p = gi.embed(A2, K2 + 7), gi.embed(B2, N2 + 3)        # pitches that TMA can address
+        assert (K2 + 7) % 8 == 0 and (N2 + 3) % 8 == 0
+        assert B.select_variant(M2, N2, K2, K2 + 7, N2 + 3, N2, 1, gi.F32) == code
+        vals, raw, guards = G.run_gemm(A2p, B2p, M2, N2, K2, K2 + 7, N2 + 3, N2, gi.F32)
+        Cref2, S2 = oracle.gemm(A2, B2, M2, N2, K2)
+        assert guards and oracle.check(vals[0], Cref2, S2, G.tol_for(gi.F32)).ok
     finally:
         B.dispatch_clear()
+        B.dispatch_load_packaged()
 
 
 def test_bounded_wait_runs_out_and_the_library_recovers():
