@@ -345,7 +345,7 @@ def run_ours(args):
     cfg = gi.CONFIGS["C2"]
     A, Bm = cfg.make()
     prob = H.DeviceProblem(cfg, A, Bm, min_bytes=3.2 * L2_BYTES)
-    vname = B.variant_name(B.select_variant(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_,
+    vname = B.describe_code(B.select_variant(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_,
                                             cfg.batch, cfg.out_dtype))
     sampler = ClockSampler(local)
     total, kern_avg = time_steps(lambda i: prob.launch(i, stream=stream), args.steps, args.warmup,
@@ -365,7 +365,7 @@ def run_ours(args):
                                         args.sustained_seconds, peaks["bf16_tflops_sustained"], local, barrier)
         c3 = gi.CONFIGS["C3"]
         c3p = H.DeviceProblem(c3, nsets=1)             # one set is 338 MB > L2
-        c3_name = B.variant_name(B.select_variant(c3.M, c3.N, c3.K, c3.lda_, c3.ldb_, c3.ldc_, c3.batch, c3.out_dtype))
+        c3_name = B.describe_code(B.select_variant(c3.M, c3.N, c3.K, c3.lda_, c3.ldb_, c3.ldc_, c3.batch, c3.out_dtype))
         _, c3_avg = time_steps(lambda i: c3p.launch(i, stream=stream), 20, 3, barrier)
         sustained["C3"] = sustained_run(lambda i: c3p.launch(i, stream=stream), c3.flops, c3_avg,
                                         args.sustained_seconds, peaks["bf16_tflops_sustained"], local, barrier)
@@ -398,7 +398,7 @@ def run_ours(args):
     sk = gi.CONFIGS["C5a"]
     sA, sB = sk.make()
     skp = H.DeviceProblem(sk, sA, sB, min_bytes=2.2 * L2_BYTES)
-    sk_name = B.variant_name(B.select_variant(sk.M, sk.N, sk.K, sk.lda_, sk.ldb_, sk.ldc_, sk.batch,
+    sk_name = B.describe_code(B.select_variant(sk.M, sk.N, sk.K, sk.lda_, sk.ldb_, sk.ldc_, sk.batch,
                                               sk.out_dtype))
     sk_steps = max(args.steps, 20)
     sk_total, sk_avg = time_steps(lambda i: skp.launch(i, stream=stream), sk_steps, args.warmup, barrier)

@@ -127,7 +127,7 @@ def test_variant_support_rules():
 def test_selection_and_workspace_queries():
     for cfg in gi.CONFIGS.values():
         v = B.select_variant(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype)
-        assert 0 < v < B.num_variants()
+        assert 0 < (v & 0xFF) < B.num_variants() and B.variant_name(v) is not None      # an id or a code
         assert B.variant_supports(v, cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch,
                                   cfg.out_dtype) == 1
         ws = B.workspace_bytes(cfg.M, cfg.N, cfg.K, cfg.lda_, cfg.ldb_, cfg.ldc_, cfg.batch, cfg.out_dtype)

@@ -344,3 +344,29 @@ def test_short_a_boundaries(out_dtype):
                 if B.variant_supports(v, M, N, K, K, N, N, 1, out_dtype) != 1:
                     continue
                 check_case(A.ravel(), Bm.ravel(), M, N, K, out_dtype, v, ref=ref)
+
+
+@pytest.mark.parametrize("out_dtype", [gi.F32, gi.BF16])
+def test_large_unaligned_operands(out_dtype):
+    """Larger products whose operands TMA cannot address (repacked by the warp-per-row-piece
+    copy kernel): either operand or both unaligned (odd pitch, or a base two bytes off a
+    16-byte boundary), row lengths that end inside a 512-element piece or right after one,
+    lone-CTA, CTA-pair, split-K and tail-split kernels."""
+    rng = np.random.default_rng(606 + out_dtype)
+    cases = [(700, 900, 3000, 1, 3, 0, 0),        # (M, N, K, pad_a, pad_b, lead_a, lead_b)
+             (1300, 1000, 2100, 3, 0, 0, 0),      # only A unaligned
+             (520, 2100, 1800, 0, 5, 0, 0),       # only B unaligned
+             (640, 1024, 2560, 0, 0, 1, 1),       # pitches fine, bases 2 bytes off
+             (300, 513, 1025, 1, 1, 1, 0),        # one element past a 512-element piece
+             (200, 1536, 512, 3, 3, 0, 1)]        # rows end exactly on a piece boundary
+    names = ("umma_n64", "umma_n128_ts", "umma_n256_k2", "umma2_n256", "umma2_n256_ts", "umma2_n256_sk2",
+             "umma_n128_sk4")
+    for (M, N, K, pa, pb, la, lb) in cases:
+        A = bits(rng.standard_normal((M, K))); Bm = bits(rng.standard_normal((K, N)))
+        ref = oracle.gemm(A, Bm, M, N, K)
+        lda, ldb = K + pa, N + pb
+        Ap, Bp = gi.embed(A, lda), gi.embed(Bm, ldb)           # NaN padding
+        for v in [B.VARIANT_AUTO] + variant_ids(*names):
+            if v >= 0 and B.variant_supports(v, M, N, K, lda, ldb, N, 1, out_dtype) != 1:
+                continue
+            check_case(Ap, Bp, M, N, K, out_dtype, v, lda, ldb, N, ref=ref, lead_a=la, lead_b=lb)
