@@ -3,8 +3,7 @@
 //    alignment (bring-up cross-check on the device; also serves K == 0).
 //  * pack_rows_kernel  -- copies operands whose leading dimension or base
 //    is not 16-byte aligned into an aligned workspace so that TMA can read them
-//    (small or batched products; large single products repack inside the GEMM
-//    kernel, see row_copy.cuh).
+//    (the row copies themselves are in row_copy.cuh).
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>

@@ -1458,6 +1458,7 @@ int cudallm_dispatch_get_class(int64_t M, int64_t N, int64_t K, int64_t batch, i
 
 int cudallm_dispatch_clear(void)
 {
+    build_variants();                  // (the packaged entries are entered on first use: before, not after, this)
     std::lock_guard<std::mutex> lock(g_dispatch_mutex);
     const int n = (int)(g_dispatch.size() + g_dispatch_class.size());
     g_dispatch.clear();

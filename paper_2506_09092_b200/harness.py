@@ -331,13 +331,20 @@ def search_config(cfg, candidates=None, iters: int = 10, passes: int = 3, cases=
 
     prob = DeviceProblem(cfg)
     samples = {}
+    batch = {}
 
     def time_round(todo):
+        # every sample brackets enough back-to-back calls to last about 200 us: a short kernel is
+        # then timed as a stream of launches (what a caller's pipeline sees), not as one launch
+        # plus its latency
         for v in todo:
             samples[v] = []
+            if v not in batch:
+                est = performance_profiler(lambda i: prob.launch(i, v), iters=3, warmup=2)["median_s"]
+                batch[v] = max(1, min(64, int(math.ceil(200e-6 / max(est, 1e-7)))))
         for _ in range(passes):
             for v in todo:
-                t = performance_profiler(lambda i: prob.launch(i, v), iters=iters, warmup=2)
+                t = performance_profiler(lambda i: prob.launch(i, v), iters=iters, warmup=2, batch_calls=batch[v])
                 samples[v].append(t["median_s"])
         for v in todo:
             samples[v] = statistics.median(samples[v])
