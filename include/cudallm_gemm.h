@@ -347,14 +347,19 @@ int cudallm_shutdown(void);
  *   CUDALLM_DEBUG_WAIT_LIMIT_NS          value = the wall-clock limit of every
  *       in-kernel wait in nanoseconds (0 restores the default of 2 s).
  *   CUDALLM_DEBUG_MISS_NEXT_SPLIT_FLAGS  value != 0: the next launch that splits
- *       tiles along K raises its hand-over flags to a value that no unit waits
- *       for, so every such wait runs out after the limit; the kernel then
- *       returns normally, C is unspecified, and cudallm_device_status reports
- *       CUDALLM_ERR_DEVICE_TIMEOUT.  One launch only.
- * Returns CUDALLM_ERR_INVALID_VARIANT for an unknown `what`.
+ *       tiles along K (or the next one-pass cudallm_layernorm_f32 launch,
+ *       whichever comes first) raises its hand-over flags to a value that
+ *       nobody waits for, so every such wait runs out after the limit; the
+ *       kernel then returns normally, its output is unspecified, and
+ *       cudallm_device_status reports CUDALLM_ERR_DEVICE_TIMEOUT.  One launch only.
+ *   CUDALLM_DEBUG_LAYERNORM_PATH         value = 0: cudallm_layernorm_f32 picks its
+ *       kernel by size; 1: always the two-kernel path; 2: the one-pass kernel
+ *       whenever the samples fit in shared memory, however small.
+ * Returns CUDALLM_ERR_INVALID_VARIANT for an unknown `what` or value.
  */
 #define CUDALLM_DEBUG_WAIT_LIMIT_NS          1
 #define CUDALLM_DEBUG_MISS_NEXT_SPLIT_FLAGS  2
+#define CUDALLM_DEBUG_LAYERNORM_PATH         3
 int cudallm_debug_set(int what, unsigned long long value);
 
 /*

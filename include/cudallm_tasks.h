@@ -12,8 +12,8 @@
  * caller, pitches in elements, calls enqueue on `stream` and return without
  * synchronising, negative CUDALLM_ERR_* status codes, argument errors found
  * before any CUDA call, compute capability 10.0 only, no CPU fallback).  The
- * status codes are those of cudallm_gemm.h.  None of these kernels waits for
- * another CTA.
+ * status codes are those of cudallm_gemm.h.  Only the one-pass LayerNorm kernel
+ * (see cudallm_layernorm_f32) has CTAs that wait for one another.
  *
  * cudallm_sum_f32 / cudallm_dot_f32 keep their per-block partial sums in one
  * fixed scratch area per device, and cudallm_layernorm_f32 keeps its per-sample
@@ -85,6 +85,18 @@ int cudallm_dot_f32(const float *a, const float *b, int64_t n, float *result, vo
  * not dominated by a few outliers; squared deviations must stay inside the fp32
  * range (|x - mean| below about 1e19).  batch == 0 or m == 0: success, nothing
  * written.
+ * Kernels: when x, y, gamma and beta are 32-byte aligned, m is a multiple of 8
+ * and a sample is neither tiny nor larger than about 4.2 M elements, ONE
+ * persistent kernel (one CTA per SM) keeps every SM's slice of the samples in
+ * shared memory between the moments and the normalisation, so x is read from
+ * DRAM once; its CTAs exchange their partial moments through the workspace and
+ * wait for one another with a bound (default 2 s; all CTAs must be resident,
+ * i.e. no other kernel may hold SMs for that long).  If a wait runs out the
+ * kernel returns, y is unspecified and cudallm_device_status(stream, ...)
+ * reports CUDALLM_ERR_DEVICE_TIMEOUT.  Everything else takes two plain kernels
+ * (moments, then normalisation; x is read twice, the second time from L2 when
+ * it fits).  Both give results within the bound above; they differ in the
+ * last bits because the partial moments are grouped differently.
  * Errors: INVALID_DIM (negative, batch >= 2^31, m > 2^40, eps negative or not
  * finite), INVALID_POINTER (x or y NULL), MISALIGNED (4 bytes), WORKSPACE (an
  * external workspace is set and too small), UNSUPPORTED_DEVICE, CUDA.

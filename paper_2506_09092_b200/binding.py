@@ -295,7 +295,7 @@ def shutdown(check=True):
     return _check(lib().cudallm_shutdown(), "cudallm_shutdown", check)
 
 
-DEBUG_WAIT_LIMIT_NS, DEBUG_MISS_NEXT_SPLIT_FLAGS = 1, 2
+DEBUG_WAIT_LIMIT_NS, DEBUG_MISS_NEXT_SPLIT_FLAGS, DEBUG_LAYERNORM_PATH = 1, 2, 3
 
 
 def debug_set(what: int, value: int, check=True):

@@ -408,6 +408,7 @@ struct DeviceState {
     Workspace ws;                // the device's default workspace
     std::unordered_map<cudaStream_t, Workspace> stream_ws;   // cudallm_set_workspace_for_stream
     bool smem_attr_set[40] = {};
+    bool layernorm_attr_set = false;
     int max_pairs = 0;           // co-resident 2-CTA clusters of the pair kernel (0 = not asked yet)
     int epoch = 0;               // last split-K flag value used on this device
 };
@@ -419,6 +420,7 @@ std::mutex g_mutex;
 // waits for, so that every such wait runs out (the self-test of the timeout path).
 std::atomic<unsigned long long> g_wait_limit_ns{kWaitLimitNs};
 std::atomic<int> g_skew_next_flags{0};
+std::atomic<int> g_layernorm_path{0};      // 0 = by size, 1 = always the two-kernel path, 2 = one-pass whenever it fits
 
 // The workspace calls on `stream` use: the one attached to the stream, else the device's.
 Workspace &workspace_for(DeviceState &d, cudaStream_t stream)
@@ -1626,6 +1628,10 @@ int cudallm_debug_set(int what, unsigned long long value)
         return CUDALLM_OK;
     case CUDALLM_DEBUG_MISS_NEXT_SPLIT_FLAGS:
         g_skew_next_flags.store(value ? 1 : 0);
+        return CUDALLM_OK;
+    case CUDALLM_DEBUG_LAYERNORM_PATH:
+        if (value > 2) return CUDALLM_ERR_INVALID_VARIANT;
+        g_layernorm_path.store((int)value);
         return CUDALLM_OK;
     default:
         return CUDALLM_ERR_INVALID_VARIANT;

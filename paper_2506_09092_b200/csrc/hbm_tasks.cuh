@@ -221,7 +221,8 @@ reduce_kernel(const float *__restrict__ a, const float *__restrict__ b, long lon
 // y[s][i] = (x[s][i] - mean_s) / sqrt(var_s + eps) * gamma[i] + beta[i] with the
 // mean and the (biased) variance taken over the m elements of sample s.
 //
-// Two plain kernels of many small CTAs (no CTA waits for another):
+// General path: two plain kernels of many small CTAs (no CTA waits for another;
+// the one-pass kernel for samples that fit in shared memory follows further down):
 //  * layernorm_moments_kernel: CTA (s, part) takes the moments of one part of
 //    sample s and publishes them;
 //  * layernorm_apply_kernel: CTA (pair of samples, chunk) combines the published
@@ -480,6 +481,469 @@ layernorm_apply_kernel(const LayerNorm2Params p)
             const float cv = two ? __ldcg(xc + i) : 0.f;             // read before the stores: y may be x
             ya[i] = ln_apply(a, mha, mla, ra, gm, bt);
             if (two) yc[i] = ln_apply(cv, mhc, mlc, rc, gm, bt);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// LayerNorm as ONE persistent kernel that reads x from DRAM once: the second
+// read of a sample comes out of L2, a few samples after the first.  G CTAs (one
+// per SM); CTA i owns positions [i * slice_len, (i + 1) * slice_len) of EVERY
+// sample (so each line of x, gamma and beta is only ever asked for by one SM),
+// cut into 16 KB chunks.  All loads are bulk asynchronous copies into shared
+// memory: what is in flight is bounded by shared memory (5 + 6 chunks), not by
+// registers.  Roles:
+//
+//   loader A (one lane): chunk after chunk of x, sample after sample, from DRAM
+//     into ring A ("evict last": wanted again soon); never more than `lead` chunks ahead of the normalisation,
+//     so that what it fetched is still in L2 when it is read again;
+//   8 moments warps: take the chunks from ring A, hand each sample's moments to
+//     the exchange warp;
+//   4 exchange warps (warp w serves samples w, w + 4, ...): publish this CTA's
+//     moments of a sample, wait for the G entries of the sample, combine them
+//     (the same arithmetic in the same order in every CTA), hand mean and
+//     1 / sqrt(var + eps) on; one round trip to L2 takes microseconds while
+//     the SM streams, so several samples' exchanges must be in flight;
+//   loader B (one lane): for every chunk of a sample whose moments are done,
+//     x again (now from L2, "evict first": its last use) and the chunk's gamma
+//     and beta (from L2, "evict last") into ring B;
+//   8 normalising warps: take the stages from ring B, store y (streaming).
+//
+// DRAM reads and writes therefore run side by side all the time, a CTA meets
+// the others' moments a sample or more after it published its own, and no
+// kernel boundary drains the memory system.  In place (y == x) is safe: an
+// element of y is stored after both copies of that element of x have landed.
+//
+// All G CTAs must be resident at the same time (G <= number of SMs, one CTA per
+// SM by shared memory); every wait is bounded, gives up with a status word
+// (role 5: 0x10 + kind of wait) and lets the kernel drain and return.
+constexpr int kLnRoleWarps = 8;
+constexpr int kLnRoleThreads = kLnRoleWarps * 32;
+constexpr int kLnExchangeWarps = 4;                               // exchange warp w serves samples w, w + 4, ...
+constexpr int kLnStreamThreads = 2 * kLnRoleThreads + (2 + kLnExchangeWarps) * 32;     // + loader A, loader B, exchange
+constexpr int kLnChunkElems = 4096;
+constexpr int kLnChunkBytes = kLnChunkElems * 4;                  // 16 KB
+constexpr int kLnRingA = 5;                                       // chunks of x on their way from DRAM
+constexpr int kLnRingB = 3;                                       // stages of (x, gamma, beta) on their way from L2
+constexpr int kLnStreamSmem = (kLnRingA + 3 * kLnRingB) * kLnChunkBytes;      // 224 KB
+constexpr int kLnSlots = 16;                             // samples in flight between the roles (see `lead`)
+constexpr int kRoleLayerNorm = 5;
+
+struct LayerNormStreamParams {
+    const float *x, *gamma, *beta;
+    float *y;
+    long long m;             // elements per sample
+    long long slice_len;     // elements per CTA (a multiple of 8)
+    int batch, ctas;
+    int lead;                // chunks loader A may run ahead of loader B (at most kLnSlots - 8 samples' worth)
+    double eps, inv_m;
+    unsigned long long *entries;   // [batch][ctas][6]: the published moments, every word tagged (see LnEntry)
+    int epoch;               // the tag of this launch's entries (never 0)
+    int tag_post;            // the tag this launch writes: epoch (anything else only in the host's
+                             // self-test of the wait limit)
+    int *status;
+    unsigned long long wait_limit_ns;
+};
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+// `bytes` (a multiple of 16) from global to this CTA's shared memory; completion is counted on `bar`.
+__device__ __forceinline__ void bulk_load_hint(uint32_t smem_dst, const void *src, uint32_t bytes, uint32_t bar,
+                                               uint64_t policy)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+                 "[%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ Float8 lds8(uint32_t addr)
+{
+    Float8 r;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "r"(addr) : "memory");
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7]) : "r"(addr + 16) : "memory");
+    return r;
+}
+constexpr int kLnMaxCtas = 160;                          // entries per sample: at most five per lane of a warp
+
+// What a CTA publishes for its n elements of a sample, in the form the other CTAs read it:
+// six 8-byte words, each a 32-bit payload under a 32-bit tag (the launch's epoch).  A naturally
+// aligned 8-byte store is indivisible, so a reader that finds the tag has the payload too: no
+// flag, no fence, one round trip to L2.  Payloads: A = sum x (double, two words), the CTA's
+// own mean A / n (double, two words), B = sum of squared deviations about that mean (float),
+// n (int).
+struct LnEntry {
+    double A, mean;
+    float B;
+    int n;
+};
+__device__ __forceinline__ void ln_entry_store(unsigned long long *dst, int n, float c, double s1, double s2,
+                                               int tag, int word)
+{
+    const double nd = static_cast<double>(n);
+    const double A = nd * static_cast<double>(c) + s1;
+    const double mean = n > 0 ? A / nd : 0.0;
+    double B = n > 0 ? s2 - s1 * s1 / nd : 0.0;
+    B = B > 0.0 ? B : 0.0;
+    const unsigned long long a = static_cast<unsigned long long>(__double_as_longlong(A));
+    const unsigned long long mu = static_cast<unsigned long long>(__double_as_longlong(mean));
+    unsigned int payload;
+    switch (word) {
+    case 0: payload = static_cast<unsigned int>(a); break;
+    case 1: payload = static_cast<unsigned int>(a >> 32); break;
+    case 2: payload = static_cast<unsigned int>(mu); break;
+    case 3: payload = static_cast<unsigned int>(mu >> 32); break;
+    case 4: payload = __float_as_uint(static_cast<float>(B)); break;
+    default: payload = static_cast<unsigned int>(n); break;
+    }
+    const unsigned long long v = (static_cast<unsigned long long>(static_cast<unsigned int>(tag)) << 32) | payload;
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(dst + word), "l"(v) : "memory");
+}
+// Reads one entry; false if any of its words does not carry `tag` yet.
+__device__ __forceinline__ bool ln_entry_load(const unsigned long long *src, int tag, LnEntry &e)
+{
+    unsigned long long w[6];
+#pragma unroll
+    for (int i = 0; i < 3; ++i)
+        asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];"
+                     : "=l"(w[2 * i]), "=l"(w[2 * i + 1]) : "l"(src + 2 * i) : "memory");
+    bool ok = true;
+#pragma unroll
+    for (int i = 0; i < 6; ++i) ok = ok && static_cast<int>(w[i] >> 32) == tag;
+    e.A = __longlong_as_double(static_cast<long long>((w[1] << 32) | (w[0] & 0xffffffffull)));
+    e.mean = __longlong_as_double(static_cast<long long>((w[3] << 32) | (w[2] & 0xffffffffull)));
+    e.B = __uint_as_float(static_cast<unsigned int>(w[4]));
+    e.n = static_cast<int>(static_cast<unsigned int>(w[5]));
+    return ok;
+}
+
+__device__ __forceinline__ void ln_report(int *status, int what)
+{
+    if (atomicCAS(status, 0, -9 /* CUDALLM_ERR_DEVICE_TIMEOUT */) == 0) status[1] = (kRoleLayerNorm << 8) | what;
+}
+
+// Bounded wait until the shared counter `*counter` exceeds `value`.
+__device__ __forceinline__ bool ln_wait_counter(const volatile int *counter, int value, volatile int *abort_flag,
+                                                uint64_t limit_ns)
+{
+    if (*counter > value) return true;
+    const uint64_t t0 = globaltimer_ns();
+    while (*counter <= value) {
+        __nanosleep(20);
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > limit_ns) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+    return true;
+}
+
+__global__ void __launch_bounds__(kLnStreamThreads, 1)
+layernorm_stream_kernel(const LayerNormStreamParams p)
+{
+    extern __shared__ __align__(128) uint8_t ln_smem[];  // ring A, then ring B's stages of (x, gamma, beta)
+    __shared__ __align__(8) uint64_t bars[2 * (kLnRingA + kLnRingB)];
+    __shared__ double warp_part[2][2][kLnRoleWarps];
+    __shared__ double moments_of[kLnSlots][2];           // a sample's sums about its pilot, from the moments warps
+    __shared__ float pilot_of[kLnSlots];
+    __shared__ float stat_of[kLnSlots][4];               // a sample's (mean high, mean low, 1 / sqrt(var + eps))
+    __shared__ volatile int stat_ready[kLnSlots];        // sample + 1 once stat_of holds its statistics
+    __shared__ volatile int moments_done;                // samples the moments warps have finished
+    __shared__ volatile int b_issued;                    // chunks loader B has started
+    __shared__ int abort_word;
+    volatile int *abort_flag = &abort_word;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x, G = p.ctas;
+    const uint32_t ring_a = smem_u32(ln_smem);
+    const uint32_t ring_b = ring_a + kLnRingA * kLnChunkBytes;
+    const uint32_t bar_base = smem_u32(bars);
+    auto full_a = [&](int i) { return bar_base + 8u * i; };
+    auto empty_a = [&](int i) { return bar_base + 8u * (kLnRingA + i); };
+    auto full_b = [&](int i) { return bar_base + 8u * (2 * kLnRingA + i); };
+    auto empty_b = [&](int i) { return bar_base + 8u * (2 * kLnRingA + kLnRingB + i); };
+    if (tid == 0) {
+        abort_word = 0;
+        moments_done = 0;
+        b_issued = 0;
+        for (int i = 0; i < kLnSlots; ++i) stat_ready[i] = 0;
+        for (int i = 0; i < kLnRingA; ++i) {
+            mbar_init(full_a(i), 1);
+            mbar_init(empty_a(i), kLnRoleWarps);
+        }
+        for (int i = 0; i < kLnRingB; ++i) {
+            mbar_init(full_b(i), 1);
+            mbar_init(empty_b(i), kLnRoleWarps);
+        }
+        fence_mbar_init();
+    }
+    __syncthreads();
+    grid_launch_dependents();
+    grid_dependency_wait();
+
+    const long long lo = static_cast<long long>(cta) * p.slice_len;
+    const long long n_ll = min(p.m, lo + p.slice_len) - lo;
+    const int n = n_ll > 0 ? static_cast<int>(n_ll) : 0;                   // this CTA's elements of a sample
+    const int C = (n + kLnChunkElems - 1) / kLnChunkElems;                 // ... in chunks (the last may be short)
+    auto chunk_bytes = [&](int j) { return 4u * static_cast<uint32_t>(min(kLnChunkElems, n - j * kLnChunkElems)); };
+    const int kinds = 1 + (p.gamma ? 1 : 0) + (p.beta ? 1 : 0);            // arrays per stage of ring B
+
+    int last_a = -1, last_b = -1;                        // loader lanes: the last chunk whose copies they started
+    if (n == 0) {
+        // nothing of any sample lies here: publish empty entries, so that nobody waits for this CTA
+        if (tid < 6)
+            for (int s = 0; s < p.batch; ++s)
+                ln_entry_store(p.entries + (static_cast<long long>(s) * G + cta) * 6, 0, 0.f, 0.0, 0.0, p.tag_post, tid);
+    } else if (warp < kLnRoleWarps) {
+        // ------------------------------------------------------------- moments
+        bool ok = true;
+        const uint32_t off0 = static_cast<uint32_t>(tid) * 32u, off1 = off0 + kLnRoleThreads * 32u;
+        int t = 0;
+        for (int s = 0; s < p.batch; ++s) {
+            double s1 = 0.0, s2 = 0.0;
+            float c = 0.f;
+            for (int j = 0; j < C; ++j, ++t) {
+                const int use = t / kLnRingA, slot = t - use * kLnRingA;
+                if (ok && !mbar_wait(full_a(slot), use & 1, abort_flag, p.wait_limit_ns)) {
+                    if (lane == 0) ln_report(p.status, 0x11);
+                    ok = false;
+                }
+                if (ok) {
+                    const uint32_t chunk = ring_a + slot * kLnChunkBytes;
+                    if (j == 0) c = ln_pilot(lds8(chunk));
+                    const int e = j * kLnChunkElems + tid * 8;
+                    float f1 = 0.f, f2 = 0.f;
+                    if (e < n) ln_add_piece(lds8(chunk + off0), c, f1, f2);
+                    if (e + kLnRoleThreads * 8 < n) ln_add_piece(lds8(chunk + off1), c, f1, f2);
+                    ln_flush(f1, f2, s1, s2);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_a(slot));
+            }
+            s1 = warp_sum(s1);
+            s2 = warp_sum(s2);
+            if (lane == 0) {
+                warp_part[s & 1][0][warp] = s1;
+                warp_part[s & 1][1][warp] = s2;
+            }
+            named_bar_sync(1, kLnRoleThreads);
+            if (tid == 0) {
+                // the sample's sums in a fixed order, handed to the exchange warp (which is at most
+                // kLnSlots - 2 samples behind: loader A waits for loader B, which waits for it)
+                double t1 = 0.0, t2 = 0.0;
+                for (int w = 0; w < kLnRoleWarps; ++w) {
+                    t1 += warp_part[s & 1][0][w];
+                    t2 += warp_part[s & 1][1][w];
+                }
+                const int k = s % kLnSlots;
+                moments_of[k][0] = t1;
+                moments_of[k][1] = t2;
+                pilot_of[k] = c;
+                __threadfence_block();
+                moments_done = ok ? s + 1 : 0;
+            }
+        }
+    } else if (warp < 2 * kLnRoleWarps) {
+        // ------------------------------------------------------- normalisation
+        const int at = tid - kLnRoleThreads;
+        bool ok = true;
+        int t = 0;
+        for (int q = 0; q < p.batch; ++q) {
+            if (ok && !ln_wait_counter(&stat_ready[q % kLnSlots], q, abort_flag, p.wait_limit_ns)) {
+                if (lane == 0) ln_report(p.status, 0x13);
+                ok = false;
+            }
+            __threadfence_block();
+            const int k = q % kLnSlots;
+            const float mh = stat_of[k][0], ml = stat_of[k][1], rstd = stat_of[k][2];
+            float *yq = p.y + static_cast<long long>(q) * p.m + lo;
+            for (int j = 0; j < C; ++j, ++t) {
+                const int use = t / kLnRingB, stage = t - use * kLnRingB;
+                if (ok && !mbar_wait(full_b(stage), use & 1, abort_flag, p.wait_limit_ns)) {
+                    if (lane == 0) ln_report(p.status, 0x14);
+                    ok = false;
+                }
+                if (ok) {
+                    const uint32_t sx = ring_b + stage * (3 * kLnChunkBytes);
+                    const uint32_t sg = sx + kLnChunkBytes, sb = sg + (p.gamma ? kLnChunkBytes : 0);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int piece = at + h * kLnRoleThreads;
+                        const int e = j * kLnChunkElems + piece * 8;
+                        if (e < n) {
+                            Float8 v = lds8(sx + piece * 32), gm, bt;
+                            if (p.gamma) gm = lds8(sg + piece * 32);
+                            if (p.beta) bt = lds8(sb + piece * 32);
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                v.v[u] = ln_apply(v.v[u], mh, ml, rstd, p.gamma ? gm.v[u] : 1.f, p.beta ? bt.v[u] : 0.f);
+                            st8_stream(yq + e, v);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_b(stage));
+            }
+        }
+    } else if (warp == 2 * kLnRoleWarps) {
+        // ------------------------------------------------------------ loader A
+        if (lane == 0) {
+            const uint64_t keep = l2_policy_evict_last();        // these lines are wanted again, `lead` chunks later
+            int t = 0;
+            for (int s = 0; s < p.batch && t >= 0; ++s) {
+                const float *src = p.x + static_cast<long long>(s) * p.m + lo;
+                for (int j = 0; j < C; ++j, ++t) {
+                    const int use = t / kLnRingA, slot = t - use * kLnRingA;
+                    if (t >= p.lead && !ln_wait_counter(&b_issued, t - p.lead, abort_flag, p.wait_limit_ns)) {
+                        ln_report(p.status, 0x10);
+                        t = -1;
+                        break;
+                    }
+                    if (use > 0 && !mbar_wait(empty_a(slot), (use - 1) & 1, abort_flag, p.wait_limit_ns)) {
+                        ln_report(p.status, 0x15);
+                        t = -1;
+                        break;
+                    }
+                    fence_proxy_async_smem();            // the warps' reads of the slot come before the copy's writes
+                    mbar_expect_tx(full_a(slot), chunk_bytes(j));
+                    bulk_load_hint(ring_a + slot * kLnChunkBytes, src + j * kLnChunkElems, chunk_bytes(j), full_a(slot), keep);
+                    last_a = t;
+                }
+            }
+        }
+    } else if (warp == 2 * kLnRoleWarps + 1) {
+        // ------------------------------------------------------------ loader B
+        if (lane == 0) {
+            const uint64_t once = l2_policy_evict_first(), keep = l2_policy_evict_last();
+            int t = 0;
+            for (int q = 0; q < p.batch && t >= 0; ++q) {
+                // x of sample q has passed through the moments warps: it is in L2 (and, in place,
+                // may now be overwritten once this copy of it has landed)
+                if (!ln_wait_counter(&moments_done, q, abort_flag, p.wait_limit_ns)) {
+                    ln_report(p.status, 0x16);
+                    break;
+                }
+                const float *src = p.x + static_cast<long long>(q) * p.m + lo;
+                for (int j = 0; j < C; ++j, ++t) {
+                    const int use = t / kLnRingB, stage = t - use * kLnRingB;
+                    if (use > 0 && !mbar_wait(empty_b(stage), (use - 1) & 1, abort_flag, p.wait_limit_ns)) {
+                        ln_report(p.status, 0x17);
+                        t = -1;
+                        break;
+                    }
+                    const uint32_t bytes = chunk_bytes(j);
+                    const uint32_t sx = ring_b + stage * (3 * kLnChunkBytes);
+                    const uint32_t sg = sx + kLnChunkBytes, sb = sg + (p.gamma ? kLnChunkBytes : 0);
+                    fence_proxy_async_smem();
+                    mbar_expect_tx(full_b(stage), bytes * kinds);
+                    bulk_load_hint(sx, src + j * kLnChunkElems, bytes, full_b(stage), once);
+                    if (p.gamma) bulk_load_hint(sg, p.gamma + lo + j * kLnChunkElems, bytes, full_b(stage), keep);
+                    if (p.beta) bulk_load_hint(sb, p.beta + lo + j * kLnChunkElems, bytes, full_b(stage), keep);
+                    last_b = t;
+                    b_issued = t + 1;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ exchange
+        // The only warps that talk to the other CTAs.  (An acquire or a release in a warp that
+        // has loads and stores in flight waits for those, microseconds per sample.)  Each
+        // publishes this CTA's moments of its next sample s as soon as the moments warps have
+        // handed them over, and works out the statistics of its sample q as soon as all G
+        // entries of q are there; neither duty ever blocks the other.
+        const int first = warp - (2 * kLnRoleWarps + 2);
+        int s = first, q = first;
+        uint64_t t_idle = globaltimer_ns();
+        while (q < p.batch) {
+            bool progress = false;
+            if (s < p.batch && moments_done > s) {
+                __threadfence_block();
+                const int k = s % kLnSlots;
+                if (lane < 6)
+                    ln_entry_store(p.entries + (static_cast<long long>(s) * G + cta) * 6, n, pilot_of[k],
+                                   moments_of[k][0], moments_of[k][1], p.tag_post, lane);
+                s += kLnExchangeWarps;
+                progress = true;
+            }
+            if (q < s) {
+                // entries lane, lane + 32, ... of sample q: all their loads are in flight together
+                const unsigned long long *base = p.entries + static_cast<long long>(q) * G * 6;
+                LnEntry e[kLnMaxCtas / 32];
+                bool all = true;
+#pragma unroll
+                for (int u = 0; u < kLnMaxCtas / 32; ++u) {
+                    const int k = lane + 32 * u;
+                    e[u].A = 0.0; e[u].mean = 0.0; e[u].B = 0.f; e[u].n = 0;
+                    if (k < G) all = ln_entry_load(base + k * 6, p.epoch, e[u]) && all;
+                }
+                if (__all_sync(0xffffffffu, all)) {
+                    // mean = sum A_k / m, then M2 = sum (B_k + n_k (mean_k - mean)^2): the same
+                    // arithmetic in the same order in every CTA
+                    double a = 0.0;
+#pragma unroll
+                    for (int u = 0; u < kLnMaxCtas / 32; ++u) a += e[u].A;
+                    const double mean = warp_sum(a) * p.inv_m;
+                    float m2 = 0.f;
+#pragma unroll
+                    for (int u = 0; u < kLnMaxCtas / 32; ++u) {
+                        const float dm = static_cast<float>(e[u].mean - mean);
+                        m2 += e[u].B + static_cast<float>(e[u].n) * dm * dm;
+                    }
+                    m2 = warp_sum_f32(m2);
+                    if (lane == 0) {
+                        const double var = static_cast<double>(m2) * p.inv_m;
+                        const float mh = static_cast<float>(mean);
+                        float *out = stat_of[q % kLnSlots];
+                        out[0] = mh;
+                        out[1] = static_cast<float>(mean - static_cast<double>(mh));
+                        out[2] = static_cast<float>(rsqrt(var + p.eps));
+                        __threadfence_block();
+                        stat_ready[q % kLnSlots] = q + 1;
+                    }
+                    q += kLnExchangeWarps;
+                    progress = true;
+                }
+            }
+            if (progress) {
+                t_idle = globaltimer_ns();
+            } else {
+                __nanosleep(40);
+                if (*abort_flag) break;
+                if (globaltimer_ns() - t_idle > p.wait_limit_ns) {
+                    *abort_flag = 1;
+                    if (lane == 0) ln_report(p.status, 0x12);
+                    break;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // After a wait that ran out the warps may have left chunks unread: their copies must still
+    // land before the CTA gives up its shared memory.  Each loader lane polls (bounded) the
+    // chunks it started last; on the normal path every copy was awaited by the warps.
+    if (*abort_flag) {
+        for (int t = last_a; t >= 0 && t > last_a - kLnRingA; --t) {
+            const int use = t / kLnRingA, slot = t - use * kLnRingA;
+            for (int k = 0; k < 20000 && !mbar_try_wait(full_a(slot), use & 1); ++k) __nanosleep(100);
+        }
+        for (int t = last_b; t >= 0 && t > last_b - kLnRingB; --t) {
+            const int use = t / kLnRingB, stage = t - use * kLnRingB;
+            for (int k = 0; k < 20000 && !mbar_try_wait(full_b(stage), use & 1); ++k) __nanosleep(100);
         }
     }
 }

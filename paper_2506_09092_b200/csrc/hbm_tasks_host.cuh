@@ -112,6 +112,57 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
 
     const bool vec = (all & 31) == 0 && m % 8 == 0;            // 32-byte loads and stores
     const int sms = d.sm_count;
+    // The persistent kernel (x read from DRAM once): one CTA per SM, each with its slice of every
+    // sample.  Taken where it was measured faster than the two kernels below: samples of 8 to
+    // 20 MB (4 MB with 32 or more of them) -- smaller ones finish before the exchange of the
+    // moments between the CTAs (several microseconds) is amortised, larger ones do not stay in
+    // L2 between their two reads -- and at least four samples.
+    const int ln_path = g_layernorm_path.load();
+    if (vec && ln_path != 1) {
+        const int64_t G = std::min<int64_t>({int64_t(sms), int64_t(kLnMaxCtas), std::max<int64_t>(1, m / 1024)});
+        const int64_t slice_len = round_up(cdiv(m, G), 8);
+        const bool worth = (batch >= 4 && m <= (int64_t(5) << 20) && (m >= (int64_t(1) << 21) || (m >= (int64_t(1) << 20) && batch >= 32)))
+                        || ln_path == 2;
+        if (worth && slice_len < (int64_t(1) << 30)) {
+            // Loader A runs ahead of loader B by what keeps about 34 MB of x in L2 between its two
+            // reads, at least one sample and a half, at most 8 samples (loader B is at most 3
+            // chunks ahead of the normalisation, and the roles hand samples over in 16 slots).
+            const int64_t chunks = cdiv(slice_len, kLnChunkElems);
+            const int64_t lead = std::max<int64_t>(chunks + (chunks + 1) / 2,
+                                                   std::min<int64_t>((kLnSlots - 8) * chunks,
+                                                                     (int64_t(34) << 20) / (G * kLnChunkBytes)));
+            // The entries live in the flag area of the workspace header, where every 32-bit word is
+            // either zero or an epoch of an earlier launch: a stale word cannot pass for this
+            // launch's tag.  The area holds kFlagBytes / 48 entries; larger batches go in pieces.
+            const int64_t per_launch = std::max<int64_t>(1, int64_t(kFlagBytes / 48) / G);
+            Workspace &w = workspace_for(d, stream);
+            st = ensure_workspace(w, kHeaderBytes, stream);
+            if (st != CUDALLM_OK) return st;
+            uint8_t *ws = static_cast<uint8_t *>(w.ptr);
+            if (!d.layernorm_attr_set) {
+                CUDA_TRY(cudaFuncSetAttribute(layernorm_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              kLnStreamSmem));
+                d.layernorm_attr_set = true;
+            }
+            for (int64_t s0 = 0; s0 < batch; s0 += per_launch) {
+                LayerNormStreamParams sp{};
+                sp.x = x + s0 * m; sp.gamma = gamma; sp.beta = beta; sp.y = y + s0 * m;
+                sp.m = m; sp.slice_len = slice_len;
+                sp.batch = (int)std::min<int64_t>(per_launch, batch - s0); sp.ctas = (int)G; sp.lead = (int)lead;
+                sp.eps = (double)eps;
+                sp.inv_m = 1.0 / (double)m;
+                sp.entries = reinterpret_cast<unsigned long long *>(ws + 256);
+                sp.epoch = next_epoch(d);
+                sp.tag_post = g_skew_next_flags.exchange(0) ? (sp.epoch ^ 0x40000000) : sp.epoch;
+                sp.status = reinterpret_cast<int *>(ws);
+                sp.wait_limit_ns = g_wait_limit_ns.load();
+                st = launch_serialised_smem(layernorm_stream_kernel, dim3((unsigned)G), dim3(kLnStreamThreads),
+                                            (size_t)kLnStreamSmem, stream, sp);
+                if (st != CUDALLM_OK) return st;
+            }
+            return CUDALLM_OK;
+        }
+    }
     // first kernel: about four CTAs per SM in total (what is resident at once: one wave), at
     // least 4096 elements each, at most 256 parts
     int64_t parts = std::max<int64_t>(1, std::min<int64_t>(cdiv(int64_t(4) * sms, batch), m / 4096));

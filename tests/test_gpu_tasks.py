@@ -210,10 +210,86 @@ def check_layernorm(got, x, gamma, beta, batch, m, eps=1e-5):
 
 
 @pytest.mark.parametrize("batch,m", [(1, 4), (3, 7), (16, 4 * 64 * 64), (16, 4 * 128 * 128), (5, 4096 * 3 + 4),
-                                     (2, 1 << 20), (200, 1000), (7, 100003), (16, 4 * 256 * 256),
+                                     (2, 1 << 20), (200, 1000), (7, 100003), (16, 4 * 256 * 256), (5, 1 << 21),
                                      (40, 200000), (33, 100024), (1, 8)])
 def test_layernorm_against_oracle(batch, m):
     x, gamma, beta = gi.layernorm_inputs(4, batch, m)
+    check_layernorm(run_layernorm(x, gamma, beta, batch, m), x, gamma, beta, batch, m)
+
+
+@pytest.fixture
+def layernorm_path():
+    """Forces cudallm_layernorm_f32 onto one of its two kernels for the test's duration."""
+    def force(path):
+        B.debug_set(B.DEBUG_LAYERNORM_PATH, path)
+    yield force
+    B.debug_set(B.DEBUG_LAYERNORM_PATH, 0)
+
+
+# Sizes that exercise the persistent kernel's rings and hand-over slots: one CTA; a few CTAs with
+# a ragged last slice; 148 slices of 1, 2 (ragged), 3 and 7 chunks of 16 KB with more samples
+# than the rings hold; one sample with slices of 10 chunks; more samples than one launch has
+# room for in the exchange area (148 CTAs: 147 samples); many samples of one short chunk.
+@pytest.mark.parametrize("batch,m", [(1, 8), (3, 8000), (16, 4 * 64 * 64), (9, 148 * 4096),
+                                     (6, 148 * 4096 * 2 - 4096 * 5 + 24), (5, 148 * 4096 * 3),
+                                     (3, 148 * 4096 * 7 - 40), (1, 148 * 4096 * 10 - 8), (7, 100000),
+                                     (150, 148 * 1024), (45, 148 * 1024 + 8)])
+def test_layernorm_one_pass_kernel_against_oracle(layernorm_path, batch, m):
+    x, gamma, beta = gi.layernorm_inputs(14, batch, m)
+    layernorm_path(2)
+    got = run_layernorm(x, gamma, beta, batch, m)
+    check_layernorm(got, x, gamma, beta, batch, m)
+    assert np.array_equal(got, run_layernorm(x, gamma, beta, batch, m))          # repeatable bit for bit
+    layernorm_path(1)
+    check_layernorm(run_layernorm(x, gamma, beta, batch, m), x, gamma, beta, batch, m)
+
+
+def test_layernorm_one_pass_kernel_variants_of_the_call(layernorm_path):
+    layernorm_path(2)
+    batch, m = 6, 148 * 1024 + 64
+    x, gamma, beta = gi.layernorm_inputs(45, batch, m)
+    check_layernorm(run_layernorm(x, None, None, batch, m), x, None, None, batch, m)
+    check_layernorm(run_layernorm(x, gamma, None, batch, m), x, gamma, None, batch, m)
+    check_layernorm(run_layernorm(x, gamma, beta, batch, m, in_place=True), x, gamma, beta, batch, m)
+    check_layernorm(run_layernorm(x, gamma, beta, batch, m, eps=0.5), x, gamma, beta, batch, m, eps=0.5)
+    # closed forms: a constant sample returns beta exactly; a large common offset does not cancel
+    m = 148 * 2048
+    beta = np.linspace(-1, 1, m).astype(np.float32)
+    gamma = np.full(m, 3.0, np.float32)
+    got = run_layernorm(np.full(2 * m, 7.25, np.float32), gamma, beta, 2, m)
+    assert np.array_equal(got[0], beta.astype(np.float64)) and np.array_equal(got[1], got[0])
+    sign = np.where(np.arange(m) % 2 == 0, -1.0, 1.0).astype(np.float32)
+    y = (np.float32(4096.0) + sign * np.float32(2.0 ** -6)).astype(np.float32)
+    got = run_layernorm(y, None, None, 1, m)
+    ref, _, _ = oracle.layernorm_f32(y, None, None, 1, m)
+    assert np.allclose(got, ref, rtol=2e-7, atol=0)
+
+
+def test_layernorm_one_pass_kernel_wait_limit(layernorm_path):
+    """The CTAs of the persistent kernel wait for one another's moments; with the entries tagged
+    with a value nobody waits for, every such wait runs out after the (shortened) limit, the
+    kernel returns, the status word says so, and the next call is unaffected."""
+    layernorm_path(2)
+    batch, m = 4, 1 << 20
+    x, gamma, beta = gi.layernorm_inputs(46, batch, m)
+    s = torch.cuda.current_stream()
+    dx, dg, db = dev(x), dev(gamma), dev(beta)
+    dy = torch.zeros(batch * m, dtype=torch.float32, device="cuda")
+    assert B.device_status(s) == (B.OK, 0)
+    try:
+        B.debug_set(B.DEBUG_WAIT_LIMIT_NS, 1_000_000)
+        B.debug_set(B.DEBUG_MISS_NEXT_SPLIT_FLAGS, 1)
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        B.layernorm_f32(dx, dg, db, dy, batch, m, 1e-5, s)
+        t1.record()
+        code, detail = B.device_status(s)
+        assert code == B.ERR_DEVICE_TIMEOUT and detail >> 8 == 5 and detail & 0xF0 == 0x10, (code, hex(detail))
+        assert 0.9 <= t0.elapsed_time(t1) < 500.0
+        assert B.device_status(s) == (B.OK, 0)
+    finally:
+        B.debug_set(B.DEBUG_WAIT_LIMIT_NS, 0)
+        B.debug_set(B.DEBUG_MISS_NEXT_SPLIT_FLAGS, 0)
     check_layernorm(run_layernorm(x, gamma, beta, batch, m), x, gamma, beta, batch, m)
 
 
