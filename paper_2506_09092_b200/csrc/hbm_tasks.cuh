@@ -569,6 +569,31 @@ __device__ __forceinline__ void bulk_load_hint(uint32_t smem_dst, const void *sr
                  "[%0], [%1], %2, [%3], %4;"
                  ::"r"(smem_dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
 }
+// 16-byte accesses for the persistent LayerNorm kernel: consecutive lanes touch consecutive
+// 16 bytes of shared memory (a 32-byte piece per lane costs every access two passes through
+// the banks, and with the copies' own writes that made shared memory the kernel's bound).
+__device__ __forceinline__ float4 lds4(uint32_t addr)
+{
+    float4 r;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr) : "memory");
+    return r;
+}
+__device__ __forceinline__ void st4_stream(float *p, const float4 &r, uint64_t policy)
+{
+    asm volatile("st.global.L1::no_allocate.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
+                 ::"l"(p), "f"(r.x), "f"(r.y), "f"(r.z), "f"(r.w), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void ln_add_piece4(const float4 &v, float c, float &f1, float &f2)
+{
+    const float d0 = v.x - c, d1 = v.y - c, d2 = v.z - c, d3 = v.w - c;
+    f1 += (d0 + d1) + (d2 + d3);
+    float q = d0 * d0;
+    q = fmaf(d1, d1, q);
+    q = fmaf(d2, d2, q);
+    q = fmaf(d3, d3, q);
+    f2 += q;
+}
 __device__ __forceinline__ Float8 lds8(uint32_t addr)
 {
     Float8 r;
@@ -712,7 +737,6 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
     } else if (warp < kLnRoleWarps) {
         // ------------------------------------------------------------- moments
         bool ok = true;
-        const uint32_t off0 = static_cast<uint32_t>(tid) * 32u, off1 = off0 + kLnRoleThreads * 32u;
         int t = 0;
         for (int s = 0; s < p.batch; ++s) {
             double s1 = 0.0, s2 = 0.0;
@@ -726,10 +750,12 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
                 if (ok) {
                     const uint32_t chunk = ring_a + slot * kLnChunkBytes;
                     if (j == 0) c = ln_pilot(lds8(chunk));
-                    const int e = j * kLnChunkElems + tid * 8;
                     float f1 = 0.f, f2 = 0.f;
-                    if (e < n) ln_add_piece(lds8(chunk + off0), c, f1, f2);
-                    if (e + kLnRoleThreads * 8 < n) ln_add_piece(lds8(chunk + off1), c, f1, f2);
+#pragma unroll
+                    for (int h = 0; h < kLnChunkElems / (4 * kLnRoleThreads); ++h) {
+                        const int off = h * kLnRoleThreads * 4 + tid * 4;        // element of the chunk
+                        if (j * kLnChunkElems + off < n) ln_add_piece4(lds4(chunk + off * 4), c, f1, f2);
+                    }
                     ln_flush(f1, f2, s1, s2);
                 }
                 __syncwarp();
@@ -761,6 +787,7 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
     } else if (warp < 2 * kLnRoleWarps) {
         // ------------------------------------------------------- normalisation
         const int at = tid - kLnRoleThreads;
+        const uint64_t stream_out = l2_policy_evict_first();      // y is not read again
         bool ok = true;
         int t = 0;
         for (int q = 0; q < p.batch; ++q) {
@@ -782,17 +809,19 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
                     const uint32_t sx = ring_b + stage * (3 * kLnChunkBytes);
                     const uint32_t sg = sx + kLnChunkBytes, sb = sg + (p.gamma ? kLnChunkBytes : 0);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int piece = at + h * kLnRoleThreads;
-                        const int e = j * kLnChunkElems + piece * 8;
+                    for (int h = 0; h < kLnChunkElems / (4 * kLnRoleThreads); ++h) {
+                        const int off = h * kLnRoleThreads * 4 + at * 4;         // element of the chunk
+                        const int e = j * kLnChunkElems + off;
                         if (e < n) {
-                            Float8 v = lds8(sx + piece * 32), gm, bt;
-                            if (p.gamma) gm = lds8(sg + piece * 32);
-                            if (p.beta) bt = lds8(sb + piece * 32);
-#pragma unroll
-                            for (int u = 0; u < 8; ++u)
-                                v.v[u] = ln_apply(v.v[u], mh, ml, rstd, p.gamma ? gm.v[u] : 1.f, p.beta ? bt.v[u] : 0.f);
-                            st8_stream(yq + e, v);
+                            float4 v = lds4(sx + off * 4);
+                            float4 gm = make_float4(1.f, 1.f, 1.f, 1.f), bt = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (p.gamma) gm = lds4(sg + off * 4);
+                            if (p.beta) bt = lds4(sb + off * 4);
+                            v.x = ln_apply(v.x, mh, ml, rstd, gm.x, bt.x);
+                            v.y = ln_apply(v.y, mh, ml, rstd, gm.y, bt.y);
+                            v.z = ln_apply(v.z, mh, ml, rstd, gm.z, bt.z);
+                            v.w = ln_apply(v.w, mh, ml, rstd, gm.w, bt.w);
+                            st4_stream(yq + e, v, stream_out);
                         }
                     }
                 }

@@ -45,23 +45,21 @@ def check_case(A, Bm, M, N, K, out_dtype, variant, lda=None, ldb=None, ldc=None,
 
 @pytest.mark.parametrize("M", DIMS)
 def test_shape_grid(M):
-    """Every N of the grid, K cycling through the list, both output types,
-    on the automatic choice, the CUDA-core kernel and one tcgen05 variant per
-    tile width (plus a split-K one where K allows)."""
+    """Every (N, K) of the grid, both output types, on the automatic choice, the CUDA-core
+    kernel and every listed tcgen05 variant that supports the shape (one per tile width and
+    ring arrangement, lone CTAs and pairs, two CTAs per SM, split-K and tail-split ones)."""
     rng = np.random.default_rng(1000 + M)
     names = ["simt", "umma_n64", "umma_n128", "umma_n256", "umma_n64_sk2", "umma_n256_sk4",
              "umma2_n256", "umma2_n256_sk2", "umma_n256_ts", "umma2_n256_ts", "umma_n64_x2", "umma_n128_x2",
              "umma_n128_k1", "umma_n256_k2_ts", "umma2_n256_k1", "umma2_n256_k1_ts"]
-    for ni, N in enumerate(DIMS):
-        for ki in range(3):
-            K = KS[(ni * 3 + ki + M) % len(KS)]
+    ids = variant_ids(*names)
+    for N in DIMS:
+        for K in KS:
             A = bits(rng.standard_normal((M, K)))
             Bm = bits(rng.uniform(-1, 1, (K, N)))
             ref = oracle.gemm(A, Bm, M, N, K)
             for out_dtype in (gi.F32, gi.BF16):
-                vs = [B.VARIANT_AUTO] + [v for v in variant_ids(*names)
-                                         if B.variant_supports(v, M, N, K, K, N, N, 1, out_dtype) == 1]
-                for v in vs[:: 1 if (ni + ki) % 4 == 0 else 3] + [B.VARIANT_AUTO]:
+                for v in [B.VARIANT_AUTO] + [v for v in ids if B.variant_supports(v, M, N, K, K, N, N, 1, out_dtype) == 1]:
                     check_case(A.ravel(), Bm.ravel(), M, N, K, out_dtype, v, ref=ref)
 
 
