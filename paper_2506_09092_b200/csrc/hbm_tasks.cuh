@@ -491,8 +491,8 @@ layernorm_apply_kernel(const LayerNorm2Params p)
 // per SM); CTA i owns positions [i * slice_len, (i + 1) * slice_len) of EVERY
 // sample (so each line of x, gamma and beta is only ever asked for by one SM),
 // cut into 16 KB chunks.  All loads are bulk asynchronous copies into shared
-// memory: what is in flight is bounded by shared memory (5 + 6 chunks), not by
-// registers.  Roles:
+// memory: what is in flight is bounded by shared memory (5 chunks from DRAM, 6 to
+// 8 from L2), not by registers.  Roles:
 //
 //   loader A (one lane): chunk after chunk of x, sample after sample, from DRAM
 //     into ring A ("evict last": wanted again soon); never more than `lead` chunks ahead of the normalisation,
@@ -506,7 +506,8 @@ layernorm_apply_kernel(const LayerNorm2Params p)
 //     the SM streams, so several samples' exchanges must be in flight;
 //   loader B (one lane): for every chunk of a sample whose moments are done,
 //     x again (now from L2, "evict first": its last use) and the chunk's gamma
-//     and beta (from L2, "evict last") into ring B;
+//     and beta (from L2, "evict last") into ring B (3 stages of 48 KB; 4 or 9
+//     stages when gamma and / or beta are absent);
 //   8 normalising warps: take the stages from ring B, store y (streaming).
 //
 // DRAM reads and writes therefore run side by side all the time, a CTA meets
@@ -524,8 +525,9 @@ constexpr int kLnStreamThreads = 2 * kLnRoleThreads + (2 + kLnExchangeWarps) * 3
 constexpr int kLnChunkElems = 4096;
 constexpr int kLnChunkBytes = kLnChunkElems * 4;                  // 16 KB
 constexpr int kLnRingA = 5;                                       // chunks of x on their way from DRAM
-constexpr int kLnRingB = 3;                                       // stages of (x, gamma, beta) on their way from L2
-constexpr int kLnStreamSmem = (kLnRingA + 3 * kLnRingB) * kLnChunkBytes;      // 224 KB
+constexpr int kLnRingBChunks = 9;                                 // chunks of shared memory for ring B: 9 stages of x alone,
+                                                                  // 4 of (x, gamma) or (x, beta), 3 of (x, gamma, beta)
+constexpr int kLnStreamSmem = (kLnRingA + kLnRingBChunks) * kLnChunkBytes;    // 224 KB
 constexpr int kLnSlots = 16;                             // samples in flight between the roles (see `lead`)
 constexpr int kRoleLayerNorm = 5;
 
@@ -682,7 +684,7 @@ __global__ void __launch_bounds__(kLnStreamThreads, 1)
 layernorm_stream_kernel(const LayerNormStreamParams p)
 {
     extern __shared__ __align__(128) uint8_t ln_smem[];  // ring A, then ring B's stages of (x, gamma, beta)
-    __shared__ __align__(8) uint64_t bars[2 * (kLnRingA + kLnRingB)];
+    __shared__ __align__(8) uint64_t bars[2 * (kLnRingA + kLnRingBChunks)];
     __shared__ double warp_part[2][2][kLnRoleWarps];
     __shared__ double moments_of[kLnSlots][2];           // a sample's sums about its pilot, from the moments warps
     __shared__ float pilot_of[kLnSlots];
@@ -701,7 +703,7 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
     auto full_a = [&](int i) { return bar_base + 8u * i; };
     auto empty_a = [&](int i) { return bar_base + 8u * (kLnRingA + i); };
     auto full_b = [&](int i) { return bar_base + 8u * (2 * kLnRingA + i); };
-    auto empty_b = [&](int i) { return bar_base + 8u * (2 * kLnRingA + kLnRingB + i); };
+    auto empty_b = [&](int i) { return bar_base + 8u * (2 * kLnRingA + kLnRingBChunks + i); };
     if (tid == 0) {
         abort_word = 0;
         moments_done = 0;
@@ -711,7 +713,7 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
             mbar_init(full_a(i), 1);
             mbar_init(empty_a(i), kLnRoleWarps);
         }
-        for (int i = 0; i < kLnRingB; ++i) {
+        for (int i = 0; i < kLnRingBChunks; ++i) {
             mbar_init(full_b(i), 1);
             mbar_init(empty_b(i), kLnRoleWarps);
         }
@@ -727,6 +729,7 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
     const int C = (n + kLnChunkElems - 1) / kLnChunkElems;                 // ... in chunks (the last may be short)
     auto chunk_bytes = [&](int j) { return 4u * static_cast<uint32_t>(min(kLnChunkElems, n - j * kLnChunkElems)); };
     const int kinds = 1 + (p.gamma ? 1 : 0) + (p.beta ? 1 : 0);            // arrays per stage of ring B
+    const int NB = kLnRingBChunks / kinds;                                 // stages of ring B
 
     int last_a = -1, last_b = -1;                        // loader lanes: the last chunk whose copies they started
     if (n == 0) {
@@ -800,13 +803,13 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
             const float mh = stat_of[k][0], ml = stat_of[k][1], rstd = stat_of[k][2];
             float *yq = p.y + static_cast<long long>(q) * p.m + lo;
             for (int j = 0; j < C; ++j, ++t) {
-                const int use = t / kLnRingB, stage = t - use * kLnRingB;
+                const int use = t / NB, stage = t - use * NB;
                 if (ok && !mbar_wait(full_b(stage), use & 1, abort_flag, p.wait_limit_ns)) {
                     if (lane == 0) ln_report(p.status, 0x14);
                     ok = false;
                 }
                 if (ok) {
-                    const uint32_t sx = ring_b + stage * (3 * kLnChunkBytes);
+                    const uint32_t sx = ring_b + stage * (kinds * kLnChunkBytes);
                     const uint32_t sg = sx + kLnChunkBytes, sb = sg + (p.gamma ? kLnChunkBytes : 0);
 #pragma unroll
                     for (int h = 0; h < kLnChunkElems / (4 * kLnRoleThreads); ++h) {
@@ -869,14 +872,14 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
                 }
                 const float *src = p.x + static_cast<long long>(q) * p.m + lo;
                 for (int j = 0; j < C; ++j, ++t) {
-                    const int use = t / kLnRingB, stage = t - use * kLnRingB;
+                    const int use = t / NB, stage = t - use * NB;
                     if (use > 0 && !mbar_wait(empty_b(stage), (use - 1) & 1, abort_flag, p.wait_limit_ns)) {
                         ln_report(p.status, 0x17);
                         t = -1;
                         break;
                     }
                     const uint32_t bytes = chunk_bytes(j);
-                    const uint32_t sx = ring_b + stage * (3 * kLnChunkBytes);
+                    const uint32_t sx = ring_b + stage * (kinds * kLnChunkBytes);
                     const uint32_t sg = sx + kLnChunkBytes, sb = sg + (p.gamma ? kLnChunkBytes : 0);
                     fence_proxy_async_smem();
                     mbar_expect_tx(full_b(stage), bytes * kinds);
@@ -970,8 +973,8 @@ layernorm_stream_kernel(const LayerNormStreamParams p)
             const int use = t / kLnRingA, slot = t - use * kLnRingA;
             for (int k = 0; k < 20000 && !mbar_try_wait(full_a(slot), use & 1); ++k) __nanosleep(100);
         }
-        for (int t = last_b; t >= 0 && t > last_b - kLnRingB; --t) {
-            const int use = t / kLnRingB, stage = t - use * kLnRingB;
+        for (int t = last_b; t >= 0 && t > last_b - NB; --t) {
+            const int use = t / NB, stage = t - use * NB;
             for (int k = 0; k < 20000 && !mbar_try_wait(full_b(stage), use & 1); ++k) __nanosleep(100);
         }
     }

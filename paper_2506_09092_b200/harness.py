@@ -522,6 +522,9 @@ def _main(argv=None):
     ap.add_argument("--size", type=int, default=None,
                     help="with --task: N (transpose: N x N; sum, dot: N elements; layernorm: (16, 4, N, N); "
                          "attention: N queries and keys)")
+    ap.add_argument("--layernorm-kernels", default="auto", choices=["auto", "two", "persistent"],
+                    help="with --task layernorm: let the library choose by size, or force the two plain "
+                         "kernels / the persistent kernel (cudallm_debug_set)")
     args = ap.parse_args(argv)
     if args.task:
         return _task_main(args)
@@ -619,6 +622,8 @@ def _task_main(args):
 
     default = {"transpose": 8192, "sum": 1 << 28, "dot": 1 << 27, "layernorm": 512, "attention": 512}
     size = args.size or default[args.task]
+    if args.task == "layernorm":
+        B.debug_set(B.DEBUG_LAYERNORM_PATH, {"auto": 0, "two": 1, "persistent": 2}[args.layernorm_kernels])
     launch, bytes_, what = task_problem(args.task, size, args.sets)
     t = performance_profiler(launch, iters=args.iters, warmup=args.warmup)
     code, detail = B.device_status(torch.cuda.current_stream())
