@@ -98,7 +98,7 @@ def run_config(cfg: gi.GemmConfig, variant=B.VARIANT_AUTO, operands=None):
 def log_observed_error(family: str, case: str, observed: float, bound: float, what: str, **extra):
     """Append the largest error a parity test observed (in the units of its tolerance) to
     ``observed_errors.jsonl`` in the directory the environment variable CUDALLM_ERROR_LOG_DIR
-    names (default: ``gpurun_out`` at the repository root, created on demand), so that the
+    names (default: the scratch output directory at the repository root, created on demand), so that the
     share of each tolerance that is actually used can be read off."""
     import json
     import os
