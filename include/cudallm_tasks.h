@@ -85,18 +85,19 @@ int cudallm_dot_f32(const float *a, const float *b, int64_t n, float *result, vo
  * not dominated by a few outliers; squared deviations must stay inside the fp32
  * range (|x - mean| below about 1e19).  batch == 0 or m == 0: success, nothing
  * written.
- * Kernels: when x, y, gamma and beta are 32-byte aligned, m is a multiple of 8
- * and a sample is neither tiny nor larger than about 4.2 M elements, ONE
- * persistent kernel (one CTA per SM) keeps every SM's slice of the samples in
- * shared memory between the moments and the normalisation, so x is read from
- * DRAM once; its CTAs exchange their partial moments through the workspace and
- * wait for one another with a bound (default 2 s; all CTAs must be resident,
- * i.e. no other kernel may hold SMs for that long).  If a wait runs out the
- * kernel returns, y is unspecified and cudallm_device_status(stream, ...)
- * reports CUDALLM_ERR_DEVICE_TIMEOUT.  Everything else takes two plain kernels
- * (moments, then normalisation; x is read twice, the second time from L2 when
- * it fits).  Both give results within the bound above; they differ in the
- * last bits because the partial moments are grouped differently.
+ * Kernels: when x, y, gamma and beta are 32-byte aligned, m is a multiple of 8,
+ * a sample has 8 to 20 MB (from 4 MB with 32 or more samples) and there are at
+ * least four samples, ONE persistent kernel (one CTA per SM) takes the moments
+ * of a sample and, a sample or two later, reads it again while it is still in
+ * L2, so x crosses DRAM once; its CTAs exchange their partial moments through
+ * the workspace and wait for one another with a bound (default 2 s; all CTAs
+ * must be resident, i.e. no other kernel may hold SMs for that long).  If a
+ * wait runs out the kernel returns, y is unspecified and
+ * cudallm_device_status(stream, ...) reports CUDALLM_ERR_DEVICE_TIMEOUT.
+ * Everything else takes two plain kernels (moments, then normalisation; x is
+ * read twice, the second time from L2 when all of it fits).  Both give results
+ * within the bound above; they differ in the last bits because the partial
+ * moments are grouped differently.  Equal inputs give equal bits on either.
  * Errors: INVALID_DIM (negative, batch >= 2^31, m > 2^40, eps negative or not
  * finite), INVALID_POINTER (x or y NULL), MISALIGNED (4 bytes), WORKSPACE (an
  * external workspace is set and too small), UNSUPPORTED_DEVICE, CUDA.
