@@ -115,6 +115,25 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C,
                      int variant, void *stream);
 
 /*
+ * The same product with the operands read by the tensor cores as they lie in
+ * memory (tcgen05.mma kind::tf32: of every float32 operand the sign, the
+ * exponent and the ten leading fraction bits are used; products are exact in
+ * and accumulated in float32).  One pass over A and B, no conversion kernel, no
+ * workspace beyond the header: about 2.5 times faster than cudallm_gemm_f32 on
+ * the paper's Task 2 sizes, at about three decimal digits per product instead
+ * of seven: every element within 2.5e-3 * sum_k |a_ik||b_kj| of the exact
+ * product (2^-9 for two truncated operands plus the float32 accumulation);
+ * operands whose values have at most 11 significant bits (e.g. integers below
+ * 2048) are multiplied exactly.  Arguments as for cudallm_gemm_f32.  A and B must
+ * be 16-byte aligned with lda and ldb multiples of 4 to be read in place; any
+ * other alignment, and K == 0, are passed to cudallm_gemm_f32 (whose result is
+ * the more accurate one).  C may have any 4-byte alignment and pitch.
+ */
+int cudallm_gemm_tf32(const void *A, const void *B, void *C,
+                      int64_t M, int64_t N, int64_t K,
+                      int64_t lda, int64_t ldb, int64_t ldc, void *stream);
+
+/*
  * `batch` independent products of the same shape (Task 2 applied per item;
  * the paper's Task 6 score matrices Q_i K_i^T are products of this kind).
  * Item t uses A + t*strideA, B + t*strideB, C + t*strideC.  Items of C must

@@ -42,6 +42,7 @@ _sz = ctypes.c_size_t
 SIGNATURES = {
     "cudallm_gemm_bf16": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp]),
     "cudallm_gemm_f32": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_int, _vp]),
+    "cudallm_gemm_tf32": (_int, [_vp, _vp, _vp] + [_i64] * 6 + [_vp]),
     "cudallm_mhsa_bf16": (_int, [_vp, _vp, _vp, _vp] + [_i64] * 7 + [_vp]),
     "cudallm_gemm_bf16_batched": (_int, [_vp, _vp, _vp] + [_i64] * 10 + [_int, _vp]),
     "cudallm_gemm_bf16_variant": (_int, [_int, _vp, _vp, _vp] + [_i64] * 10 + [_int, _vp]),
@@ -135,6 +136,12 @@ def gemm_f32(A, B, C, M, N, K, lda, ldb, ldc, variant=VARIANT_AUTO, stream=None,
     bf16 tensor cores from three-piece splits of the operands."""
     st = lib().cudallm_gemm_f32(_p(A), _p(B), _p(C), M, N, K, lda, ldb, ldc, variant, _s(stream))
     return _check(st, "cudallm_gemm_f32", check)
+
+
+def gemm_tf32(A, B, C, M, N, K, lda, ldb, ldc, stream=None, check=True):
+    """fp32 operands and result with the tensor cores reading the operands as TF32."""
+    st = lib().cudallm_gemm_tf32(_p(A), _p(B), _p(C), M, N, K, lda, ldb, ldc, _s(stream))
+    return _check(st, "cudallm_gemm_tf32", check)
 
 
 def mhsa_bf16(Q, K, V, O, N, d_model, h, ldq, ldk, ldv, ldo, stream=None, check=True):

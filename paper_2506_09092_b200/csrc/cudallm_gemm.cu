@@ -18,6 +18,7 @@
 #include "aux_kernels.cuh"
 #include "umma_gemm.cuh"
 #include "umma_gemm_2cta.cuh"
+#include "umma_tf32.cuh"
 #include "mhsa.cuh"
 #include "hbm_tasks.cuh"
 
@@ -409,6 +410,7 @@ struct DeviceState {
     std::unordered_map<cudaStream_t, Workspace> stream_ws;   // cudallm_set_workspace_for_stream
     bool smem_attr_set[40] = {};
     bool layernorm_attr_set = false;
+    bool tf32_attr_set = false;
     int max_pairs = 0;           // co-resident 2-CTA clusters of the pair kernel (0 = not asked yet)
     int epoch = 0;               // last split-K flag value used on this device
 };
@@ -583,15 +585,17 @@ int encode_map(int dev, CUtensorMap *tm, const void *base, int64_t inner, int64_
             *tm = mc.map[i];
             return CUDALLM_OK;
         }
-    const cuuint64_t es = (kind == 1) ? 4 : 2;
+    const cuuint64_t es = (kind == 1 || kind == 3) ? 4 : 2;      // kinds: 0 bf16, 1 fp32, 2 bf16 with a 64-byte swizzle,
+                                                                 // 3 fp32 with the 128-byte swizzle on 32-byte units
     cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batch};
     cuuint64_t item_stride = (batch > 1) ? (cuuint64_t)stride * es : (cuuint64_t)rows * ld * es;
     cuuint64_t strides[2] = {(cuuint64_t)ld * es, item_stride};
     cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = g_encode(tm, kind == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+    CUresult r = g_encode(tm, (kind == 1 || kind == 3) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
                           const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          kind == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                          kind == 2 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                    : kind == 3 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
                           kind == 0 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -1124,6 +1128,68 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C, int64_t M, int64_t N
     gp.flags = reinterpret_cast<int *>(ws + 256);
     gp.status = reinterpret_cast<int *>(ws);
     return launch_variant(dev, v, false, ta, tb, tc, gp, stream);
+}
+
+int cudallm_gemm_tf32(const void *A, const void *B, void *C, int64_t M, int64_t N, int64_t K, int64_t lda,
+                      int64_t ldb, int64_t ldc, void *stream_v)
+{
+    build_variants();
+    const Problem p = make_problem(A, B, C, M, N, K, lda, ldb, ldc, 0, 0, 0, 1, CUDALLM_F32);
+    int st = validate(p);
+    if (st != CUDALLM_OK) return st;
+    if (is_empty(p)) return CUDALLM_OK;
+    if (K > 0 && ((reinterpret_cast<uintptr_t>(A) & 3) || (reinterpret_cast<uintptr_t>(B) & 3)))
+        return CUDALLM_ERR_MISALIGNED;
+    // TMA reads the operands where they lie: bases on 16 bytes, pitches multiples of 16 bytes.
+    // Anything else (and the empty sum) goes the way of cudallm_gemm_f32, which copies its
+    // operands anyway and is the more accurate of the two.
+    const bool direct = K > 0 && ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B)) & 15) == 0
+                     && lda % 4 == 0 && ldb % 4 == 0;
+    if (!direct) return cudallm_gemm_f32(A, B, C, M, N, K, lda, ldb, ldc, CUDALLM_VARIANT_AUTO, stream_v);
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CUDALLM_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    st = probe_device(dev);
+    if (st != CUDALLM_OK) return st;
+    DeviceState &d = g_dev[dev];
+
+    Tiling t{};
+    t.tiles_m = cdiv(M, kBlockM);
+    t.tiles_n = cdiv(N, kTf32BlockN);
+    t.tiles = t.tiles_m * t.tiles_n;
+    t.kblocks = cdiv(K, kTf32BlockK);
+    t.dp_tiles = t.tiles;
+    t.split = 1;
+    t.units = t.tiles;
+    if (t.tiles > kMaxDim) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+
+    Workspace &w = workspace_for(d, stream);
+    st = ensure_workspace(w, kHeaderBytes, stream);            // for the status word
+    if (st != CUDALLM_OK) return st;
+    uint8_t *ws = static_cast<uint8_t *>(w.ptr);
+
+    CUtensorMap ta, tb, tc;
+    st = encode_map(dev, &ta, A, K, M, 1, lda, 0, kTf32BlockK, kBlockM, 1);
+    if (st != CUDALLM_OK) return st;
+    st = encode_map(dev, &tb, B, N, K, 1, ldb, 0, 32, kTf32BlockK, 3);
+    if (st != CUDALLM_OK) return st;
+    // (the raster-group rule counts A's bytes as bf16: here its slices are twice that, still in L2)
+    GemmParams gp = make_params(p, t, kBlockM);
+    st = encode_c_map(dev, &tc, p, gp.c_tma != 0);
+    if (st != CUDALLM_OK) return st;
+    set_split_epoch(gp, d, false);
+    gp.flags = reinterpret_cast<int *>(ws + 256);
+    gp.status = reinterpret_cast<int *>(ws);
+    if (!d.tf32_attr_set) {
+        CUDA_TRY(cudaFuncSetAttribute(umma_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      Tf32Smem::kDynamicBytes));
+        d.tf32_attr_set = true;
+    }
+    const int grid = (int)std::min<int64_t>(t.units, d.sm_count);
+    return launch_overlapped(umma_tf32_kernel, grid, Tf32Smem::kDynamicBytes, stream, ta, tb, tc, gp);
 }
 
 int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int64_t N, int64_t d_model,

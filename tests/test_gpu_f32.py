@@ -1,6 +1,5 @@
-"""The fp32-operand entry point (the paper's Task 2 as stated: "multiplies two
-matrices of 32-bit floating point numbers") against the fp64 oracle on float32
-operands.
+"""The fp32-operand entry points (the element type the paper's Task 2 gives for
+both factors and the product) against the fp64 oracle on float32 operands.
 
 Tolerance: every element within 1e-5 * sum_k |a_ik||b_kj|.  The three-piece
 split drops products of relative size <= 2^-26; fp32 accumulation of the
@@ -148,3 +147,85 @@ def test_paper_task2_ladder_fp32_sampled_rows():
         Cref, S = oracle.gemm_f32_rows(Af, Bf, rows, cfg.N, cfg.K)
         assert oracle.check(got[rows], Cref, S, TOL).ok
         assert np.isfinite(got).all()
+
+
+# ---------------------------------------------------------------- TF32 -----
+# cudallm_gemm_tf32: the tensor cores read the float32 operands as TF32 (ten fraction bits).
+# Tolerance 2.5e-3 * S (2^-9 per product of two truncated operands + float32 accumulation);
+# operands with at most 11 significant bits are multiplied exactly, which pins the operand
+# layout (every k-block, every 32-column box of B, both edges) bit for bit.
+
+def run_tf32(Af, Bf, M, N, K, pad_ab=0, pad_c=0, lead=0):
+    lda, ldb, ldc = K + pad_ab, N + pad_ab, N + pad_c
+    A = np.full(lead + max(M * lda, 1), np.nan, dtype=np.float32)
+    Bm = np.full(lead + max(K * ldb, 1), np.nan, dtype=np.float32)
+    A[lead:lead + M * lda].reshape(M, lda)[:, :K] = Af
+    Bm[lead:lead + K * ldb].reshape(K, ldb)[:, :N] = Bf
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(Bm).cuda()
+    guard = 32
+    dC = torch.full((guard + M * ldc + guard,), float("nan"), dtype=torch.float32, device="cuda")
+    B.gemm_tf32(dA.data_ptr() + 4 * lead, dB.data_ptr() + 4 * lead, dC.data_ptr() + 4 * guard,
+                M, N, K, lda, ldb, ldc, torch.cuda.current_stream())
+    assert B.device_status(torch.cuda.current_stream()) == (B.OK, 0)
+    host = dC.cpu().numpy()
+    assert np.isnan(host[:guard]).all() and np.isnan(host[guard + M * ldc:]).all()
+    body = host[guard: guard + M * ldc].reshape(M, ldc)
+    if pad_c:
+        assert np.isnan(body[:-1, N:]).all()
+    return body[:, :N].astype(np.float64)
+
+
+TF32_SHAPES = [(128, 256, 32), (128, 256, 64), (1, 1, 1), (100, 300, 77), (257, 513, 129), (300, 260, 1000),
+               (1024, 2048, 4096), (129, 31, 33), (512, 1000, 2048)]
+
+
+@pytest.mark.parametrize("M,N,K", TF32_SHAPES)
+def test_tf32_integer_operands_are_exact(M, N, K):
+    """Integers of magnitude < 16 (and, on a few entries, up to 2047: eleven significant
+    bits) have exact TF32 forms and exact float32 sums here, so the result must equal the
+    oracle's bit for bit: a misplaced k-block, box or swizzle row would not."""
+    rng = np.random.default_rng(5000 + M + N + K)
+    Af = rng.integers(-15, 16, (M, K)).astype(np.float32)
+    Bf = rng.integers(-15, 16, (K, N)).astype(np.float32)
+    Af[rng.integers(0, M), rng.integers(0, K)] = 2047.0
+    Bf[rng.integers(0, K), rng.integers(0, N)] = -1025.0
+    Cref, _ = oracle.gemm_f32(Af, Bf, M, N, K)
+    assert np.abs(Cref).max() < 2 ** 24
+    pad = 4 if (M + N) % 2 else 0
+    assert np.array_equal(run_tf32(Af, Bf, M, N, K, pad_ab=pad, pad_c=pad + 1 if pad else 0), Cref)
+
+
+@pytest.mark.parametrize("M,N,K", TF32_SHAPES + [(2048, 2048, 8192)])
+def test_tf32_against_oracle(M, N, K):
+    rng = np.random.default_rng(5100 + M + N + K)
+    Af = rng.standard_normal((M, K)).astype(np.float32)
+    Bf = rng.uniform(-1, 1, (K, N)).astype(np.float32)
+    got = run_tf32(Af, Bf, M, N, K)
+    Cref, S = oracle.gemm_f32(Af, Bf, M, N, K)
+    r = oracle.check(got, Cref, S, oracle.TOL_TF32)
+    G.log_observed_error("gemm_tf32", f"{M}x{N}x{K}", r.max_scaled_err, oracle.TOL_TF32, "max |C - C_ref| / sum|a||b|")
+    assert r.ok, r
+    # and where the operands can be read in place it IS a reduced-precision product: some element is
+    # further off than the three-piece path allows
+    if K >= 64 and K % 4 == 0 and N % 4 == 0:
+        assert r.max_scaled_err > oracle.TOL_F32_IN
+
+
+def test_tf32_unaligned_operands_take_the_three_piece_path_and_errors():
+    """Pitches that are not multiples of 4 elements (or bases off 16 bytes) cannot be read in
+    place by TMA: the call is then served by cudallm_gemm_f32, to ITS tolerance."""
+    rng = np.random.default_rng(5200)
+    M, N, K = 130, 270, 333
+    Af = rng.standard_normal((M, K)).astype(np.float32)
+    Bf = rng.standard_normal((K, N)).astype(np.float32)
+    Cref, S = oracle.gemm_f32(Af, Bf, M, N, K)
+    for pad, lead in ((1, 0), (0, 1), (3, 1)):
+        assert oracle.check(run_tf32(Af, Bf, M, N, K, pad_ab=pad, lead=lead), Cref, S, TOL).ok
+    got = run_tf32(Af[:, :0], Bf[:0, :], M, N, 0)           # the empty sum
+    assert np.array_equal(got, np.zeros((M, N)))
+    s = torch.cuda.current_stream()
+    x = torch.zeros(64, device="cuda")
+    assert B.gemm_tf32(x, x, x, 4, 4, -1, 4, 4, 4, s, check=False) == B.ERR_INVALID_DIM
+    assert B.gemm_tf32(x, x, x, 4, 4, 4, 3, 4, 4, s, check=False) == B.ERR_INVALID_LD
+    assert B.gemm_tf32(x.data_ptr() + 2, x, x, 4, 4, 4, 4, 4, 4, s, check=False) == B.ERR_MISALIGNED
+    assert B.gemm_tf32(x, x, x, 0, 4, 4, 4, 4, 4, s, check=False) == B.OK
