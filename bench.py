@@ -414,6 +414,11 @@ def run_ours(args):
         lambda i: B.gemm_f32(fa, fb, fcs[i & 1], t2.M, t2.N, t2.K, t2.K, t2.N, t2.N, -1, stream),
         f_steps, 3, barrier)
     f_tflops = t2.flops / f_avg / 1e12
+    tf_steps = max(3, min(args.steps, 20))
+    tf_total, tf_avg = time_steps(
+        lambda i: B.gemm_tf32(fa, fb, fcs[i & 1], t2.M, t2.N, t2.K, t2.K, t2.N, t2.N, stream),
+        tf_steps, 3, barrier)
+    tf_tflops = t2.flops / tf_avg / 1e12
 
     # ---------- the paper's Task 6 at its largest size: N = 512, d_model = 512, h = 16 ----------
     aN, aD, aH = 512, 512, 16
@@ -485,7 +490,13 @@ def run_ours(args):
             "value": f_tflops, "unit": "TFLOP/s (2MNK)", "us_per_call": f_avg * 1e6, "steps": f_steps,
             "tensor_rate": {"value": 6 * f_tflops, "unit": "TFLOP/s of bf16 MMA work (6 x 2MNK)",
                             "frac_of_measured_bf16_peak": 6 * f_tflops / peaks["bf16_tflops"]},
-            "note": "inputs 436 MB > L2; fp32-grade accuracy (<= 1e-5 * sum|a||b|, observed ~1e-7)"}
+            "note": "inputs 436 MB > L2; fp32-grade accuracy (<= 1e-5 * sum|a||b|, observed ~1e-7)",
+            "tf32": {"call": "cudallm_gemm_tf32 (operands read in place, tcgen05.mma kind::tf32)",
+                     "value": tf_tflops, "unit": "TFLOP/s (2MNK)", "us_per_call": tf_avg * 1e6, "steps": tf_steps,
+                     "peak": peaks["bf16_tflops"] * 0.5,
+                     "frac": tf_tflops / (peaks["bf16_tflops"] * 0.5),
+                     "peak_source": f"half of the bf16 peak {peak_src} (the nominal ratio of the two dense rates)",
+                     "note": "<= 2.5e-3 * sum|a||b| (ten fraction bits per operand)"}}
         line["task6_attention"] = {
             "workload": f"paper Task 6, largest size: N={aN}, d_model={aD}, h={aH} (d_k={aD // aH}), bf16 in, fp32 out",
             "call": "cudallm_mhsa_bf16 (one fused kernel, 64 CTAs)", "us_per_call": a_avg * 1e6,
