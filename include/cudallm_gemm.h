@@ -119,7 +119,7 @@ int cudallm_gemm_f32(const void *A, const void *B, void *C,
  * memory (tcgen05.mma kind::tf32: of every float32 operand the sign, the
  * exponent and the ten leading fraction bits are used; products are exact in
  * and accumulated in float32).  One pass over A and B, no conversion kernel, no
- * workspace beyond the header: about 2.5 times faster than cudallm_gemm_f32 on
+ * workspace beyond the header: about 3 times faster than cudallm_gemm_f32 on
  * the paper's Task 2 sizes, at about three decimal digits per product instead
  * of seven: every element within 2.5e-3 * sum_k |a_ik||b_kj| of the exact
  * product (2^-9 for two truncated operands plus the float32 accumulation);

@@ -1156,8 +1156,14 @@ int cudallm_gemm_tf32(const void *A, const void *B, void *C, int64_t M, int64_t 
     if (st != CUDALLM_OK) return st;
     DeviceState &d = g_dev[dev];
 
+    // CTA pairs (256 x 256 tiles) from two tile rows up; lone CTAs (128 x 256) for one
+    const bool pair = M > kBlockM;
+    if (pair && d.max_pairs == 0) {
+        st = prepare_umma_pair<3, 2, false>(dev, 7);           // asks how many pairs the device holds at once
+        if (st != CUDALLM_OK) return st;
+    }
     Tiling t{};
-    t.tiles_m = cdiv(M, kBlockM);
+    t.tiles_m = cdiv(M, pair ? kPairM : kBlockM);
     t.tiles_n = cdiv(N, kTf32BlockN);
     t.tiles = t.tiles_m * t.tiles_n;
     t.kblocks = cdiv(K, kTf32BlockK);
@@ -1186,7 +1192,13 @@ int cudallm_gemm_tf32(const void *A, const void *B, void *C, int64_t M, int64_t 
     if (!d.tf32_attr_set) {
         CUDA_TRY(cudaFuncSetAttribute(umma_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       Tf32Smem::kDynamicBytes));
+        CUDA_TRY(cudaFuncSetAttribute(umma_tf32_2cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      Tf32PairSmem::kDynamicBytes));
         d.tf32_attr_set = true;
+    }
+    if (pair) {
+        const int pairs = (int)std::min<int64_t>(t.units, d.max_pairs);
+        return launch_overlapped(umma_tf32_2cta_kernel, 2 * pairs, Tf32PairSmem::kDynamicBytes, stream, ta, tb, tc, gp);
     }
     const int grid = (int)std::min<int64_t>(t.units, d.sm_count);
     return launch_overlapped(umma_tf32_kernel, grid, Tf32Smem::kDynamicBytes, stream, ta, tb, tc, gp);

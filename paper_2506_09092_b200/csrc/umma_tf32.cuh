@@ -27,6 +27,7 @@
 // pipe the bound here.
 #pragma once
 #include "umma_gemm.cuh"
+#include "umma_gemm_2cta.cuh"
 
 namespace cudallm {
 
@@ -252,6 +253,221 @@ umma_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// The same product on CTA pairs (cta_group::2), as umma_gemm_2cta_kernel does it
+// for bf16: a cluster of two CTAs owns a 256 x 256 tile, CTA r stages rows
+// [128 r, 128 r + 128) of A and columns [128 r, 128 r + 128) of B (32 instead of
+// 48 KiB per k-block and SM, six stages instead of four), the leader issues
+// 256 x 256 x 8 MMAs for both, and the barriers are laid out as there (the
+// leader's `full`, each CTA's `empty`, no multicast).
+constexpr int kTf32PairStages = 6;
+
+struct Tf32PairSmem {
+    static constexpr int kABytes = kBlockM * kTf32BlockK * 4;        // 16 KiB: this CTA's 128 rows of A
+    static constexpr int kBoxBytes = 32 * kTf32BlockK * 4;
+    static constexpr int kBBytes = (kPairN / 2 / 32) * kBoxBytes;    // 16 KiB: this CTA's 128 columns of B
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kEpiOffset = kTf32PairStages * kStageBytes;
+    static constexpr int kBarOffset = kEpiOffset + kEpiStageBytes;
+    static constexpr int kNumBars = 2 * kTf32PairStages + 4;
+    static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
+    static constexpr int kDynamicBytes = kMiscOffset + 64;
+};
+
+// TMA load whose bytes are counted on a barrier of the pair's leader (cluster address).
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t smem_dst, const CUtensorMap *tm, int x, int y, int z,
+                                                 uint32_t bar_cluster_addr)
+{
+    asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+                 "[%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z),
+                   "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void umma_tf32_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile("{\n\t"
+                 ".reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t"
+                 "}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
+umma_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                      const __grid_constant__ CUtensorMap tmap_c, const GemmParams p)
+{
+    using L = Tf32PairSmem;
+    constexpr int STAGES = kTf32PairStages;
+    constexpr uint32_t kTmemCols = 2 * kPairN;
+
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *smem = smem_raw;
+    const uint32_t smem_base = smem_u32(smem);
+    if (smem_base & 1023u) {                             // (the same in both CTAs of a pair)
+        if (threadIdx.x == 0) report_timeout(p.status, 0, 0x7F);
+        return;
+    }
+    const uint32_t bar_base = smem_base + L::kBarOffset;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L::kMiscOffset);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kMiscOffset + 4);
+
+    const int warp_idx = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                         // 0 = leader
+    const int pair = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);       // leader's is used: one expect_tx arrival + both CTAs' bytes
+            mbar_init(empty_bar(s), 1);      // one commit from the leader
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);      // one commit from the leader
+            mbar_init(tempty_bar(a), 8);     // leader's is used: 4 epilogue warps x 2 CTAs
+        }
+        fence_mbar_init();
+        fence_proxy_async_smem();
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+        if (p.c_tma) prefetch_tensormap(&tmap_c);
+    }
+    if (warp_idx == 1) {
+        tmem_alloc_2cta(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+        tmem_relinquish_2cta();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();              // both CTAs' barriers exist before anyone signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    grid_launch_dependents();
+
+    if (warp_idx == 0) {
+        // ------------------------------------------------ TMA producer ----
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
+            constexpr int half = kPairN / 2;             // columns of B this CTA stages
+            grid_dependency_wait();
+            for (int u = pair; ok && u < p.num_units; u += num_pairs) {
+                const UnitCoord c = decode_unit(p, u);
+                const int row0 = c.m_tile * kPairM + static_cast<int>(rank) * kBlockM;
+                const int col0 = c.n_tile * kPairN + static_cast<int>(rank) * half;
+                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                    if (!mbar_wait<true>(empty_bar(stage), phase ^ 1, abort_flag, p.wait_limit_ns)) {
+                        report_timeout(p.status, kRoleProducer, stage);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t sa = smem_base + stage * L::kStageBytes, sb = sa + L::kABytes;
+                    const uint32_t bar = leader_full0 + 8u * stage;
+                    if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * L::kStageBytes);
+                    tma_load_3d_pair(sa, &tmap_a, kb * kTf32BlockK, row0, c.b, bar);
+#pragma unroll
+                    for (int j = 0; j < half / 32; ++j)
+                        tma_load_3d_pair(sb + j * L::kBoxBytes, &tmap_b, col0 + 32 * j, kb * kTf32BlockK, c.b, bar);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp_idx == 1) {
+        // ------------------------------------- MMA issuer (leader only) ----
+        if (lane == 0 && rank == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            constexpr uint32_t idesc = make_idesc_tf32(kPairM, kPairN);
+            const uint32_t empty0_cta0 = map_to_cta(empty_bar(0), 0);
+            const uint32_t empty0_cta1 = map_to_cta(empty_bar(0), 1);
+            const uint32_t tfull0_cta0 = map_to_cta(tfull_bar(0), 0);
+            const uint32_t tfull0_cta1 = map_to_cta(tfull_bar(0), 1);
+            for (int u = pair; ok && u < p.num_units; u += num_pairs) {
+                const UnitCoord c = decode_unit(p, u);
+                if (!mbar_wait<true>(tempty_bar(acc), acc_phase ^ 1, abort_flag, p.wait_limit_ns)) {
+                    report_timeout(p.status, kRoleMma, 0x40 + acc);
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kPairN;
+                uint32_t accumulate = 0;
+                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                    if (!mbar_wait<true>(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) {
+                        report_timeout(p.status, kRoleMma, stage);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = smem_base + stage * L::kStageBytes, sb = sa + L::kABytes;
+#pragma unroll
+                    for (int i = 0; i < kTf32BlockK / 8; ++i) {
+                        umma_tf32_pair(d_tmem, make_smem_desc_sw128(sa + 32 * i, 16, 1024),
+                                       make_smem_desc_sw128_32b(sb + 1024 * i, L::kBoxBytes, 512), idesc, accumulate);
+                        accumulate = 1;
+                    }
+                    umma_commit_pair(empty0_cta0 + 8u * stage);      // frees the stage in both CTAs
+                    umma_commit_pair(empty0_cta1 + 8u * stage);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                umma_commit_pair(tfull0_cta0 + 8u * acc);
+                umma_commit_pair(tfull0_cta1 + 8u * acc);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ---------------------------------------------------- epilogue ----
+        const int quad = warp_idx & 3;
+        const int epi_tid = quad * 32 + lane;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        uint32_t sel = 0;
+        const uint32_t stage_addr = smem_base + L::kEpiOffset + quad * kEpiWarpBytes;
+        grid_dependency_wait();
+        for (int u = pair; u < p.num_units; u += num_pairs) {
+            const UnitCoord c = decode_unit(p, u);
+            bool ok = mbar_wait<true>(tfull_bar(acc), acc_phase, abort_flag, p.wait_limit_ns);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0x80 + acc);
+                break;
+            }
+            tc_fence_after();
+            if (!epilogue_tile<kPairN, false>(p, c, c.m_tile * kPairM + static_cast<int>(rank) * kBlockM + epi_tid,
+                                              tmem_base + acc * kPairN + (static_cast<uint32_t>(quad * 32) << 16),
+                                              quad, lane, static_cast<int>(rank), 2, abort_flag, &tmap_c,
+                                              stage_addr, sel)) {
+                if (lane == 0) report_timeout(p.status, kRoleEpilogue, 0xC0);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(map_to_cta(tempty_bar(acc), 0));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+        if (lane == 0) bulk_wait_group_read<0>();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();              // nobody leaves while the peer may still signal or read it
+    if (warp_idx == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc_2cta(tmem_base, kTmemCols);
     }
 }
 

@@ -175,8 +175,11 @@ def run_tf32(Af, Bf, M, N, K, pad_ab=0, pad_c=0, lead=0):
     return body[:, :N].astype(np.float64)
 
 
+# lone CTAs up to M = 128, CTA pairs above; (100, 300, 77), (257, 513, 129) and (129, 31, 33) have
+# pitches that are not multiples of 4 and take the three-piece path
 TF32_SHAPES = [(128, 256, 32), (128, 256, 64), (1, 1, 1), (100, 300, 77), (257, 513, 129), (300, 260, 1000),
-               (1024, 2048, 4096), (129, 31, 33), (512, 1000, 2048)]
+               (1024, 2048, 4096), (129, 31, 33), (512, 1000, 2048), (64, 512, 256), (128, 1000, 516),
+               (129, 260, 36), (384, 256, 32), (256, 256, 8), (1000, 4, 4)]
 
 
 @pytest.mark.parametrize("M,N,K", TF32_SHAPES)
