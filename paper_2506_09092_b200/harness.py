@@ -517,11 +517,12 @@ def _main(argv=None):
     ap.add_argument("--table", default=None, help="with --search: JSON file to record the winner in")
     ap.add_argument("--dispatch", default=None,
                     help="a table file, or 'packaged': enter its records into the library's dispatch table first")
-    ap.add_argument("--task", default=None, choices=["transpose", "sum", "dot", "layernorm", "attention"],
-                    help="time one of the other tasks (8, 14, 15, 4, 6) instead of a GEMM configuration")
+    ap.add_argument("--task", default=None, choices=["transpose", "sum", "dot", "layernorm", "attention", "tf32", "f32"],
+                    help="time one of the other tasks (8, 14, 15, 4, 6; tf32 / f32: Task 2 with float32 operands "
+                         "through cudallm_gemm_tf32 / cudallm_gemm_f32) instead of a GEMM configuration")
     ap.add_argument("--size", type=int, default=None,
                     help="with --task: N (transpose: N x N; sum, dot: N elements; layernorm: (16, 4, N, N); "
-                         "attention: N queries and keys)")
+                         "attention: N queries and keys; tf32, f32: A (N x 4096) x B (4096 x 2048))")
     ap.add_argument("--layernorm-kernels", default="auto", choices=["auto", "two", "persistent"],
                     help="with --task layernorm: let the library choose by size, or force the two plain "
                          "kernels / the persistent kernel (cudallm_debug_set)")
@@ -577,6 +578,20 @@ def task_problem(task: str, size: int, nsets: int | None = None):
     from . import inputs as gi
 
     st = torch.cuda.current_stream()
+    if task in ("tf32", "f32"):
+        # the paper's Task 2 ladder: A (size x 4096) x B (4096 x 2048), float32
+        M, K, N = size, 4096, 2048
+        bytes_ = 4 * (M * K + K * N + M * N)
+        n = nsets or max(2, min(8, (400 << 20) // bytes_ + 1))
+        gen = torch.Generator(device="cuda").manual_seed(700)
+        A = [torch.randn(M, K, device="cuda", generator=gen) for _ in range(n)]
+        Bm = [torch.randn(K, N, device="cuda", generator=gen) for _ in range(n)]
+        C = [torch.empty(M, N, device="cuda") for _ in range(n)]
+        if task == "tf32":
+            return (lambda i: B.gemm_tf32(A[i % n], Bm[i % n], C[i % n], M, N, K, K, N, N, st)), bytes_, \
+                f"A ({M} x {K}) x B ({K} x {N}), float32 as TF32"
+        return (lambda i: B.gemm_f32(A[i % n], Bm[i % n], C[i % n], M, N, K, K, N, N, -1, st)), bytes_, \
+            f"A ({M} x {K}) x B ({K} x {N}), float32 in three bf16 pieces"
     if task == "attention":
         # Task 6: the paper's (N, d_model, h) with this N, else about N columns, 32 per head
         paper = {64: (32, 4), 128: (64, 8), 256: (128, 8), 384: (256, 16), 512: (512, 16)}
@@ -620,15 +635,19 @@ def _task_main(args):
     import torch
     from . import binding as B
 
-    default = {"transpose": 8192, "sum": 1 << 28, "dot": 1 << 27, "layernorm": 512, "attention": 512}
+    default = {"transpose": 8192, "sum": 1 << 28, "dot": 1 << 27, "layernorm": 512, "attention": 512,
+               "tf32": 1 << 14, "f32": 1 << 14}
     size = args.size or default[args.task]
     if args.task == "layernorm":
         B.debug_set(B.DEBUG_LAYERNORM_PATH, {"auto": 0, "two": 1, "persistent": 2}[args.layernorm_kernels])
     launch, bytes_, what = task_problem(args.task, size, args.sets)
     t = performance_profiler(launch, iters=args.iters, warmup=args.warmup)
     code, detail = B.device_status(torch.cuda.current_stream())
-    print(json.dumps({"task": args.task, "input": what, "status": code, "us_min": t["min_s"] * 1e6,
-                      "us_median": t["median_s"] * 1e6, "gbs": bytes_ / t["median_s"] / 1e9}), flush=True)
+    rec = {"task": args.task, "input": what, "status": code, "us_min": t["min_s"] * 1e6,
+           "us_median": t["median_s"] * 1e6, "gbs": bytes_ / t["median_s"] / 1e9}
+    if args.task in ("tf32", "f32"):
+        rec["tflops"] = 2.0 * size * 4096 * 2048 / t["median_s"] / 1e12
+    print(json.dumps(rec), flush=True)
 
 
 if __name__ == "__main__":
