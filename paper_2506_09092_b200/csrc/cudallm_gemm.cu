@@ -1162,18 +1162,21 @@ int cudallm_gemm_tf32(const void *A, const void *B, void *C, int64_t M, int64_t 
         st = prepare_umma_pair<3, 2, false>(dev, 7);           // asks how many pairs the device holds at once
         if (st != CUDALLM_OK) return st;
     }
-    Tiling t{};
-    t.tiles_m = cdiv(M, pair ? kPairM : kBlockM);
-    t.tiles_n = cdiv(N, kTf32BlockN);
-    t.tiles = t.tiles_m * t.tiles_n;
-    t.kblocks = cdiv(K, kTf32BlockK);
-    t.dp_tiles = t.tiles;
-    t.split = 1;
-    t.units = t.tiles;
-    if (t.tiles > kMaxDim) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+    // Tiles as for the bf16 kernels of the same shape (a k-block is 128 bytes of a row of A in
+    // both), the tiles of a ragged last wave split along K.
+    Variant tv{};
+    tv.family = pair ? kUmmaPair : kUmma;
+    tv.block_n = kTf32BlockN;
+    tv.split_k = kTailSplit;
+    tv.per_sm = 1;
+    Problem q = p;
+    q.K = 2 * K;                                               // in 2-byte elements
+    const Tiling t = tiling_for(tv, q, pair ? d.max_pairs : d.sm_count);
+    if (t.units > kMaxDim || t.helper_tiles > kMaxHelperTiles || t.partial_bytes > kMaxPartialBytes)
+        return CUDALLM_ERR_UNSUPPORTED_SHAPE;
 
     Workspace &w = workspace_for(d, stream);
-    st = ensure_workspace(w, kHeaderBytes, stream);            // for the status word
+    st = ensure_workspace(w, kHeaderBytes + (size_t)t.partial_bytes, stream);
     if (st != CUDALLM_OK) return st;
     uint8_t *ws = static_cast<uint8_t *>(w.ptr);
 
@@ -1186,7 +1189,8 @@ int cudallm_gemm_tf32(const void *A, const void *B, void *C, int64_t M, int64_t 
     GemmParams gp = make_params(p, t, kBlockM);
     st = encode_c_map(dev, &tc, p, gp.c_tma != 0);
     if (st != CUDALLM_OK) return st;
-    set_split_epoch(gp, d, false);
+    set_split_epoch(gp, d, t.split > 1);
+    gp.partials = reinterpret_cast<float *>(ws + kHeaderBytes);
     gp.flags = reinterpret_cast<int *>(ws + 256);
     gp.status = reinterpret_cast<int *>(ws);
     if (!d.tf32_attr_set) {
