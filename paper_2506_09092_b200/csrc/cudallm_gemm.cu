@@ -387,9 +387,15 @@ int select_variant(const Problem &p, bool no_waits = false)
 }
 
 // --------------------------------------------------------------- workspace --
-// Layout: [status 256 B][split-K flags][split-K partial tiles][packed A][packed B]
+// Layout: [status 256 B][split-K flags][LayerNorm entries][split-K partial tiles][packed A][packed B]
+// The two areas of the header are kept apart because of what their words may hold: a flag word
+// is zero or the epoch of some launch, and a kernel takes it for raised when it equals ITS
+// epoch; an entry word is a 32-bit payload (any bits) under a 32-bit epoch tag.  A payload
+// left behind in a flag word could one day equal the epoch of a later launch.
 constexpr size_t kFlagBytes = kMaxHelperTiles * 4 * sizeof(int);
-constexpr size_t kHeaderBytes = 256 + kFlagBytes;    // zeroed when a workspace is created
+constexpr size_t kEntryBytes = size_t(1) << 20;      // the persistent LayerNorm kernel's exchange area
+constexpr size_t kEntryOffset = 256 + kFlagBytes;
+constexpr size_t kHeaderBytes = kEntryOffset + kEntryBytes;   // zeroed when a workspace is created
 constexpr int kMaxDevices = 64;
 
 // A workspace: the device's default one (allocated and grown by the library unless the

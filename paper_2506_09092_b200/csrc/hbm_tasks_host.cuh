@@ -131,10 +131,10 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
             const int64_t lead = std::max<int64_t>(chunks + (chunks + 1) / 2,
                                                    std::min<int64_t>((kLnSlots - 8) * chunks,
                                                                      (int64_t(34) << 20) / (G * kLnChunkBytes)));
-            // The entries live in the flag area of the workspace header, where every 32-bit word is
-            // either zero or an epoch of an earlier launch: a stale word cannot pass for this
-            // launch's tag.  The area holds kFlagBytes / 48 entries; larger batches go in pieces.
-            const int64_t per_launch = std::max<int64_t>(1, int64_t(kFlagBytes / 48) / G);
+            // The entries live in their own area of the workspace header, whose 8-byte words are
+            // zero or an earlier launch's (payload, epoch) pairs: a stale word cannot pass for
+            // this launch's tag.  The area holds kEntryBytes / 48 entries; larger batches go in pieces.
+            const int64_t per_launch = std::max<int64_t>(1, int64_t(kEntryBytes / 48) / G);
             Workspace &w = workspace_for(d, stream);
             st = ensure_workspace(w, kHeaderBytes, stream);
             if (st != CUDALLM_OK) return st;
@@ -151,7 +151,7 @@ int cudallm_layernorm_f32(const float *x, const float *gamma, const float *beta,
                 sp.batch = (int)std::min<int64_t>(per_launch, batch - s0); sp.ctas = (int)G; sp.lead = (int)lead;
                 sp.eps = (double)eps;
                 sp.inv_m = 1.0 / (double)m;
-                sp.entries = reinterpret_cast<unsigned long long *>(ws + 256);
+                sp.entries = reinterpret_cast<unsigned long long *>(ws + kEntryOffset);
                 sp.epoch = next_epoch(d);
                 sp.tag_post = g_skew_next_flags.exchange(0) ? (sp.epoch ^ 0x40000000) : sp.epoch;
                 sp.status = reinterpret_cast<int *>(ws);

@@ -44,7 +44,7 @@ def test_caller_provided_workspace():
         for vn in ("umma_n128_sk4", "umma2_n256_sk2", "umma_n64"):
             vals, _, g = G.run_gemm(Ap, Bp, M, N, K, lda, ldb, ldc, gi.F32, variant=names[vn])
             assert g and oracle.check(vals[0], Cref, S, G.tol_for(gi.F32)).ok, vn
-        small = torch.zeros(1 << 21, dtype=torch.uint8, device="cuda")   # header fits, the rest does not
+        small = torch.zeros(3 << 20, dtype=torch.uint8, device="cuda")   # the header (2 MiB + 256 B) fits, the rest does not
         B.set_workspace(small, small.numel())
         dA = G.to_device_bits(gi.embed(bits(np.ones((600, 1030))), 1031))
         dB = G.to_device_bits(gi.embed(bits(np.ones((1030, 3000))), 3003))
