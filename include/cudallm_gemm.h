@@ -229,18 +229,20 @@ int cudallm_gemm_bf16_splitk_noalloc(const void *A, const void *B, void *C,
                                      int out_dtype, int split_k, void *stream);
 
 /*
- * Multi-head self-attention for short sequences: the paper's benchmark Task 6,
+ * Multi-head self-attention: the paper's benchmark Task 6,
  *   O = Concat(head_1, ..., head_h),  head_i = softmax(Q_i K_i^T / sqrt(d_k)) V_i,
  * with d_k = d_model / h and Q_i, K_i, V_i the i-th head's partition (columns
  * [i d_k, (i+1) d_k)) of Q, K, V.  The softmax runs over the keys.
  *   Q, K, V : bf16, N x d_model, row strides ldq, ldk, ldv >= d_model (read only)
  *   O       : fp32, N x d_model, row stride ldo >= d_model; padding untouched
  * One fused kernel: scores in tensor memory, softmax in registers,
- * probabilities rounded to bf16 for the second product, fp32 accumulation.
- * Limits (the paper's sizes go up to N = 512, d_model = 512, h = 16):
- * 1 <= N <= 512; h divides d_model; d_k a multiple of 8, at most 32; Q, K, V
- * 16-byte aligned with ldq, ldk, ldv multiples of 8; O 4-byte aligned.
- * Shapes outside these limits return CUDALLM_ERR_UNSUPPORTED_SHAPE.
+ * probabilities rounded to bf16 for the second product, fp32 accumulation.  Up
+ * to 512 keys (the paper's sizes go up to N = 512, d_model = 512, h = 16) are
+ * handled in one pass; longer sequences in blocks of 512 keys with a running
+ * maximum, the accumulated row rescaled from block to block.
+ * Limits: h divides d_model; d_k a multiple of 8, at most 32; Q, K, V 16-byte
+ * aligned with ldq, ldk, ldv multiples of 8; O 4-byte aligned.  Shapes outside
+ * these limits return CUDALLM_ERR_UNSUPPORTED_SHAPE.
  * N == 0 or d_model == 0 is a successful no-op.
  */
 int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O,

@@ -1226,7 +1226,8 @@ int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int6
     if ((reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V)) & 1)
         return CUDALLM_ERR_MISALIGNED;
     const int64_t dk = d_model / h;
-    if (N > kMhsaMaxKeys || dk > kMhsaMaxDk || dk % 8 || h > 65535) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
+    if (N > kMaxDim) return CUDALLM_ERR_INVALID_DIM;
+    if (dk > kMhsaMaxDk || dk % 8 || h > 65535) return CUDALLM_ERR_UNSUPPORTED_SHAPE;
     if (((reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V)) & 15)
         || ldq % 8 || ldk % 8 || ldv % 8)
         return CUDALLM_ERR_UNSUPPORTED_SHAPE;
@@ -1249,7 +1250,7 @@ int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int6
     mp.V = static_cast<const __nv_bfloat16 *>(V);
     mp.O = static_cast<float *>(O);
     mp.N = (int)N; mp.h = (int)h; mp.dk = (int)dk;
-    mp.keys_pad = (int)round_up(N, 32);
+    mp.keys_pad = N <= kMhsaMaxKeys ? (int)round_up(N, 32) : kMhsaMaxKeys;   // keys per block
     mp.dkp = (int)round_up(dk, 16);
     mp.tmem_cols = 64;                                  // the second product writes dkp + 16 <= 48 columns
     while (mp.tmem_cols < mp.keys_pad) mp.tmem_cols *= 2;
@@ -1258,11 +1259,14 @@ int cudallm_mhsa_bf16(const void *Q, const void *K, const void *V, void *O, int6
     mp.status = static_cast<int *>(w.ptr);
     const MhsaSmem L = mhsa_smem_layout(mp.keys_pad, mp.dkp);
     if (!d.smem_attr_set[8]) {
-        CUDA_TRY(cudaFuncSetAttribute(mhsa_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(mhsa_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(mhsa_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         d.smem_attr_set[8] = true;
     }
     dim3 grid((unsigned)cdiv(N, kMhsaRows), (unsigned)h);
-    return launch_serialised_smem(mhsa_kernel, grid, dim3(kMhsaThreads), (size_t)L.total, stream, mp);
+    if (N > kMhsaMaxKeys)
+        return launch_serialised_smem(mhsa_kernel<true>, grid, dim3(kMhsaThreads), (size_t)L.total, stream, mp);
+    return launch_serialised_smem(mhsa_kernel<false>, grid, dim3(kMhsaThreads), (size_t)L.total, stream, mp);
 }
 
 size_t cudallm_host_staging_bytes(int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,

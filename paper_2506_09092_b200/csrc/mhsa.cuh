@@ -3,8 +3,12 @@
 //   head_i = softmax(Q_i K_i^T / sqrt(d_k)) V_i,   O = Concat(head_1 .. head_h)
 //
 // Q, K, V are N x d_model bf16, row-major; head i owns columns [i d_k, (i+1) d_k).
-// One CTA computes 128 query rows of one head, for N <= 512 keys and d_k <= 32
-// (the paper's sizes go up to N = 512, d_model = 512, h = 16):
+// One CTA computes 128 query rows of one head for d_k <= 32 (the paper's sizes go up
+// to N = 512, d_model = 512, h = 16).  Up to 512 keys are handled in one pass, steps
+// 1 to 5 below; longer sequences in blocks of 512 keys with a running maximum: a
+// block's probabilities are taken relative to the maximum so far, the row's
+// accumulated output and sum (registers) are scaled by exp(old max - new max) and the
+// block's product is added (step 6).
 //
 //   1. all threads copy Q_i (128 x d_k), K_i (N x d_k) and V_i (N x d_k) into
 //      shared memory, directly in the tensor core's unswizzled operand layouts
@@ -29,8 +33,12 @@
 //      the block goes through shared memory so that a warp's store covers whole
 //      rows of the head's columns.
 //
-// The two waits on tensor-core completion are bounded like those of the GEMM
-// kernels.
+//   6. (N > 512) the next block of keys: K_i and V_i rows again (step 1), S (2), the
+//      block's maximum joined with the running one, P relative to the new maximum (3),
+//      the block's O and row sum (4) added to the scaled accumulators.
+//
+// The two waits on tensor-core completion per block are bounded like those of the
+// GEMM kernels.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -47,7 +55,7 @@ struct MhsaParams {
     const __nv_bfloat16 *Q, *K, *V;
     float *O;
     int N, h, dk;
-    int keys_pad;           // N rounded up to 32
+    int keys_pad;           // keys per block: N rounded up to 32, or 512 when N > 512
     int dkp;                // d_k rounded up to 16 (K of the first product, N of the second)
     int tmem_cols;          // power of two >= max(keys_pad, 64): tensor-memory columns to allocate
     long long ldq, ldk, ldv, ldo;
@@ -134,6 +142,8 @@ __device__ __forceinline__ void mhsa_exp_chunk(const uint32_t (&r)[32], float sc
     }
 }
 
+// MULTI: more than one block of keys (N > 512); the one-block instance keeps no accumulators.
+template <bool MULTI>
 __global__ void __launch_bounds__(kMhsaThreads, 1)
 mhsa_kernel(const MhsaParams p)
 {
@@ -166,145 +176,190 @@ mhsa_kernel(const MhsaParams p)
     grid_launch_dependents();
     grid_dependency_wait();                           // (launched with programmatic stream serialisation)
 
-    // ---- 1. operands -> shared memory, in core-matrix order -------------------
-    // One list of 16-byte pieces: the rows of Q, then K's, then V's, the d_k chunks of a
-    // row on neighbouring lanes (at the largest size, N = 512 and d_k = 32, eighteen per thread).
+    const uint32_t t_row_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const int kshift = kchunks == 4 ? 2 : 1;          // kchunks is 2 or 4
-    const int total = (kMhsaRows + 2 * p.keys_pad) << kshift;
-    // Asynchronous 16-byte copies straight into shared memory (a piece outside the
-    // operand -- a padding row or d_k chunk -- copies zero source bytes: it is zero-filled).
-    for (int i = tid; i < total; i += kMhsaThreads) {
-        const __nv_bfloat16 *src = p.Q;               // (any valid address: no byte of it is read)
-        uint32_t bytes = 0;
-        int dst;
-        const int c = i & (kchunks - 1);
-        int r = i >> kshift;
-        const bool live = c * 8 < p.dk;
-        if (r < kMhsaRows) {                          // Q: row within the block
-            const int row = q0 + r;
-            dst = L.q + c * L.lbo_q + r * 16;
-            if (row < p.N && live) { src = p.Q + row * p.ldq + col0 + c * 8; bytes = 16; }
-        } else if (r < kMhsaRows + p.keys_pad) {
-            r -= kMhsaRows;                           // K: key
-            dst = L.k + c * L.lbo_k + r * 16;
-            if (r < p.N && live) { src = p.K + r * p.ldk + col0 + c * 8; bytes = 16; }
-        } else {
-            r -= kMhsaRows + p.keys_pad;              // V: key
-            dst = L.v + (r >> 3) * L.lbo_v + c * L.sbo_v + (r & 7) * 16;
-            if (r < p.N && live) { src = p.V + r * p.ldv + col0 + c * 8; bytes = 16; }
-        }
-        cp_async_16(sbase + dst, src, bytes);
-    }
-    cp_async_wait_all();
-    // behind V's d_k chunks: a column of ones (bf16 1.0 in element 0 of the chunk)
-    for (int j = tid; j < p.keys_pad; j += kMhsaThreads)
-        *reinterpret_cast<uint4 *>(smem + L.v + (j >> 3) * L.lbo_v + kchunks * L.sbo_v + (j & 7) * 16) =
-            make_uint4(0x3F80u, 0, 0, 0);
-    fence_proxy_async_smem();                         // make the writes visible to the tensor core
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-
-    // ---- 2. S = Q K^T ---------------------------------------------------------
-    const int n1 = p.keys_pad < 256 ? p.keys_pad : 256;
-    const int n2 = p.keys_pad - n1;
-    if (tid == 0) {
-        for (int part = 0; part < 2; ++part) {
-            const int n = part ? n2 : n1;
-            if (n == 0) break;
-            const uint32_t idesc = make_idesc_bf16(kMhsaRows, n, 0, 0);      // both operands K-major
-            for (int ks = 0; ks < p.dkp / 16; ++ks) {
-                const uint64_t da = make_smem_desc_plain(sbase + L.q + ks * 2 * L.lbo_q, L.lbo_q, 128);
-                const uint64_t db = make_smem_desc_plain(sbase + L.k + ks * 2 * L.lbo_k + part * (256 / 8) * 128,
-                                                         L.lbo_k, 128);
-                umma_bf16_1cta(tmem + part * 256, da, db, idesc, ks > 0 ? 1u : 0u);
-            }
-        }
-        umma_commit(bar);
-    }
-    bool ok = mbar_wait(bar, 0, abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    tc_fence_after();
-
-    // ---- 3. softmax: this thread's half of its row ------------------------------
-    const uint32_t t_row = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-    // Four 32-column loads are in flight per wait: a TMEM round trip costs far
-    // more than the arithmetic on 32 values.
-    float row_max = -INFINITY;
     const int nch = p.keys_pad / 32;
     const int ch_lo = half ? (nch + 1) / 2 : 0, ch_hi = half ? nch : (nch + 1) / 2;
-    if (ok) {
+    const int nblocks = MULTI ? (p.N + p.keys_pad - 1) / p.keys_pad : 1;
+    constexpr int kInFlight = MULTI ? 2 : 4;          // 32-column loads of S per wait (the accumulators need registers too)
+    // running maximum, sum and this thread's half of the row of O (blocks of keys: step 6)
+    float m_run = -INFINITY, l_acc = 0.f;
+    float o_acc[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) o_acc[k] = 0.f;
+    uint32_t tmem = 0;
+    bool ok = true;
+
 #pragma unroll 1
-        for (int ch0 = ch_lo; ch0 < ch_hi; ch0 += 4) {
-            uint32_t r[4][32];
+    for (int kb = 0; kb < nblocks; ++kb) {
+        const int key0 = kb * p.keys_pad;
+        const int nvalid = min(p.keys_pad, p.N - key0);       // keys of this block that exist (>= 1)
+
+        // ---- 1. operands -> shared memory, in core-matrix order -------------------
+        // One list of 16-byte pieces: the rows of Q (first block only), then K's, then V's, the
+        // d_k chunks of a row on neighbouring lanes (at N = 512 and d_k = 32, eighteen per thread).
+        // Asynchronous 16-byte copies straight into shared memory (a piece outside the
+        // operand -- a padding row or d_k chunk -- copies zero source bytes: it is zero-filled).
+        const int first = kb == 0 ? 0 : kMhsaRows << kshift;
+        const int total = (kMhsaRows + 2 * p.keys_pad) << kshift;
+        for (int i = first + tid; i < total; i += kMhsaThreads) {
+            const __nv_bfloat16 *src = p.Q;           // (any valid address: no byte of it is read)
+            uint32_t bytes = 0;
+            int dst;
+            const int c = i & (kchunks - 1);
+            int r = i >> kshift;
+            const bool live = c * 8 < p.dk;
+            if (r < kMhsaRows) {                      // Q: row within the block
+                const int row = q0 + r;
+                dst = L.q + c * L.lbo_q + r * 16;
+                if (row < p.N && live) { src = p.Q + row * p.ldq + col0 + c * 8; bytes = 16; }
+            } else if (r < kMhsaRows + p.keys_pad) {
+                r -= kMhsaRows;                       // K: key of the block
+                dst = L.k + c * L.lbo_k + r * 16;
+                if (r < nvalid && live) { src = p.K + (key0 + r) * p.ldk + col0 + c * 8; bytes = 16; }
+            } else {
+                r -= kMhsaRows + p.keys_pad;          // V: key of the block
+                dst = L.v + (r >> 3) * L.lbo_v + c * L.sbo_v + (r & 7) * 16;
+                if (r < nvalid && live) { src = p.V + (key0 + r) * p.ldv + col0 + c * 8; bytes = 16; }
+            }
+            cp_async_16(sbase + dst, src, bytes);
+        }
+        cp_async_wait_all();
+        // behind V's d_k chunks: a column of ones (bf16 1.0 in element 0 of the chunk)
+        if (kb == 0)
+            for (int j = tid; j < p.keys_pad; j += kMhsaThreads)
+                *reinterpret_cast<uint4 *>(smem + L.v + (j >> 3) * L.lbo_v + kchunks * L.sbo_v + (j & 7) * 16) =
+                    make_uint4(0x3F80u, 0, 0, 0);
+        fence_proxy_async_smem();                     // make the writes visible to the tensor core
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        tmem = *tmem_slot;
+        const uint32_t t_row = tmem + t_row_off;
+
+        // ---- 2. S = Q K^T ---------------------------------------------------------
+        const int n1 = p.keys_pad < 256 ? p.keys_pad : 256;
+        const int n2 = p.keys_pad - n1;
+        if (tid == 0 && ok) {
+            for (int part = 0; part < 2; ++part) {
+                const int n = part ? n2 : n1;
+                if (n == 0) break;
+                const uint32_t idesc = make_idesc_bf16(kMhsaRows, n, 0, 0);      // both operands K-major
+                for (int ks = 0; ks < p.dkp / 16; ++ks) {
+                    const uint64_t da = make_smem_desc_plain(sbase + L.q + ks * 2 * L.lbo_q, L.lbo_q, 128);
+                    const uint64_t db = make_smem_desc_plain(sbase + L.k + ks * 2 * L.lbo_k + part * (256 / 8) * 128,
+                                                             L.lbo_k, 128);
+                    umma_bf16_1cta(tmem + part * 256, da, db, idesc, ks > 0 ? 1u : 0u);
+                }
+            }
+            umma_commit(bar);
+        }
+        if (ok) ok = mbar_wait(bar, 0, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        tc_fence_after();
+
+        // ---- 3. softmax: this thread's half of its row ------------------------------
+        // Several 32-column loads are in flight per wait: a TMEM round trip costs far
+        // more than the arithmetic on 32 values.
+        float blk_max = -INFINITY;
+        if (ok) {
+#pragma unroll 1
+            for (int ch0 = ch_lo; ch0 < ch_hi; ch0 += kInFlight) {
+                uint32_t r[kInFlight][32];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (ch0 + u < ch_hi) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
-            tmem_ld_wait();
+                for (int u = 0; u < kInFlight; ++u)
+                    if (ch0 + u < ch_hi) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
+                tmem_ld_wait();
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (ch0 + u < ch_hi) {
-                    if ((ch0 + u) * 32 + 32 <= p.N) {                        // all 32 keys exist
+                for (int u = 0; u < kInFlight; ++u) {
+                    if (ch0 + u < ch_hi) {
+                        if ((ch0 + u) * 32 + 32 <= nvalid) {                     // all 32 keys exist
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) row_max = fmaxf(row_max, __uint_as_float(r[u][j]));
-                    } else {
+                            for (int j = 0; j < 32; ++j) blk_max = fmaxf(blk_max, __uint_as_float(r[u][j]));
+                        } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if ((ch0 + u) * 32 + j < p.N) row_max = fmaxf(row_max, __uint_as_float(r[u][j]));
+                            for (int j = 0; j < 32; ++j)
+                                if ((ch0 + u) * 32 + j < nvalid) blk_max = fmaxf(blk_max, __uint_as_float(r[u][j]));
+                        }
                     }
                 }
             }
         }
-    }
-    xch[tid] = row_max;
-    __syncthreads();
-    row_max = fmaxf(xch[row_in], xch[row_in + kMhsaRows]);          // the first half always has a key < N
-    const float neg_max_scaled = -row_max * p.scale_log2;
-    if (ok) {
-        const int r_off = (row_in >> 3) * 128 + (row_in & 7) * 16;           // this row inside a chunk of P
+        xch[tid] = blk_max;
+        __syncthreads();
+        blk_max = fmaxf(xch[row_in], xch[row_in + kMhsaRows]);      // the first half always has a key that exists
+        const float m_new = fmaxf(m_run, blk_max);
+        // what the accumulators of the earlier blocks are worth relative to the new maximum
+        const float alpha = (!MULTI || kb == 0) ? 0.f : fast_exp2((m_run - m_new) * p.scale_log2);
+        m_run = m_new;
+        const float neg_max_scaled = -m_new * p.scale_log2;
+        if (ok) {
+            const int r_off = (row_in >> 3) * 128 + (row_in & 7) * 16;           // this row inside a chunk of P
 #pragma unroll 1
-        for (int ch0 = ch_lo; ch0 < ch_hi; ch0 += 4) {
-            uint32_t r[4][32];
+            for (int ch0 = ch_lo; ch0 < ch_hi; ch0 += kInFlight) {
+                uint32_t r[kInFlight][32];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (ch0 + u < ch_hi) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
-            tmem_ld_wait();
+                for (int u = 0; u < kInFlight; ++u)
+                    if (ch0 + u < ch_hi) tmem_ld_32x32b_x32(t_row + (ch0 + u) * 32, r[u]);
+                tmem_ld_wait();
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int ch = ch0 + u;
-                if (ch < ch_hi) {
-                    uint32_t w[16];
-                    if (ch * 32 + 32 <= p.N) mhsa_exp_chunk<false>(r[u], p.scale_log2, neg_max_scaled, 32, w);
-                    else                     mhsa_exp_chunk<true>(r[u], p.scale_log2, neg_max_scaled, p.N - ch * 32, w);
+                for (int u = 0; u < kInFlight; ++u) {
+                    const int ch = ch0 + u;
+                    if (ch < ch_hi) {
+                        uint32_t w[16];
+                        if (ch * 32 + 32 <= nvalid) mhsa_exp_chunk<false>(r[u], p.scale_log2, neg_max_scaled, 32, w);
+                        else                        mhsa_exp_chunk<true>(r[u], p.scale_log2, neg_max_scaled, nvalid - ch * 32, w);
 #pragma unroll
-                    for (int g = 0; g < 4; ++g)                              // 8 keys = one 16-byte chunk
-                        *reinterpret_cast<uint4 *>(smem + L.p + (ch * 4 + g) * 2048 + r_off) =
-                            make_uint4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+                        for (int g = 0; g < 4; ++g)                              // 8 keys = one 16-byte chunk
+                            *reinterpret_cast<uint4 *>(smem + L.p + (ch * 4 + g) * 2048 + r_off) =
+                                make_uint4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+                    }
                 }
             }
         }
-    }
-    fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();                                   // everyone is done reading S and writing P
-    tc_fence_after();
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();                               // everyone is done reading S and writing P
+        tc_fence_after();
 
-    // ---- 4. O = P V -------------------------------------------------------------
-    if (tid == 0 && ok) {
-        const uint32_t idesc = make_idesc_bf16(kMhsaRows, p.dkp + 16, 0, 1); // [V | 1 | unused]: MN-major
-        for (int ks = 0; ks < p.keys_pad / 16; ++ks) {
-            const uint64_t da = make_smem_desc_plain(sbase + L.p + ks * 2 * 2048, 2048, 128);
-            const uint64_t db = make_smem_desc_plain(sbase + L.v + ks * 2 * L.lbo_v, L.lbo_v, L.sbo_v);
-            umma_bf16_1cta(tmem, da, db, idesc, ks > 0 ? 1u : 0u);
+        // ---- 4. O = P V -------------------------------------------------------------
+        if (tid == 0 && ok) {
+            const uint32_t idesc = make_idesc_bf16(kMhsaRows, p.dkp + 16, 0, 1); // [V | 1 | unused]: MN-major
+            for (int ks = 0; ks < p.keys_pad / 16; ++ks) {
+                const uint64_t da = make_smem_desc_plain(sbase + L.p + ks * 2 * 2048, 2048, 128);
+                const uint64_t db = make_smem_desc_plain(sbase + L.v + ks * 2 * L.lbo_v, L.lbo_v, L.sbo_v);
+                umma_bf16_1cta(tmem, da, db, idesc, ks > 0 ? 1u : 0u);
+            }
+            umma_commit(bar);
         }
-        umma_commit(bar);
+        if (ok) {
+            ok = mbar_wait(bar, 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        tc_fence_after();
+
+        // ---- 6. the block's O and row sum join the accumulators ---------------------
+        if (ok) {
+            uint32_t r[32], r2[32];
+            tmem_ld_32x32b_x32(t_row, r);              // d_k <= 32 columns of O ...
+            if (p.dkp == 32) tmem_ld_32x32b_x32(t_row + 32, r2);             // ... and the row sum in column dkp
+            tmem_ld_wait();
+            if (MULTI) {
+                l_acc = fmaf(l_acc, alpha, __uint_as_float(p.dkp == 32 ? r2[0] : r[16]));
+#pragma unroll
+                for (int k = 0; k < 16; ++k) o_acc[k] = fmaf(o_acc[k], alpha, __uint_as_float(half ? r[16 + k] : r[k]));
+            } else {
+                l_acc = __uint_as_float(p.dkp == 32 ? r2[0] : r[16]);
+#pragma unroll
+                for (int k = 0; k < 16; ++k) o_acc[k] = __uint_as_float(half ? r[16 + k] : r[k]);
+            }
+        }
+        if (MULTI && kb + 1 < nblocks) {
+            tc_fence_before();
+            __syncthreads();                           // O has been read: the next block may overwrite S, K, V and P
+            tc_fence_after();
+        }
     }
-    if (ok) {
-        ok = mbar_wait(bar, 1, abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-    }
-    tc_fence_after();
 
     // ---- 5. normalise and store (each of the row's two threads: half of d_k) -----
     // P's shared memory is free now and takes the 128 x d_k block of O, rows 36 floats
@@ -313,15 +368,11 @@ mhsa_kernel(const MhsaParams p)
     const bool vec_out = ((reinterpret_cast<uintptr_t>(p.O) & 15) == 0) && (p.ldo % 4 == 0);
     float *stage = reinterpret_cast<float *>(smem + L.p);
     if (ok) {
-        uint32_t r[32], r2[32];
-        tmem_ld_32x32b_x32(t_row, r);                  // d_k <= 32 columns of O ...
-        if (p.dkp == 32) tmem_ld_32x32b_x32(t_row + 32, r2);                 // ... and the row sum in column dkp
-        tmem_ld_wait();
         const int row = q0 + row_in;
-        const float inv = 1.f / __uint_as_float(p.dkp == 32 ? r2[0] : r[16]);
+        const float inv = 1.f / l_acc;
         float o[16];                                   // this thread's half of the row
 #pragma unroll
-        for (int k = 0; k < 16; ++k) o[k] = __uint_as_float(half ? r[16 + k] : r[k]) * inv;
+        for (int k = 0; k < 16; ++k) o[k] = o_acc[k] * inv;
         if (vec_out) {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
