@@ -96,7 +96,7 @@ def test_attention_entry_point_validates_first():
     assert f(p, p, p, p, 64, 32, 4, 32, 31, 32, 32) == B.ERR_INVALID_LD
     assert f(p, None, p, p, 64, 32, 4, 32, 32, 32, 32) == B.ERR_INVALID_POINTER
     assert f(p, p, p, p + 2, 64, 32, 4, 32, 32, 32, 32) == B.ERR_MISALIGNED
-    assert f(p, p, p, p, 513, 32, 4, 32, 32, 32, 32) == B.ERR_UNSUPPORTED_SHAPE    # more than 512 keys
+    assert f(p, p, p, p, 1 << 31, 32, 4, 32, 32, 32, 32) == B.ERR_INVALID_DIM      # any sequence length below 2^31 - 1024
     assert f(p, p, p, p, 64, 160, 4, 160, 160, 160, 160) == B.ERR_UNSUPPORTED_SHAPE  # d_k = 40
     assert f(p + 2, p, p, p, 64, 32, 4, 32, 32, 32, 32) == B.ERR_UNSUPPORTED_SHAPE  # Q not 16-byte aligned
     assert f(None, None, None, None, 0, 32, 4, 32, 32, 32, 32) == B.OK
