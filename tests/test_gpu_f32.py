@@ -232,3 +232,21 @@ def test_tf32_unaligned_operands_take_the_three_piece_path_and_errors():
     assert B.gemm_tf32(x, x, x, 4, 4, 4, 3, 4, 4, s, check=False) == B.ERR_INVALID_LD
     assert B.gemm_tf32(x.data_ptr() + 2, x, x, 4, 4, 4, 4, 4, 4, s, check=False) == B.ERR_MISALIGNED
     assert B.gemm_tf32(x, x, x, 0, 4, 4, 4, 4, 4, s, check=False) == B.OK
+
+
+@pytest.mark.parametrize("step", [2, 3])
+def test_tf32_paper_task2_ladder_closed_form(step):
+    """The paper's Task 2 shapes A (size x 4096) x B (4096 x 2048), size = 2^14 and 2^16, as
+    float32 through the TF32 kernel (CTA pairs, the last wave split along K): rank-one integer
+    operands with at most 8 significant bits, every element exact."""
+    cfg = gi.task2_ladder(step)
+    u, v_, p, q = gi.rank1_int_factors(cfg.M, cfg.N, cfg.K, seed=60 + step)
+    dA = torch.outer(torch.from_numpy(u.astype(np.float32)).cuda(), torch.from_numpy(p.astype(np.float32)).cuda())
+    dB = torch.outer(torch.from_numpy(q.astype(np.float32)).cuda(), torch.from_numpy(v_.astype(np.float32)).cuda())
+    dC = torch.full((cfg.M * cfg.N,), float("nan"), dtype=torch.float32, device="cuda")
+    B.gemm_tf32(dA, dB, dC, cfg.M, cfg.N, cfg.K, cfg.K, cfg.N, cfg.N, torch.cuda.current_stream())
+    assert B.device_status(torch.cuda.current_stream()) == (B.OK, 0)
+    scale = float(np.dot(p, q))
+    want = torch.outer(torch.from_numpy(u.astype(np.float32)).cuda(),
+                       torch.from_numpy(v_.astype(np.float32)).cuda()) * scale      # exact in fp32
+    assert torch.equal(dC.view(cfg.M, cfg.N), want)
