@@ -1191,8 +1191,12 @@ int cudallm_gemm_tf32(const void *A, const void *B, void *C, int64_t M, int64_t 
     if (st != CUDALLM_OK) return st;
     st = encode_map(dev, &tb, B, N, K, 1, ldb, 0, 32, kTf32BlockK, 3);
     if (st != CUDALLM_OK) return st;
-    // (the raster-group rule counts A's bytes as bf16: here its slices are twice that, still in L2)
-    GemmParams gp = make_params(p, t, kBlockM);
+    // raster groups as for bf16, but A's elements are four bytes: as many tile rows as keep the
+    // group's slice of A within about 32 MB, rounded down to a power of two (the knob's unit)
+    int64_t group = (int64_t(32) << 20) / (cdiv(M, t.tiles_m) * K * 4 + 1);
+    int knob = 1;
+    while (knob < 15 && (int64_t(2) << (knob - 1)) <= group) ++knob;
+    GemmParams gp = make_params(p, t, kBlockM, knob);
     st = encode_c_map(dev, &tc, p, gp.c_tma != 0);
     if (st != CUDALLM_OK) return st;
     set_split_epoch(gp, d, t.split > 1);

@@ -260,16 +260,19 @@ umma_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 // The same product on CTA pairs (cta_group::2), as umma_gemm_2cta_kernel does it
 // for bf16: a cluster of two CTAs owns a 256 x 256 tile, CTA r stages rows
 // [128 r, 128 r + 128) of A and columns [128 r, 128 r + 128) of B (32 instead of
-// 48 KiB per k-block and SM, six stages instead of four), the leader issues
+// 48 KiB per k-block and SM; three stages of two k-blocks each, so that producer and
+// MMA thread pay one barrier round trip per 64 of K), the leader issues
 // 256 x 256 x 8 MMAs for both, and the barriers are laid out as there (the
 // leader's `full`, each CTA's `empty`, no multicast).
-constexpr int kTf32PairStages = 6;
+constexpr int kTf32PairStages = 3;
+constexpr int kTf32PairSub = 2;                                       // k-blocks per stage: one barrier round trip per 64 of K
 
 struct Tf32PairSmem {
     static constexpr int kABytes = kBlockM * kTf32BlockK * 4;        // 16 KiB: this CTA's 128 rows of A
     static constexpr int kBoxBytes = 32 * kTf32BlockK * 4;
     static constexpr int kBBytes = (kPairN / 2 / 32) * kBoxBytes;    // 16 KiB: this CTA's 128 columns of B
-    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kSubBytes = kABytes + kBBytes;              // one k-block
+    static constexpr int kStageBytes = kTf32PairSub * kSubBytes;
     static constexpr int kEpiOffset = kTf32PairStages * kStageBytes;
     static constexpr int kBarOffset = kEpiOffset + kEpiStageBytes;
     static constexpr int kNumBars = 2 * kTf32PairStages + 4;
@@ -366,19 +369,23 @@ umma_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 const UnitCoord c = decode_unit(p, u);
                 const int row0 = c.m_tile * kPairM + static_cast<int>(rank) * kBlockM;
                 const int col0 = c.n_tile * kPairN + static_cast<int>(rank) * half;
-                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                for (int kb = c.kb_begin; kb < c.kb_end; kb += kTf32PairSub) {
                     if (!mbar_wait<true>(empty_bar(stage), phase ^ 1, abort_flag, p.wait_limit_ns)) {
                         report_timeout(p.status, kRoleProducer, stage);
                         ok = false;
                         break;
                     }
-                    const uint32_t sa = smem_base + stage * L::kStageBytes, sb = sa + L::kABytes;
+                    const int nsub = min(kTf32PairSub, c.kb_end - kb);
                     const uint32_t bar = leader_full0 + 8u * stage;
-                    if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * L::kStageBytes);
-                    tma_load_3d_pair(sa, &tmap_a, kb * kTf32BlockK, row0, c.b, bar);
+                    if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * nsub * L::kSubBytes);
+                    for (int sub = 0; sub < nsub; ++sub) {
+                        const uint32_t sa = smem_base + stage * L::kStageBytes + sub * L::kSubBytes, sb = sa + L::kABytes;
+                        const int k = (kb + sub) * kTf32BlockK;
+                        tma_load_3d_pair(sa, &tmap_a, k, row0, c.b, bar);
 #pragma unroll
-                    for (int j = 0; j < half / 32; ++j)
-                        tma_load_3d_pair(sb + j * L::kBoxBytes, &tmap_b, col0 + 32 * j, kb * kTf32BlockK, c.b, bar);
+                        for (int j = 0; j < half / 32; ++j)
+                            tma_load_3d_pair(sb + j * L::kBoxBytes, &tmap_b, col0 + 32 * j, k, c.b, bar);
+                    }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
@@ -405,19 +412,22 @@ umma_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kPairN;
                 uint32_t accumulate = 0;
-                for (int kb = c.kb_begin; kb < c.kb_end; ++kb) {
+                for (int kb = c.kb_begin; kb < c.kb_end; kb += kTf32PairSub) {
                     if (!mbar_wait<true>(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) {
                         report_timeout(p.status, kRoleMma, stage);
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t sa = smem_base + stage * L::kStageBytes, sb = sa + L::kABytes;
+                    const int nsub = min(kTf32PairSub, c.kb_end - kb);
+                    for (int sub = 0; sub < nsub; ++sub) {
+                        const uint32_t sa = smem_base + stage * L::kStageBytes + sub * L::kSubBytes, sb = sa + L::kABytes;
 #pragma unroll
-                    for (int i = 0; i < kTf32BlockK / 8; ++i) {
-                        umma_tf32_pair(d_tmem, make_smem_desc_sw128(sa + 32 * i, 16, 1024),
-                                       make_smem_desc_sw128_32b(sb + 1024 * i, L::kBoxBytes, 512), idesc, accumulate);
-                        accumulate = 1;
+                        for (int i = 0; i < kTf32BlockK / 8; ++i) {
+                            umma_tf32_pair(d_tmem, make_smem_desc_sw128(sa + 32 * i, 16, 1024),
+                                           make_smem_desc_sw128_32b(sb + 1024 * i, L::kBoxBytes, 512), idesc, accumulate);
+                            accumulate = 1;
+                        }
                     }
                     umma_commit_pair(empty0_cta0 + 8u * stage);      // frees the stage in both CTAs
                     umma_commit_pair(empty0_cta1 + 8u * stage);
