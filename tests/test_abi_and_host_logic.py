@@ -88,6 +88,21 @@ def test_fp32_entry_point_validates_first():
     assert f(None, None, None, 0, 4, 4, 4, 4, 4) == B.OK
 
 
+def test_tf32_entry_point_and_debug_hooks_validate_first():
+    p = 4096
+    f = lambda *a: B.gemm_tf32(*a, check=False)
+    assert f(None, p, p, 4, 4, 4, 4, 4, 4) == B.ERR_INVALID_POINTER
+    assert f(p, p, p, 4, 4, 4, 3, 4, 4) == B.ERR_INVALID_LD
+    assert f(p, p, p, 4, -4, 4, 4, 4, 4) == B.ERR_INVALID_DIM
+    assert f(p + 2, p, p, 4, 4, 4, 4, 4, 4) == B.ERR_MISALIGNED
+    assert f(p, p, p + 2, 4, 4, 4, 4, 4, 4) == B.ERR_MISALIGNED
+    assert f(None, None, None, 0, 4, 4, 4, 4, 4) == B.OK
+    # the hooks are host-side switches: unknown ones and values out of range are refused
+    assert B.debug_set(B.DEBUG_LAYERNORM_PATH, 3, check=False) == B.ERR_INVALID_VARIANT
+    assert B.debug_set(B.DEBUG_LAYERNORM_PATH, 0, check=False) == B.OK
+    assert B.debug_set(99, 0, check=False) == B.ERR_INVALID_VARIANT
+
+
 def test_attention_entry_point_validates_first():
     p = 4096
     f = lambda *a: B.mhsa_bf16(*a, check=False)
