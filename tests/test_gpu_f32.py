@@ -250,3 +250,16 @@ def test_tf32_paper_task2_ladder_closed_form(step):
     want = torch.outer(torch.from_numpy(u.astype(np.float32)).cuda(),
                        torch.from_numpy(v_.astype(np.float32)).cuda()) * scale      # exact in fp32
     assert torch.equal(dC.view(cfg.M, cfg.N), want)
+
+
+def test_tf32_random_shapes():
+    rng = np.random.default_rng(5300)
+    for it in range(40):
+        M = int(np.exp(rng.uniform(0, np.log(700)))); N = 4 * int(np.exp(rng.uniform(0, np.log(200))))
+        K = 4 * int(np.exp(rng.uniform(0, np.log(400))))
+        Af = rng.standard_normal((M, K)).astype(np.float32)
+        Bf = rng.uniform(-1, 1, (K, N)).astype(np.float32)
+        got = run_tf32(Af, Bf, M, N, K, pad_ab=4 * int(rng.integers(0, 3)), pad_c=int(rng.integers(0, 4)))
+        Cref, S = oracle.gemm_f32(Af, Bf, M, N, K)
+        r = oracle.check(got, Cref, S, oracle.TOL_TF32)
+        assert r.ok, (M, N, K, r)

@@ -87,6 +87,17 @@ def test_sequences_longer_than_one_block_of_keys(N, dm, h, pad):
     assert oracle.check(run(Q2, K2, V, N, dm, h, pad), ref2, T2, oracle.TOL_MHSA).ok
 
 
+def test_random_lengths_and_head_shapes():
+    rng = np.random.default_rng(77)
+    for it in range(30):
+        h = int(rng.choice([1, 2, 3, 4, 8])); dk = int(rng.choice([8, 16, 24, 32])); dm = h * dk
+        N = int(np.exp(rng.uniform(0, np.log(1800))))
+        Q, K, V = (bits(rng.standard_normal((N, dm))) for _ in range(3))
+        ref, T = oracle.mhsa(Q, K, V, N, dm, h)
+        r = oracle.check(run(Q, K, V, N, dm, h, int(rng.integers(0, 2))), ref, T, oracle.TOL_MHSA)
+        assert r.ok, (N, dm, h, r)
+
+
 def test_closed_forms_over_several_blocks():
     rng = np.random.default_rng(3)
     N, dm, h = 1500, 64, 2

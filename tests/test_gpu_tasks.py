@@ -244,6 +244,15 @@ def test_layernorm_one_pass_kernel_against_oracle(layernorm_path, batch, m):
     check_layernorm(run_layernorm(x, gamma, beta, batch, m), x, gamma, beta, batch, m)
 
 
+def test_layernorm_random_sizes_on_both_paths(layernorm_path):
+    rng = np.random.default_rng(4400)
+    for it in range(24):
+        batch = int(rng.integers(1, 12)); m = 8 * int(np.exp(rng.uniform(0, np.log(60000))))
+        x, gamma, beta = gi.layernorm_inputs(4400 + it, batch, m)
+        layernorm_path(int(rng.choice([1, 2])))
+        check_layernorm(run_layernorm(x, gamma, beta, batch, m), x, gamma, beta, batch, m)
+
+
 def test_layernorm_one_pass_kernel_variants_of_the_call(layernorm_path):
     layernorm_path(2)
     batch, m = 6, 148 * 1024 + 64
