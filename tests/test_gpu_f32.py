@@ -234,9 +234,9 @@ def test_tf32_unaligned_operands_take_the_three_piece_path_and_errors():
     assert B.gemm_tf32(x, x, x, 0, 4, 4, 4, 4, 4, s, check=False) == B.OK
 
 
-@pytest.mark.parametrize("step", [2, 3])
+@pytest.mark.parametrize("step", [2, 3, 4])
 def test_tf32_paper_task2_ladder_closed_form(step):
-    """The paper's Task 2 shapes A (size x 4096) x B (4096 x 2048), size = 2^14 and 2^16, as
+    """The paper's Task 2 shapes A (size x 4096) x B (4096 x 2048), size = 2^14, 2^16 and 2^18 (4 GiB of A), as
     float32 through the TF32 kernel (CTA pairs, the last wave split along K): rank-one integer
     operands with at most 8 significant bits, every element exact."""
     cfg = gi.task2_ladder(step)
