@@ -258,6 +258,26 @@ __device__ __forceinline__ void stage_row_swizzled(uint32_t blk, int lane, const
     }
 }
 
+// One thread's row of 32 floats -> its row of a staging block (36 floats per row), moved
+// right by A elements: position A + i holds v[i], so that the 16-byte pieces of the row
+// in shared memory are the 16-byte-aligned pieces of the row in a C whose element (row, col0)
+// lies A elements behind a 16-byte boundary.  (Positions outside A .. A + 31 get zeros that
+// nobody stores.)
+template <int A>
+__device__ __forceinline__ void stage_row_shifted(uint32_t row_addr, const float (&v)[32])
+{
+#pragma unroll
+    for (int q = 0; q < (A ? 9 : 8); ++q) {
+        float w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = 4 * q + j - A;
+            w[j] = (i >= 0 && i < 32) ? v[i < 0 ? 0 : (i > 31 ? 31 : i)] : 0.f;
+        }
+        st_shared_v4(row_addr + 16 * q, w[0], w[1], w[2], w[3]);
+    }
+}
+
 // Stores one 32 x 32 block of the accumulator (this warp's 32 rows, 32
 // consecutive columns from col0) to C.  Each thread arrives with the 32 values
 // of ITS row (v); writing them as they are would make every store instruction
@@ -298,6 +318,57 @@ __device__ __forceinline__ void store_block_staged(const GemmParams &p, const CU
     if (p.c_tma) {                                       // earlier TMA stores may still read the staging blocks
         if (lane == 0) bulk_wait_group_read<0>();
         __syncwarp();
+    }
+    if (!OUT_BF16 && col0 + 32 <= p.N) {
+        // fp32 rows that are only 4-byte aligned: each row's 16-byte-aligned body goes out in
+        // 16-byte stores (four rows per instruction), the up to three elements before and
+        // after it in element stores (eight rows per instruction).
+        const long long e0 = static_cast<long long>(reinterpret_cast<uintptr_t>(p.C) >> 2)
+                           + static_cast<long long>(b) * p.strideC + static_cast<long long>(row0) * p.ldc + col0;
+        const uint32_t my_row = stage + lane * (kEpiPitch * 4);
+        switch (static_cast<int>((e0 + lane * p.ldc) & 3)) {
+        case 0:  stage_row_shifted<0>(my_row, v); break;
+        case 1:  stage_row_shifted<1>(my_row, v); break;
+        case 2:  stage_row_shifted<2>(my_row, v); break;
+        default: stage_row_shifted<3>(my_row, v); break;
+        }
+        __syncwarp();
+        const int rows = min(32, p.M - row0);
+        float *c0 = reinterpret_cast<float *>(p.C) + (static_cast<long long>(b) * p.strideC
+                                                      + static_cast<long long>(row0) * p.ldc + col0);
+        float4 body[8];
+        float edge[4];
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {                    // rows 4g .. 4g + 3, lane k of a row: piece k (+ 1)
+            const int r = 4 * g + (lane >> 3);
+            const int a = static_cast<int>((e0 + r * p.ldc) & 3);
+            const int piece = (lane & 7) + (a ? 1 : 0);
+            const uint32_t src = stage + (r * kEpiPitch + 4 * piece) * 4;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                         : "=f"(body[g].x), "=f"(body[g].y), "=f"(body[g].z), "=f"(body[g].w) : "r"(src) : "memory");
+        }
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {                    // rows 8g .. 8g + 7, lane e of a row: its e-th edge element
+            const int r = 8 * g + (lane >> 2), e = lane & 3;
+            const int a = static_cast<int>((e0 + r * p.ldc) & 3);
+            edge[g] = ld_shared_f32(stage + (r * kEpiPitch + (e >= a ? e : 32 + e)) * 4);
+        }
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            const int r = 4 * g + (lane >> 3);
+            const int a = static_cast<int>((e0 + r * p.ldc) & 3);
+            const int piece = (lane & 7) + (a ? 1 : 0);
+            if (r < rows && piece < 8)
+                *reinterpret_cast<float4 *>(c0 + r * p.ldc - a + 4 * piece) = body[g];
+        }
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int r = 8 * g + (lane >> 2), e = lane & 3;
+            const int a = static_cast<int>((e0 + r * p.ldc) & 3);
+            if (r < rows && a) c0[r * p.ldc - a + (e >= a ? e : 32 + e)] = edge[g];
+        }
+        __syncwarp();                                    // the block is reused for the next chunk
+        return;
     }
 #pragma unroll
     for (int q = 0; q < 8; ++q)
