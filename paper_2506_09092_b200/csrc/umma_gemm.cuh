@@ -292,8 +292,15 @@ __device__ __forceinline__ void stage_row_shifted(uint32_t row_addr, const float
 //    store to have read it.  The clipping works in units of 16 bytes (measured:
 //    with N = 127 column 127 is written), so a box that straddles an N whose
 //    row length is not a multiple of 16 bytes takes the other path.
-//  * otherwise: rows 36 floats apart, read back one row per instruction and
-//    written with element stores that are contiguous per row.
+//  * fp32 C that TMA cannot address (rows only 4-byte aligned), block inside N: the
+//    thread writes its row moved right by the row's own misalignment (0 to 3
+//    elements), so that the 16-byte pieces of the staged row are the 16-byte-aligned
+//    pieces of the row of C; those go out in 16-byte stores, four rows per
+//    instruction, and the up to three elements before and after them in element
+//    stores, eight rows per instruction (12 store instructions per block, not 32).
+//  * otherwise (bf16 C, or the block that straddles column N): rows 36 floats apart,
+//    read back one row per instruction and written with element stores that are
+//    contiguous per row.
 // `stage` = shared-memory address of the warp's 8 KiB; `sel` alternates between
 // its two blocks; row0 = global row of lane 0; b = batch item.
 template <bool OUT_BF16>
